@@ -1,0 +1,327 @@
+"""Pins for the oracle's transformer and for the whole speculative loop on real (tiny) models.
+
+The paper prints no architecture values, so the forward pass is pinned by special cases with closed
+forms, an independent matrix-form restatement, invariances, and parallel == sequential scoring
+(section "Conditional Scoring").  The loop is pinned end to end by Theorem 1: the first tokens SpS
+emits follow the target's own autoregressive law exactly."""
+import numpy as np
+import pytest
+import torch
+from scipy.stats import chi2
+
+import oracle
+import sps_synth
+from test_oracle_sampler import chi_square_p, sm
+
+TINY = sps_synth.CONFIGS["tiny"]
+
+
+def np_weights(cfg, seed=0, tag="target", **kw):
+    return sps_synth.weights_to_numpy(sps_synth.make_weights(cfg, seed=seed, tag=tag, **kw))
+
+
+def as_f64(a):
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).double().numpy()
+    return a.astype(np.float64)
+
+
+def round_storage(x, dtype):
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    if dtype == 0:
+        return t.float().double().numpy()
+    return t.to(torch.bfloat16).double().numpy()
+
+
+def gelu_tanh(v):
+    return 0.5 * v * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (v + 0.044715 * v ** 3)))
+
+
+def matrix_forward(cfg, w, tokens):
+    """Whole-sequence, matrix-form forward pass (positions 0..n-1), written independently of the oracle."""
+    d, H, dh, eps = cfg["d_model"], cfg["n_heads"], cfg["d_head"], cfg["rms_eps"]
+    n = len(tokens)
+    x = as_f64(w["tok_embed"])[tokens]
+    pos = np.arange(n)[:, None]
+    freq = cfg["rope_base"] ** (-2.0 * np.arange(dh // 2) / dh)[None, :]
+    cos, sin = np.cos(pos * freq), np.sin(pos * freq)
+
+    def norm(v, g):
+        return g.astype(np.float64) * v / np.sqrt((v ** 2).mean(-1, keepdims=True) + eps)
+
+    def rope(a):  # a [n, H, dh]
+        a0, a1 = a[..., 0::2], a[..., 1::2]
+        out = np.empty_like(a)
+        out[..., 0::2] = a0 * cos[:, None, :] - a1 * sin[:, None, :]
+        out[..., 1::2] = a0 * sin[:, None, :] + a1 * cos[:, None, :]
+        return out
+
+    mask = np.tril(np.ones((n, n), dtype=bool))
+    for lw in w["layers"]:
+        h = norm(x, lw["attn_norm"])
+        q = rope((h @ as_f64(lw["wq"]).T).reshape(n, H, dh))
+        k = round_storage(rope((h @ as_f64(lw["wk"]).T).reshape(n, H, dh)), cfg["dtype"])
+        v = round_storage((h @ as_f64(lw["wv"]).T).reshape(n, H, dh), cfg["dtype"])
+        sc = np.einsum("ihd,jhd->hij", q, k) / np.sqrt(dh)
+        sc = np.where(mask[None], sc, -np.inf)
+        pr = np.exp(sc - sc.max(-1, keepdims=True))
+        pr /= pr.sum(-1, keepdims=True)
+        o = np.einsum("hij,jhd->ihd", pr, v).reshape(n, d)
+        x = x + o @ as_f64(lw["wo"]).T
+        h = norm(x, lw["ffn_norm"])
+        x = x + gelu_tanh(h @ as_f64(lw["w_up"]).T) @ as_f64(lw["w_down"]).T
+    return norm(x, w["final_norm"]) @ as_f64(w["unembed"]).T
+
+
+@pytest.mark.parametrize("name,tag", [("tiny", "target"), ("tiny", "draft"), ("tiny_bf16", "target")])
+def test_forward_matches_matrix_restatement(name, tag):
+    cfg = sps_synth.CONFIGS[name][tag]
+    w = np_weights(cfg, seed=0, tag=tag, std=0.08)   # larger std so attention is far from uniform
+    toks = sps_synth.make_prompt(3, 12, cfg["vocab"])
+    m = oracle.Transformer(cfg, w, max_seq=32)
+    got = m.forward64(toks, np.arange(12))
+    want = matrix_forward(cfg, w, toks)
+    assert np.abs(got - want).max() < 1e-9 * max(1.0, np.abs(want).max())
+
+
+def test_parallel_scoring_equals_sequential_scoring():
+    """K+1 rows in one call give the K+1 conditionals that single-row calls give (Conditional Scoring)."""
+    cfg = TINY["target"]
+    w = np_weights(cfg)
+    toks = sps_synth.make_prompt(1, 14, cfg["vocab"])
+    a = oracle.Transformer(cfg, w, max_seq=32)
+    b = oracle.Transformer(cfg, w, max_seq=32)
+    a.forward(toks[:9], np.arange(9), want_logits=False)
+    par = a.forward64(toks[9:14], np.arange(9, 14))
+    for i in range(9):
+        b.forward(toks[i:i + 1], [i], want_logits=False)
+    for i in range(9, 14):
+        seq = b.forward64(toks[i:i + 1], [i])
+        assert np.abs(seq[0] - par[i - 9]).max() < 1e-12
+
+
+def test_rollback_is_a_length_rewind():
+    """Rows written for rejected drafts are never read again: after accepting 2 of 5 drafts and feeding
+    other tokens at the following positions, logits equal those of a fresh pass over the true sequence."""
+    cfg = TINY["target"]
+    w = np_weights(cfg)
+    V = cfg["vocab"]
+    toks = sps_synth.make_prompt(2, 10, V)
+    drafts = sps_synth.make_prompt(3, 5, V)
+    nxt = sps_synth.make_prompt(4, 3, V)
+    a = oracle.Transformer(cfg, w, max_seq=32)
+    a.forward(toks, np.arange(10), want_logits=False)
+    a.forward(drafts, np.arange(10, 15), want_logits=False)     # positions 10..14 speculative
+    got = a.forward64(nxt, np.arange(12, 15))                   # keep 10, 11; overwrite from 12
+    b = oracle.Transformer(cfg, w, max_seq=32)
+    true_seq = np.concatenate([toks, drafts[:2], nxt])
+    want = b.forward64(true_seq, np.arange(15))[12:]
+    assert np.abs(got - want).max() < 1e-12
+
+
+def test_special_cases_with_closed_forms():
+    cfg = dict(TINY["draft"], n_layers=1)
+    d, V = cfg["d_model"], cfg["vocab"]
+    rng = np.random.default_rng(0)
+    base = np_weights(cfg, tag="draft", std=0.1)
+    toks = sps_synth.make_prompt(5, 6, V)
+    E, U = base["tok_embed"].astype(np.float64), base["unembed"].astype(np.float64)
+
+    def rms(v):
+        return v / np.sqrt((v ** 2).mean(-1, keepdims=True) + cfg["rms_eps"])
+
+    def run(w):
+        return oracle.Transformer(cfg, w, max_seq=16).forward64(toks, np.arange(6))
+
+    zero = {k: np.zeros_like(v) if k not in ("attn_norm", "ffn_norm") else v for k, v in base["layers"][0].items()}
+    # (a) every layer matrix zero: logits = U rmsnorm(E[tok])
+    w = dict(base, layers=[dict(zero)])
+    assert np.abs(run(w) - rms(E[toks]) @ U.T).max() < 1e-12
+    # (b) wq = wk = 0: attention is a uniform average over positions <= i;  x_i += Wo mean_{j<=i} Wv h_j
+    lw = dict(zero)
+    lw["wv"] = (rng.normal(size=(d, d)) * 0.1).astype(np.float32)
+    lw["wo"] = (rng.normal(size=(d, d)) * 0.1).astype(np.float32)
+    h = rms(E[toks])
+    vals = np.float32(h @ lw["wv"].astype(np.float64).T).astype(np.float64)  # cache holds fp32
+    x = E[toks] + np.stack([vals[: i + 1].mean(0) for i in range(6)]) @ lw["wo"].astype(np.float64).T
+    got = run(dict(base, layers=[lw]))
+    assert np.abs(got - rms(x) @ U.T).max() < 1e-6
+    # (c) attention off, FFN on: x += Wdown gelu(Wup rmsnorm(x))
+    lw = dict(zero)
+    lw["w_up"] = (rng.normal(size=(cfg["d_ff"], d)) * 0.2).astype(np.float32)
+    lw["w_down"] = (rng.normal(size=(d, cfg["d_ff"])) * 0.2).astype(np.float32)
+    x = E[toks] + gelu_tanh(rms(E[toks]) @ lw["w_up"].astype(np.float64).T) @ lw["w_down"].astype(np.float64).T
+    assert np.abs(run(dict(base, layers=[lw])) - rms(x) @ U.T).max() < 1e-10
+    # (d) a norm gain of g scales that norm's output: with zero layers, final gain 2 doubles the logits
+    w = dict(base, layers=[dict(zero)], final_norm=np.full(d, 2.0, dtype=np.float32))
+    assert np.abs(run(w) - 2 * rms(E[toks]) @ U.T).max() < 1e-12
+
+
+def test_invariances():
+    cfg = TINY["target"]
+    w = np_weights(cfg, std=0.08)
+    toks = sps_synth.make_prompt(6, 8, cfg["vocab"])
+    m = oracle.Transformer(cfg, w, max_seq=64)
+    base = m.forward64(toks, np.arange(8))
+    # rotary: the layer-0 key of one token cached at two positions differs by a rotation of each
+    # adjacent pair (2i, 2i+1) through (p2 - p1) * base^(-2i/d_head); values carry no position
+    dh, H = cfg["d_head"], cfg["n_heads"]
+    m2 = oracle.Transformer(cfg, w, max_seq=64)
+    m.forward(toks[:1], [3], want_logits=False)
+    m2.forward(toks[:1], [10], want_logits=False)
+    k3, v3 = m.kv(0, 3)
+    k10, v10 = m2.kv(0, 10)
+    assert np.array_equal(v3, v10)
+    ang = 7.0 * cfg["rope_base"] ** (-2.0 * np.arange(dh // 2) / dh)
+    k3h = k3.astype(np.float64).reshape(H, dh // 2, 2)
+    rot = np.stack([k3h[..., 0] * np.cos(ang) - k3h[..., 1] * np.sin(ang),
+                    k3h[..., 0] * np.sin(ang) + k3h[..., 1] * np.cos(ang)], axis=-1).reshape(-1)
+    assert np.abs(rot - k10).max() < 1e-6 * np.abs(k10).max() + 1e-7
+    assert np.abs(base).max() > 0
+    # scaling the embedding by c > 0 leaves the first norm's output (hence, with zero layers, the logits)
+    # unchanged up to eps
+    cfg0 = dict(cfg, n_layers=0)
+    w0 = dict(w, layers=[])
+    a = oracle.Transformer(cfg0, w0, max_seq=16).forward64(toks, np.arange(8))
+    w1 = dict(w0, tok_embed=(w0["tok_embed"] * 8).astype(np.float32))
+    b = oracle.Transformer(cfg0, w1, max_seq=16).forward64(toks, np.arange(8))
+    assert np.abs(a - b).max() < 1e-3 * np.abs(a).max()
+
+
+def test_layerwise_pass_equals_whole_pass():
+    cfg = sps_synth.CONFIGS["tiny_bf16"]["target"]
+    w = np_weights(cfg)
+    toks = sps_synth.make_prompt(9, 5, cfg["vocab"])
+    a = oracle.Transformer(cfg, w, max_seq=16)
+    want = a.forward64(toks, np.arange(5))
+    b = oracle.Transformer(cfg, None, max_seq=16)
+    b.begin_rows(w["tok_embed"][toks], np.arange(5))
+    for l, lw in enumerate(w["layers"]):
+        b.layer(l, lw)
+    got = b.end(w["final_norm"], w["unembed"])
+    assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------ the loop on the tiny pair
+def tiny_pair(name="tiny", max_seq=128):
+    c = sps_synth.CONFIGS[name]
+    wt = np_weights(c["target"], tag="target")
+    wd = np_weights(c["draft"], tag="draft")
+    return oracle.Transformer(c["target"], wt, max_seq), oracle.Transformer(c["draft"], wd, max_seq)
+
+
+def test_loop_on_transformers_invariants_and_K0():
+    tgt, drf = tiny_pair()
+    c = TINY
+    prompt = sps_synth.make_prompt(0, c["prompt_len"], c["target"]["vocab"])
+    sps = oracle.Sps(tgt, drf)
+    out = sps.generate(prompt, 24, c["K"], c["T"], seed=0)
+    h = out["hist_emitted"]
+    assert h[0] == 0 and h.sum() == out["loops"] and 24 <= sum(j * h[j] for j in range(len(h))) <= 24 + c["K"]
+    # K = 0 on the transformer: token i = plain draw from the target's next-token law
+    ar = oracle.Sps(tgt, None).generate(prompt, 6, 0, 1.0, seed=5)
+    seq = list(prompt)
+    ref = oracle.Transformer(c["target"], np_weights(c["target"], tag="target"), 64)
+    for i in range(6):
+        lg = ref.forward64(np.array(seq, dtype=np.int32), np.arange(len(seq)))[-1]
+        w = sm(np.float32(lg))
+        cum = np.cumsum(w)
+        tok = int(np.nonzero(cum > oracle.uniforms(5, 0, i, 0)[2] * cum[-1])[0][0])
+        assert ar["tokens"][i] == tok
+        seq.append(tok)
+
+
+def test_draft_equal_to_target_accepts_all():
+    c = TINY
+    wt = np_weights(c["target"], tag="target")
+    a = oracle.Transformer(c["target"], wt, 128)
+    b = oracle.Transformer(c["target"], wt, 128)
+    sps = oracle.Sps(a, b)
+    prompt = sps_synth.make_prompt(0, 16, c["target"]["vocab"])
+    sps.reset(prompt)
+    for s in range(4):
+        r = sps.loop(4, 1.0, 3, 0, s)
+        # identical weights: q/p differs from 1 only through the order rows were scored in, and
+        # in double that leaves nothing outside a flagged near tie
+        assert r["n_accepted"] == 4 or r["flags"] & oracle.FLAG_NEAR_ACCEPT
+        assert not r["flags"] & oracle.FLAG_FALLBACK
+
+
+def context_tables(model_cfg, weights, prompt, V, depth):
+    """logits after prompt + every suffix of length <= depth, in TableModel row order"""
+    rows = []
+    ref = oracle.Transformer(model_cfg, weights, len(prompt) + depth + 1)
+    P = len(prompt)
+    ref.forward(prompt, np.arange(P), want_logits=False)
+    import itertools
+    for L in range(depth + 1):
+        for suf in itertools.product(range(V), repeat=L):
+            if L == 0:
+                lg = ref.forward(prompt[-1:], [P - 1])[0]
+            else:
+                lg = ref.forward(np.array(suf, dtype=np.int32), np.arange(P, P + L))[-1]
+            rows.append(lg)
+    return np.stack(rows)
+
+
+@pytest.fixture(scope="module")
+def tiny16_tables():
+    c = sps_synth.CONFIGS["tiny16"]
+    prompt = sps_synth.make_prompt(0, c["prompt_len"], 16)
+    wt = np_weights(c["target"], tag="target")
+    wd = np_weights(c["draft"], tag="draft")
+    tq = context_tables(c["target"], wt, prompt, 16, 2)
+    tp = context_tables(c["draft"], wd, prompt, 16, 2)
+    return c, prompt, wt, wd, tq, tp
+
+
+def target_law_3(tq, T):
+    law = np.zeros((16, 16, 16))
+    q0 = sm(tq[0], T)
+    for a in range(16):
+        q1 = sm(tq[1 + a], T)
+        for b in range(16):
+            law[a, b] = q0[a] * q1[b] * sm(tq[1 + 16 + a * 16 + b], T)
+    return law
+
+
+@pytest.mark.parametrize("K,T,logit_gain", [(1, 1.0, 1.0), (2, 1.0, 1.0), (4, 1.0, 1.0), (2, 0.25, 1.0),
+                                            (4, 1.0, 12.0)])
+def test_end_to_end_distribution_vocab16(tiny16_tables, K, T, logit_gain):
+    """Theorem 1 applied along the sequence: the first 3 tokens SpS emits follow
+    q(x1) q(x2|x1) q(x3|x1 x2), here enumerated exactly from the target's own logits (10^6 trials).
+    Only contexts of <= 2 generated tokens can influence those 3 tokens, so lookup tables of that
+    depth stand in for the two transformers; the next test ties the tables to the real loop."""
+    c, prompt, wt, wd, tq, tp = tiny16_tables
+    # random-init logits are nearly flat (std ~0.3); a gain sharpens them so the test has teeth
+    tq, tp = tq * logit_gain, tp * logit_gain
+    n = 1_000_000
+    P = len(prompt)
+    mq, mp = oracle.TableModel(tq, 2, P), oracle.TableModel(tp, 2, P)
+    r = oracle.trials(mq, mp, prompt, n_new=3, K=K, T=T, seed=2024, n_trials=n)
+    t = r["tokens"]
+    counts = np.bincount(t[:, 0] * 256 + t[:, 1] * 16 + t[:, 2], minlength=4096)
+    law = target_law_3(tq, T)
+    assert chi_square_p(counts, law) > 1e-3
+    # negative control with the wrong resampling rule must fail wherever p and q differ enough
+    if logit_gain > 1.0 or T < 1.0:
+        rw = oracle.trials(mq, mp, prompt, n_new=3, K=K, T=T, seed=2024, n_trials=n, wrong_rule=True)
+        tw = rw["tokens"]
+        cw = np.bincount(tw[:, 0] * 256 + tw[:, 1] * 16 + tw[:, 2], minlength=4096)
+        assert chi_square_p(cw, law) < 1e-6
+
+
+def test_table_trials_equal_real_loop(tiny16_tables):
+    c, prompt, wt, wd, tq, tp = tiny16_tables
+    P = len(prompt)
+    mq, mp = oracle.TableModel(tq, 2, P), oracle.TableModel(tp, 2, P)
+    tgt = oracle.Transformer(c["target"], wt, 64)
+    drf = oracle.Transformer(c["draft"], wd, 64)
+    sps = oracle.Sps(tgt, drf)
+    n = 150
+    for K in (1, 2, 4):
+        r = oracle.trials(mq, mp, prompt, n_new=3, K=K, T=1.0, seed=9, n_trials=n)
+        for b in range(n):
+            out = sps.generate(prompt, 3, K, 1.0, seed=9, b=b)
+            same = np.array_equal(out["tokens"], r["tokens"][b])
+            assert same or out["flags"] & (oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF)
