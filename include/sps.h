@@ -1,0 +1,211 @@
+/*
+ * sps.h -- C ABI of the B200 speculative-sampling library (libsps_b200.so).
+ *
+ * The library implements the hot path of speculative sampling (Chen et al.,
+ * "Accelerating Large Language Model Decoding with Speculative Sampling"):
+ * K single-row draft-model steps, one (K+1)-row target-model scoring pass and
+ * the modified rejection sampler, as CUDA kernels for sm_100a.  Notation is
+ * the paper's: q = TARGET model, p = DRAFT model, K = lookahead.
+ *
+ * Conventions
+ *   - every function returns an int status: SPS_OK (0) or a negative error.
+ *     Nothing throws, aborts or prints.  sps_last_error() describes the last
+ *     failure on a handle (or, with a NULL handle, of the handle-less calls).
+ *   - "host" / "device" in a comment says where the pointer must point.
+ *   - weight and logit buffers passed in are caller-owned and never written
+ *     unless stated; the handle owns its KV caches, work buffers and graphs.
+ *   - one handle = one CUDA stream; calls on a handle are not re-entrant.
+ *
+ * Random numbers.  Algorithm 2 draws r ~ U[0,1] and samples tokens; this
+ * library fixes the generator so results can be reproduced elsewhere:
+ * Philox4x32-10, key = (seed low 32, seed high 32), counter =
+ * (t, s, b, 0) with t the position inside the loop (0..K-1 drafts, K the extra
+ * token), s the loop index, b the sequence index.  Word 0 -> u_draft (draw of
+ * draft token t), word 1 -> u_acc (accept test), word 2 -> u_res (resample at
+ * t, or extra-token draw at t = K).  u = (word >> 8) * 2^-24.
+ * Every draw is an inverse-CDF draw in index order on unnormalised weights.
+ */
+#ifndef SPS_B200_H
+#define SPS_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPS_OK 0
+#define SPS_EINVAL (-1)   /* bad argument or unsupported shape                     */
+#define SPS_ENOMEM (-2)   /* device or host allocation failed                      */
+#define SPS_ECUDA (-3)    /* a CUDA call failed; sps_last_error has its message    */
+#define SPS_ERANGE (-4)   /* token id >= vocab, or sequence would exceed max_seq   */
+#define SPS_ESTATE (-5)   /* call order (e.g. step before prefill)                 */
+#define SPS_ETIMEOUT (-6) /* reserved: a bounded device-side wait ran out          */
+
+#define SPS_MAX_K 15      /* K + 1 rows <= 16 per sequence                         */
+
+/* sps_accept / sps_step flag bits (per sequence) */
+#define SPS_FLAG_RESAMPLED 1u /* a draft was rejected; token drawn from norm(max(0, q - p)) */
+#define SPS_FLAG_BONUS 2u     /* all K drafts accepted; extra token drawn from q_{K+1}       */
+#define SPS_FLAG_FALLBACK 4u  /* rejected with sum max(0, q - p) == 0: token drawn from q_t  */
+
+/* sps_cfg.flags */
+#define SPS_CFG_NO_GRAPH 1u   /* launch kernels one by one instead of replaying CUDA graphs  */
+
+typedef struct sps_handle sps_handle;
+
+/* One decoder-only transformer: pre-RMSNorm, multi-head attention with
+ * n_heads * d_head == d_model, rotary positions on adjacent pairs over the
+ * whole head, non-gated FFN with tanh-GeLU, no biases, untied (un)embedding.
+ * (The paper's Hyperparams table fixes d_model / heads / layers only.)
+ * dtype: 0 = fp32, 1 = bf16; it is the storage type of the weight matrices,
+ * the embeddings and the KV cache.  Norm gains are always fp32.
+ * bf16 models need d_model and d_ff to be multiples of 128; d_head is 64 or 128. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, d_head, d_ff, vocab;
+  int32_t dtype;
+  float rms_eps, rope_base;
+} sps_model_cfg;
+
+typedef struct {
+  sps_model_cfg target, draft;
+  int32_t max_seq;   /* longest sequence (prompt + generated + K) a cache row exists for */
+  int32_t max_batch; /* sequences decoded together; max_batch * (max_K + 1) <= 16        */
+  int32_t max_K;     /* largest lookahead that will be asked for, <= SPS_MAX_K           */
+  int32_t device;    /* CUDA device ordinal                                              */
+  void* stream;      /* cudaStream_t to run on; NULL = the library creates its own       */
+  uint32_t flags;    /* SPS_CFG_*                                                        */
+} sps_cfg;
+
+/* Weights of one model.  All pointers are DEVICE pointers, borrowed for the
+ * life of the handle and never written.  Matrices are row-major [out, in]
+ * (y = W x), in the model's dtype.  The per-layer members are HOST arrays of
+ * n_layers device pointers. */
+typedef struct {
+  const void* tok_embed;  /* [vocab, d_model]            */
+  const void* unembed;    /* [vocab, d_model]            */
+  const void* final_norm; /* [d_model] fp32              */
+  const void* const* attn_norm; /* each [d_model] fp32   */
+  const void* const* ffn_norm;  /* each [d_model] fp32   */
+  const void* const* wq;        /* each [d_model, d_model] */
+  const void* const* wk;
+  const void* const* wv;
+  const void* const* wo;
+  const void* const* w_up;      /* each [d_ff, d_model]  */
+  const void* const* w_down;    /* each [d_model, d_ff]  */
+} sps_weights;
+
+/* What a generation did ("we log the amount of tokens generated for each
+ * speculative loop", Results). */
+typedef struct {
+  int32_t loops;         /* target calls                                             */
+  int32_t draft_calls;   /* draft forward passes                                     */
+  int32_t emitted;       /* tokens produced before truncation to n_new               */
+  int32_t accepted;      /* draft tokens accepted                                    */
+  int32_t resampled;     /* loops that ended in a residual resample                  */
+  int32_t bonus;         /* loops that accepted all K drafts and drew the extra token */
+  int32_t fallback;      /* loops that took the sum max(0, q-p) == 0 fallback         */
+  int32_t overshoot;     /* tokens of the last loop dropped to return exactly n_new  */
+  int32_t hist_emitted[SPS_MAX_K + 2]; /* hist_emitted[j] = loops that emitted j tokens */
+  float ms_prefill;      /* device time of the prompt pass                           */
+  float ms_decode;       /* device time of all loops                                 */
+  float ms_draft, ms_verify, ms_accept; /* split of ms_decode by phase               */
+} sps_stats;
+
+/* Build a handle for a (target, draft) pair.  Algorithm 2's preamble: "given
+ * lookahead K ..., target model q, draft model p".  draft_w may be NULL, then
+ * only K = 0 (Algorithm 1) is available.  Allocates the KV caches
+ * [layer][sequence][head][position][d_head] in the model dtype, work buffers
+ * and rotary tables on cfg->device.  *out receives the handle. */
+int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sps_cfg* cfg, sps_handle** out);
+int sps_destroy(sps_handle* h);
+/* NUL-terminated text owned by the handle (or by the library when h is NULL). */
+const char* sps_last_error(sps_handle* h);
+
+/* Algorithm 2 (K >= 1) or Algorithm 1 (K == 0) for one sequence: ingest the
+ * prompt, then loop { draft K tokens; score K+1 positions; accept / resample /
+ * extra token } until n_new tokens exist.  "T" of the algorithms is a minimum
+ * length: the last loop may overshoot and is truncated to exactly n_new.
+ *   prompt      host  [prompt_len], prompt_len >= 1, ids < vocab
+ *   out_tokens  host  [n_new]
+ *   out_stats   host, may be NULL
+ * temperature > 0 scales both models' logits before the rejection scheme
+ * ("adjusting temperature ... modify the probabilities accordingly").
+ * SPS_ERANGE if prompt_len + n_new + K > max_seq. */
+int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K,
+                 float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
+
+/* Same for B sequences with equal prompt lengths, advanced in lock-step with
+ * ragged progress; sequence b uses Philox sequence index b.
+ *   prompts host [B, prompt_len]; out_tokens host [B, n_new]; out_stats host [B] or NULL. */
+int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new,
+                       int32_t K, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
+
+/* Pieces of sps_generate, for tests that drive the loop themselves. */
+/* forget every sequence and both caches' lengths */
+int sps_reset(sps_handle* h);
+/* make toks[0..n-1] (host) the sequence so far of a batch-1 run; both caches take positions 0..n-2 */
+int sps_prefill(sps_handle* h, const int32_t* toks, int32_t n);
+/* one loop iteration with loop index `step`; out_tokens host [K+1] (emitted first, -1 after),
+ * *out_n_emitted = n_accepted + 1, *out_flags SPS_FLAG_* (may be NULL) */
+int sps_step(sps_handle* h, int32_t K, float temperature, uint64_t seed, uint32_t step, int32_t* out_tokens,
+             int32_t* out_n_emitted, uint32_t* out_flags);
+/* copy what the last sps_step saw to HOST buffers (any may be NULL):
+ * q_logits [K+1, V], p_logits [K, V], drafts [K] */
+int sps_last_logits(sps_handle* h, int32_t K, float* q_logits, float* p_logits, int32_t* drafts);
+
+/* The scoring pass alone ("In parallel, compute K+1 sets of logits from
+ * drafts", Algorithm 2): feeds rows[0..K] (host) to the TARGET at positions
+ * len..len+K where len is the target cache's valid length, appends their
+ * keys/values, and writes logits.  Does not move the valid length (calling it
+ * again overwrites the same positions), so it can be timed repeatedly.
+ *   out_logits DEVICE fp32 [K+1, vocab], caller-owned; out_ms host, device time, may be NULL.
+ * which: 0 = target, 1 = draft. */
+int sps_verify(sps_handle* h, const int32_t* rows, int32_t K, float* out_logits, float* out_ms);
+int sps_score(sps_handle* h, int32_t which, const int32_t* rows, int32_t n_rows, float* out_logits, float* out_ms);
+
+/* The modified rejection sampler alone (Algorithm 2's second for-loop and its
+ * extra-token line; section "Modified Rejection Sampling"), one fused kernel:
+ * softmax statistics of q_0..q_K and p_0..p_{K-1} at `temperature`; for
+ * t = 0..K-1 accept draft t iff u_acc < min(1, q_t(d_t) / p_t(d_t)); at the
+ * first rejection draw from max(0, q_t - p_t) / sum max(0, q_t - p_t) and stop;
+ * if none, draw from q_K.
+ *   q_logits      device fp32 [B, K+1, V]
+ *   p_logits      device fp32 [B, K, V]   (the logits the drafts were drawn from)
+ *   draft_tokens  device int32 [B, K]
+ *   stream        cudaStream_t (NULL = default stream); the call only enqueues
+ *   out_n_accepted device int32 [B]
+ *   out_tokens    device int32 [B, K+1]: accepted drafts, then the resampled / extra token, then -1
+ *   out_flags     device uint32 [B], SPS_FLAG_*
+ * Sequence b uses Philox counter (t, step, b, 0).  0 <= K <= SPS_MAX_K, V >= 1. */
+int sps_accept(const float* q_logits, const float* p_logits, const int32_t* draft_tokens, int32_t B, int32_t K,
+               int32_t V, float temperature, uint64_t seed, uint32_t step, void* stream, int32_t* out_n_accepted,
+               int32_t* out_tokens, uint32_t* out_flags);
+
+/* One inverse-CDF draw per row from softmax(logits / temperature) with
+ * u_draft of counter (t, step, b, 0): Algorithm 2's "sample draft
+ * auto-regressively" for given logits.  logits device fp32 [B, V];
+ * out_tokens device int32 [B]. */
+int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uint64_t seed, uint32_t step, uint32_t t,
+               void* stream, int32_t* out_tokens);
+
+/* The memory-bound linear layer alone ("dense matrix multiplies ... become
+ * memory bound", Conditional Scoring): Y[M, N] = X[M, D] W[N, D]^T with fp32
+ * accumulation.  W device, row-major [N, D], dtype 0 fp32 / 1 bf16; X device
+ * fp32 [M, D]; Y device fp32 [M, N]; 1 <= M <= 16.  bf16 needs D % 128 == 0 and
+ * 16-byte aligned W.  workspace: device scratch of sps_linear_workspace_bytes()
+ * bytes for the same (dtype, M, N, D), zero-filled once before its first use
+ * (the kernel leaves it ready for the next call).
+ * out_ms: host, device time of the kernel, may be NULL. */
+int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
+               void* workspace, void* stream, float* out_ms);
+int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D);
+
+/* Philox4x32-10 on the device, for known-answer tests: ctr device uint32 [n,4],
+ * key device uint32 [n,2], out device uint32 [n,4]. */
+int sps_philox(const uint32_t* ctr, const uint32_t* key, int32_t n, void* stream, uint32_t* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

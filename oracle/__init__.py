@@ -79,6 +79,7 @@ def lib():
         L.orc_sps_generate.restype = i32
         L.orc_sps_trials.argtypes = [vp, vp, vp, i32, i32, i32, f64, u64, u32, i64, i32, vp, vp, vp, vp]
         L.orc_num_threads.restype = i32
+        L.orc_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -97,6 +98,17 @@ def _i32(a):
 
 def num_threads() -> int:
     return int(lib().orc_num_threads())
+
+
+def linear(W, X):
+    """Y = X W^T in double.  W [N,D] float32 or uint16 (bf16 bits); X [M,D] float32."""
+    W = np.ascontiguousarray(W)
+    X = _f32(X)
+    dtype = 0 if W.dtype == np.float32 else 1
+    N, D = W.shape
+    out = np.zeros((X.shape[0], N), dtype=np.float64)
+    lib().orc_linear(_p(W), dtype, _p(X), X.shape[0], N, D, _p(out))
+    return out
 
 
 # --------------------------------------------------------------------------- RNG

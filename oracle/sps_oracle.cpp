@@ -686,6 +686,17 @@ extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t*
   orc_sps_destroy(c);
 }
 
+// Y[m][n] = sum_k X[m][k] W[n][k]: the linear layer by its definition, in double.
+extern "C" void orc_linear(const void* W, int dtype, const float* X, int M, int N, int D, double* Y) {
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int m = 0; m < M; ++m) {
+      double acc = 0.0;
+      for (int k = 0; k < D; ++k) acc += load_w(W, (size_t)n * D + k, dtype) * (double)X[(size_t)m * D + k];
+      Y[(size_t)m * N + n] = acc;
+    }
+}
+
 extern "C" int orc_num_threads() {
 #ifdef _OPENMP
   return omp_get_max_threads();

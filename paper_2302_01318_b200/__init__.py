@@ -1,0 +1,244 @@
+"""Thin Python binding of libsps_b200.so (the C ABI of include/sps.h).
+
+Argument marshalling only: torch supplies device memory and streams, every step of the path runs in
+the library's CUDA kernels.  There is no CPU fallback: if the library is missing or there is no CUDA
+device, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+SPS_OK, SPS_EINVAL, SPS_ENOMEM, SPS_ECUDA, SPS_ERANGE, SPS_ESTATE, SPS_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+SPS_MAX_K = 15
+FLAG_RESAMPLED, FLAG_BONUS, FLAG_FALLBACK = 1, 2, 4
+CFG_NO_GRAPH = 1
+LAYER_KEYS = ("attn_norm", "ffn_norm", "wq", "wk", "wv", "wo", "w_up", "w_down")
+
+
+class SpsError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"sps error {code}: {msg}")
+        self.code = code
+
+
+class sps_model_cfg(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32), ("d_head", C.c_int32),
+                ("d_ff", C.c_int32), ("vocab", C.c_int32), ("dtype", C.c_int32), ("rms_eps", C.c_float),
+                ("rope_base", C.c_float)]
+
+
+class sps_cfg(C.Structure):
+    _fields_ = [("target", sps_model_cfg), ("draft", sps_model_cfg), ("max_seq", C.c_int32), ("max_batch", C.c_int32),
+                ("max_K", C.c_int32), ("device", C.c_int32), ("stream", C.c_void_p), ("flags", C.c_uint32)]
+
+
+class sps_weights(C.Structure):
+    _fields_ = [("tok_embed", C.c_void_p), ("unembed", C.c_void_p), ("final_norm", C.c_void_p)] + \
+               [(k, C.POINTER(C.c_void_p)) for k in LAYER_KEYS]
+
+
+class sps_stats(C.Structure):
+    _fields_ = [("loops", C.c_int32), ("draft_calls", C.c_int32), ("emitted", C.c_int32), ("accepted", C.c_int32),
+                ("resampled", C.c_int32), ("bonus", C.c_int32), ("fallback", C.c_int32), ("overshoot", C.c_int32),
+                ("hist_emitted", C.c_int32 * (SPS_MAX_K + 2)), ("ms_prefill", C.c_float), ("ms_decode", C.c_float),
+                ("ms_draft", C.c_float), ("ms_verify", C.c_float), ("ms_accept", C.c_float)]
+
+    def as_dict(self):
+        d = {k: getattr(self, k) for k, _ in self._fields_ if k != "hist_emitted"}
+        d["hist_emitted"] = list(self.hist_emitted)
+        return d
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Load the CUDA library, building it first if the sources are newer.  Raises if that fails."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        vp, i32, u32, u64, f32, i64 = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64, C.c_float, C.c_int64
+        L.sps_create.argtypes = [C.POINTER(sps_weights), C.POINTER(sps_weights), C.POINTER(sps_cfg), C.POINTER(vp)]
+        L.sps_destroy.argtypes = [vp]
+        L.sps_last_error.argtypes = [vp]
+        L.sps_last_error.restype = C.c_char_p
+        L.sps_generate.argtypes = [vp, vp, i32, i32, i32, f32, u64, vp, C.POINTER(sps_stats)]
+        L.sps_generate_batch.argtypes = [vp, vp, i32, i32, i32, i32, f32, u64, vp, C.POINTER(sps_stats)]
+        L.sps_reset.argtypes = [vp]
+        L.sps_prefill.argtypes = [vp, vp, i32]
+        L.sps_step.argtypes = [vp, i32, f32, u64, u32, vp, vp, vp]
+        L.sps_last_logits.argtypes = [vp, i32, vp, vp, vp]
+        L.sps_verify.argtypes = [vp, vp, i32, vp, C.POINTER(f32)]
+        L.sps_score.argtypes = [vp, i32, vp, i32, vp, C.POINTER(f32)]
+        L.sps_accept.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp]
+        L.sps_sample.argtypes = [vp, i32, i32, f32, u64, u32, u32, vp, vp]
+        L.sps_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
+        L.sps_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.sps_linear_workspace_bytes.restype = i64
+        L.sps_philox.argtypes = [vp, vp, i32, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _check(rc, h=None):
+    if rc != SPS_OK:
+        msg = lib().sps_last_error(h)
+        raise SpsError(rc, msg.decode() if msg else "")
+
+
+def _np_ptr(a):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _model_cfg(c: dict) -> sps_model_cfg:
+    return sps_model_cfg(c["n_layers"], c["d_model"], c["n_heads"], c["d_head"], c["d_ff"], c["vocab"], c["dtype"],
+                         c.get("rms_eps", 1e-5), c.get("rope_base", 10000.0))
+
+
+def _weights(w: dict, keep: list) -> sps_weights:
+    sw = sps_weights()
+    sw.tok_embed, sw.unembed, sw.final_norm = w["tok_embed"].data_ptr(), w["unembed"].data_ptr(), w["final_norm"].data_ptr()
+    n = len(w["layers"])
+    for k in LAYER_KEYS:
+        arr = (C.c_void_p * max(n, 1))(*[lw[k].data_ptr() for lw in w["layers"]])
+        keep.append(arr)
+        setattr(sw, k, C.cast(arr, C.POINTER(C.c_void_p)))
+    return sw
+
+
+class Handle:
+    """sps_create / sps_destroy and the calls that take a handle.  `target_w` / `draft_w` are dicts of
+    CUDA torch tensors (tok_embed, unembed, final_norm, layers=[{attn_norm, ffn_norm, wq, wk, wv, wo,
+    w_up, w_down}]); they must stay alive as long as the handle."""
+
+    def __init__(self, target_cfg, target_w, draft_cfg=None, draft_w=None, max_seq=1024, max_batch=1, max_K=4,
+                 device=0, stream=None, flags=0):
+        self._keep = [target_w, draft_w]
+        cfg = sps_cfg()
+        cfg.target = _model_cfg(target_cfg)
+        if draft_cfg is not None:
+            cfg.draft = _model_cfg(draft_cfg)
+        cfg.max_seq, cfg.max_batch, cfg.max_K, cfg.device = max_seq, max_batch, max_K, device
+        cfg.stream = stream
+        cfg.flags = flags
+        tw = _weights(target_w, self._keep)
+        dw = _weights(draft_w, self._keep) if draft_w is not None else None
+        h = C.c_void_p()
+        rc = lib().sps_create(C.byref(tw), C.byref(dw) if dw is not None else None, C.byref(cfg), C.byref(h))
+        _check(rc, None)
+        self._h = h
+        self.vocab = target_cfg["vocab"]
+        self.max_K = max_K
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().sps_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def sps_generate(self, prompt, n_new, K, temperature, seed):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        out = np.zeros(n_new, dtype=np.int32)
+        st = sps_stats()
+        _check(lib().sps_generate(self._h, _np_ptr(p), p.shape[0], n_new, K, temperature, seed, _np_ptr(out), C.byref(st)),
+               self._h)
+        return out, st.as_dict()
+
+    def sps_generate_batch(self, prompts, n_new, K, temperature, seed):
+        p = np.ascontiguousarray(prompts, dtype=np.int32)
+        B, P = p.shape
+        out = np.zeros((B, n_new), dtype=np.int32)
+        st = (sps_stats * B)()
+        _check(lib().sps_generate_batch(self._h, _np_ptr(p), B, P, n_new, K, temperature, seed, _np_ptr(out), st), self._h)
+        return out, [s.as_dict() for s in st]
+
+    def sps_reset(self):
+        _check(lib().sps_reset(self._h), self._h)
+
+    def sps_prefill(self, toks):
+        t = np.ascontiguousarray(toks, dtype=np.int32)
+        _check(lib().sps_prefill(self._h, _np_ptr(t), t.shape[0]), self._h)
+
+    def sps_step(self, K, temperature, seed, step):
+        out = np.full(K + 1, -1, dtype=np.int32)
+        n = np.zeros(1, dtype=np.int32)
+        fl = np.zeros(1, dtype=np.uint32)
+        _check(lib().sps_step(self._h, K, temperature, seed, step, _np_ptr(out), _np_ptr(n), _np_ptr(fl)), self._h)
+        return out, int(n[0]), int(fl[0])
+
+    def sps_last_logits(self, K):
+        q = np.zeros((K + 1, self.vocab), dtype=np.float32)
+        p = np.zeros((K, self.vocab), dtype=np.float32)
+        d = np.zeros(K, dtype=np.int32)
+        _check(lib().sps_last_logits(self._h, K, _np_ptr(q), _np_ptr(p) if K else None, _np_ptr(d) if K else None), self._h)
+        return q, p, d
+
+    def sps_verify(self, rows, K, out_logits):
+        r = np.ascontiguousarray(rows, dtype=np.int32)
+        ms = C.c_float(0)
+        _check(lib().sps_verify(self._h, _np_ptr(r), K, out_logits.data_ptr(), C.byref(ms)), self._h)
+        return ms.value
+
+    def sps_score(self, which, rows, out_logits):
+        r = np.ascontiguousarray(rows, dtype=np.int32)
+        ms = C.c_float(0)
+        _check(lib().sps_score(self._h, which, _np_ptr(r), r.shape[0], out_logits.data_ptr(), C.byref(ms)), self._h)
+        return ms.value
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream
+
+
+def sps_accept(q_logits, p_logits, draft_tokens, temperature, seed, step, out_n_accepted, out_tokens, out_flags,
+               stream=None):
+    """q_logits [B,K+1,V] fp32, p_logits [B,K,V] fp32, draft_tokens [B,K] int32: CUDA torch tensors;
+    outputs CUDA int32 [B], int32 [B,K+1], int32-sized [B].  Enqueues one kernel on `stream`."""
+    B, K1, V = q_logits.shape
+    K = K1 - 1
+    _check(lib().sps_accept(q_logits.data_ptr(), p_logits.data_ptr() if K else None,
+                            draft_tokens.data_ptr() if K else None, B, K, V, temperature, seed, step,
+                            _stream_ptr(stream), out_n_accepted.data_ptr(), out_tokens.data_ptr(), out_flags.data_ptr()))
+
+
+def sps_sample(logits, temperature, seed, step, t, out_tokens, stream=None):
+    B, V = logits.shape
+    _check(lib().sps_sample(logits.data_ptr(), B, V, temperature, seed, step, t, _stream_ptr(stream), out_tokens.data_ptr()))
+
+
+def sps_linear_workspace_bytes(dtype, M, N, D):
+    return int(lib().sps_linear_workspace_bytes(dtype, M, N, D))
+
+
+def sps_linear(W, X, Y, workspace, stream=None, timed=False):
+    """Y[M,N] = X[M,D] W[N,D]^T.  W CUDA fp32 or bf16, X/Y CUDA fp32, workspace CUDA uint8 (zeroed once)."""
+    import torch
+    dtype = 0 if W.dtype == torch.float32 else 1
+    N, D = W.shape
+    M = X.shape[0]
+    ms = C.c_float(0)
+    _check(lib().sps_linear(W.data_ptr(), dtype, X.data_ptr(), M, N, D, Y.data_ptr(), workspace.data_ptr(),
+                            _stream_ptr(stream), C.byref(ms) if timed else None))
+    return ms.value
+
+
+def sps_philox(ctr, key, out, stream=None):
+    _check(lib().sps_philox(ctr.data_ptr(), key.data_ptr(), ctr.shape[0], _stream_ptr(stream), out.data_ptr()))

@@ -1,0 +1,197 @@
+// Shared declarations of the CUDA library: argument blocks of the kernels, their host launchers,
+// and small device helpers (counter-based random numbers, warp/block reductions, bf16 packing).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define SPS_MAX_ROWS 16   // activation rows one pass may carry (two 8-column MMA tiles)
+#define SPS_NUM_SM_FALLBACK 148
+
+// ------------------------------------------------------------------------------------------------
+// Random numbers (see include/sps.h): Philox4x32-10, counter (t, s, b, 0), key (seed lo, seed hi).
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t a = (uint64_t)0xD2511F53u * c0;
+    const uint64_t b = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(b >> 32) ^ c1 ^ k0;
+    const uint32_t n1 = (uint32_t)b;
+    const uint32_t n2 = (uint32_t)(a >> 32) ^ c3 ^ k1;
+    const uint32_t n3 = (uint32_t)a;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// 24-bit grid in [0,1): exact in fp32
+__host__ __device__ inline float u01_from_word(uint32_t w) { return (float)(w >> 8) * (1.0f / 16777216.0f); }
+
+struct Uniforms { float u_draft, u_acc, u_res; };
+__device__ inline Uniforms sps_uniforms(uint64_t seed, uint32_t b, uint32_t s, uint32_t t) {
+  uint32_t w[4];
+  philox4x32_10(t, s, b, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), w);
+  Uniforms u;
+  u.u_draft = u01_from_word(w[0]);
+  u.u_acc = u01_from_word(w[1]);
+  u.u_res = u01_from_word(w[2]);
+  return u;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Reductions with a fixed tree (results are bit-reproducible run to run).
+// ------------------------------------------------------------------------------------------------
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ inline float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ inline int warp_min_int(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ inline int warp_max_int(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Device-resident state of a handle: everything a loop iteration reads or advances, so that a
+// captured graph can be replayed with no host patching.
+// ------------------------------------------------------------------------------------------------
+struct DevState {
+  // per-call parameters, written by the host before a loop / generation
+  float temperature;
+  float inv_temperature;
+  uint32_t step;      // loop index s, advanced on the device after each loop
+  uint32_t pad0;
+  uint64_t seed;
+  int32_t B;          // live sequences
+  int32_t max_seq;
+  // per sequence
+  int32_t* n;         // [B] tokens known so far
+  int32_t* limit;     // [B] a sequence that has reached this many tokens stops advancing
+  int32_t* tokens;    // [B][max_seq]
+  int32_t* drafts;    // [B][max_K]
+  // rows of the pass in flight
+  int32_t* row_tok;   // [SPS_MAX_ROWS]
+  int32_t* row_pos;   // [SPS_MAX_ROWS]
+  // loop results
+  int32_t* n_acc;     // [B]
+  int32_t* out_tok;   // [B][max_K+1]
+  uint32_t* flags;    // [B]
+  int32_t* err;       // [1] sticky device-side error word (token out of range ...)
+  int32_t max_K;
+  int32_t done_counter_pad;
+  uint32_t* done_counter;  // [1] CTAs of the accept kernel that finished (for the step advance)
+};
+
+// which rows a pass feeds (per sequence)
+enum PassMode : int {
+  PASS_PREFILL = 0,   // rows = tokens[c0 .. c0+m) of the sequence, positions the same
+  PASS_DRAFT0 = 1,    // 2 rows: positions max(n-2,0), n-1          (catches the draft cache up)
+  PASS_DRAFT_T = 2,   // 1 row : draft t-1 at position n-1+t
+  PASS_VERIFY = 3,    // K+1 rows: x[n-1], d_0..d_{K-1} at positions n-1..n-1+K
+  PASS_EXPLICIT = 4   // rows already written to row_tok / row_pos by the host
+};
+
+// ------------------------------------------------------------------------------------------------
+// Linear layer  Y[M,N] = f(X)[M,D] W[N,D]^T  with fused prologue f and epilogue.
+// ------------------------------------------------------------------------------------------------
+enum { PRO_NONE = 0, PRO_RMSNORM = 1, PRO_GELU = 2 };
+enum { EPI_STORE = 0, EPI_RESIDUAL = 1 };
+
+struct LinArgs {
+  const void* W[3];       // up to three stacked matrices (fused Q,K,V), each [rows_per_mat][D]
+  int rows_per_mat;
+  int N;                  // total output features = n_mats * rows_per_mat
+  int D;                  // input features
+  int M;                  // activation rows, 1..16
+  const float* X;         // [*, ldx] fp32; row of activation m is x_row0 + m * x_rowstep
+  int ldx, x_row0, x_rowstep;
+  int pro;                // PRO_*
+  const float* gain;      // [D] fp32 (PRO_RMSNORM)
+  const float* ssq_in;    // [rows] sum of squares of each X row (PRO_RMSNORM)
+  float eps;
+  int epi;                // EPI_*
+  float* Y;               // EPI_STORE: Y[m*ldy + n] = y.  EPI_RESIDUAL: Y[m*ldy + n] += y
+  long long ldy;
+  float* ssq_out;         // EPI_RESIDUAL: [M] sum over n of the updated Y[m][n]^2
+  // scratch (owned by the handle / caller): split-K partials and arrival counters
+  float* part;            // [S][SPS_MAX_ROWS][N]
+  float* ssq_part;        // [R][SPS_MAX_ROWS]
+  int* counters;          // [R + 1], zero between launches (the kernel re-zeroes them)
+  int R, S, WC;           // row ranges, K splits, warps per CTA
+  int PR;                 // rows per shared-memory pass (multiple of 32)
+};
+
+struct LinPlan { int R, S, WC, PR, NT; size_t smem; };
+LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
+cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
+size_t lin_part_floats(int N, int S_max);
+#define LIN_MAX_R 512
+#define LIN_MAX_S 64
+
+// ------------------------------------------------------------------------------------------------
+// Rows / embedding, attention, samplers
+// ------------------------------------------------------------------------------------------------
+struct EmbedArgs {
+  DevState* st;
+  const void* tok_embed;  // [V][d]
+  int dtype, d, V;
+  int mode, t, K, c0, rows_per_seq, B;
+  float* x;               // [rows][d] fp32 residual stream
+  float* ssq;             // [rows]
+};
+cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st);
+
+struct AttnArgs {
+  const DevState* st;
+  const float* qkv;       // [rows][3d]
+  float* out;             // [rows][d]
+  void* kcache;           // this layer: [B][H][max_seq][dh]
+  void* vcache;
+  const float2* rope;     // [max_seq][dh/2] (cos, sin)
+  int dtype, H, dh, d, max_seq, rows_per_seq, B;
+};
+cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
+size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh);
+
+struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(logits/T)
+  const DevState* st;      // T, seed, step come from here when st != nullptr
+  const float* logits;     // row b at logits + b*ld
+  long long ld;
+  int V, B;
+  uint32_t t;              // Philox position
+  int32_t* out;            // out[b*out_ld]
+  int out_ld;
+  float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+};
+cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st);
+
+struct AcceptArgs {
+  DevState* st;            // when non-null: T/seed/step from the state, and the loop is advanced
+  const float* q_logits;   // [B][K+1][V]
+  const float* p_logits;   // [B][K][V]
+  const int32_t* drafts;   // [B][drafts_ld]
+  int drafts_ld;
+  int B, K, V;
+  int32_t* n_acc;          // [B]
+  int32_t* out_tok;        // [B][out_ld]
+  int out_ld;
+  uint32_t* flags;         // [B]
+  float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+};
+cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);
+cudaError_t philox_launch(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out, cudaStream_t st);

@@ -1,0 +1,709 @@
+// The C ABI of include/sps.h: handle, passes over a model, the speculative loop and its pieces.
+// Host code only enqueues kernels (or replays graphs of them) and reads back a few integers per loop;
+// every step of the path runs in the kernels of linear.cu, attention.cu and sampler.cu.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/sps.h"
+#include "common.cuh"
+
+namespace {
+
+std::string g_err;  // last error of the handle-less entry points
+
+struct ModelDev {
+  sps_model_cfg cfg{};
+  bool present = false;
+  const void *tok_embed = nullptr, *unembed = nullptr, *final_norm = nullptr;
+  std::vector<const void*> attn_norm, ffn_norm, wq, wk, wv, wo, w_up, w_down;
+  char* kcache = nullptr;  // [L][B][H][max_seq][dh] in the storage type
+  char* vcache = nullptr;
+  size_t layer_bytes = 0;
+  float2* rope = nullptr;  // [max_seq][dh/2]
+};
+
+struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uint64_t seed; };
+
+}  // namespace
+
+struct sps_handle {
+  sps_cfg cfg{};
+  cudaStream_t stream = nullptr;
+  bool own_stream = false;
+  int num_sm = SPS_NUM_SM_FALLBACK;
+  ModelDev tgt, drf;
+  DevState hst{};          // host image of the device state block
+  DevState* dst = nullptr;
+  float *x = nullptr, *qkv = nullptr, *attn = nullptr, *up = nullptr, *ssqA = nullptr, *ssqB = nullptr;
+  float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr, *ssq_part = nullptr;
+  int* counters = nullptr;
+  int32_t* res = nullptr;    // device: [n_acc B][flags B][out_tok B*(maxK+1)][err 1]
+  int32_t* h_res = nullptr;  // pinned mirror
+  HostParams* h_par = nullptr;  // pinned
+  int32_t* h_rows = nullptr;    // pinned [2][16]
+  size_t res_words = 0;
+  int B = 0;
+  int seq_len[SPS_MAX_ROWS] = {0};   // host view of n per sequence
+  bool ready = false;
+  std::map<int, cudaGraphExec_t> g_draft, g_verify;  // key = K * 32 + B
+  std::map<int, int> warm;                          // key -> eager runs done
+  cudaEvent_t ev[5]{};
+  std::string err;
+  int last_K = -1;
+};
+
+namespace {
+
+int fail(sps_handle* h, int code, const std::string& msg) {
+  if (h) h->err = msg; else g_err = msg;
+  return code;
+}
+#define CU(h, call)                                                                         \
+  do {                                                                                      \
+    cudaError_t e__ = (call);                                                               \
+    if (e__ != cudaSuccess)                                                                 \
+      return fail(h, SPS_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e__));       \
+  } while (0)
+
+size_t esize(int dtype) { return dtype == 0 ? 4 : 2; }
+
+int check_model_cfg(const sps_model_cfg& c, std::string& why) {
+  if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.d_ff <= 0 || c.vocab <= 0) { why = "non-positive model dimension"; return 0; }
+  if (c.n_heads * c.d_head != c.d_model) { why = "n_heads * d_head must equal d_model"; return 0; }
+  if (c.d_head != 64 && c.d_head != 128) { why = "d_head must be 64 or 128"; return 0; }
+  if (c.dtype != 0 && c.dtype != 1) { why = "dtype must be 0 (fp32) or 1 (bf16)"; return 0; }
+  if (c.dtype == 1 && (c.d_model % 128 || c.d_ff % 128)) { why = "bf16 models need d_model and d_ff multiples of 128"; return 0; }
+  if (c.dtype == 0 && ((size_t)SPS_MAX_ROWS * (size_t)(c.d_ff > c.d_model ? c.d_ff : c.d_model) * 4 > 200 * 1024)) { why = "fp32 model too wide for the fp32 kernel"; return 0; }
+  if (c.d_model % 4 || c.d_ff % 4) { why = "d_model and d_ff must be multiples of 4"; return 0; }
+  return 1;
+}
+
+int load_model(sps_handle* h, ModelDev& m, const sps_model_cfg& c, const sps_weights* w, int max_seq, int max_batch) {
+  m.cfg = c;
+  m.present = true;
+  m.tok_embed = w->tok_embed; m.unembed = w->unembed; m.final_norm = w->final_norm;
+  if (!m.tok_embed || !m.unembed || !m.final_norm) return fail(h, SPS_EINVAL, "null embedding / unembedding / final_norm");
+  const void* const* srcs[8] = {w->attn_norm, w->ffn_norm, w->wq, w->wk, w->wv, w->wo, w->w_up, w->w_down};
+  std::vector<const void*>* dsts[8] = {&m.attn_norm, &m.ffn_norm, &m.wq, &m.wk, &m.wv, &m.wo, &m.w_up, &m.w_down};
+  for (int i = 0; i < 8; ++i) {
+    if (c.n_layers > 0 && !srcs[i]) return fail(h, SPS_EINVAL, "null per-layer pointer array");
+    dsts[i]->assign(c.n_layers, nullptr);
+    for (int l = 0; l < c.n_layers; ++l) {
+      if (!srcs[i][l]) return fail(h, SPS_EINVAL, "null layer weight pointer");
+      if (((uintptr_t)srcs[i][l]) & 15) return fail(h, SPS_EINVAL, "weight pointers must be 16-byte aligned");
+      (*dsts[i])[l] = srcs[i][l];
+    }
+  }
+  m.layer_bytes = (size_t)max_batch * c.n_heads * (size_t)max_seq * c.d_head * esize(c.dtype);
+  const size_t total = m.layer_bytes * (size_t)(c.n_layers > 0 ? c.n_layers : 1);
+  if (cudaMalloc(&m.kcache, total) != cudaSuccess || cudaMalloc(&m.vcache, total) != cudaSuccess)
+    return fail(h, SPS_ENOMEM, "KV cache allocation failed");
+  CU(h, cudaMemsetAsync(m.kcache, 0, total, h->stream));
+  CU(h, cudaMemsetAsync(m.vcache, 0, total, h->stream));
+  // rotary table: angle = pos * base^(-2i/dh), computed in double, stored as fp32 (cos, sin)
+  const int half = c.d_head / 2;
+  std::vector<float2> tab((size_t)max_seq * half);
+  for (int p = 0; p < max_seq; ++p)
+    for (int i = 0; i < half; ++i) {
+      const double ang = (double)p * std::pow((double)c.rope_base, -2.0 * i / c.d_head);
+      tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+    }
+  if (cudaMalloc(&m.rope, tab.size() * sizeof(float2)) != cudaSuccess) return fail(h, SPS_ENOMEM, "rope table allocation failed");
+  CU(h, cudaMemcpy(m.rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice));
+  return SPS_OK;
+}
+
+void free_model(ModelDev& m) {
+  if (m.kcache) cudaFree(m.kcache);
+  if (m.vcache) cudaFree(m.vcache);
+  if (m.rope) cudaFree(m.rope);
+  m.kcache = m.vcache = nullptr; m.rope = nullptr;
+}
+
+// scratch need of one model's linear layers, over every row count the handle may use
+size_t model_part_floats(const ModelDev& m, int num_sm) {
+  if (!m.present) return 0;
+  const sps_model_cfg& c = m.cfg;
+  size_t need = 0;
+  const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  for (int M : {1, SPS_MAX_ROWS})
+    for (auto& s : shapes) {
+      const LinPlan p = lin_plan(c.dtype, M, s[0], s[1], num_sm);
+      const size_t f = lin_part_floats(s[0], p.S);
+      if (f > need) need = f;
+    }
+  return need;
+}
+
+struct PassSpec {
+  int mode, t, K, c0, rows_per_seq;
+  float* logits;        // null: skip the unembedding
+  long long logits_ld;  // stride between logits rows
+  int lrow0, lrowstep, lrows;  // which residual rows get logits
+};
+
+// one forward pass of a model over the rows `ps` describes, for the handle's B live sequences
+int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
+  const sps_model_cfg& c = m.cfg;
+  const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff;
+  cudaStream_t st = h->stream;
+  EmbedArgs ea{};
+  ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = c.dtype; ea.d = d; ea.V = c.vocab;
+  ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
+  ea.x = h->x; ea.ssq = h->ssqA;
+  CU(h, embed_launch(ea, st));
+  LinArgs base{};
+  base.part = h->part; base.ssq_part = h->ssq_part; base.counters = h->counters; base.eps = c.rms_eps;
+  for (int l = 0; l < c.n_layers; ++l) {
+    {  // q, k, v = Wq h, Wk h, Wv h with h = rmsnorm(x, g_attn), one launch over the three matrices
+      LinArgs a = base;
+      a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
+      a.rows_per_mat = d; a.N = 3 * d; a.D = d; a.M = rows;
+      a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
+      a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA;
+      a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = 3 * d;
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+    }
+    {
+      AttnArgs aa{};
+      aa.st = h->dst; aa.qkv = h->qkv; aa.out = h->attn;
+      aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
+      aa.rope = m.rope; aa.dtype = c.dtype; aa.H = c.n_heads; aa.dh = c.d_head; aa.d = d;
+      aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
+      CU(h, attn_launch(aa, st));
+    }
+    {  // x += Wo o ; also sum(x^2) for the FFN norm
+      LinArgs a = base;
+      a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = d; a.M = rows;
+      a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
+      a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+    }
+    {  // up = Wup rmsnorm(x, g_ffn)
+      LinArgs a = base;
+      a.W[0] = m.w_up[l]; a.rows_per_mat = dff; a.N = dff; a.D = d; a.M = rows;
+      a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
+      a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB;
+      a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+    }
+    {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
+      LinArgs a = base;
+      a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
+      a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
+      a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+    }
+  }
+  if (ps.logits) {
+    LinArgs a = base;
+    a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
+    a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
+    a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA;
+    a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
+    CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm), st));
+  }
+  return SPS_OK;
+}
+
+// K draft steps: step 0 feeds two rows per sequence (positions n-2, n-1) so that a draft cache left
+// one token behind by a fully accepted loop catches up in the same fixed-shape pass
+int enqueue_draft(sps_handle* h, int K) {
+  const int V = h->tgt.cfg.vocab, B = h->B;
+  for (int t = 0; t < K; ++t) {
+    PassSpec ps{};
+    ps.mode = t == 0 ? PASS_DRAFT0 : PASS_DRAFT_T; ps.t = t; ps.K = K; ps.rows_per_seq = t == 0 ? 2 : 1;
+    ps.logits = h->p_logits + (size_t)t * V; ps.logits_ld = (long long)K * V;
+    ps.lrow0 = t == 0 ? 1 : 0; ps.lrowstep = t == 0 ? 2 : 1; ps.lrows = B;
+    int rc = run_pass(h, h->drf, ps);
+    if (rc) return rc;
+    SampleArgs sa{};
+    sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = V; sa.B = B; sa.t = (uint32_t)t;
+    sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
+    CU(h, sample_launch(sa, h->stream));
+  }
+  return SPS_OK;
+}
+
+int enqueue_verify(sps_handle* h, int K) {
+  PassSpec ps{};
+  ps.mode = PASS_VERIFY; ps.K = K; ps.rows_per_seq = K + 1;
+  ps.logits = h->q_logits; ps.logits_ld = h->tgt.cfg.vocab; ps.lrow0 = 0; ps.lrowstep = 1; ps.lrows = h->B * (K + 1);
+  return run_pass(h, h->tgt, ps);
+}
+
+int enqueue_accept(sps_handle* h, int K) {
+  AcceptArgs aa{};
+  aa.st = h->dst; aa.q_logits = h->q_logits; aa.p_logits = h->p_logits; aa.drafts = h->hst.drafts;
+  aa.drafts_ld = h->hst.max_K; aa.B = h->B; aa.K = K; aa.V = h->tgt.cfg.vocab;
+  aa.n_acc = h->hst.n_acc; aa.out_tok = h->hst.out_tok; aa.out_ld = h->hst.max_K + 1; aa.flags = h->hst.flags;
+  CU(h, accept_launch(aa, h->stream));
+  return SPS_OK;
+}
+
+// replay (or, the first two times, run eagerly and then capture) one phase
+int launch_phase(sps_handle* h, std::map<int, cudaGraphExec_t>& cache, int K, int (*enq)(sps_handle*, int), int tag) {
+  if (h->cfg.flags & SPS_CFG_NO_GRAPH) return enq(h, K);
+  const int key = K * 32 + h->B;
+  auto it = cache.find(key);
+  if (it != cache.end()) { CU(h, cudaGraphLaunch(it->second, h->stream)); return SPS_OK; }
+  int& w = h->warm[key * 2 + tag];
+  if (w == 0) { ++w; return enq(h, K); }   // first use runs eagerly (it also sets kernel attributes)
+  cudaGraph_t g = nullptr;
+  CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+  int rc = enq(h, K);
+  cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+  if (rc) { if (g) cudaGraphDestroy(g); return rc; }
+  if (e != cudaSuccess) return fail(h, SPS_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
+  cudaGraphExec_t ge = nullptr;
+  e = cudaGraphInstantiate(&ge, g, 0);
+  cudaGraphDestroy(g);
+  if (e != cudaSuccess) return fail(h, SPS_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+  cache[key] = ge;
+  CU(h, cudaGraphLaunch(ge, h->stream));
+  return SPS_OK;
+}
+
+int write_params(sps_handle* h, float T, uint64_t seed, uint32_t step) {
+  h->h_par->temperature = T; h->h_par->inv_temperature = 1.0f / T; h->h_par->step = step; h->h_par->pad0 = 0;
+  h->h_par->seed = seed;
+  CU(h, cudaMemcpyAsync(h->dst, h->h_par, sizeof(HostParams), cudaMemcpyHostToDevice, h->stream));
+  return SPS_OK;
+}
+
+// one loop iteration for all live sequences; results land in h->h_res after the sync
+int loop_once(sps_handle* h, int K, bool timed) {
+  int rc;
+  if (timed) CU(h, cudaEventRecord(h->ev[0], h->stream));
+  if (K > 0 && (rc = launch_phase(h, h->g_draft, K, enqueue_draft, 0))) return rc;
+  if (timed) CU(h, cudaEventRecord(h->ev[1], h->stream));
+  if ((rc = launch_phase(h, h->g_verify, K, enqueue_verify, 1))) return rc;
+  if (timed) CU(h, cudaEventRecord(h->ev[2], h->stream));
+  if ((rc = enqueue_accept(h, K))) return rc;
+  if (timed) CU(h, cudaEventRecord(h->ev[3], h->stream));
+  CU(h, cudaMemcpyAsync(h->h_res, h->res, h->res_words * 4, cudaMemcpyDeviceToHost, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  h->last_K = K;
+  if (h->h_res[h->res_words - 1] != 0) return fail(h, SPS_ERANGE, "device flagged a token id or position out of range");
+  return SPS_OK;
+}
+
+int set_sequences(sps_handle* h, const int32_t* toks, int B, int n) {
+  const int max_seq = h->cfg.max_seq;
+  if (B < 1 || B > h->cfg.max_batch) return fail(h, SPS_EINVAL, "batch outside 1..max_batch");
+  if (n < 1) return fail(h, SPS_EINVAL, "a sequence needs at least one token");
+  if (n > max_seq) return fail(h, SPS_ERANGE, "sequence longer than max_seq");
+  const int V = h->tgt.cfg.vocab;
+  for (long long i = 0; i < (long long)B * n; ++i)
+    if (toks[i] < 0 || toks[i] >= V) return fail(h, SPS_ERANGE, "token id outside the vocabulary");
+  h->B = B;
+  std::vector<int32_t> nn(B, n);
+  CU(h, cudaMemcpy2DAsync(h->hst.tokens, (size_t)max_seq * 4, toks, (size_t)n * 4, (size_t)n * 4, B, cudaMemcpyHostToDevice, h->stream));
+  CU(h, cudaMemcpyAsync(h->hst.n, nn.data(), B * 4, cudaMemcpyHostToDevice, h->stream));
+  int32_t Bv = B;
+  CU(h, cudaMemcpyAsync(&h->dst->B, &Bv, 4, cudaMemcpyHostToDevice, h->stream));
+  std::vector<int32_t> lim(B, 0x7fffffff);
+  CU(h, cudaMemcpyAsync(h->hst.limit, lim.data(), B * 4, cudaMemcpyHostToDevice, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));  // nn / lim are stack-lifetime host buffers
+  for (int b = 0; b < B; ++b) h->seq_len[b] = n;
+  return SPS_OK;
+}
+
+// both caches ingest positions 0..n-2 of every live sequence
+int prefill_all(sps_handle* h, int n) {
+  const int per = SPS_MAX_ROWS / h->B;
+  for (int which = 0; which < 2; ++which) {
+    ModelDev& m = which == 0 ? h->tgt : h->drf;
+    if (!m.present) continue;
+    for (int c0 = 0; c0 < n - 1; c0 += per) {
+      PassSpec ps{};
+      ps.mode = PASS_PREFILL; ps.c0 = c0; ps.rows_per_seq = (n - 1 - c0) < per ? (n - 1 - c0) : per;
+      int rc = run_pass(h, m, ps);
+      if (rc) return rc;
+    }
+  }
+  h->ready = true;
+  return SPS_OK;
+}
+
+void add_loop_stats(sps_stats* s, int K, int a, uint32_t fl) {
+  s->loops += 1;
+  s->draft_calls += K;
+  s->emitted += a + 1;
+  s->accepted += a;
+  if (fl & SPS_FLAG_RESAMPLED) s->resampled += 1;
+  if (fl & SPS_FLAG_BONUS) s->bonus += 1;
+  if (fl & SPS_FLAG_FALLBACK) s->fallback += 1;
+  s->hist_emitted[a + 1] += 1;
+}
+
+int check_K(sps_handle* h, int K) {
+  if (K < 0 || K > h->cfg.max_K) return fail(h, SPS_EINVAL, "K outside 0..max_K");
+  if (K > 0 && !h->drf.present) return fail(h, SPS_EINVAL, "K > 0 needs a draft model");
+  if (h->B * (K + 1) > SPS_MAX_ROWS) return fail(h, SPS_EINVAL, "batch * (K + 1) exceeds 16 rows");
+  return SPS_OK;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+const char* sps_last_error(sps_handle* h) { return h ? h->err.c_str() : g_err.c_str(); }
+
+int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sps_cfg* cfg, sps_handle** out) {
+  if (!target_w || !cfg || !out) return fail(nullptr, SPS_EINVAL, "null argument");
+  *out = nullptr;
+  std::string why;
+  if (!check_model_cfg(cfg->target, why)) return fail(nullptr, SPS_EINVAL, "target: " + why);
+  if (draft_w) {
+    if (!check_model_cfg(cfg->draft, why)) return fail(nullptr, SPS_EINVAL, "draft: " + why);
+    if (cfg->draft.vocab != cfg->target.vocab) return fail(nullptr, SPS_EINVAL, "draft and target vocabularies differ");
+  }
+  if (cfg->max_K < 0 || cfg->max_K > SPS_MAX_K) return fail(nullptr, SPS_EINVAL, "max_K outside 0..15");
+  if (cfg->max_batch < 1 || cfg->max_batch * (cfg->max_K + 1) > SPS_MAX_ROWS || cfg->max_batch * 2 > SPS_MAX_ROWS)
+    return fail(nullptr, SPS_EINVAL, "max_batch * (max_K + 1) must be <= 16");
+  if (cfg->max_seq < 2) return fail(nullptr, SPS_EINVAL, "max_seq too small");
+  {
+    const int dh_max = (draft_w && cfg->draft.d_head > cfg->target.d_head) ? cfg->draft.d_head : cfg->target.d_head;
+    if (attn_smem_bytes(SPS_MAX_ROWS / cfg->max_batch, cfg->max_seq, dh_max) > 220 * 1024)
+      return fail(nullptr, SPS_EINVAL, "max_seq too large for the attention kernel's score buffer");
+  }
+  cudaError_t e = cudaSetDevice(cfg->device);
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("cudaSetDevice: ") + cudaGetErrorString(e));
+  sps_handle* h = new sps_handle();
+  h->cfg = *cfg;
+  int rc = SPS_OK;
+  auto bail = [&](int code) { g_err = h->err; sps_destroy(h); return code; };
+  cudaDeviceGetAttribute(&h->num_sm, cudaDevAttrMultiProcessorCount, cfg->device);
+  if (cfg->stream) h->stream = (cudaStream_t)cfg->stream;
+  else {
+    if (cudaStreamCreateWithFlags(&h->stream, cudaStreamNonBlocking) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "stream creation failed"));
+    h->own_stream = true;
+  }
+  for (auto& ev : h->ev) if (cudaEventCreate(&ev) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "event creation failed"));
+  if ((rc = load_model(h, h->tgt, cfg->target, target_w, cfg->max_seq, cfg->max_batch))) return bail(rc);
+  if (draft_w && (rc = load_model(h, h->drf, cfg->draft, draft_w, cfg->max_seq, cfg->max_batch))) return bail(rc);
+
+  const int V = cfg->target.vocab, maxK = cfg->max_K > 0 ? cfg->max_K : 1, MB = cfg->max_batch;
+  int dmax = cfg->target.d_model, fmax = cfg->target.d_ff;
+  if (draft_w) { if (cfg->draft.d_model > dmax) dmax = cfg->draft.d_model; if (cfg->draft.d_ff > fmax) fmax = cfg->draft.d_ff; }
+  size_t part_floats = model_part_floats(h->tgt, h->num_sm);
+  const size_t pf2 = model_part_floats(h->drf, h->num_sm);
+  if (pf2 > part_floats) part_floats = pf2;
+  if (part_floats == 0) part_floats = 1;
+  h->res_words = (size_t)MB * 2 + (size_t)MB * (maxK + 1) + 1;
+  struct Want { void** p; size_t bytes; };
+  DevState& s = h->hst;
+  const Want wants[] = {
+      {(void**)&h->x, sizeof(float) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->qkv, sizeof(float) * SPS_MAX_ROWS * 3 * (size_t)dmax},
+      {(void**)&h->attn, sizeof(float) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->up, sizeof(float) * SPS_MAX_ROWS * (size_t)fmax},
+      {(void**)&h->ssqA, sizeof(float) * SPS_MAX_ROWS},
+      {(void**)&h->ssqB, sizeof(float) * SPS_MAX_ROWS},
+      {(void**)&h->q_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
+      {(void**)&h->p_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
+      {(void**)&h->part, sizeof(float) * part_floats},
+      {(void**)&h->ssq_part, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
+      {(void**)&h->counters, sizeof(int) * (LIN_MAX_R + 1)},
+      {(void**)&h->res, 4 * h->res_words},
+      {(void**)&h->dst, sizeof(DevState)},
+      {(void**)&s.n, 4 * (size_t)MB},
+      {(void**)&s.limit, 4 * (size_t)MB},
+      {(void**)&s.tokens, 4 * (size_t)MB * cfg->max_seq},
+      {(void**)&s.drafts, 4 * (size_t)MB * maxK},
+      {(void**)&s.row_tok, 4 * SPS_MAX_ROWS},
+      {(void**)&s.row_pos, 4 * SPS_MAX_ROWS},
+      {(void**)&s.done_counter, 4},
+  };
+  for (const Want& w : wants) {
+    if (cudaMalloc(w.p, w.bytes) != cudaSuccess) return bail(fail(h, SPS_ENOMEM, "device allocation failed"));
+    if (cudaMemsetAsync(*w.p, 0, w.bytes, h->stream) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "memset failed"));
+  }
+  if (cudaMallocHost(&h->h_res, 4 * h->res_words) != cudaSuccess || cudaMallocHost(&h->h_par, sizeof(HostParams)) != cudaSuccess ||
+      cudaMallocHost(&h->h_rows, 4 * 2 * SPS_MAX_ROWS) != cudaSuccess)
+    return bail(fail(h, SPS_ENOMEM, "pinned host allocation failed"));
+  s.temperature = 1.f; s.inv_temperature = 1.f; s.step = 0; s.seed = 0; s.B = 1; s.max_seq = cfg->max_seq; s.max_K = maxK;
+  s.n_acc = h->res;
+  s.flags = (uint32_t*)(h->res + MB);
+  s.out_tok = h->res + 2 * MB;
+  s.err = h->res + (h->res_words - 1);
+  if (cudaMemcpyAsync(h->dst, &h->hst, sizeof(DevState), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return bail(fail(h, SPS_ECUDA, "state upload failed"));
+  h->B = 1;
+  *out = h;
+  return SPS_OK;
+}
+
+int sps_destroy(sps_handle* h) {
+  if (!h) return SPS_OK;
+  cudaSetDevice(h->cfg.device);
+  if (h->stream) cudaStreamSynchronize(h->stream);
+  for (auto& kv : h->g_draft) cudaGraphExecDestroy(kv.second);
+  for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
+  free_model(h->tgt);
+  free_model(h->drf);
+  void* bufs[] = {h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part, h->ssq_part,
+                  h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
+                  h->hst.row_pos, h->hst.done_counter};
+  for (void* p : bufs) if (p) cudaFree(p);
+  if (h->h_res) cudaFreeHost(h->h_res);
+  if (h->h_par) cudaFreeHost(h->h_par);
+  if (h->h_rows) cudaFreeHost(h->h_rows);
+  for (auto& ev : h->ev) if (ev) cudaEventDestroy(ev);
+  if (h->own_stream && h->stream) cudaStreamDestroy(h->stream);
+  delete h;
+  return SPS_OK;
+}
+
+int sps_reset(sps_handle* h) {
+  if (!h) return fail(nullptr, SPS_EINVAL, "null handle");
+  CU(h, cudaSetDevice(h->cfg.device));
+  h->ready = false;
+  h->B = 1;
+  for (int& v : h->seq_len) v = 0;
+  CU(h, cudaMemsetAsync(h->hst.n, 0, 4 * (size_t)h->cfg.max_batch, h->stream));
+  CU(h, cudaMemsetAsync(h->res, 0, 4 * h->res_words, h->stream));
+  CU(h, cudaMemsetAsync(h->hst.done_counter, 0, 4, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+int sps_prefill(sps_handle* h, const int32_t* toks, int32_t n) {
+  if (!h || !toks) return fail(h, SPS_EINVAL, "null argument");
+  CU(h, cudaSetDevice(h->cfg.device));
+  int rc = set_sequences(h, toks, 1, n);
+  if (rc) return rc;
+  if ((rc = prefill_all(h, n))) return rc;
+  CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+int sps_step(sps_handle* h, int32_t K, float temperature, uint64_t seed, uint32_t step, int32_t* out_tokens,
+             int32_t* out_n_emitted, uint32_t* out_flags) {
+  if (!h || !out_tokens || !out_n_emitted) return fail(h, SPS_EINVAL, "null argument");
+  if (!h->ready) return fail(h, SPS_ESTATE, "sps_step before sps_prefill");
+  if (!(temperature > 0.f)) return fail(h, SPS_EINVAL, "temperature must be > 0");
+  CU(h, cudaSetDevice(h->cfg.device));
+  int rc = check_K(h, K);
+  if (rc) return rc;
+  for (int b = 0; b < h->B; ++b)
+    if (h->seq_len[b] + K + 1 > h->cfg.max_seq) return fail(h, SPS_ERANGE, "sequence would exceed max_seq");
+  if ((rc = write_params(h, temperature, seed, step))) return rc;
+  if ((rc = loop_once(h, K, false))) return rc;
+  const int MB = h->cfg.max_batch, ld = h->hst.max_K + 1;
+  for (int b = 0; b < h->B; ++b) {
+    const int a = h->h_res[b];
+    out_n_emitted[b] = a + 1;
+    if (out_flags) out_flags[b] = (uint32_t)h->h_res[MB + b];
+    for (int i = 0; i <= K; ++i) out_tokens[b * (K + 1) + i] = h->h_res[2 * MB + b * ld + i];
+    h->seq_len[b] += a + 1;
+  }
+  return SPS_OK;
+}
+
+int sps_last_logits(sps_handle* h, int32_t K, float* q_logits, float* p_logits, int32_t* drafts) {
+  if (!h) return fail(nullptr, SPS_EINVAL, "null handle");
+  if (K != h->last_K) return fail(h, SPS_ESTATE, "K differs from the last step's");
+  CU(h, cudaSetDevice(h->cfg.device));
+  const size_t V = h->tgt.cfg.vocab;
+  if (q_logits) CU(h, cudaMemcpyAsync(q_logits, h->q_logits, 4 * V * h->B * (K + 1), cudaMemcpyDeviceToHost, h->stream));
+  if (p_logits && K > 0) CU(h, cudaMemcpyAsync(p_logits, h->p_logits, 4 * V * h->B * K, cudaMemcpyDeviceToHost, h->stream));
+  if (drafts && K > 0)
+    CU(h, cudaMemcpy2DAsync(drafts, (size_t)K * 4, h->hst.drafts, (size_t)h->hst.max_K * 4, (size_t)K * 4, h->B, cudaMemcpyDeviceToHost, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, int n_new, int K, float T, uint64_t seed,
+                         int32_t* out_tokens, sps_stats* out_stats) {
+  if (!h || !prompts || !out_tokens) return fail(h, SPS_EINVAL, "null argument");
+  if (n_new < 1) return fail(h, SPS_EINVAL, "n_new must be >= 1");
+  if (!(T > 0.f)) return fail(h, SPS_EINVAL, "temperature must be > 0");
+  CU(h, cudaSetDevice(h->cfg.device));
+  if (P < 1) return fail(h, SPS_EINVAL, "prompt_len must be >= 1");
+  if ((long long)P + n_new + K > h->cfg.max_seq) return fail(h, SPS_ERANGE, "prompt_len + n_new + K exceeds max_seq");
+  int rc = sps_reset(h);
+  if (rc) return rc;
+  h->B = B;
+  if ((rc = check_K(h, K))) return rc;
+  CU(h, cudaEventRecord(h->ev[4], h->stream));
+  if ((rc = set_sequences(h, prompts, B, P))) return rc;
+  {
+    std::vector<int32_t> lim(B, P + n_new);
+    CU(h, cudaMemcpy(h->hst.limit, lim.data(), B * 4, cudaMemcpyHostToDevice));
+  }
+  cudaEvent_t e_pre0 = h->ev[4];
+  CU(h, cudaEventRecord(e_pre0, h->stream));
+  if ((rc = prefill_all(h, P))) return rc;
+  if ((rc = write_params(h, T, seed, 0u))) return rc;
+  std::vector<sps_stats> st(B);
+  for (auto& s : st) std::memset(&s, 0, sizeof(s));
+  std::vector<int> made(B, 0);
+  const int MB = h->cfg.max_batch, ld = h->hst.max_K + 1;
+  float ms_draft = 0.f, ms_verify = 0.f, ms_accept = 0.f, ms_prefill = 0.f;
+  bool first = true;
+  for (;;) {
+    bool all = true;
+    for (int b = 0; b < B; ++b) all = all && made[b] >= n_new;
+    if (all) break;
+    if ((rc = loop_once(h, K, true))) return rc;
+    float a01 = 0, a12 = 0, a23 = 0;
+    if (first) { cudaEventElapsedTime(&ms_prefill, e_pre0, h->ev[0]); first = false; }
+    cudaEventElapsedTime(&a01, h->ev[0], h->ev[1]);
+    cudaEventElapsedTime(&a12, h->ev[1], h->ev[2]);
+    cudaEventElapsedTime(&a23, h->ev[2], h->ev[3]);
+    ms_draft += a01; ms_verify += a12; ms_accept += a23;
+    for (int b = 0; b < B; ++b) {
+      if (made[b] >= n_new) continue;
+      const int a = h->h_res[b];
+      const uint32_t fl = (uint32_t)h->h_res[MB + b];
+      add_loop_stats(&st[b], K, a, fl);
+      for (int i = 0; i <= a; ++i) {
+        const int32_t tok = h->h_res[2 * MB + b * ld + i];
+        if (made[b] < n_new) out_tokens[(size_t)b * n_new + made[b]++] = tok;
+        else st[b].overshoot += 1;
+      }
+      h->seq_len[b] += a + 1;
+    }
+  }
+  if (out_stats)
+    for (int b = 0; b < B; ++b) {
+      st[b].ms_prefill = ms_prefill; st[b].ms_draft = ms_draft; st[b].ms_verify = ms_verify; st[b].ms_accept = ms_accept;
+      st[b].ms_decode = ms_draft + ms_verify + ms_accept;
+      out_stats[b] = st[b];
+    }
+  return SPS_OK;
+}
+
+int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K, float temperature,
+                 uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
+  return generate_impl(h, prompt, 1, prompt_len, n_new, K, temperature, seed, out_tokens, out_stats);
+}
+
+int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new, int32_t K,
+                       float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
+  if (h && (B < 1 || B > h->cfg.max_batch)) return fail(h, SPS_EINVAL, "batch outside 1..max_batch");
+  return generate_impl(h, prompts, B, prompt_len, n_new, K, temperature, seed, out_tokens, out_stats);
+}
+
+int sps_score(sps_handle* h, int32_t which, const int32_t* rows, int32_t n_rows, float* out_logits, float* out_ms) {
+  if (!h || !rows || !out_logits) return fail(h, SPS_EINVAL, "null argument");
+  if (!h->ready) return fail(h, SPS_ESTATE, "sps_score before sps_prefill");
+  if (h->B != 1) return fail(h, SPS_ESTATE, "sps_score works on a batch-1 handle");
+  if (n_rows < 1 || n_rows > SPS_MAX_ROWS) return fail(h, SPS_EINVAL, "n_rows outside 1..16");
+  ModelDev& m = which == 0 ? h->tgt : h->drf;
+  if (!m.present) return fail(h, SPS_EINVAL, "model not loaded");
+  CU(h, cudaSetDevice(h->cfg.device));
+  const int len = h->seq_len[0] - 1;
+  if (len + n_rows > h->cfg.max_seq) return fail(h, SPS_ERANGE, "rows would exceed max_seq");
+  for (int i = 0; i < n_rows; ++i) {
+    if (rows[i] < 0 || rows[i] >= m.cfg.vocab) return fail(h, SPS_ERANGE, "token id outside the vocabulary");
+    h->h_rows[i] = rows[i];
+    h->h_rows[SPS_MAX_ROWS + i] = len + i;
+  }
+  CU(h, cudaMemcpyAsync(h->hst.row_tok, h->h_rows, 4 * n_rows, cudaMemcpyHostToDevice, h->stream));
+  CU(h, cudaMemcpyAsync(h->hst.row_pos, h->h_rows + SPS_MAX_ROWS, 4 * n_rows, cudaMemcpyHostToDevice, h->stream));
+  PassSpec ps{};
+  ps.mode = PASS_EXPLICIT; ps.rows_per_seq = n_rows; ps.logits = out_logits; ps.logits_ld = m.cfg.vocab;
+  ps.lrow0 = 0; ps.lrowstep = 1; ps.lrows = n_rows;
+  CU(h, cudaEventRecord(h->ev[0], h->stream));
+  int rc = run_pass(h, m, ps);
+  if (rc) return rc;
+  CU(h, cudaEventRecord(h->ev[1], h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  if (out_ms) CU(h, cudaEventElapsedTime(out_ms, h->ev[0], h->ev[1]));
+  return SPS_OK;
+}
+
+int sps_verify(sps_handle* h, const int32_t* rows, int32_t K, float* out_logits, float* out_ms) {
+  if (K < 0 || K > SPS_MAX_K) return fail(h, SPS_EINVAL, "K outside 0..15");
+  return sps_score(h, 0, rows, K + 1, out_logits, out_ms);
+}
+
+int sps_accept(const float* q_logits, const float* p_logits, const int32_t* draft_tokens, int32_t B, int32_t K, int32_t V,
+               float temperature, uint64_t seed, uint32_t step, void* stream, int32_t* out_n_accepted,
+               int32_t* out_tokens, uint32_t* out_flags) {
+  if (!q_logits || !out_n_accepted || !out_tokens || !out_flags) return fail(nullptr, SPS_EINVAL, "null argument");
+  if (K > 0 && (!p_logits || !draft_tokens)) return fail(nullptr, SPS_EINVAL, "K > 0 needs p_logits and draft_tokens");
+  if (B < 1 || K < 0 || K > SPS_MAX_K || V < 1) return fail(nullptr, SPS_EINVAL, "B, K or V out of range");
+  if (!(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "temperature must be > 0");
+  AcceptArgs a{};
+  a.st = nullptr; a.q_logits = q_logits; a.p_logits = p_logits ? p_logits : q_logits;
+  a.drafts = draft_tokens ? draft_tokens : out_tokens; a.drafts_ld = K;
+  a.B = B; a.K = K; a.V = V; a.n_acc = out_n_accepted; a.out_tok = out_tokens; a.out_ld = K + 1; a.flags = out_flags;
+  a.temperature = temperature; a.seed = seed; a.step = step;
+  cudaError_t e = accept_launch(a, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("accept launch: ") + cudaGetErrorString(e));
+  return SPS_OK;
+}
+
+int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uint64_t seed, uint32_t step, uint32_t t,
+               void* stream, int32_t* out_tokens) {
+  if (!logits || !out_tokens) return fail(nullptr, SPS_EINVAL, "null argument");
+  if (B < 1 || V < 1 || !(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "B, V or temperature out of range");
+  SampleArgs a{};
+  a.st = nullptr; a.logits = logits; a.ld = V; a.V = V; a.B = B; a.t = t; a.out = out_tokens; a.out_ld = 1;
+  a.temperature = temperature; a.seed = seed; a.step = step;
+  cudaError_t e = sample_launch(a, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("sample launch: ") + cudaGetErrorString(e));
+  return SPS_OK;
+}
+
+static int cur_num_sm() {
+  int dev = 0, n = SPS_NUM_SM_FALLBACK;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  return n;
+}
+
+int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
+  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return -1;
+  const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
+  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (LIN_MAX_R + 1) + 256);
+}
+
+int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace,
+               void* stream, float* out_ms) {
+  if (!W || !X || !Y || !workspace) return fail(nullptr, SPS_EINVAL, "null argument");
+  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return fail(nullptr, SPS_EINVAL, "M, N or D out of range");
+  if (dtype == 1 && D % 128) return fail(nullptr, SPS_EINVAL, "bf16 needs D to be a multiple of 128");
+  if (dtype == 0 && (size_t)M * D * 4 > 200 * 1024) return fail(nullptr, SPS_EINVAL, "fp32: M * D too large");
+  if (dtype != 0 && dtype != 1) return fail(nullptr, SPS_EINVAL, "dtype must be 0 or 1");
+  const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
+  LinArgs a{};
+  a.W[0] = W; a.rows_per_mat = N; a.N = N; a.D = D; a.M = M; a.X = X; a.ldx = D; a.x_row0 = 0; a.x_rowstep = 1;
+  a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
+  char* ws = (char*)workspace;
+  a.counters = (int*)ws;
+  size_t off = ((sizeof(int) * (LIN_MAX_R + 1) + 255) / 256) * 256;
+  a.ssq_part = (float*)(ws + off);
+  off += sizeof(float) * (size_t)LIN_MAX_R * SPS_MAX_ROWS;
+  a.part = (float*)(ws + off);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (out_ms) { cudaEventCreate(&e0); cudaEventCreate(&e1); cudaEventRecord(e0, st); }
+  cudaError_t e = lin_launch(dtype, a, p, st);
+  if (out_ms) {
+    cudaEventRecord(e1, st);
+    cudaEventSynchronize(e1);
+    cudaEventElapsedTime(out_ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+  }
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("linear launch: ") + cudaGetErrorString(e));
+  return SPS_OK;
+}
+
+int sps_philox(const uint32_t* ctr, const uint32_t* key, int32_t n, void* stream, uint32_t* out) {
+  if (!ctr || !key || !out || n < 1) return fail(nullptr, SPS_EINVAL, "bad argument");
+  cudaError_t e = philox_launch(ctr, key, n, out, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("philox launch: ") + cudaGetErrorString(e));
+  return SPS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,293 @@
+// Sampling kernels: the inverse-CDF draw used for draft tokens, and the fused modified rejection
+// sampler of Algorithm 2 (accept test, residual resample, extra token) -- one CTA per sequence,
+// warp shuffles plus a block prefix sum over the vocabulary.
+#include <limits.h>
+
+#include "common.cuh"
+
+#define SAMPLER_THREADS 1024
+#define SAMPLER_WARPS (SAMPLER_THREADS / 32)
+
+struct ScanSmem {
+  float warp_part[SAMPLER_WARPS];
+  float total;
+  int ired[SAMPLER_WARPS];
+  int ires;
+};
+
+__device__ inline int block_min_int(int v, ScanSmem& sm) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_min_int(v);
+  __syncthreads();
+  if (lane == 0) sm.ired[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    int x = (lane < (int)(blockDim.x >> 5)) ? sm.ired[lane] : INT_MAX;
+    x = warp_min_int(x);
+    if (lane == 0) sm.ires = x;
+  }
+  __syncthreads();
+  return sm.ires;
+}
+__device__ inline int block_max_int(int v, ScanSmem& sm) { return -block_min_int(-v, sm); }
+
+// Inverse-CDF draw in index order on unnormalised weights w(0..V-1): the smallest i whose inclusive
+// running sum exceeds u * total; if rounding leaves none, the largest i with w(i) > 0.
+// Thread t owns the contiguous chunk [t*c, (t+1)*c); chunk sums are combined by a warp scan and a
+// scan of the warp totals, so the result does not depend on timing.  Returns the token to all threads.
+template <class F>
+__device__ int block_invcdf(F w, int V, float u, ScanSmem& sm, float* total_out) {
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk = (V + nt - 1) / nt;
+  const int i0 = min(tid * chunk, V), i1 = min(i0 + chunk, V);
+  float local = 0.f;
+  for (int i = i0; i < i1; ++i) local += w(i);
+  float incl = local;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const float v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  __syncthreads();
+  if (lane == 31) sm.warp_part[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = nt >> 5;
+    const float v = (lane < nw) ? sm.warp_part[lane] : 0.f;
+    float iv = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float x = __shfl_up_sync(0xffffffffu, iv, o);
+      if (lane >= o) iv += x;
+    }
+    if (lane < nw) sm.warp_part[lane] = iv - v;  // exclusive prefix of the warp
+    if (lane == nw - 1) sm.total = iv;
+  }
+  __syncthreads();
+  const float pre = sm.warp_part[warp] + (incl - local);
+  const float total = sm.total;
+  if (total_out) *total_out = total;
+  const float target = u * total;
+  int cand = INT_MAX;
+  float c = pre;
+  for (int i = i0; i < i1; ++i) {
+    c += w(i);
+    if (c > target) { cand = i; break; }
+  }
+  int tok = block_min_int(cand, sm);
+  if (tok == INT_MAX) {
+    int last = -1;
+    for (int i = i0; i < i1; ++i) if (w(i) > 0.f) last = i;
+    tok = block_max_int(last, sm);
+    if (tok < 0) tok = V - 1;
+  }
+  return tok;
+}
+
+__device__ inline float block_max_f(float v, float* s_part, float* s_out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_max(v);
+  __syncthreads();
+  if (lane == 0) s_part[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    float x = (lane < (int)(blockDim.x >> 5)) ? s_part[lane] : -INFINITY;
+    x = warp_max(x);
+    if (lane == 0) *s_out = x;
+  }
+  __syncthreads();
+  return *s_out;
+}
+__device__ inline float block_sum_f(float v, float* s_part, float* s_out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) s_part[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    float x = (lane < (int)(blockDim.x >> 5)) ? s_part[lane] : 0.f;
+    x = warp_sum(x);
+    if (lane == 0) *s_out = x;
+  }
+  __syncthreads();
+  return *s_out;
+}
+
+// ------------------------------------------------------------------------------------------------
+// x ~ softmax(logits / T) by inverse CDF with u_draft(b, s, t)  (Algorithm 2: "sample draft
+// auto-regressively"; with t = 0 and u_res it is Algorithm 1's sample).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
+  __shared__ ScanSmem sm;
+  __shared__ float s_part[SAMPLER_WARPS];
+  __shared__ float s_val;
+  const int b = blockIdx.x;
+  float T = a.temperature;
+  uint64_t seed = a.seed;
+  uint32_t step = a.step;
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; }
+  const float invT = 1.0f / T;
+  const float* row = a.logits + (long long)b * a.ld;
+  float m = -INFINITY;
+  for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
+  m = block_max_f(m, s_part, &s_val);
+  const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, a.t);
+  auto w = [&](int i) { return expf((row[i] - m) * invT); };
+  const int tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+  if (threadIdx.x == 0) a.out[(long long)b * a.out_ld] = tok;
+}
+
+cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st) {
+  sample_kernel<<<a.B, SAMPLER_THREADS, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Modified rejection sampling, fused (Algorithm 2, second for-loop and extra-token line).
+// Phase 1: max and sum-exp of all 2K+1 rows.  Phase 2: thread 0 walks the accept chain.
+// Phase 3: one vocabulary-wide prefix sum, over max(0, q_t - p_t) at the rejected position or over
+// q_K when every draft was accepted.  When a DevState is given the loop is advanced in place.
+// ------------------------------------------------------------------------------------------------
+#define ACC_MAX_ROWS (2 * 15 + 1)
+
+__global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
+  __shared__ ScanSmem sm;
+  __shared__ float s_red[SAMPLER_WARPS][ACC_MAX_ROWS + 1];
+  __shared__ float s_max[ACC_MAX_ROWS], s_sum[ACC_MAX_ROWS];
+  __shared__ int s_stop, s_mode;
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = a.K, V = a.V, R = 2 * K + 1;
+  float T = a.temperature;
+  uint64_t seed = a.seed;
+  uint32_t step = a.step;
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; }
+  const float invT = 1.0f / T;
+  const float* qrow = a.q_logits + (long long)b * (K + 1) * V;
+  const float* prow = a.p_logits + (long long)b * K * V;
+  auto rowptr = [&](int r) { return r <= K ? qrow + (long long)r * V : prow + (long long)(r - K - 1) * V; };
+
+  // ---- phase 1a: maxima
+  for (int r = 0; r < R; ++r) {
+    const float* row = rowptr(r);
+    float m = -INFINITY;
+    for (int i = tid; i < V; i += SAMPLER_THREADS) m = fmaxf(m, row[i]);
+    m = warp_max(m);
+    if (lane == 0) s_red[warp][r] = m;
+  }
+  __syncthreads();
+  if (tid < R) {
+    float m = -INFINITY;
+    for (int w = 0; w < SAMPLER_WARPS; ++w) m = fmaxf(m, s_red[w][tid]);
+    s_max[tid] = m;
+  }
+  __syncthreads();
+  // ---- phase 1b: sums of exp((l - max) / T)
+  for (int r = 0; r < R; ++r) {
+    const float* row = rowptr(r);
+    const float m = s_max[r];
+    float s = 0.f;
+    for (int i = tid; i < V; i += SAMPLER_THREADS) s += expf((row[i] - m) * invT);
+    s = warp_sum(s);
+    if (lane == 0) s_red[warp][r] = s;
+  }
+  __syncthreads();
+  if (tid < R) {
+    float s = 0.f;
+    for (int w = 0; w < SAMPLER_WARPS; ++w) s += s_red[w][tid];
+    s_sum[tid] = s;
+  }
+  __syncthreads();
+
+  // ---- phase 2: accept chain, left to right
+  const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
+  if (tid == 0) {
+    int stop = K;
+    for (int t = 0; t < K; ++t) {
+      int d = drafts[t];
+      if (d < 0 || d >= V) { d = 0; if (a.st) atomicExch(a.st->err, 1); }
+      const float qd = expf((qrow[(long long)t * V + d] - s_max[t]) * invT) / s_sum[t];
+      const float pd = expf((prow[(long long)t * V + d] - s_max[K + 1 + t]) * invT) / s_sum[K + 1 + t];
+      // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
+      const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
+      const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)t);
+      if (!(u.u_acc < ratio)) { stop = t; break; }
+    }
+    s_stop = stop;
+  }
+  __syncthreads();
+  const int stop = s_stop;
+  uint32_t fl = 0;
+  int tok;
+  if (stop < K) {
+    // ---- rejected at `stop`: x ~ max(0, q - p) / sum max(0, q - p)
+    const float* ql = qrow + (long long)stop * V;
+    const float* pl = prow + (long long)stop * V;
+    const float mq = s_max[stop], mp = s_max[K + 1 + stop];
+    const float iq = 1.0f / s_sum[stop], ip = 1.0f / s_sum[K + 1 + stop];
+    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)stop);
+    auto wres = [&](int i) {
+      return fmaxf(0.f, expf((ql[i] - mq) * invT) * iq - expf((pl[i] - mp) * invT) * ip);
+    };
+    float total;
+    tok = block_invcdf(wres, V, u.u_res, sm, &total);
+    fl |= 1u;
+    if (!(total > 0.f)) {
+      auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
+      tok = block_invcdf(wq, V, u.u_res, sm, nullptr);
+      fl |= 4u;
+    }
+  } else {
+    // ---- every draft accepted: extra token from the (K+1)-th target distribution
+    const float* ql = qrow + (long long)K * V;
+    const float mq = s_max[K];
+    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)K);
+    auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
+    tok = block_invcdf(wq, V, u.u_res, sm, nullptr);
+    fl |= 2u;
+  }
+  (void)s_mode;
+  // ---- results
+  int32_t* out = a.out_tok + (long long)b * a.out_ld;
+  if (tid <= K) out[tid] = (tid < stop) ? drafts[tid] : (tid == stop ? tok : -1);
+  if (tid == 0) {
+    a.n_acc[b] = stop;
+    a.flags[b] = fl;
+  }
+  if (a.st) {
+    // advance the sequence in place: accepted drafts, then the resampled / extra token
+    DevState* st = a.st;
+    const int n = st->n[b];
+    const bool live = n < st->limit[b];   // a finished sequence of a batch keeps its length
+    __syncthreads();
+    if (live && tid <= stop && n + tid < st->max_seq)
+      st->tokens[(long long)b * st->max_seq + n + tid] = (tid < stop) ? drafts[tid] : tok;
+    __syncthreads();
+    if (tid == 0) {
+      if (live) st->n[b] = n + stop + 1;
+      __threadfence();
+      // the last sequence to finish moves the loop counter
+      const uint32_t done = atomicAdd(st->done_counter, 1u);
+      if (done == (uint32_t)gridDim.x - 1) {
+        *st->done_counter = 0u;
+        st->step = step + 1u;
+      }
+    }
+  }
+}
+
+cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st) {
+  accept_kernel<<<a.B, SAMPLER_THREADS, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+__global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t w[4];
+  philox4x32_10(ctr[4 * i], ctr[4 * i + 1], ctr[4 * i + 2], ctr[4 * i + 3], key[2 * i], key[2 * i + 1], w);
+  for (int j = 0; j < 4; ++j) out[4 * i + j] = w[j];
+}
+cudaError_t philox_launch(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out, cudaStream_t st) {
+  philox_kernel<<<(n + 127) / 128, 128, 0, st>>>(ctr, key, n, out);
+  return cudaGetLastError();
+}

@@ -1,0 +1,72 @@
+"""GPU parity of the memory-bound linear layer (sps_linear) with its definition in the oracle.
+
+Tolerance: fp32 accumulation of D products against a double sum.  With |w| ~ 0.02..1 and |x| ~ 1 the
+result y has magnitude ~ sqrt(D)*|w|; the bound used is 2e-5 * sqrt(D) * max|w| * max|x| + 1e-6, far
+inside the 1e-3 (fp32) / 5e-2 (bf16) logit tolerances; bf16 weights are exact inputs on both sides and
+activations keep ~16 mantissa bits through the hi/lo split."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2302_01318_b200 as sps
+import sps_synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def run_linear(W, X):
+    N, D = W.shape
+    M = X.shape[0]
+    dtype = 0 if W.dtype == torch.float32 else 1
+    ws = torch.zeros(sps.sps_linear_workspace_bytes(dtype, M, N, D), dtype=torch.uint8, device=DEV)
+    Y = torch.full((M, N), float("nan"), device=DEV)
+    sps.sps_linear(W, X, Y, ws)
+    # second call on the same workspace: the kernel must have left its counters ready
+    Y2 = torch.full((M, N), float("nan"), device=DEV)
+    sps.sps_linear(W, X, Y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2)       # and results are bit-reproducible
+    return Y.cpu().numpy()
+
+
+def tol(W, X, D):
+    return 2e-5 * np.sqrt(D) * float(W.abs().max()) * float(X.abs().max()) + 1e-6
+
+
+@pytest.mark.parametrize("M", [1, 2, 5, 8, 9, 16])
+@pytest.mark.parametrize("N,D", [(1000, 256), (77, 128), (4099, 1024), (2048, 2048), (1536, 6144)])
+def test_linear_bf16_small(M, N, D):
+    g = torch.Generator().manual_seed(N + D + M)
+    W = (torch.randn((N, D), generator=g) * 0.05).to(torch.bfloat16)
+    X = torch.randn((M, D), generator=g)
+    got = run_linear(W.to(DEV), X.to(DEV))
+    want = oracle.linear(sps_synth.to_numpy(W), X.numpy())
+    assert np.abs(got - want).max() <= tol(W.float(), X, D)
+
+
+@pytest.mark.parametrize("M", [1, 5, 9])
+@pytest.mark.parametrize("N,D", [(1024, 256), (130, 128), (515, 1024)])
+def test_linear_fp32(M, N, D):
+    g = torch.Generator().manual_seed(N + D + M)
+    W = torch.randn((N, D), generator=g) * 0.05
+    X = torch.randn((M, D), generator=g)
+    got = run_linear(W.to(DEV), X.to(DEV))
+    want = oracle.linear(W.numpy(), X.numpy())
+    assert np.abs(got - want).max() <= tol(W, X, D)
+
+
+@pytest.mark.parametrize("N,D", [(8192, 8192), (8192, 32768), (32000, 8192), (24576, 6144)])
+def test_linear_full_size_sampled_rows(N, D):
+    """the 70B-shaped layers at full size, M = 5 as in the bench: 64 sampled output rows checked
+    one by one against the oracle's double dot products"""
+    g = torch.Generator(device=DEV).manual_seed(N + D)
+    W = torch.empty((N, D), device=DEV, dtype=torch.bfloat16).normal_(0, 0.02, generator=g)
+    X = torch.randn((5, D), device=DEV, generator=g)
+    got = run_linear(W, X)
+    rows = np.unique(np.concatenate([[0, 1, 15, 16, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 58)]))
+    Wr = sps_synth.to_numpy(W[torch.from_numpy(rows).to(DEV)])
+    want = oracle.linear(Wr, X.cpu().numpy())
+    assert np.abs(got[:, rows] - want).max() <= tol(W[:64].float(), X, D)
+    assert np.isfinite(got).all()
