@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-sampling hot path on B200.
+
+One "step" = one whole generation through the library (`sps_generate`): prompt of P tokens, then
+n_new tokens by speculative sampling with lookahead K at batch 1, i.e. every row of the hot path (K
+draft steps, one K+1-row scoring pass, the fused accept / resample kernel, cache rollback, loop
+control) run ~n_new/(tokens per loop) times.  Default workload: the 70B-shaped target with the 4B-shaped
+draft (random-init bf16 weights generated on the device, shared (un)embedding), P = 128, n_new = 128,
+K = 4, temperature 1 -- the configuration the headline metric is quoted on.
+
+  value : tokens/s over the decode loops, timed with CUDA events on the library's stream (inputs resident)
+  e2e   : tokens/s of the same calls by wall clock, prompt upload, prompt pass and result read-back included
+  ar    : the same library's autoregressive decode (K = 0) on the same models
+
+N > 1 (torchrun): independent replicas, one per GPU, no collective on the data path; the time is the
+max over ranks.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import sps_synth  # noqa: E402
+
+METRIC = "batch-1 tokens/s SpS vs AR decode; verify-pass HBM GB/s vs peak"
+UNIT = "tokens/s"
+# mean tokens per speculative loop measured by this bench's own arm on each workload (seeded weights and
+# prompts make it repeatable); the CPU arm cannot run whole generations of the 70B pair, so it uses these
+ASSUMED_TOKENS_PER_LOOP = {"70b": 1.30, "mid": 1.9, "tiny": 3.0, "tiny_bf16": 3.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, device copy)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region"""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_models(cfgname, device):
+    c = sps_synth.CONFIGS[cfgname]
+    wt = sps_synth.make_weights(c["target"], seed=0, tag="target", device=device)
+    share = wt if cfgname == "70b" else None
+    wd = sps_synth.make_weights(c["draft"], seed=0, tag="draft", device=device, share_embed_from=share)
+    return c, wt, wd
+
+
+def kv_bytes_per_token(cfg):
+    return cfg["n_layers"] * 2 * cfg["d_model"] * (4 if cfg["dtype"] == 0 else 2)
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_seconds(c, K, wt_layer, wd_layer, wt_unembed, wd_unembed, P):
+    """Time the oracle, as it stands, on the pieces one loop is made of: one target layer over K+1 rows,
+    the target unembedding over K+1 rows, one draft layer and the draft unembedding over 1 row."""
+    import oracle
+    tc, dc = c["target"], c["draft"]
+    rng = np.random.default_rng(0)
+    out = {}
+    for tag, mc, lw, un, rows in (("target", tc, wt_layer, wt_unembed, K + 1), ("draft", dc, wd_layer, wd_unembed, 1)):
+        m = oracle.Transformer(dict(mc, n_layers=1), None, P + K + 2)
+        emb = un[rng.integers(0, mc["vocab"], rows)]
+        pos = np.arange(P - 1, P - 1 + rows, dtype=np.int32)
+        m.begin_rows(np.ascontiguousarray(emb), pos)
+        t0 = time.perf_counter()
+        m.layer(0, lw)
+        t1 = time.perf_counter()
+        m.end(np.ones(mc["d_model"], dtype=np.float32), un)
+        t2 = time.perf_counter()
+        out[tag + "_layer_s"] = t1 - t0
+        out[tag + "_unembed_s"] = t2 - t1
+        m.close()
+    return out
+
+
+def oracle_loop_seconds(c, K, s):
+    tc, dc = c["target"], c["draft"]
+    verify = tc["n_layers"] * s["target_layer_s"] + s["target_unembed_s"]
+    draft_row = dc["n_layers"] * s["draft_layer_s"] + s["draft_unembed_s"]
+    return verify + (K + 1) * draft_row if K > 0 else verify / (K + 1)
+
+
+def layer_numpy(lw):
+    return {k: sps_synth.to_numpy(v) for k, v in lw.items()}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfgname = args.config
+    c = sps_synth.CONFIGS[cfgname]
+    K, P, n_new = args.K, c["prompt_len"], c["n_new"]
+    tc, dc = c["target"], c["draft"]
+    one_t = sps_synth.make_weights(dict(tc, n_layers=1), seed=0, tag="target", device="cpu")
+    one_d = sps_synth.make_weights(dict(dc, n_layers=1), seed=0, tag="draft", device="cpu")
+    lt, ld = layer_numpy(one_t["layers"][0]), layer_numpy(one_d["layers"][0])
+    ut, ud = sps_synth.to_numpy(one_t["unembed"]), sps_synth.to_numpy(one_d["unembed"])
+    times = []
+    for i in range(args.warmup + args.steps):
+        s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
+        if i >= args.warmup:
+            times.append(oracle_loop_seconds(c, K, s))
+    loop_s = statistics.mean(times)
+    tpl = ASSUMED_TOKENS_PER_LOOP.get(cfgname, 1.0) if K > 0 else 1.0
+    value = tpl / loop_s
+    sample = (f"per step: 1 of {tc['n_layers']} target layers over {K + 1} rows + target unembedding + 1 of "
+              f"{dc['n_layers']} draft layers and draft unembedding over 1 row, context {P}; scaled to one loop "
+              f"(x layers, x{K + 1} draft rows) at {tpl} tokens per loop")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * loop_s * (n_new / tpl), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cfgname, K, P, n_new)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_name(cfgname, K, P, n_new):
+    c = sps_synth.CONFIGS[cfgname]
+    t, d = c["target"], c["draft"]
+    return (f"{cfgname}: target L{t['n_layers']}/d{t['d_model']}/ff{t['d_ff']}/V{t['vocab']}, draft L{d['n_layers']}/"
+            f"d{d['d_model']}/ff{d['d_ff']}, {'bf16' if t['dtype'] else 'fp32'} random-init N(0,0.02) "
+            f"(shared (un)embedding), prompt {P}, generate {n_new}, K={K}, T=1.0, batch 1")
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import paper_2302_01318_b200 as sps
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    cfgname, K = args.config, args.K
+    c, wt, wd = build_models(cfgname, dev)
+    P, n_new, T = c["prompt_len"], c["n_new"], 1.0
+    V = c["target"]["vocab"]
+    max_seq = ((P + n_new + max(K, 8) + 63) // 64) * 64
+    h = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=max_seq, max_batch=1, max_K=max(K, 1), device=local)
+    seeds = [1000 * rank + i for i in range(args.warmup + args.steps + 8)]
+
+    def gen(i, k):
+        prompt = sps_synth.make_prompt(seeds[i], P, V)
+        t0 = time.perf_counter()
+        out, st = h.sps_generate(prompt, n_new, k, T, seeds[i])
+        return out, st, time.perf_counter() - t0
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        gen(i, K)
+    clk = ClockSampler(local)
+    barrier()
+    clk.start()
+    stats, walls = [], []
+    for i in range(args.steps):
+        _, st, w = gen(args.warmup + i, K)
+        stats.append(st); walls.append(w)
+    barrier()
+    clocks = clk.stop()
+    dec_ms = sum(s["ms_decode"] for s in stats)
+    wall_s = sum(walls)
+    if dist is not None:
+        tt = torch.tensor([dec_ms, wall_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        dec_ms, wall_s = float(tt[0]), float(tt[1])
+    tokens = args.steps * n_new * world
+    value = tokens / (dec_ms / 1e3)
+    e2e = tokens / wall_s
+    loops = sum(s["loops"] for s in stats)
+    emitted = sum(s["emitted"] for s in stats)
+    accepted = sum(s["accepted"] for s in stats)
+    hist = [sum(s["hist_emitted"][j] for s in stats) for j in range(K + 2)]
+    ms_verify = sum(s["ms_verify"] for s in stats)
+    ms_draft = sum(s["ms_draft"] for s in stats)
+    ms_accept = sum(s["ms_accept"] for s in stats)
+    peak, peak_src = measured_peaks()
+    # algorithmic bytes: every weight of the model once per pass, plus the cached keys/values read
+    ctx = P + n_new / 2.0
+    vbytes = sps_synth.weight_bytes(c["target"]) + kv_bytes_per_token(c["target"]) * ctx
+    dbytes = sps_synth.weight_bytes(c["draft"]) + kv_bytes_per_token(c["draft"]) * ctx
+    v_gbs = vbytes * loops / (ms_verify / 1e3) / 1e9 if ms_verify > 0 else None
+    d_gbs = dbytes * loops * K / (ms_draft / 1e3) / 1e9 if ms_draft > 0 and K > 0 else None
+    n_lin_verify = 5 * c["target"]["n_layers"] + 1
+    roofline = {"bound": "hbm", "kernel": "lin_bf16_kernel (weight-streaming linear layer) inside the scoring pass",
+                "achieved": v_gbs, "peak": peak, "unit": "GB/s", "frac": (v_gbs / peak) if v_gbs else None,
+                "frac_of_8000_nominal": (v_gbs / 8000.0) if v_gbs else None, "peak_source": peak_src,
+                "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
+                "traffic": args.traffic}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dec_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if c["target"]["dtype"] else "f32", "data": "synthetic",
+            "config": {"workload": workload_name(cfgname, K, P, n_new), "l2": "weights streamed per pass exceed L2 by >1000x",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e, "unit": UNIT, "h2d_bytes_per_step": 4 * P + 24 + 16,
+                    "d2h_bytes_per_step": int(loops / args.steps * 4 * (2 + K + 2))},
+            "gpu_launches": sum(s["kernel_launches"] for s in stats),
+            "roofline": roofline,
+            "roofline_draft": {"bound": "hbm", "achieved": d_gbs, "peak": peak, "unit": "GB/s", "frac": (d_gbs / peak) if d_gbs else None},
+            "loop": {"loops": loops, "tokens_per_loop": emitted / loops if loops else None,
+                     "accept_rate": accepted / (loops * K) if loops and K else None, "hist_emitted": hist,
+                     "ms_verify_per_loop": ms_verify / loops if loops else None,
+                     "ms_draft_per_step": ms_draft / loops / K if loops and K else None,
+                     "ms_accept_per_loop": ms_accept / loops if loops else None,
+                     "ms_prefill": stats[-1]["ms_prefill"]}}
+    if rank == 0 and world == 1:
+        # the same library's autoregressive decode on the same models
+        ar_stats = []
+        gen(0, 0)
+        for i in range(args.ar_steps):
+            _, st, _ = gen(args.warmup + i, 0)
+            ar_stats.append(st)
+        ar_ms = sum(s["ms_decode"] for s in ar_stats)
+        ar_tps = args.ar_steps * n_new / (ar_ms / 1e3)
+        ar_gbs = sps_synth.weight_bytes(c["target"]) * args.ar_steps * n_new / (ar_ms / 1e3) / 1e9
+        line["ar"] = {"value": ar_tps, "unit": UNIT, "ms_per_token": ar_ms / (args.ar_steps * n_new), "hbm_gbs": ar_gbs,
+                      "frac": ar_gbs / peak}
+        line["speedup_vs_ar"] = value / ar_tps
+        if not args.no_cpu:
+            import oracle
+            lt = layer_numpy(wt["layers"][0])
+            ld = layer_numpy(wd["layers"][0])
+            ut, ud = sps_synth.to_numpy(wt["unembed"]), sps_synth.to_numpy(wd["unembed"])
+            s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
+            loop_s = oracle_loop_seconds(c, K, s)
+            tpl = emitted / loops if K > 0 else 1.0
+            line["cpu_baseline"] = {"value": tpl / loop_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                    "sample": (f"oracle timed on 1 of {c['target']['n_layers']} target layers over {K + 1} rows + "
+                                               f"target unembedding + 1 of {c['draft']['n_layers']} draft layers + draft "
+                                               f"unembedding over 1 row (context {P}), scaled to one loop and divided into the "
+                                               f"measured {tpl:.3f} tokens per loop"), "seconds": s}
+    h.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="70b", choices=list(sps_synth.CONFIGS))
+    ap.add_argument("--K", type=int, default=4)
+    ap.add_argument("--ar-steps", type=int, default=2)
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None, help="ncu dram bytes per launch of the dominant kernel, if known")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

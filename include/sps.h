@@ -40,7 +40,7 @@ extern "C" {
 #define SPS_ECUDA (-3)    /* a CUDA call failed; sps_last_error has its message    */
 #define SPS_ERANGE (-4)   /* token id >= vocab, or sequence would exceed max_seq   */
 #define SPS_ESTATE (-5)   /* call order (e.g. step before prefill)                 */
-#define SPS_ETIMEOUT (-6) /* reserved: a bounded device-side wait ran out          */
+#define SPS_ETIMEOUT (-6) /* a bounded device-side wait ran out                    */
 
 #define SPS_MAX_K 15      /* K + 1 rows <= 16 per sequence                         */
 
@@ -108,8 +108,10 @@ typedef struct {
   int32_t overshoot;     /* tokens of the last loop dropped to return exactly n_new  */
   int32_t hist_emitted[SPS_MAX_K + 2]; /* hist_emitted[j] = loops that emitted j tokens */
   float ms_prefill;      /* device time of the prompt pass                           */
-  float ms_decode;       /* device time of all loops                                 */
-  float ms_draft, ms_verify, ms_accept; /* split of ms_decode by phase               */
+  float ms_decode;       /* device time from the first loop's start to the last loop's end,
+                            host turnaround between loops included                   */
+  float ms_draft, ms_verify, ms_accept; /* device time inside the three phases       */
+  int32_t kernel_launches; /* kernels the loops launched (graph nodes counted per replay) */
 } sps_stats;
 
 /* Build a handle for a (target, draft) pair.  Algorithm 2's preamble: "given
@@ -196,7 +198,8 @@ int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uin
  * 16-byte aligned W.  workspace: device scratch of sps_linear_workspace_bytes()
  * bytes for the same (dtype, M, N, D), zero-filled once before its first use
  * (the kernel leaves it ready for the next call).
- * out_ms: host, device time of the kernel, may be NULL. */
+ * out_ms: host, device time of the kernel, may be NULL; when given the call
+ * waits for the kernel and returns SPS_ETIMEOUT if a bounded wait inside it ran out. */
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
                void* workspace, void* stream, float* out_ms);
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D);

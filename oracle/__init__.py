@@ -31,7 +31,7 @@ FLAG_NEAR_CDF = 512
 def build(force: bool = False) -> str:
     """Compile the oracle with the host compiler (no CUDA involved)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        cmd = ["g++", "-O2", "-std=c++17", "-fopenmp", "-shared", "-fPIC", "-o", _LIB, _SRC]
+        cmd = ["g++", "-O2", "-std=c++17", "-pthread", "-shared", "-fPIC", "-o", _LIB, _SRC]
         subprocess.check_call(cmd)
     return _LIB
 

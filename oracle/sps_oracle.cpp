@@ -30,10 +30,32 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <thread>
 #include <vector>
-#ifdef _OPENMP
-#include <omp.h>
-#endif
+
+// Rows of a large mat-vec are split over plain std::threads (no OpenMP runtime: the host process
+// usually carries another one already).  Small problems run on the calling thread.
+static int hw_threads() {
+  static const int n = [] {
+    unsigned h = std::thread::hardware_concurrency();
+    int v = h ? (int)h : 1;
+    return v > 64 ? 64 : v;
+  }();
+  return n;
+}
+template <class F>
+static void parallel_rows(int N, long long work_per_row, F fn) {
+  const int T = hw_threads();
+  if (T <= 1 || (long long)N * work_per_row < (1ll << 22)) { fn(0, N); return; }
+  std::vector<std::thread> th;
+  const int per = (N + T - 1) / T;
+  for (int t = 0; t < T; ++t) {
+    const int a = t * per, b = std::min(N, a + per);
+    if (a >= b) break;
+    th.emplace_back([=] { fn(a, b); });
+  }
+  for (auto& x : th) x.join();
+}
 
 // ---------------------------------------------------------------------------
 // Random numbers.  Algorithm 2 draws r ~ U[0,1] and "samples" tokens without
@@ -342,13 +364,15 @@ struct Transformer : OrcModel {
 
   // y[n] = sum_k W[n][k] v[k],  W row-major [N][D]
   void matvec(const void* W, const double* v, int N, int D, double* y) const {
-#pragma omp parallel for schedule(static)
-    for (int n = 0; n < N; ++n) {
-      double acc = 0.0;
-      const size_t base = (size_t)n * D;
-      for (int k = 0; k < D; ++k) acc += load_w(W, base + k, dtype) * v[k];
-      y[n] = acc;
-    }
+    const int dt = dtype;
+    parallel_rows(N, D, [=](int n0, int n1) {
+      for (int n = n0; n < n1; ++n) {
+        double acc = 0.0;
+        const size_t base = (size_t)n * D;
+        for (int k = 0; k < D; ++k) acc += load_w(W, base + k, dt) * v[k];
+        y[n] = acc;
+      }
+    });
   }
   void rmsnorm(const double* v, const void* gain, double* out) const {
     double ss = 0.0;
@@ -688,19 +712,14 @@ extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t*
 
 // Y[m][n] = sum_k X[m][k] W[n][k]: the linear layer by its definition, in double.
 extern "C" void orc_linear(const void* W, int dtype, const float* X, int M, int N, int D, double* Y) {
-#pragma omp parallel for schedule(static)
-  for (int n = 0; n < N; ++n)
-    for (int m = 0; m < M; ++m) {
-      double acc = 0.0;
-      for (int k = 0; k < D; ++k) acc += load_w(W, (size_t)n * D + k, dtype) * (double)X[(size_t)m * D + k];
-      Y[(size_t)m * N + n] = acc;
-    }
+  parallel_rows(N, (long long)D * M, [=](int n0, int n1) {
+    for (int n = n0; n < n1; ++n)
+      for (int m = 0; m < M; ++m) {
+        double acc = 0.0;
+        for (int k = 0; k < D; ++k) acc += load_w(W, (size_t)n * D + k, dtype) * (double)X[(size_t)m * D + k];
+        Y[(size_t)m * N + n] = acc;
+      }
+  });
 }
 
-extern "C" int orc_num_threads() {
-#ifdef _OPENMP
-  return omp_get_max_threads();
-#else
-  return 1;
-#endif
-}
+extern "C" int orc_num_threads() { return hw_threads(); }

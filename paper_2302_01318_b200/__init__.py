@@ -46,7 +46,7 @@ class sps_stats(C.Structure):
     _fields_ = [("loops", C.c_int32), ("draft_calls", C.c_int32), ("emitted", C.c_int32), ("accepted", C.c_int32),
                 ("resampled", C.c_int32), ("bonus", C.c_int32), ("fallback", C.c_int32), ("overshoot", C.c_int32),
                 ("hist_emitted", C.c_int32 * (SPS_MAX_K + 2)), ("ms_prefill", C.c_float), ("ms_decode", C.c_float),
-                ("ms_draft", C.c_float), ("ms_verify", C.c_float), ("ms_accept", C.c_float)]
+                ("ms_draft", C.c_float), ("ms_verify", C.c_float), ("ms_accept", C.c_float), ("kernel_launches", C.c_int32)]
 
     def as_dict(self):
         d = {k: getattr(self, k) for k, _ in self._fields_ if k != "hist_emitted"}

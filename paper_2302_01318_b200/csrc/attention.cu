@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a) {
   __shared__ float s_part[8];
   const int row = blockIdx.x, tid = threadIdx.x;
   const int rps = a.rows_per_seq;
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = row / rps, i = row - b * rps;
   DevState* st = a.st;
   const int max_seq = st->max_seq;
@@ -62,32 +64,147 @@ __global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a) {
 }
 
 cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st) {
-  embed_kernel<<<a.B * a.rows_per_seq, 256, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_k(embed_kernel, dim3(a.B * a.rows_per_seq), dim3(256), 0, st, a);
 }
 
 // ------------------------------------------------------------------------------------------------
-// attention: one CTA per (head, sequence)
+// attention: one CTA per (head, sequence), flash-decoding style.
+//
+// The cached keys / values of a (sequence, head) are one contiguous span, so a tile of TP positions is
+// brought into shared memory by two bulk async copies (one for K, one for V) that are issued before the
+// kernel waits for its predecessor: old cache rows do not depend on it.  The rows of this pass (rotary
+// applied, rounded to the storage type, appended to the cache) are patched into the tile from shared
+// memory, so the tile never depends on reading back what this CTA just wrote.  Per tile: scores with
+// one thread per (position, row group), running max / sum per row (online softmax), then P.V with one
+// thread per (dim, position group).  Loops over rows are the only unrolled ones: the code stays small
+// enough for the instruction cache, which is what a kernel that runs for microseconds lives or dies by.
 // ------------------------------------------------------------------------------------------------
-#define ATTN_THREADS 256
-#define ATTN_WARPS 8
+#define ATTN_THREADS 512
+#define ATTN_WARPS 16
+#define ATTN_TILE_BYTES 32768
 
-template <int DH, typename CT>
+__device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool a_mbar_wait(uint32_t bar, uint32_t parity, int* err) {
+  unsigned long long t0 = 0;
+  for (int spin = 0;; ++spin) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((spin & 255) == 255) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > 2000000000ull) { atomicExch(err, 3); return false; }
+    }
+  }
+}
+
+template <typename CT> __device__ __forceinline__ float ct_to_f(CT v);
+template <> __device__ __forceinline__ float ct_to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float ct_to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename CT> __device__ __forceinline__ CT f_to_ct(float v);
+template <> __device__ __forceinline__ float f_to_ct<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 f_to_ct<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// position of row i of sequence b in this pass (the same rule as embed_kernel)
+__device__ __forceinline__ int row_position(const AttnArgs& a, int b, int i) {
+  const DevState* st = a.st;
+  const int n = st->n[b];
+  int pos;
+  switch (a.mode) {
+    case PASS_PREFILL: pos = a.c0 + i; break;
+    case PASS_DRAFT0: pos = (i == 0) ? max(n - 2, 0) : n - 1; break;
+    case PASS_DRAFT_T: pos = n - 1 + a.t; break;
+    case PASS_VERIFY: pos = n - 1 + i; break;
+    default: pos = st->row_pos[b * a.rows_per_seq + i]; break;
+  }
+  return max(0, min(pos, a.max_seq - 1));
+}
+
+template <int DH, typename CT, int MR>
 __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
-  extern __shared__ float sm[];
+  constexpr int TP = ATTN_TILE_BYTES / (DH * (int)sizeof(CT));   // positions per tile
+  constexpr int SG = ATTN_THREADS / TP;                          // row groups in the score phase (1, 2 or 4)
+  constexpr int RPG = (MR + SG - 1) / SG;                        // rows per score thread
+  constexpr int PG = ATTN_THREADS / DH;                          // position groups in the P.V phase (2 or 4)
+  constexpr int VEC = 16 / (int)sizeof(CT);                      // elements per 128-bit chunk
+  constexpr int NCH = DH / VEC;                                  // chunks per row
+  extern __shared__ __align__(128) unsigned char asm_[];
+  CT* Ks = reinterpret_cast<CT*>(asm_);                          // [TP][DH]
+  CT* Vs = Ks + TP * DH;                                         // [TP][DH]
+  CT* knew = Vs + TP * DH;                                       // [MR][DH]  this pass's keys (storage-rounded)
+  CT* vnew = knew + MR * DH;                                     // [MR][DH]
+  float* q_s = reinterpret_cast<float*>(vnew + MR * DH);         // [MR][DH]
+  float* sc = q_s + MR * DH;                                     // [MR][TP]
+  float* red = sc + MR * TP;                                     // [PG][MR][DH]
+  float* row_m = red + PG * MR * DH;                             // [MR] running max
+  float* row_l = row_m + MR;                                     // [MR] running sum
+  float* row_a = row_l + MR;                                     // [MR] rescale of this tile
+  int* pos_s = reinterpret_cast<int*>(row_a + MR);               // [MR]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(pos_s + MR);       // 8-byte aligned by construction
+
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Mb = a.rows_per_seq, row0 = b * Mb, d = a.d, max_seq = a.max_seq;
-  float* q_s = sm;                                  // [Mb][DH]
-  float* red = q_s + Mb * DH;                       // [ATTN_WARPS][Mb][DH]
-  float* inv_sum = red + ATTN_WARPS * Mb * DH;      // [16]
-  int* pos_s = reinterpret_cast<int*>(inv_sum + 16);  // [16]
-  float* sc = inv_sum + 32;                         // [Mb][max_seq]
   CT* kc = reinterpret_cast<CT*>(a.kcache) + ((size_t)b * a.H + h) * (size_t)max_seq * DH;
   CT* vc = reinterpret_cast<CT*>(a.vcache) + ((size_t)b * a.H + h) * (size_t)max_seq * DH;
   const float scale = rsqrtf((float)DH);
+  const uint32_t bar_addr = a_smem_u32(bar);
 
-  if (tid < Mb) pos_s[tid] = a.st->row_pos[row0 + tid];
+  if (tid < MR) {
+    pos_s[tid] = tid < Mb ? row_position(a, b, tid) : -1;
+    row_m[tid] = -INFINITY;
+    row_l[tid] = 0.f;
+  }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_addr) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   __syncthreads();
+  int n_ctx = 0, n_old = max_seq;
+  for (int i = 0; i < Mb; ++i) { n_ctx = max(n_ctx, pos_s[i] + 1); n_old = min(n_old, pos_s[i]); }
+  // Rows [0, n_old) were cached by earlier passes; rows >= n_old of a tile come from knew / vnew.
+  // Of the old rows, [0, n_safe) were written before the host last waited for the stream (the host
+  // waits once per loop and after the prompt pass), so they may be fetched before this kernel waits
+  // for its predecessor; rows written by earlier passes of the SAME loop may not: under programmatic
+  // launch only the immediate predecessor is known to be complete, and only after the wait.
+  int n_safe = 0;
+  if (a.mode == PASS_VERIFY) n_safe = max(a.st->n[b] - 1, 0);
+  else if (a.mode == PASS_DRAFT0 || a.mode == PASS_DRAFT_T) n_safe = max(a.st->n[b] - 2, 0);
+  n_safe = min(n_safe, n_old);
+  auto copy_rows = [&](int r0, int r1) {   // cache rows [r0, r1) of tile 0 .. into the tile buffers
+    const uint32_t bytes = (uint32_t)(r1 - r0) * DH * (uint32_t)sizeof(CT);
+    const int tr = r0 % TP;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(a_smem_u32(Ks + tr * DH)), "l"(kc + (size_t)r0 * DH), "r"(bytes), "r"(bar_addr) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(a_smem_u32(Vs + tr * DH)), "l"(vc + (size_t)r0 * DH), "r"(bytes), "r"(bar_addr) : "memory");
+    return 2 * bytes;
+  };
+  // the part of a tile that is fetched after the wait; it also arrives on the tile's barrier
+  auto issue_tile = [&](int t0, int from) {
+    const int r1 = min(t0 + TP, n_old);
+    if (r1 > from) {
+      const uint32_t bytes = 2u * (uint32_t)(r1 - from) * DH * (uint32_t)sizeof(CT);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
+      copy_rows(from, r1);
+    } else {
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+    }
+  };
+  const int pre = min(TP, n_safe);   // rows of tile 0 fetched right away
+  if (tid == 0 && pre > 0) {
+    const uint32_t bytes = 2u * (uint32_t)pre * DH * (uint32_t)sizeof(CT);
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
+    copy_rows(0, pre);
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (tid == 0) issue_tile(0, pre);
+
   // ---- rotary on q and k (adjacent pairs, angle = pos * base^(-2i/dh)); append k, v at the row's position
   for (int idx = tid; idx < Mb * (DH / 2); idx += ATTN_THREADS) {
     const int i = idx / (DH / 2), pr = idx - i * (DH / 2);
@@ -99,125 +216,163 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
     const float v0 = src[2 * d], v1 = src[2 * d + 1];
     q_s[i * DH + 2 * pr] = (q0 * cs.x - q1 * cs.y) * scale;
     q_s[i * DH + 2 * pr + 1] = (q0 * cs.y + q1 * cs.x) * scale;
-    CT* kd = kc + (size_t)pos * DH + 2 * pr;
-    CT* vd = vc + (size_t)pos * DH + 2 * pr;
-    CacheIO<CT>::st(kd, k0 * cs.x - k1 * cs.y);
-    CacheIO<CT>::st(kd + 1, k0 * cs.y + k1 * cs.x);
-    CacheIO<CT>::st(vd, v0);
-    CacheIO<CT>::st(vd + 1, v1);
+    const CT ka = f_to_ct<CT>(k0 * cs.x - k1 * cs.y), kb = f_to_ct<CT>(k0 * cs.y + k1 * cs.x);
+    const CT va = f_to_ct<CT>(v0), vb = f_to_ct<CT>(v1);
+    knew[i * DH + 2 * pr] = ka; knew[i * DH + 2 * pr + 1] = kb;
+    vnew[i * DH + 2 * pr] = va; vnew[i * DH + 2 * pr + 1] = vb;
+    kc[(size_t)pos * DH + 2 * pr] = ka; kc[(size_t)pos * DH + 2 * pr + 1] = kb;
+    vc[(size_t)pos * DH + 2 * pr] = va; vc[(size_t)pos * DH + 2 * pr + 1] = vb;
   }
-  __syncthreads();
-  int n_ctx = 0;
-  for (int i = 0; i < Mb; ++i) n_ctx = max(n_ctx, pos_s[i] + 1);
+  for (int idx = tid; idx < (MR - Mb) * DH; idx += ATTN_THREADS) q_s[Mb * DH + idx] = 0.f;
 
-  // ---- scores: one thread per cached position, all rows at once
-  for (int j = tid; j < n_ctx; j += ATTN_THREADS) {
-    float acc[SPS_MAX_ROWS];
+  float o[MR];   // P.V accumulators: this thread's dim, its position group
 #pragma unroll
-    for (int i = 0; i < SPS_MAX_ROWS; ++i) acc[i] = 0.f;
-    const CT* kr = kc + (size_t)j * DH;
+  for (int i = 0; i < MR; ++i) o[i] = 0.f;
+  const int dim = tid % DH, pg = tid / DH;
+  bool ok = true;
+  int phase = 0;
+  for (int t0 = 0; t0 < n_ctx; t0 += TP, phase ^= 1) {
+    const int tn = min(TP, n_ctx - t0);   // positions of this tile
+    if (!a_mbar_wait(bar_addr, (uint32_t)phase, a.st->err)) ok = false;
+    __syncthreads();   // also: phase A's shared writes are visible
+    // patch in the rows of this pass that fall into the tile
+    for (int idx = tid; idx < Mb * DH; idx += ATTN_THREADS) {
+      const int i = idx / DH, e = idx - i * DH;
+      const int j = pos_s[i] - t0;
+      if (j >= 0 && j < TP) { Ks[j * DH + e] = knew[idx]; Vs[j * DH + e] = vnew[idx]; }
+    }
+    __syncthreads();
+    // ---- scores: thread = (position j, row group sg); chunks are visited in a per-position rotated
+    // order so that neighbouring positions hit different banks
+    {
+      const int j = tid % TP, sg = tid / TP;
+      if (j < tn) {
+        float acc[RPG];
+#pragma unroll
+        for (int r = 0; r < RPG; ++r) acc[r] = 0.f;
+        const CT* kr = Ks + j * DH;
 #pragma unroll 2
-    for (int c = 0; c < DH; c += 8) {
-      float kv[8];
-      if (sizeof(CT) == 2) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(kr + c);
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        for (int c = 0; c < NCH; ++c) {
+          const int cc = (c + j) % NCH;
+          const uint4 raw = *reinterpret_cast<const uint4*>(kr + cc * VEC);
+          float kv[VEC];
+          if (sizeof(CT) == 2) {
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          kv[2 * e] = __uint_as_float(w[e] << 16);
-          kv[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            for (int e = 0; e < 4; ++e) {
+              kv[2 * e] = __uint_as_float(w[e] << 16);
+              kv[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+          } else {
+            kv[0] = __uint_as_float(raw.x); kv[1] = __uint_as_float(raw.y);
+            kv[2] = __uint_as_float(raw.z); kv[3] = __uint_as_float(raw.w);
+          }
+#pragma unroll
+          for (int r = 0; r < RPG; ++r) {
+            const int i = sg * RPG + r;
+            if (i < MR) {
+              const float* qp = q_s + i * DH + cc * VEC;
+              const float4 qa = *reinterpret_cast<const float4*>(qp);
+              float t = kv[0] * qa.x + kv[1] * qa.y + kv[2] * qa.z + kv[3] * qa.w;
+              if (VEC == 8) {
+                const float4 qb = *reinterpret_cast<const float4*>(qp + 4);
+                t += kv[VEC - 4] * qb.x + kv[VEC - 3] * qb.y + kv[VEC - 2] * qb.z + kv[VEC - 1] * qb.w;
+              }
+              acc[r] += t;
+            }
+          }
         }
-      } else {
-        const float4 r0 = *reinterpret_cast<const float4*>(kr + c);
-        const float4 r1 = *reinterpret_cast<const float4*>(kr + c + 4);
-        kv[0] = r0.x; kv[1] = r0.y; kv[2] = r0.z; kv[3] = r0.w;
-        kv[4] = r1.x; kv[5] = r1.y; kv[6] = r1.z; kv[7] = r1.w;
-      }
 #pragma unroll
-      for (int i = 0; i < SPS_MAX_ROWS; ++i) {
-        if (i < Mb) {
-          const float4 qa = *reinterpret_cast<const float4*>(q_s + i * DH + c);
-          const float4 qb = *reinterpret_cast<const float4*>(q_s + i * DH + c + 4);
-          acc[i] += kv[0] * qa.x + kv[1] * qa.y + kv[2] * qa.z + kv[3] * qa.w + kv[4] * qb.x + kv[5] * qb.y +
-                    kv[6] * qb.z + kv[7] * qb.w;
+        for (int r = 0; r < RPG; ++r) {
+          const int i = sg * RPG + r;
+          if (i < Mb) sc[i * TP + j] = (t0 + j <= pos_s[i]) ? acc[r] : -INFINITY;
         }
       }
     }
-#pragma unroll
-    for (int i = 0; i < SPS_MAX_ROWS; ++i)
-      if (i < Mb) sc[(size_t)i * max_seq + j] = (j <= pos_s[i]) ? acc[i] : -INFINITY;
-  }
-  __syncthreads();
-  // ---- softmax over positions, one warp per row
-  for (int i = warp; i < Mb; i += ATTN_WARPS) {
-    float* s = sc + (size_t)i * max_seq;
-    float m = -INFINITY;
-    for (int j = lane; j < n_ctx; j += 32) m = fmaxf(m, s[j]);
-    m = warp_max(m);
-    float sum = 0.f;
-    for (int j = lane; j < n_ctx; j += 32) { const float e = expf(s[j] - m); s[j] = e; sum += e; }
-    sum = warp_sum(sum);
-    if (lane == 0) inv_sum[i] = 1.0f / sum;
-  }
-  __syncthreads();
-  // ---- o = sum_j p_j v_j: a lane owns DH/32 dims, warps split the positions
-  constexpr int DPT = DH / 32;
-  float o[SPS_MAX_ROWS][DPT];
-#pragma unroll
-  for (int i = 0; i < SPS_MAX_ROWS; ++i)
-#pragma unroll
-    for (int e = 0; e < DPT; ++e) o[i][e] = 0.f;
-  for (int j = warp; j < n_ctx; j += ATTN_WARPS) {
-    float vv[DPT];
-    const CT* vr = vc + (size_t)j * DH + lane * DPT;
-#pragma unroll
-    for (int e = 0; e < DPT; ++e) vv[e] = CacheIO<CT>::ld(vr + e);
-#pragma unroll
-    for (int i = 0; i < SPS_MAX_ROWS; ++i) {
-      if (i < Mb) {
-        const float p = sc[(size_t)i * max_seq + j];
-#pragma unroll
-        for (int e = 0; e < DPT; ++e) o[i][e] += p * vv[e];
+    __syncthreads();
+    // ---- online softmax: warp per row
+    for (int i = warp; i < Mb; i += ATTN_WARPS) {
+      float* srow = sc + i * TP;
+      float m = -INFINITY;
+      for (int j = lane; j < tn; j += 32) m = fmaxf(m, srow[j]);
+      m = warp_max(m);
+      const float m_old = row_m[i];
+      const float m_new = fmaxf(m_old, m);
+      float sum = 0.f;
+      for (int j = lane; j < tn; j += 32) {
+        const float e = (m_new == -INFINITY) ? 0.f : expf(srow[j] - m_new);
+        srow[j] = e;
+        sum += e;
+      }
+      sum = warp_sum(sum);
+      if (lane == 0) {
+        const float alpha = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
+        row_a[i] = alpha;
+        row_l[i] = row_l[i] * alpha + sum;
+        row_m[i] = m_new;
       }
     }
+    __syncthreads();
+    // ---- o = alpha * o + sum_j p_j v_j: thread = (dim, position group)
+#pragma unroll
+    for (int i = 0; i < MR; ++i) if (i < Mb) o[i] *= row_a[i];
+#pragma unroll 2
+    for (int j = pg; j < tn; j += PG) {
+      const float v = ct_to_f<CT>(Vs[j * DH + dim]);
+#pragma unroll
+      for (int i = 0; i < MR; ++i) if (i < Mb) o[i] += sc[i * TP + j] * v;
+    }
+    __syncthreads();   // the tile buffers and sc are free again
+    if (tid == 0 && t0 + TP < n_ctx) issue_tile(t0 + TP, t0 + TP);
   }
 #pragma unroll
-  for (int i = 0; i < SPS_MAX_ROWS; ++i)
-    if (i < Mb)
-#pragma unroll
-      for (int e = 0; e < DPT; ++e) red[((size_t)warp * Mb + i) * DH + lane * DPT + e] = o[i][e];
+  for (int i = 0; i < MR; ++i) if (i < Mb) red[(pg * MR + i) * DH + dim] = o[i];
   __syncthreads();
   for (int idx = tid; idx < Mb * DH; idx += ATTN_THREADS) {
-    const int i = idx / DH, dim = idx - i * DH;
+    const int i = idx / DH, e = idx - i * DH;
     float t = 0.f;
 #pragma unroll
-    for (int w = 0; w < ATTN_WARPS; ++w) t += red[((size_t)w * Mb + i) * DH + dim];
-    a.out[(size_t)(row0 + i) * d + h * DH + dim] = t * inv_sum[i];
+    for (int g = 0; g < PG; ++g) t += red[(g * MR + i) * DH + e];
+    a.out[(size_t)(row0 + i) * d + h * DH + e] = ok ? t / row_l[i] : 0.f;
   }
+}
+
+template <int DH, typename CT, int MR>
+static size_t attn_smem_t() {
+  constexpr int TP = ATTN_TILE_BYTES / (DH * (int)sizeof(CT));
+  constexpr int PG = ATTN_THREADS / DH;
+  return 2 * (size_t)ATTN_TILE_BYTES + 2 * (size_t)MR * DH * sizeof(CT) + sizeof(float) * ((size_t)MR * DH + (size_t)MR * TP + (size_t)PG * MR * DH + 3 * MR) +
+         sizeof(int) * MR + 16;
 }
 
 size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh) {
-  return sizeof(float) * ((size_t)rows_per_seq * dh + (size_t)ATTN_WARPS * rows_per_seq * dh + 32 +
-                          (size_t)rows_per_seq * max_seq);
+  (void)rows_per_seq; (void)max_seq; (void)dh;
+  return attn_smem_t<128, float, 16>();   // the largest instantiation
 }
 
-template <int DH, typename CT>
-static cudaError_t attn_go(const AttnArgs& a, cudaStream_t st, size_t& cached) {
-  const size_t smem = attn_smem_bytes(a.rows_per_seq, a.max_seq, DH);
+template <int DH, typename CT, int MR>
+static cudaError_t attn_go(const AttnArgs& a, cudaStream_t st) {
+  static size_t cached = 48 * 1024;
+  const size_t smem = attn_smem_t<DH, CT, MR>();
   if (smem > cached) {
-    cudaError_t e = cudaFuncSetAttribute(attn_kernel<DH, CT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_kernel<DH, CT, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     cached = smem;
   }
-  attn_kernel<DH, CT><<<dim3(a.H, a.B), ATTN_THREADS, smem, st>>>(a);
-  return cudaGetLastError();
+  return launch_k(attn_kernel<DH, CT, MR>, dim3(a.H, a.B), dim3(ATTN_THREADS), smem, st, a);
+}
+
+template <int DH, typename CT>
+static cudaError_t attn_rows(const AttnArgs& a, cudaStream_t st) {
+  if (a.rows_per_seq <= 2) return attn_go<DH, CT, 2>(a, st);
+  if (a.rows_per_seq <= 8) return attn_go<DH, CT, 8>(a, st);
+  return attn_go<DH, CT, 16>(a, st);
 }
 
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st) {
-  static size_t c0 = 48 * 1024, c1 = 48 * 1024, c2 = 48 * 1024, c3 = 48 * 1024;
-  if (a.dh == 64 && a.dtype == 0) return attn_go<64, float>(a, st, c0);
-  if (a.dh == 128 && a.dtype == 0) return attn_go<128, float>(a, st, c1);
-  if (a.dh == 64 && a.dtype == 1) return attn_go<64, __nv_bfloat16>(a, st, c2);
-  if (a.dh == 128 && a.dtype == 1) return attn_go<128, __nv_bfloat16>(a, st, c3);
+  if (a.dh == 64 && a.dtype == 0) return attn_rows<64, float>(a, st);
+  if (a.dh == 128 && a.dtype == 0) return attn_rows<128, float>(a, st);
+  if (a.dh == 64 && a.dtype == 1) return attn_rows<64, __nv_bfloat16>(a, st);
+  if (a.dh == 128 && a.dtype == 1) return attn_rows<128, __nv_bfloat16>(a, st);
   return cudaErrorInvalidValue;
 }

@@ -43,6 +43,27 @@ __device__ inline Uniforms sps_uniforms(uint64_t seed, uint32_t b, uint32_t s, u
 }
 
 // ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch: every kernel lets its successor start early (its CTAs may become
+// resident and prefetch constant data) and waits for its predecessor before touching anything the
+// predecessor wrote.  Without the launch attribute both instructions are no-ops.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+bool sps_pdl_enabled();
+template <class... KArgs, class... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = sps_pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Reductions with a fixed tree (results are bit-reproducible run to run).
 // ------------------------------------------------------------------------------------------------
 __device__ inline float warp_sum(float v) {
@@ -122,25 +143,29 @@ struct LinArgs {
   int ldx, x_row0, x_rowstep;
   int pro;                // PRO_*
   const float* gain;      // [D] fp32 (PRO_RMSNORM)
-  const float* ssq_in;    // [rows] sum of squares of each X row (PRO_RMSNORM)
+  const float* ssq_in;    // [ssq_in_n][16] partial sums of squares of each X row (PRO_RMSNORM)
+  int ssq_in_n;
   float eps;
   int epi;                // EPI_*
   float* Y;               // EPI_STORE: Y[m*ldy + n] = y.  EPI_RESIDUAL: Y[m*ldy + n] += y
   long long ldy;
-  float* ssq_out;         // EPI_RESIDUAL: [M] sum over n of the updated Y[m][n]^2
+  float* ssq_out;         // EPI_RESIDUAL: [R][16] per-range sums over n of the updated Y[m][n]^2
   // scratch (owned by the handle / caller): split-K partials and arrival counters
   float* part;            // [S][SPS_MAX_ROWS][N]
-  float* ssq_part;        // [R][SPS_MAX_ROWS]
-  int* counters;          // [R + 1], zero between launches (the kernel re-zeroes them)
+  int* counters;          // [R], zero between launches (the kernel re-zeroes them)
   int R, S, WC;           // row ranges, K splits, warps per CTA
-  int PR;                 // rows per shared-memory pass (multiple of 32)
+  int PR;                 // rows per shared-memory pass (multiple of 32)      [register-streaming variant]
+  int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
+  int* err;               // sticky error word: set to 3 if a bounded wait ran out
+  int dbg;                // experiments only: bit 0 = consumers skip the arithmetic
 };
 
-struct LinPlan { int R, S, WC, PR, NT; size_t smem; };
+struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G; size_t smem; };
 LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
 size_t lin_part_floats(int N, int S_max);
 #define LIN_MAX_R 512
+#define LIN_CONSUMER_WARPS 8
 #define LIN_MAX_S 64
 
 // ------------------------------------------------------------------------------------------------
@@ -152,7 +177,7 @@ struct EmbedArgs {
   int dtype, d, V;
   int mode, t, K, c0, rows_per_seq, B;
   float* x;               // [rows][d] fp32 residual stream
-  float* ssq;             // [rows]
+  float* ssq;             // [1][16]: one partial per row
 };
 cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st);
 
@@ -164,6 +189,7 @@ struct AttnArgs {
   void* vcache;
   const float2* rope;     // [max_seq][dh/2] (cos, sin)
   int dtype, H, dh, d, max_seq, rows_per_seq, B;
+  int mode, t, c0;        // which rows the pass feeds (PassMode), as in EmbedArgs
 };
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
 size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh);
@@ -177,6 +203,7 @@ struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(log
   int32_t* out;            // out[b*out_ld]
   int out_ld;
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+  int smem_weights;        // set by the launcher: weights are staged in shared memory
 };
 cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st);
 
@@ -192,6 +219,7 @@ struct AcceptArgs {
   int out_ld;
   uint32_t* flags;         // [B]
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+  int smem_weights;        // set by the launcher: weights are staged in shared memory
 };
 cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);
 cudaError_t philox_launch(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out, cudaStream_t st);

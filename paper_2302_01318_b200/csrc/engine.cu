@@ -2,6 +2,7 @@
 // Host code only enqueues kernels (or replays graphs of them) and reads back a few integers per loop;
 // every step of the path runs in the kernels of linear.cu, attention.cu and sampler.cu.
 #include <cmath>
+#include <cstdlib>
 #include <cstdio>
 #include <cstring>
 #include <map>
@@ -39,7 +40,7 @@ struct sps_handle {
   DevState hst{};          // host image of the device state block
   DevState* dst = nullptr;
   float *x = nullptr, *qkv = nullptr, *attn = nullptr, *up = nullptr, *ssqA = nullptr, *ssqB = nullptr;
-  float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr, *ssq_part = nullptr;
+  float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
   int32_t* res = nullptr;    // device: [n_acc B][flags B][out_tok B*(maxK+1)][err 1]
   int32_t* h_res = nullptr;  // pinned mirror
@@ -51,7 +52,9 @@ struct sps_handle {
   bool ready = false;
   std::map<int, cudaGraphExec_t> g_draft, g_verify;  // key = K * 32 + B
   std::map<int, int> warm;                          // key -> eager runs done
-  cudaEvent_t ev[5]{};
+  cudaEvent_t ev[7]{};
+  long long launches = 0;                 // kernels enqueued (graph nodes counted per replay)
+  std::map<const void*, long long> graph_launches;
   std::string err;
   int last_K = -1;
 };
@@ -155,18 +158,20 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = c.dtype; ea.d = d; ea.V = c.vocab;
   ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
   ea.x = h->x; ea.ssq = h->ssqA;
-  CU(h, embed_launch(ea, st));
+  CU(h, embed_launch(ea, st)); h->launches++;
   LinArgs base{};
-  base.part = h->part; base.ssq_part = h->ssq_part; base.counters = h->counters; base.eps = c.rms_eps;
+  base.part = h->part; base.counters = h->counters; base.eps = c.rms_eps;
+  int nA = 1, nB = 1;   // how many partial sums of squares sit in ssqA / ssqB
+  base.err = h->hst.err;
   for (int l = 0; l < c.n_layers; ++l) {
     {  // q, k, v = Wq h, Wk h, Wv h with h = rmsnorm(x, g_attn), one launch over the three matrices
       LinArgs a = base;
       a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
       a.rows_per_mat = d; a.N = 3 * d; a.D = d; a.M = rows;
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
-      a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA;
+      a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
       a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = 3 * d;
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
     }
     {
       AttnArgs aa{};
@@ -174,38 +179,44 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
       aa.rope = m.rope; aa.dtype = c.dtype; aa.H = c.n_heads; aa.dh = c.d_head; aa.d = d;
       aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
-      CU(h, attn_launch(aa, st));
+      aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
+      static const int dbg_skip = [] { const char* e = getenv("SPS_DBG_SKIP"); return e ? atoi(e) : 0; }();
+      if (!(dbg_skip & 1)) { CU(h, attn_launch(aa, st)); h->launches++; }
     }
     {  // x += Wo o ; also sum(x^2) for the FFN norm
       LinArgs a = base;
       a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = d; a.M = rows;
       a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+      nB = pl.R;
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
     }
     {  // up = Wup rmsnorm(x, g_ffn)
       LinArgs a = base;
       a.W[0] = m.w_up[l]; a.rows_per_mat = dff; a.N = dff; a.D = d; a.M = rows;
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
-      a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB;
+      a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB; a.ssq_in_n = nB;
       a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
     }
     {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
       LinArgs a = base;
       a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
       a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st));
+      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+      nA = pl.R;
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
     }
   }
   if (ps.logits) {
     LinArgs a = base;
     a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
     a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
-    a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA;
+    a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
     a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
-    CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm), st));
+    CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm), st)); h->launches++;
   }
   return SPS_OK;
 }
@@ -224,7 +235,7 @@ int enqueue_draft(sps_handle* h, int K) {
     SampleArgs sa{};
     sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = V; sa.B = B; sa.t = (uint32_t)t;
     sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
-    CU(h, sample_launch(sa, h->stream));
+    CU(h, sample_launch(sa, h->stream)); h->launches++;
   }
   return SPS_OK;
 }
@@ -241,7 +252,7 @@ int enqueue_accept(sps_handle* h, int K) {
   aa.st = h->dst; aa.q_logits = h->q_logits; aa.p_logits = h->p_logits; aa.drafts = h->hst.drafts;
   aa.drafts_ld = h->hst.max_K; aa.B = h->B; aa.K = K; aa.V = h->tgt.cfg.vocab;
   aa.n_acc = h->hst.n_acc; aa.out_tok = h->hst.out_tok; aa.out_ld = h->hst.max_K + 1; aa.flags = h->hst.flags;
-  CU(h, accept_launch(aa, h->stream));
+  CU(h, accept_launch(aa, h->stream)); h->launches++;
   return SPS_OK;
 }
 
@@ -250,12 +261,18 @@ int launch_phase(sps_handle* h, std::map<int, cudaGraphExec_t>& cache, int K, in
   if (h->cfg.flags & SPS_CFG_NO_GRAPH) return enq(h, K);
   const int key = K * 32 + h->B;
   auto it = cache.find(key);
-  if (it != cache.end()) { CU(h, cudaGraphLaunch(it->second, h->stream)); return SPS_OK; }
+  if (it != cache.end()) {
+    CU(h, cudaGraphLaunch(it->second, h->stream));
+    h->launches += h->graph_launches[(const void*)it->second];
+    return SPS_OK;
+  }
   int& w = h->warm[key * 2 + tag];
   if (w == 0) { ++w; return enq(h, K); }   // first use runs eagerly (it also sets kernel attributes)
   cudaGraph_t g = nullptr;
   CU(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+  const long long before = h->launches;
   int rc = enq(h, K);
+  const long long in_graph = h->launches - before;
   cudaError_t e = cudaStreamEndCapture(h->stream, &g);
   if (rc) { if (g) cudaGraphDestroy(g); return rc; }
   if (e != cudaSuccess) return fail(h, SPS_ECUDA, std::string("graph capture: ") + cudaGetErrorString(e));
@@ -264,6 +281,7 @@ int launch_phase(sps_handle* h, std::map<int, cudaGraphExec_t>& cache, int K, in
   cudaGraphDestroy(g);
   if (e != cudaSuccess) return fail(h, SPS_ECUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
   cache[key] = ge;
+  h->graph_launches[(const void*)ge] = in_graph;
   CU(h, cudaGraphLaunch(ge, h->stream));
   return SPS_OK;
 }
@@ -288,6 +306,7 @@ int loop_once(sps_handle* h, int K, bool timed) {
   CU(h, cudaMemcpyAsync(h->h_res, h->res, h->res_words * 4, cudaMemcpyDeviceToHost, h->stream));
   CU(h, cudaStreamSynchronize(h->stream));
   h->last_K = K;
+  if (h->h_res[h->res_words - 1] == 3) return fail(h, SPS_ETIMEOUT, "a bounded device-side wait ran out");
   if (h->h_res[h->res_words - 1] != 0) return fail(h, SPS_ERANGE, "device flagged a token id or position out of range");
   return SPS_OK;
 }
@@ -404,13 +423,12 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->qkv, sizeof(float) * SPS_MAX_ROWS * 3 * (size_t)dmax},
       {(void**)&h->attn, sizeof(float) * SPS_MAX_ROWS * (size_t)dmax},
       {(void**)&h->up, sizeof(float) * SPS_MAX_ROWS * (size_t)fmax},
-      {(void**)&h->ssqA, sizeof(float) * SPS_MAX_ROWS},
-      {(void**)&h->ssqB, sizeof(float) * SPS_MAX_ROWS},
+      {(void**)&h->ssqA, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
+      {(void**)&h->ssqB, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
       {(void**)&h->q_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
       {(void**)&h->p_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
       {(void**)&h->part, sizeof(float) * part_floats},
-      {(void**)&h->ssq_part, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
-      {(void**)&h->counters, sizeof(int) * (LIN_MAX_R + 1)},
+      {(void**)&h->counters, sizeof(int) * (LIN_MAX_R + 2)},
       {(void**)&h->res, 4 * h->res_words},
       {(void**)&h->dst, sizeof(DevState)},
       {(void**)&s.n, 4 * (size_t)MB},
@@ -449,7 +467,7 @@ int sps_destroy(sps_handle* h) {
   for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
   free_model(h->tgt);
   free_model(h->drf);
-  void* bufs[] = {h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part, h->ssq_part,
+  void* bufs[] = {h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
                   h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);
@@ -542,20 +560,25 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
   cudaEvent_t e_pre0 = h->ev[4];
   CU(h, cudaEventRecord(e_pre0, h->stream));
   if ((rc = prefill_all(h, P))) return rc;
+  // the attention kernel may fetch cache rows of earlier loops before it waits for its predecessor;
+  // that is only sound if the host has waited for the stream since those rows were written
+  CU(h, cudaStreamSynchronize(h->stream));
   if ((rc = write_params(h, T, seed, 0u))) return rc;
   std::vector<sps_stats> st(B);
   for (auto& s : st) std::memset(&s, 0, sizeof(s));
   std::vector<int> made(B, 0);
   const int MB = h->cfg.max_batch, ld = h->hst.max_K + 1;
-  float ms_draft = 0.f, ms_verify = 0.f, ms_accept = 0.f, ms_prefill = 0.f;
+  float ms_draft = 0.f, ms_verify = 0.f, ms_accept = 0.f, ms_prefill = 0.f, ms_decode = 0.f;
   bool first = true;
+  const long long launches0 = h->launches;
+  CU(h, cudaEventRecord(h->ev[5], h->stream));
   for (;;) {
     bool all = true;
     for (int b = 0; b < B; ++b) all = all && made[b] >= n_new;
     if (all) break;
     if ((rc = loop_once(h, K, true))) return rc;
     float a01 = 0, a12 = 0, a23 = 0;
-    if (first) { cudaEventElapsedTime(&ms_prefill, e_pre0, h->ev[0]); first = false; }
+    if (first) { cudaEventElapsedTime(&ms_prefill, e_pre0, h->ev[5]); first = false; }
     cudaEventElapsedTime(&a01, h->ev[0], h->ev[1]);
     cudaEventElapsedTime(&a12, h->ev[1], h->ev[2]);
     cudaEventElapsedTime(&a23, h->ev[2], h->ev[3]);
@@ -573,10 +596,14 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
       h->seq_len[b] += a + 1;
     }
   }
+  CU(h, cudaEventRecord(h->ev[6], h->stream));
+  CU(h, cudaEventSynchronize(h->ev[6]));
+  CU(h, cudaEventElapsedTime(&ms_decode, h->ev[5], h->ev[6]));
   if (out_stats)
     for (int b = 0; b < B; ++b) {
       st[b].ms_prefill = ms_prefill; st[b].ms_draft = ms_draft; st[b].ms_verify = ms_verify; st[b].ms_accept = ms_accept;
-      st[b].ms_decode = ms_draft + ms_verify + ms_accept;
+      st[b].ms_decode = ms_decode;
+      st[b].kernel_launches = (int32_t)(h->launches - launches0);
       out_stats[b] = st[b];
     }
   return SPS_OK;
@@ -665,7 +692,7 @@ static int cur_num_sm() {
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
-  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (LIN_MAX_R + 1) + 256);
+  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (LIN_MAX_R + 2) + 256);
 }
 
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace,
@@ -681,8 +708,7 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
   a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
   char* ws = (char*)workspace;
   a.counters = (int*)ws;
-  size_t off = ((sizeof(int) * (LIN_MAX_R + 1) + 255) / 256) * 256;
-  a.ssq_part = (float*)(ws + off);
+  size_t off = ((sizeof(int) * (LIN_MAX_R + 2) + 255) / 256) * 256;
   off += sizeof(float) * (size_t)LIN_MAX_R * SPS_MAX_ROWS;
   a.part = (float*)(ws + off);
   cudaStream_t st = (cudaStream_t)stream;
@@ -694,6 +720,9 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
     cudaEventSynchronize(e1);
     cudaEventElapsedTime(out_ms, e0, e1);
     cudaEventDestroy(e0); cudaEventDestroy(e1);
+    int errw = 0;
+    if (e == cudaSuccess && cudaMemcpy(&errw, a.counters + LIN_MAX_R + 1, 4, cudaMemcpyDeviceToHost) == cudaSuccess && errw == 3)
+      return fail(nullptr, SPS_ETIMEOUT, "a bounded device-side wait ran out in the linear kernel");
   }
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("linear launch: ") + cudaGetErrorString(e));
   return SPS_OK;

@@ -84,6 +84,15 @@ __device__ int block_invcdf(F w, int V, float u, ScanSmem& sm, float* total_out)
   return tok;
 }
 
+// Same draw when the weights already sit in shared memory (written once with coalesced global loads).
+// Element i lives at ws[i + (i >> 5)]: the one-word skew per 32 elements makes the chunk-order reads
+// (thread t walks i = t*c .. t*c + c - 1) conflict-free.
+__device__ __forceinline__ int skew(int i) { return i + (i >> 5); }
+__device__ int block_invcdf_smem(const float* ws, int V, float u, ScanSmem& sm, float* total_out) {
+  auto w = [&](int i) { return ws[skew(i)]; };
+  return block_invcdf(w, V, u, sm, total_out);
+}
+
 __device__ inline float block_max_f(float v, float* s_part, float* s_out) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   v = warp_max(v);
@@ -122,6 +131,8 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   __shared__ float s_part[SAMPLER_WARPS];
   __shared__ float s_val;
   const int b = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   float T = a.temperature;
   uint64_t seed = a.seed;
   uint32_t step = a.step;
@@ -132,14 +143,40 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
   m = block_max_f(m, s_part, &s_val);
   const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, a.t);
-  auto w = [&](int i) { return expf((row[i] - m) * invT); };
-  const int tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+  int tok;
+  if (a.smem_weights) {
+    extern __shared__ float ws[];
+    for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = expf((row[i] - m) * invT);
+    __syncthreads();
+    tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
+  } else {
+    auto w = [&](int i) { return expf((row[i] - m) * invT); };
+    tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+  }
   if (threadIdx.x == 0) a.out[(long long)b * a.out_ld] = tok;
 }
 
-cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st) {
-  sample_kernel<<<a.B, SAMPLER_THREADS, 0, st>>>(a);
-  return cudaGetLastError();
+// bytes of the shared weight buffer for a vocabulary, or 0 when it does not fit (weights are then recomputed)
+static size_t weights_smem(int V) {
+  const size_t bytes = sizeof(float) * ((size_t)V + (size_t)V / 32 + 32);
+  return bytes <= 200 * 1024 ? bytes : 0;
+}
+template <class Kern>
+static cudaError_t sampler_smem_attr(Kern k, size_t bytes, size_t& cached) {
+  if (bytes <= cached) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) cached = bytes;
+  return e;
+}
+
+cudaError_t sample_launch(const SampleArgs& a_in, cudaStream_t st) {
+  static size_t cached = 48 * 1024;
+  SampleArgs a = a_in;
+  const size_t smem = weights_smem(a.V);
+  a.smem_weights = smem ? 1 : 0;
+  cudaError_t e = sampler_smem_attr(sample_kernel, smem, cached);
+  if (e != cudaSuccess) return e;
+  return launch_k(sample_kernel, dim3(a.B), dim3(SAMPLER_THREADS), smem, st, a);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -154,9 +191,12 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   __shared__ ScanSmem sm;
   __shared__ float s_red[SAMPLER_WARPS][ACC_MAX_ROWS + 1];
   __shared__ float s_max[ACC_MAX_ROWS], s_sum[ACC_MAX_ROWS];
-  __shared__ int s_stop, s_mode;
+  __shared__ int s_stop;
+  extern __shared__ float ws[];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, V = a.V, R = 2 * K + 1;
+  pdl_launch_dependents();
+  pdl_wait();
   float T = a.temperature;
   uint64_t seed = a.seed;
   uint32_t step = a.step;
@@ -228,11 +268,17 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     auto wres = [&](int i) {
       return fmaxf(0.f, expf((ql[i] - mq) * invT) * iq - expf((pl[i] - mp) * invT) * ip);
     };
+    auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
     float total;
-    tok = block_invcdf(wres, V, u.u_res, sm, &total);
+    if (a.smem_weights) {
+      for (int i = tid; i < V; i += SAMPLER_THREADS) ws[skew(i)] = wres(i);
+      __syncthreads();
+      tok = block_invcdf_smem(ws, V, u.u_res, sm, &total);
+    } else {
+      tok = block_invcdf(wres, V, u.u_res, sm, &total);
+    }
     fl |= 1u;
     if (!(total > 0.f)) {
-      auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
       tok = block_invcdf(wq, V, u.u_res, sm, nullptr);
       fl |= 4u;
     }
@@ -242,10 +288,15 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     const float mq = s_max[K];
     const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)K);
     auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
-    tok = block_invcdf(wq, V, u.u_res, sm, nullptr);
+    if (a.smem_weights) {
+      for (int i = tid; i < V; i += SAMPLER_THREADS) ws[skew(i)] = wq(i);
+      __syncthreads();
+      tok = block_invcdf_smem(ws, V, u.u_res, sm, nullptr);
+    } else {
+      tok = block_invcdf(wq, V, u.u_res, sm, nullptr);
+    }
     fl |= 2u;
   }
-  (void)s_mode;
   // ---- results
   int32_t* out = a.out_tok + (long long)b * a.out_ld;
   if (tid <= K) out[tid] = (tid < stop) ? drafts[tid] : (tid == stop ? tok : -1);
@@ -275,9 +326,14 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   }
 }
 
-cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st) {
-  accept_kernel<<<a.B, SAMPLER_THREADS, 0, st>>>(a);
-  return cudaGetLastError();
+cudaError_t accept_launch(const AcceptArgs& a_in, cudaStream_t st) {
+  static size_t cached = 48 * 1024;
+  AcceptArgs a = a_in;
+  const size_t smem = weights_smem(a.V);
+  a.smem_weights = smem ? 1 : 0;
+  cudaError_t e = sampler_smem_attr(accept_kernel, smem, cached);
+  if (e != cudaSuccess) return e;
+  return launch_k(accept_kernel, dim3(a.B), dim3(SAMPLER_THREADS), smem, st, a);
 }
 
 __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out) {

@@ -28,7 +28,7 @@ def test_struct_sizes_match_header():
     assert ctypes.sizeof(sps.sps_model_cfg) == 36
     assert ctypes.sizeof(sps.sps_cfg) == 36 * 2 + 16 + 8 + 8
     assert ctypes.sizeof(sps.sps_weights) == 11 * 8
-    assert ctypes.sizeof(sps.sps_stats) == 4 * (8 + 17 + 5)
+    assert ctypes.sizeof(sps.sps_stats) == 4 * (8 + 17 + 5 + 1)
 
 
 def test_argument_errors_need_no_gpu():
