@@ -152,15 +152,16 @@ struct LinArgs {
   float* ssq_out;         // EPI_RESIDUAL: [R][16] per-range sums over n of the updated Y[m][n]^2
   // scratch (owned by the handle / caller): split-K partials and arrival counters
   float* part;            // [S][SPS_MAX_ROWS][N]
-  int* counters;          // [R], zero between launches (the kernel re-zeroes them)
+  int* counters;          // [2 * LIN_MAX_R + 2], zero between launches (the kernel re-zeroes what it used)
   int R, S, WC;           // row ranges, K splits, warps per CTA
   int PR;                 // rows per shared-memory pass (multiple of 32)      [register-streaming variant]
   int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
   int* err;               // sticky error word: set to 3 if a bounded wait ran out
   int dbg;                // experiments only: bit 0 = consumers skip the arithmetic
+  unsigned long long* dbg_t;  // experiments only: per-CTA timestamps [R*S][8]
 };
 
-struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G; size_t smem; };
+struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };
 LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
 size_t lin_part_floats(int N, int S_max);

@@ -189,7 +189,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      nB = pl.R;
+      nB = pl.ssq_parts;
       CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
     }
     {  // up = Wup rmsnorm(x, g_ffn)
@@ -206,7 +206,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      nA = pl.R;
+      nA = pl.ssq_parts;
       CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
     }
   }
@@ -428,7 +428,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->q_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
       {(void**)&h->p_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
       {(void**)&h->part, sizeof(float) * part_floats},
-      {(void**)&h->counters, sizeof(int) * (LIN_MAX_R + 2)},
+      {(void**)&h->counters, sizeof(int) * (2 * LIN_MAX_R + 2)},
       {(void**)&h->res, 4 * h->res_words},
       {(void**)&h->dst, sizeof(DevState)},
       {(void**)&s.n, 4 * (size_t)MB},
@@ -692,7 +692,7 @@ static int cur_num_sm() {
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
-  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (LIN_MAX_R + 2) + 256);
+  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256);
 }
 
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace,
@@ -708,7 +708,7 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
   a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
   char* ws = (char*)workspace;
   a.counters = (int*)ws;
-  size_t off = ((sizeof(int) * (LIN_MAX_R + 2) + 255) / 256) * 256;
+  size_t off = ((sizeof(int) * (2 * LIN_MAX_R + 2) + 255) / 256) * 256;
   off += sizeof(float) * (size_t)LIN_MAX_R * SPS_MAX_ROWS;
   a.part = (float*)(ws + off);
   cudaStream_t st = (cudaStream_t)stream;
@@ -721,7 +721,7 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
     cudaEventElapsedTime(out_ms, e0, e1);
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     int errw = 0;
-    if (e == cudaSuccess && cudaMemcpy(&errw, a.counters + LIN_MAX_R + 1, 4, cudaMemcpyDeviceToHost) == cudaSuccess && errw == 3)
+    if (e == cudaSuccess && cudaMemcpy(&errw, a.counters + 2 * LIN_MAX_R + 1, 4, cudaMemcpyDeviceToHost) == cudaSuccess && errw == 3)
       return fail(nullptr, SPS_ETIMEOUT, "a bounded device-side wait ran out in the linear kernel");
   }
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("linear launch: ") + cudaGetErrorString(e));

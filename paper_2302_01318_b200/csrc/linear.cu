@@ -18,6 +18,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdio>
 #include <cstdlib>
 #include <map>
 #include <mutex>
@@ -110,6 +111,65 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
     }
   }
   if (tid == 0) a.counters[r] = 0;
+}
+
+// Epilogue of the TMA variant.  Every CTA of a split finishes one slice of the range's rows once all
+// S partial results are in: output elements (m, n) go to threads in m-major order (neighbouring
+// threads, neighbouring n), and a thread fetches all the partials it needs before it adds them in
+// split order -- the loads are independent, the latency is paid once.  sq_s: shared scratch of
+// rows * M floats for the squares of a residual update, summed per row m in index order afterwards.
+__device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_begin, int rows, float* sq_s) {
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+  const int S = a.S, N = a.N, total = rows * a.M;
+  const bool resid = a.epi == EPI_RESIDUAL;
+  if (S <= 4) {
+    for (int e0 = tid; e0 < total; e0 += 4 * nthr) {
+      float v[4][4], old[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int e = e0 + b * nthr;
+        const int m = e < total ? e / rows : 0, n = n_begin + (e < total ? e - m * rows : 0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          v[b][j] = (e < total && j < S) ? __ldcg(a.part + ((size_t)j * SPS_MAX_ROWS + m) * N + n) : 0.f;
+        old[b] = (e < total && resid) ? a.Y[(long long)m * a.ldy + n] : 0.f;
+      }
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int e = e0 + b * nthr;
+        if (e < total) {
+          const int m = e / rows, n = n_begin + (e - m * rows);
+          float y = ((v[b][0] + v[b][1]) + v[b][2]) + v[b][3];
+          if (resid) { y += old[b]; sq_s[e] = y * y; }
+          a.Y[(long long)m * a.ldy + n] = y;
+        }
+      }
+    }
+  } else {
+    for (int e = tid; e < total; e += nthr) {
+      const int m = e / rows, n = n_begin + (e - m * rows);
+      float y = 0.f;
+      const float old = resid ? a.Y[(long long)m * a.ldy + n] : 0.f;
+      for (int s0 = 0; s0 < S; s0 += 16) {
+        float v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = (s0 + j < S) ? __ldcg(a.part + ((size_t)(s0 + j) * SPS_MAX_ROWS + m) * N + n) : 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) y += v[j];
+      }
+      if (resid) { y += old; sq_s[e] = y * y; }
+      a.Y[(long long)m * a.ldy + n] = y;
+    }
+  }
+  if (resid) {
+    __syncthreads();
+    for (int m = warp; m < a.M; m += nwarp) {
+      float t = 0.f;
+      for (int i = lane; i < rows; i += 32) t += sq_s[m * rows + i];
+      t = warp_sum(t);
+      if (lane == 0) a.ssq_out[(size_t)part_idx * SPS_MAX_ROWS + m] = t;
+    }
+  }
 }
 
 template <int NT>
@@ -358,6 +418,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   __syncthreads();
   pdl_launch_dependents();
   float* s_scale = reinterpret_cast<float*>(smem2 + 512);   // [16] 1/rms of each X row
+  unsigned long long* trace = a.dbg_t ? a.dbg_t + ((size_t)r * a.S + s) * 8 : nullptr;
+  if (trace && tid == 0) trace[0] = gtimer();
 
   const int total_it = ntiles * KSUB;
   if (warp == NCW) {
@@ -389,6 +451,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // X slab: rows 0..8*NT-1 (zeros beyond M), this CTA's k-range, bf16 hi and lo parts, natural k order.
     // Weights never change, so the producer is already streaming; X is the predecessor's output.
     pdl_wait();
+    if (trace && tid == 0) trace[1] = gtimer();
     {
       if (a.pro == PRO_RMSNORM) {
         // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
@@ -443,6 +506,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     }
+    if (trace && tid == 0) trace[2] = gtimer();
     bool alive = true;
     // Consumer warps work in groups of G: a tile goes to group (tile % NG) and its stage ks to warp
     // (ks % G) of the group, so that up to NCW warps chew on the ring at once; the G partial tiles meet
@@ -470,6 +534,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           if (!alive) { s_abort = 1; break; }
         }
         if (!mbar_wait(bar_full + 8 * slot, (uint32_t)use & 1u, a.err)) { alive = false; s_abort = 1; break; }
+        if (trace && tid == 0 && it == 0) trace[3] = gtimer();
         const uint32_t wrow = ring + slot * STAGE + g * 128;          // row g of slab 0; row g+8 is +1024
         const uint32_t xoff = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 32;  // logical chunk 2t of this stage's k-range
         const uint32_t xh_addr = xs_hi + g * XP + xoff, xl_addr = xs_lo + g * XP + xoff;
@@ -542,14 +607,45 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
     }
   }
-  // ---- arrival: the last of the S CTAs that split D for this range runs the epilogue
+  // ---- arrival.  The S CTAs that split D for this row range meet on a counter; once all partials are
+  // visible each of them finishes 1/S of the range's rows, so the reduction is S-way parallel and short.
+  // All CTAs of the grid are resident together (the grid never exceeds one CTA per SM), so the wait
+  // ends as soon as the slowest of the S is done; it is bounded all the same.
+  if (trace && tid == 0) trace[4] = gtimer();
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_flag = (atomicAdd(&a.counters[r], 1) == a.S - 1);
+  if (tid == 0) {
+    int ok = 1;
+    if (a.S > 1) {
+      atomicAdd(&a.counters[r], 1);
+      const unsigned long long t0 = gtimer();
+      while (*((volatile int*)&a.counters[r]) < a.S) {
+        __nanosleep(100);
+        if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); ok = 0; break; }
+      }
+    }
+    s_flag = ok;
+  }
   __syncthreads();
+  if (trace && tid == 0) trace[5] = gtimer();
   if (!s_flag) return;
   __threadfence();
-  lin_epilogue(a, r, row_begin, nrows, reinterpret_cast<float*>(smem2 + LIN2_HDR_BYTES));
+  {
+    // slice s of the range, cut on multiples of 4 rows
+    const int quads = (nrows + 3) >> 2;
+    const int q0 = (int)(((long long)s * quads) / a.S), q1 = (int)(((long long)(s + 1) * quads) / a.S);
+    const int b0 = min(q0 * 4, nrows), b1 = min(q1 * 4, nrows);
+    lin_epilogue_slice(a, r * a.S + s, row_begin + b0, b1 - b0, reinterpret_cast<float*>(smem2 + LIN2_HDR_BYTES));
+  }
+  if (a.S > 1) {
+    // departure: the last CTA to leave re-arms the counters for the next launch
+    __syncthreads();
+    if (tid == 0 && atomicAdd(&a.counters[LIN_MAX_R + r], 1) == a.S - 1) {
+      a.counters[r] = 0;
+      a.counters[LIN_MAX_R + r] = 0;
+    }
+  }
+  if (trace && tid == 0) trace[6] = gtimer();
 }
 
 // ---- fp32 weights: one warp per output row, X (after the prologue) in shared memory ---------------
@@ -638,6 +734,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     if (R < 1) R = 1;
     p.R = R;
     p.smem = (size_t)M * D * sizeof(float);
+    p.ssq_parts = p.R;
     return p;
   }
   static const int variant = [] {
@@ -676,6 +773,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     if (NS < 2) NS = 2;
     p.NS = NS;
     p.smem = 1024 + xbytes + (size_t)NS * stage + gscr;
+    p.ssq_parts = p.R * p.S;
     return p;
   }
   const int chunks = D / 128;
@@ -697,6 +795,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
   p.PR = pr_need < pr_fit ? pr_need : pr_fit;
   if (p.PR < 32) p.PR = 32;
   p.smem = sizeof(float) * (size_t)WC * 8 * p.NT * (p.PR + 4);
+  p.ssq_parts = p.R;
   return p;
 }
 
@@ -746,9 +845,16 @@ static cudaError_t weight_tensor_map(const void* W, int rows, int D, int KST, CU
 cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStream_t st) {
   LinArgs a = a_in;
   a.R = p.R; a.S = p.S; a.WC = p.WC; a.PR = p.PR; a.KS = p.KS; a.KST = p.KST; a.NS = p.NS; a.G = p.G;
-  if (!a.err) a.err = a.counters + LIN_MAX_R + 1;
+  if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
   static const int dbg_env = [] { const char* e = getenv("SPS_LIN_DBG"); return e ? atoi(e) : 0; }();
   a.dbg = dbg_env;
+  static unsigned long long* trace_buf = nullptr;
+  static const int trace_env = [] { const char* e = getenv("SPS_LIN_TRACE"); return e ? atoi(e) : 0; }();
+  if (trace_env && dtype == 1 && p.variant == 2) {
+    if (!trace_buf) cudaMalloc(&trace_buf, 8 * 8 * 1024);
+    cudaMemsetAsync(trace_buf, 0, 8 * 8 * 1024, st);
+    a.dbg_t = trace_buf;
+  }
   static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
   cudaError_t e;
   if (dtype == 0) {
@@ -785,5 +891,22 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     }
   }
   if (e != cudaSuccess) return e;
+  if (a.dbg_t) {
+    // experiments only: wait for the kernel and print when each phase began / ended over the CTAs (us)
+    cudaStreamSynchronize(st);
+    static unsigned long long hbuf[8 * 1024];
+    cudaMemcpy(hbuf, a.dbg_t, sizeof(hbuf), cudaMemcpyDeviceToHost);
+    const int n = p.R * p.S;
+    unsigned long long t0 = ~0ull;
+    for (int i = 0; i < n; ++i) if (hbuf[i * 8] && hbuf[i * 8] < t0) t0 = hbuf[i * 8];
+    const char* names[7] = {"entry", "waited", "slab", "tile0", "loopend", "arrived", "epidone"};
+    fprintf(stderr, "[lin trace N=%d D=%d M=%d R=%d S=%d]", a.N, a.D, a.M, p.R, p.S);
+    for (int k = 0; k < 7; ++k) {
+      double mn = 1e30, mx = 0, sum = 0; int cnt = 0;
+      for (int i = 0; i < n; ++i) if (hbuf[i * 8 + k]) { const double v = (hbuf[i * 8 + k] - t0) * 1e-3; mn = v < mn ? v : mn; mx = v > mx ? v : mx; sum += v; ++cnt; }
+      if (cnt) fprintf(stderr, " %s %.1f/%.1f/%.1f", names[k], mn, sum / cnt, mx);
+    }
+    fprintf(stderr, "\n");
+  }
   return cudaGetLastError();
 }
