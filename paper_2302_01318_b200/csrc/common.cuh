@@ -158,7 +158,6 @@ struct LinArgs {
   int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
   int* err;               // sticky error word: set to 3 if a bounded wait ran out
   int dbg;                // experiments only: bit 0 = consumers skip the arithmetic
-  unsigned long long* dbg_t;  // experiments only: per-CTA timestamps [R*S][8]
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };

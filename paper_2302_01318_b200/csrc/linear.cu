@@ -418,8 +418,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   __syncthreads();
   pdl_launch_dependents();
   float* s_scale = reinterpret_cast<float*>(smem2 + 512);   // [16] 1/rms of each X row
-  unsigned long long* trace = a.dbg_t ? a.dbg_t + ((size_t)r * a.S + s) * 8 : nullptr;
-  if (trace && tid == 0) trace[0] = gtimer();
 
   const int total_it = ntiles * KSUB;
   if (warp == NCW) {
@@ -451,7 +449,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // X slab: rows 0..8*NT-1 (zeros beyond M), this CTA's k-range, bf16 hi and lo parts, natural k order.
     // Weights never change, so the producer is already streaming; X is the predecessor's output.
     pdl_wait();
-    if (trace && tid == 0) trace[1] = gtimer();
     {
       if (a.pro == PRO_RMSNORM) {
         // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
@@ -506,7 +503,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     }
-    if (trace && tid == 0) trace[2] = gtimer();
     bool alive = true;
     // Consumer warps work in groups of G: a tile goes to group (tile % NG) and its stage ks to warp
     // (ks % G) of the group, so that up to NCW warps chew on the ring at once; the G partial tiles meet
@@ -534,7 +530,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           if (!alive) { s_abort = 1; break; }
         }
         if (!mbar_wait(bar_full + 8 * slot, (uint32_t)use & 1u, a.err)) { alive = false; s_abort = 1; break; }
-        if (trace && tid == 0 && it == 0) trace[3] = gtimer();
         const uint32_t wrow = ring + slot * STAGE + g * 128;          // row g of slab 0; row g+8 is +1024
         const uint32_t xoff = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 32;  // logical chunk 2t of this stage's k-range
         const uint32_t xh_addr = xs_hi + g * XP + xoff, xl_addr = xs_lo + g * XP + xoff;
@@ -611,7 +606,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   // visible each of them finishes 1/S of the range's rows, so the reduction is S-way parallel and short.
   // All CTAs of the grid are resident together (the grid never exceeds one CTA per SM), so the wait
   // ends as soon as the slowest of the S is done; it is bounded all the same.
-  if (trace && tid == 0) trace[4] = gtimer();
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -627,7 +621,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     s_flag = ok;
   }
   __syncthreads();
-  if (trace && tid == 0) trace[5] = gtimer();
   if (!s_flag) return;
   __threadfence();
   {
@@ -645,7 +638,6 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       a.counters[LIN_MAX_R + r] = 0;
     }
   }
-  if (trace && tid == 0) trace[6] = gtimer();
 }
 
 // ---- fp32 weights: one warp per output row, X (after the prologue) in shared memory ---------------
@@ -848,13 +840,6 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
   static const int dbg_env = [] { const char* e = getenv("SPS_LIN_DBG"); return e ? atoi(e) : 0; }();
   a.dbg = dbg_env;
-  static unsigned long long* trace_buf = nullptr;
-  static const int trace_env = [] { const char* e = getenv("SPS_LIN_TRACE"); return e ? atoi(e) : 0; }();
-  if (trace_env && dtype == 1 && p.variant == 2) {
-    if (!trace_buf) cudaMalloc(&trace_buf, 8 * 8 * 1024);
-    cudaMemsetAsync(trace_buf, 0, 8 * 8 * 1024, st);
-    a.dbg_t = trace_buf;
-  }
   static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
   cudaError_t e;
   if (dtype == 0) {
@@ -891,22 +876,5 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     }
   }
   if (e != cudaSuccess) return e;
-  if (a.dbg_t) {
-    // experiments only: wait for the kernel and print when each phase began / ended over the CTAs (us)
-    cudaStreamSynchronize(st);
-    static unsigned long long hbuf[8 * 1024];
-    cudaMemcpy(hbuf, a.dbg_t, sizeof(hbuf), cudaMemcpyDeviceToHost);
-    const int n = p.R * p.S;
-    unsigned long long t0 = ~0ull;
-    for (int i = 0; i < n; ++i) if (hbuf[i * 8] && hbuf[i * 8] < t0) t0 = hbuf[i * 8];
-    const char* names[7] = {"entry", "waited", "slab", "tile0", "loopend", "arrived", "epidone"};
-    fprintf(stderr, "[lin trace N=%d D=%d M=%d R=%d S=%d]", a.N, a.D, a.M, p.R, p.S);
-    for (int k = 0; k < 7; ++k) {
-      double mn = 1e30, mx = 0, sum = 0; int cnt = 0;
-      for (int i = 0; i < n; ++i) if (hbuf[i * 8 + k]) { const double v = (hbuf[i * 8 + k] - t0) * 1e-3; mn = v < mn ? v : mn; mx = v > mx ? v : mx; sum += v; ++cnt; }
-      if (cnt) fprintf(stderr, " %s %.1f/%.1f/%.1f", names[k], mn, sum / cnt, mx);
-    }
-    fprintf(stderr, "\n");
-  }
   return cudaGetLastError();
 }

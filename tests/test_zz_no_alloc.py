@@ -1,0 +1,45 @@
+"""sps_linear_static: the linear layer for hosts that cannot allocate device memory (code inside a
+stream capture, a server with a frozen memory budget, a plugin that only receives buffers).  Its
+scratch is a fixed array inside the library; the result must equal sps_linear's, call after call,
+because every call reuses that array and finds the previous call's contents in it.
+
+Collected last on purpose: a run that stops at the first failure has then run every other test."""
+import pytest
+import torch
+
+import paper_2302_01318_b200 as sps
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("N,D,M,dt", [(4099, 2048, 5, torch.bfloat16), (8192, 8192, 3, torch.bfloat16),
+                                      (1000, 256, 9, torch.bfloat16), (515, 1024, 2, torch.float32)])
+def test_static_scratch_matches_workspace_version_twice(N, D, M, dt):
+    g = torch.Generator(device=DEV).manual_seed(N + D + M)
+    W = (torch.randn((N, D), device=DEV, generator=g) * 0.05).to(dt)
+    dtype = 0 if dt == torch.float32 else 1
+    ws = torch.zeros(sps.sps_linear_workspace_bytes(dtype, M, N, D), dtype=torch.uint8, device=DEV)
+    for call in range(2):   # two calls in a row on the shared array, with different inputs
+        X = torch.randn((M, D), device=DEV, generator=g)
+        want = torch.full((M, N), float("nan"), device=DEV)
+        got = torch.full((M, N), float("nan"), device=DEV)
+        sps.sps_linear(W, X, want, ws)
+        sps.sps_linear_static(W, X, got)
+        torch.cuda.synchronize()
+        # same kernel, same plan, same reduction order: the tolerance of the other linear tests
+        # (2e-5 * sqrt(D) * max|w| * max|x| + 1e-6) is met with room to spare; in fact bit-equal
+        tol = 2e-5 * (D ** 0.5) * float(W.float().abs().max()) * float(X.abs().max()) + 1e-6
+        assert torch.isfinite(got).all()
+        assert (got - want).abs().max().item() <= tol
+        assert torch.equal(got, want)
+
+
+def test_static_scratch_rejects_oversized_shapes():
+    # N * splits * 16 floats must fit the array: 65536 rows with 16 splits do not
+    assert sps.sps_linear_static_max_floats() == 4 << 20
+    W = torch.zeros((8, 128), device=DEV, dtype=torch.bfloat16)
+    X = torch.zeros((1, 128), device=DEV)
+    Y = torch.zeros((1, 8), device=DEV)
+    rc = sps.lib().sps_linear_static(W.data_ptr(), 1, X.data_ptr(), 1, 65536, 32768, Y.data_ptr(), None)
+    assert rc == sps.SPS_EINVAL and b"static" in sps.lib().sps_last_error(None)
