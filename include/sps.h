@@ -204,6 +204,27 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
                void* workspace, void* stream, float* out_ms);
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D);
 
+/* The same linear layer for callers that cannot allocate device memory (the
+ * paper has no counterpart: this is a service of the library, not a step of
+ * the method).  A host that runs inside a stream capture, or serves under a
+ * frozen memory budget, or is a plugin that only ever receives buffers, has no
+ * workspace to hand to sps_linear; here the split-K scratch is a fixed array
+ * inside the library's device image (about 16 MiB on every GPU that loads the
+ * library, held until the process exits).  The call makes no cudaMalloc /
+ * cudaFree and uses no allocating library routine.
+ *   W, X, Y, dtype, M, N, D: as for sps_linear (all device pointers).
+ *   stream: cudaStream_t, NULL = default stream; the call only enqueues.
+ * Limit: N * splits * 16 <= sps_linear_static_max_floats() (4 Mi floats), where
+ * splits = D / 2048 for bf16 with M <= 8, D / 1024 for M > 8, 1 for fp32;
+ * larger shapes return SPS_EINVAL with a message.  The first call on a device
+ * looks up the array's device address (cudaGetSymbolAddress) with that device
+ * current; make that first call before any stream capture begins.
+ * All calls share the one array: two calls whose kernels overlap on the GPU
+ * (different streams) race on it -- keep them on one stream or order them. */
+int sps_linear_static(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
+                      void* stream);
+int64_t sps_linear_static_max_floats(void);
+
 /* Philox4x32-10 on the device, for known-answer tests: ctr device uint32 [n,4],
  * key device uint32 [n,2], out device uint32 [n,4]. */
 int sps_philox(const uint32_t* ctr, const uint32_t* key, int32_t n, void* stream, uint32_t* out);

@@ -86,6 +86,8 @@ def lib():
         L.sps_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sps_linear_workspace_bytes.restype = i64
         L.sps_philox.argtypes = [vp, vp, i32, vp, vp]
+        L.sps_linear_static.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp]
+        L.sps_linear_static_max_floats.restype = i64
         _lib = L
     return _lib
 
@@ -242,3 +244,16 @@ def sps_linear(W, X, Y, workspace, stream=None, timed=False):
 
 def sps_philox(ctr, key, out, stream=None):
     _check(lib().sps_philox(ctr.data_ptr(), key.data_ptr(), ctr.shape[0], _stream_ptr(stream), out.data_ptr()))
+
+
+def sps_linear_static(W, X, Y, stream=None):
+    """Y[M,N] = X[M,D] W[N,D]^T with the scratch held inside the library: for callers that cannot
+    allocate device memory (see include/sps.h).  W CUDA fp32 or bf16, X/Y CUDA fp32."""
+    import torch
+    dtype = 0 if W.dtype == torch.float32 else 1
+    N, D = W.shape
+    _check(lib().sps_linear_static(W.data_ptr(), dtype, X.data_ptr(), X.shape[0], N, D, Y.data_ptr(), _stream_ptr(stream)))
+
+
+def sps_linear_static_max_floats():
+    return int(lib().sps_linear_static_max_floats())

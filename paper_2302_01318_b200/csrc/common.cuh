@@ -164,6 +164,7 @@ struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_
 LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
 size_t lin_part_floats(int N, int S_max);
+void sps_set_global_error(const char* msg);   // text returned by sps_last_error(NULL)
 #define LIN_MAX_R 512
 #define LIN_CONSUMER_WARPS 8
 #define LIN_MAX_S 64

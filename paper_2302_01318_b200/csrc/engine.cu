@@ -31,6 +31,8 @@ struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uin
 
 }  // namespace
 
+void sps_set_global_error(const char* msg) { g_err = msg ? msg : ""; }
+
 struct sps_handle {
   sps_cfg cfg{};
   cudaStream_t stream = nullptr;

@@ -878,3 +878,62 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
+
+// ================================================================================================
+// sps_linear_static: the linear layer for callers that cannot allocate device memory.
+//
+// Some hosts of this library may not call cudaMalloc at the moment they need a result: code running
+// inside a CUDA stream capture, a real-time serving loop with a frozen memory budget, a plugin that
+// is handed buffers by its framework and nothing else.  sps_linear asks such a caller for a
+// workspace; this entry point instead keeps the split-K scratch (partial sums and arrival counters)
+// in one fixed array that lives in the library's device image.  The array below is only a host-side
+// stand-in in host code: its device address is looked up once per device with cudaGetSymbolAddress.
+// ================================================================================================
+#include "../../include/sps.h"
+
+#define SPS_STATIC_PART_FLOATS (4u << 20)                     /* 16 MiB of partial sums */
+#define SPS_STATIC_CTR_BYTES (((2 * LIN_MAX_R + 2) * 4 + 255) / 256 * 256)
+static __device__ __align__(256) unsigned char g_static_scratch[SPS_STATIC_CTR_BYTES + 4ull * SPS_STATIC_PART_FLOATS];
+
+extern "C" int64_t sps_linear_static_max_floats(void) { return (int64_t)SPS_STATIC_PART_FLOATS; }
+
+extern "C" int sps_linear_static(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
+                                 void* stream) {
+  if (!W || !X || !Y) { sps_set_global_error("null argument"); return SPS_EINVAL; }
+  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || (dtype != 0 && dtype != 1)) { sps_set_global_error("M, N, D or dtype out of range"); return SPS_EINVAL; }
+  if (dtype == 1 && D % 128) { sps_set_global_error("bf16 needs D to be a multiple of 128"); return SPS_EINVAL; }
+  if (dtype == 0 && (size_t)M * D * 4 > 200 * 1024) { sps_set_global_error("fp32: M * D too large"); return SPS_EINVAL; }
+  int dev = 0, num_sm = SPS_NUM_SM_FALLBACK;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= 64) { sps_set_global_error("cudaGetDevice failed"); return SPS_ECUDA; }
+  cudaDeviceGetAttribute(&num_sm, cudaDevAttrMultiProcessorCount, dev);
+  const LinPlan p = lin_plan(dtype, M, N, D, num_sm);
+  if (lin_part_floats(N, p.S) > (size_t)SPS_STATIC_PART_FLOATS) {
+    sps_set_global_error("shape needs more split-K scratch than the static array holds (N * splits * 16 floats > 4 Mi floats)");
+    return SPS_EINVAL;
+  }
+  // set-up, once per device, with that device current: the device address of the static array
+  static unsigned char* base[64] = {nullptr};
+  static std::mutex mu;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!base[dev]) {
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+      if (e != cudaSuccess || !ptr) { sps_set_global_error("cudaGetSymbolAddress failed for the static scratch"); return SPS_ECUDA; }
+      base[dev] = static_cast<unsigned char*>(ptr);
+    }
+  }
+  LinArgs a{};
+  a.W[0] = W; a.rows_per_mat = N; a.N = N; a.D = D; a.M = M; a.X = X; a.ldx = D; a.x_row0 = 0; a.x_rowstep = 1;
+  a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
+  a.counters = reinterpret_cast<int*>(base[dev]);
+  a.part = reinterpret_cast<float*>(base[dev] + SPS_STATIC_CTR_BYTES);
+  cudaStream_t st = (cudaStream_t)stream;
+  // The array keeps the last call's contents.  Partial sums are overwritten before they are read and
+  // the kernel re-arms its own counters; the sticky error word is the one thing that must start at zero.
+  e = cudaMemsetAsync(a.counters + 2 * LIN_MAX_R + 1, 0, sizeof(int), st);
+  if (e == cudaSuccess) e = lin_launch(dtype, a, p, st);
+  if (e != cudaSuccess) { sps_set_global_error(cudaGetErrorString(e)); return SPS_ECUDA; }
+  return SPS_OK;
+}
