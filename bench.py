@@ -38,7 +38,7 @@ METRIC = "batch-1 tokens/s SpS vs AR decode; verify-pass HBM GB/s vs peak"
 UNIT = "tokens/s"
 # mean tokens per speculative loop measured by this bench's own arm on each workload (seeded weights and
 # prompts make it repeatable); the CPU arm cannot run whole generations of the 70B pair, so it uses these
-ASSUMED_TOKENS_PER_LOOP = {"70b": 1.30, "mid": 1.9, "tiny": 3.0, "tiny_bf16": 3.0}
+ASSUMED_TOKENS_PER_LOOP = {"70b": 1.28, "mid": 1.9, "tiny": 3.0, "tiny_bf16": 3.0}
 
 
 def measured_peaks():
@@ -209,7 +209,9 @@ def run_ours(args):
     V = c["target"]["vocab"]
     max_seq = ((P + n_new + max(K, 8) + 63) // 64) * 64
     h = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=max_seq, max_batch=1, max_K=max(K, 1), device=local)
-    seeds = [1000 * rank + i for i in range(args.warmup + args.steps + 8)]
+    from paper_2302_01318_b200 import replicas
+    # independent replicas: rank r generates the global sequences r, r + world, ... (no collective on the data path)
+    seeds = replicas.shard_sequences((args.warmup + args.steps + 8) * world, rank, world)
 
     def gen(i, k):
         prompt = sps_synth.make_prompt(seeds[i], P, V)
@@ -233,13 +235,9 @@ def run_ours(args):
         stats.append(st); walls.append(w)
     barrier()
     clocks = clk.stop()
-    dec_ms = sum(s["ms_decode"] for s in stats)
-    wall_s = sum(walls)
-    if dist is not None:
-        tt = torch.tensor([dec_ms, wall_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        dec_ms, wall_s = float(tt[0]), float(tt[1])
-    tokens = args.steps * n_new * world
+    dec_s, tokens = replicas.job_time_and_tokens(sum(s["ms_decode"] for s in stats) / 1e3, args.steps * n_new, dist, dev)
+    wall_s, _ = replicas.job_time_and_tokens(sum(walls), 0, dist, dev)
+    dec_ms = dec_s * 1e3
     value = tokens / (dec_ms / 1e3)
     e2e = tokens / wall_s
     loops = sum(s["loops"] for s in stats)
@@ -257,11 +255,13 @@ def run_ours(args):
     v_gbs = vbytes * loops / (ms_verify / 1e3) / 1e9 if ms_verify > 0 else None
     d_gbs = dbytes * loops * K / (ms_draft / 1e3) / 1e9 if ms_draft > 0 and K > 0 else None
     n_lin_verify = 5 * c["target"]["n_layers"] + 1
-    roofline = {"bound": "hbm", "kernel": "lin_bf16_kernel (weight-streaming linear layer) inside the scoring pass",
+    roofline = {"bound": "hbm", "kernel": "lin_bf16_tma_kernel (weight-streaming linear layer) averaged over the scoring pass",
                 "achieved": v_gbs, "peak": peak, "unit": "GB/s", "frac": (v_gbs / peak) if v_gbs else None,
                 "frac_of_8000_nominal": (v_gbs / 8000.0) if v_gbs else None, "peak_source": peak_src,
                 "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
-                "traffic": args.traffic}
+                # profiles/lin_bf16_tma_32000x8192_M5.md: dram read + write = 1.013 x the algorithmic bytes of that launch;
+                # traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
+                "traffic": args.traffic if args.traffic is not None else 1.013 * vbytes / n_lin_verify}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dec_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if c["target"]["dtype"] else "f32", "data": "synthetic",
@@ -281,17 +281,19 @@ def run_ours(args):
                      "ms_prefill": stats[-1]["ms_prefill"]}}
     if rank == 0 and world == 1:
         # the same library's autoregressive decode on the same models
-        ar_stats = []
-        gen(0, 0)
-        for i in range(args.ar_steps):
-            _, st, _ = gen(args.warmup + i, 0)
-            ar_stats.append(st)
-        ar_ms = sum(s["ms_decode"] for s in ar_stats)
-        ar_tps = args.ar_steps * n_new / (ar_ms / 1e3)
-        ar_gbs = sps_synth.weight_bytes(c["target"]) * args.ar_steps * n_new / (ar_ms / 1e3) / 1e9
-        line["ar"] = {"value": ar_tps, "unit": UNIT, "ms_per_token": ar_ms / (args.ar_steps * n_new), "hbm_gbs": ar_gbs,
-                      "frac": ar_gbs / peak}
-        line["speedup_vs_ar"] = value / ar_tps
+        ar_tps = None
+        if args.ar_steps > 0:
+            ar_stats = []
+            gen(0, 0)
+            for i in range(args.ar_steps):
+                _, st, _ = gen(args.warmup + i, 0)
+                ar_stats.append(st)
+            ar_ms = sum(s["ms_decode"] for s in ar_stats)
+            ar_tps = args.ar_steps * n_new / (ar_ms / 1e3)
+            ar_gbs = sps_synth.weight_bytes(c["target"]) * args.ar_steps * n_new / (ar_ms / 1e3) / 1e9
+            line["ar"] = {"value": ar_tps, "unit": UNIT, "ms_per_token": ar_ms / (args.ar_steps * n_new), "hbm_gbs": ar_gbs,
+                          "frac": ar_gbs / peak}
+            line["speedup_vs_ar"] = value / ar_tps
         if not args.no_cpu:
             import oracle
             lt = layer_numpy(wt["layers"][0])
@@ -305,6 +307,25 @@ def run_ours(args):
                                                f"target unembedding + 1 of {c['draft']['n_layers']} draft layers + draft "
                                                f"unembedding over 1 row (context {P}), scaled to one loop and divided into the "
                                                f"measured {tpl:.3f} tokens per loop"), "seconds": s}
+    if rank == 0 and world == 1 and args.aligned_steps > 0 and c["target"]["dtype"] == 1:
+        # Same kernels, same shapes, but a pair whose draft agrees with its target about as often as the paper's
+        # trained pair did: both bodies' output projections are damped in place (x gamma), so that the shared
+        # (un)embedding dominates the logits.  A documented deviation from "all weights N(0, 0.02)", used only to
+        # show tokens per loop in the paper's acceptance regime; kernel times do not depend on weight values.
+        for w in (wt, wd):
+            for lw in w["layers"]:
+                lw["wo"].mul_(args.aligned_gamma)
+                lw["w_down"].mul_(args.aligned_gamma)
+        torch.cuda.synchronize()
+        gen(0, K)
+        al = [gen(args.warmup + i, K)[1] for i in range(args.aligned_steps)]
+        al_ms = sum(s["ms_decode"] for s in al)
+        al_loops = sum(s["loops"] for s in al)
+        al_tps = args.aligned_steps * n_new / (al_ms / 1e3)
+        line["variants"] = {"aligned": {"gamma": args.aligned_gamma, "value": al_tps, "unit": UNIT,
+                                        "tokens_per_loop": sum(s["emitted"] for s in al) / al_loops,
+                                        "accept_rate": sum(s["accepted"] for s in al) / (al_loops * K) if K else None,
+                                        "speedup_vs_ar": al_tps / ar_tps if ar_tps else None}}
     h.close()
     if rank == 0:
         print(json.dumps(line))
@@ -323,7 +344,10 @@ def main():
     ap.add_argument("--K", type=int, default=4)
     ap.add_argument("--ar-steps", type=int, default=2)
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--traffic", type=float, default=None, help="ncu dram bytes per launch of the dominant kernel, if known")
+    ap.add_argument("--aligned-steps", type=int, default=2)
+    ap.add_argument("--aligned-gamma", type=float, default=1e-4)
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="ncu dram bytes per launch of the dominant kernel; default: bytes_per_launch x the ratio measured in profiles/")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
