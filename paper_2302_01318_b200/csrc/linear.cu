@@ -116,60 +116,74 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
 // Epilogue of the TMA variant.  Every CTA of a split finishes one slice of the range's rows once all
 // S partial results are in: output elements (m, n) go to threads in m-major order (neighbouring
 // threads, neighbouring n), and a thread fetches all the partials it needs before it adds them in
-// split order -- the loads are independent, the latency is paid once.  sq_s: shared scratch of
-// rows * M floats for the squares of a residual update, summed per row m in index order afterwards.
-__device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_begin, int rows, float* sq_s) {
+// split order -- the loads are independent, the latency is paid once.  sq_s: shared scratch (sq_cap
+// floats; the slice is walked in chunks that fit) for the squares of a residual update, summed per row
+// m in index order afterwards; ssq_s: 16 shared floats that carry the per-row sums across chunks.
+__device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, int rows_all, float* sq_s, int sq_cap,
+                                   float* ssq_s) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
-  const int S = a.S, N = a.N, total = rows * a.M;
+  const int S = a.S, N = a.N;
   const bool resid = a.epi == EPI_RESIDUAL;
-  if (S <= 4) {
-    for (int e0 = tid; e0 < total; e0 += 4 * nthr) {
-      float v[4][4], old[4];
+  int chunk_rows = sq_cap / a.M;
+  if (chunk_rows > rows_all) chunk_rows = rows_all;
+  if (chunk_rows < 1) chunk_rows = 1;
+  if (resid) {
+    if (tid < SPS_MAX_ROWS) ssq_s[tid] = 0.f;
+    __syncthreads();
+  }
+  for (int c0 = 0; c0 < rows_all; c0 += chunk_rows) {
+    const int rows = min(chunk_rows, rows_all - c0), n_begin = n_first + c0, total = rows * a.M;
+    if (S <= 4) {
+      for (int e0 = tid; e0 < total; e0 += 4 * nthr) {
+        float v[4][4], old[4];
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int e = e0 + b * nthr;
-        const int m = e < total ? e / rows : 0, n = n_begin + (e < total ? e - m * rows : 0);
+        for (int b = 0; b < 4; ++b) {
+          const int e = e0 + b * nthr;
+          const int m = e < total ? e / rows : 0, n = n_begin + (e < total ? e - m * rows : 0);
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          v[b][j] = (e < total && j < S) ? __ldcg(a.part + ((size_t)j * SPS_MAX_ROWS + m) * N + n) : 0.f;
-        old[b] = (e < total && resid) ? a.Y[(long long)m * a.ldy + n] : 0.f;
-      }
+          for (int j = 0; j < 4; ++j)
+            v[b][j] = (e < total && j < S) ? __ldcg(a.part + ((size_t)j * SPS_MAX_ROWS + m) * N + n) : 0.f;
+          old[b] = (e < total && resid) ? a.Y[(long long)m * a.ldy + n] : 0.f;
+        }
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int e = e0 + b * nthr;
-        if (e < total) {
-          const int m = e / rows, n = n_begin + (e - m * rows);
-          float y = ((v[b][0] + v[b][1]) + v[b][2]) + v[b][3];
-          if (resid) { y += old[b]; sq_s[e] = y * y; }
-          a.Y[(long long)m * a.ldy + n] = y;
+        for (int b = 0; b < 4; ++b) {
+          const int e = e0 + b * nthr;
+          if (e < total) {
+            const int m = e / rows, n = n_begin + (e - m * rows);
+            float y = ((v[b][0] + v[b][1]) + v[b][2]) + v[b][3];
+            if (resid) { y += old[b]; sq_s[e] = y * y; }
+            a.Y[(long long)m * a.ldy + n] = y;
+          }
         }
       }
-    }
-  } else {
-    for (int e = tid; e < total; e += nthr) {
-      const int m = e / rows, n = n_begin + (e - m * rows);
-      float y = 0.f;
-      const float old = resid ? a.Y[(long long)m * a.ldy + n] : 0.f;
-      for (int s0 = 0; s0 < S; s0 += 16) {
-        float v[16];
+    } else {
+      for (int e = tid; e < total; e += nthr) {
+        const int m = e / rows, n = n_begin + (e - m * rows);
+        float y = 0.f;
+        const float old = resid ? a.Y[(long long)m * a.ldy + n] : 0.f;
+        for (int s0 = 0; s0 < S; s0 += 16) {
+          float v[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = (s0 + j < S) ? __ldcg(a.part + ((size_t)(s0 + j) * SPS_MAX_ROWS + m) * N + n) : 0.f;
+          for (int j = 0; j < 16; ++j) v[j] = (s0 + j < S) ? __ldcg(a.part + ((size_t)(s0 + j) * SPS_MAX_ROWS + m) * N + n) : 0.f;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) y += v[j];
+          for (int j = 0; j < 16; ++j) y += v[j];
+        }
+        if (resid) { y += old; sq_s[e] = y * y; }
+        a.Y[(long long)m * a.ldy + n] = y;
       }
-      if (resid) { y += old; sq_s[e] = y * y; }
-      a.Y[(long long)m * a.ldy + n] = y;
+    }
+    if (resid) {
+      __syncthreads();
+      for (int m = warp; m < a.M; m += nwarp) {   // row m always falls to the same warp: no race on ssq_s[m]
+        float t = 0.f;
+        for (int i = lane; i < rows; i += 32) t += sq_s[m * rows + i];
+        t = warp_sum(t);
+        if (lane == 0) ssq_s[m] += t;
+      }
+      __syncthreads();
     }
   }
-  if (resid) {
-    __syncthreads();
-    for (int m = warp; m < a.M; m += nwarp) {
-      float t = 0.f;
-      for (int i = lane; i < rows; i += 32) t += sq_s[m * rows + i];
-      t = warp_sum(t);
-      if (lane == 0) a.ssq_out[(size_t)part_idx * SPS_MAX_ROWS + m] = t;
-    }
-  }
+  if (resid && tid < a.M) a.ssq_out[(size_t)part_idx * SPS_MAX_ROWS + tid] = ssq_s[tid];
 }
 
 template <int NT>
@@ -393,11 +407,14 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   const int r = blockIdx.x, s = blockIdx.y;
   const int KS = a.KS, KST = a.KST, NS = a.NS, KSUB = KS / KST, D = a.D;
   const int k_base = s * KS;
-  const int T = (a.N + 15) >> 4;
-  const int tile_begin = (int)(((long long)r * T) / a.R), tile_end = (int)(((long long)(r + 1) * T) / a.R);
-  const int ntiles = tile_end - tile_begin;
-  const int row_begin = tile_begin * 16;
-  const int nrows = min(tile_end * 16, a.N) - row_begin;
+  const int T = (a.N + 15) >> 4;                       // 16-row output tiles of the whole layer
+  const int C = gridDim.x * gridDim.y, cta = r * a.S + s;
+  // Tiles are handed out at run time: the R CTAs that share k-range s draw tile numbers from one counter,
+  // so a CTA whose SM sees slower memory simply takes fewer tiles and all of them finish within a tile's
+  // time of one another.  Which CTA computed a tile leaves no trace in the result.
+  int* tileq = a.counters + 2 + s;
+  __shared__ volatile int s_issued, s_total;
+  volatile int* tile_ids = reinterpret_cast<volatile int*>(smem2 + 704);   // [64] ring: local tile -> tile number
   const uint32_t XP = (uint32_t)KS * 2 + 16, STAGE = 16u * (uint32_t)KST * 2u;
   const uint32_t xbytes = ((2u * NT * 8u * XP + 1023u) / 1024u) * 1024u;
   const uint32_t sm0 = smem_u32(smem2);
@@ -413,34 +430,53 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); consumed[i] = 0; }
     s_abort = 0;
+    s_issued = 0;
+    s_total = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   pdl_launch_dependents();
   float* s_scale = reinterpret_cast<float*>(smem2 + 512);   // [16] 1/rms of each X row
 
-  const int total_it = ntiles * KSUB;
   if (warp == NCW) {
     // ------------------------------------------------------------------ producer (one lane)
     if (lane == 0) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      int issued = 0;
-      for (int it = 0; it < total_it; ++it) {
-        const int slot = it % NS, use = it / NS;
-        if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err)) break;
-        const int tile = it / KSUB, ks = it - tile * KSUB;
-        const int row0 = row_begin + tile * 16;
+      int local = 0, it = 0;
+      bool ok = true;
+      auto issue = [&](int tile) {
+        tile_ids[local & 63] = tile;
+        const int row0 = tile * 16;
         const int mat = row0 / a.rows_per_mat;
-        mbar_expect_tx(bar_full + 8 * slot, STAGE);
-        tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, row0 - mat * a.rows_per_mat, (k_base + ks * KST) >> 6,
-                    bar_full + 8 * slot, policy);
-        issued = it + 1;
+        for (int ks = 0; ks < KSUB; ++ks, ++it) {
+          const int slot = it % NS, use = it / NS;
+          if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; return; }
+          mbar_expect_tx(bar_full + 8 * slot, STAGE);
+          tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, row0 - mat * a.rows_per_mat, (k_base + ks * KST) >> 6,
+                      bar_full + 8 * slot, policy);
+        }
+        ++local;
+        s_issued = local;
+      };
+      // The first ring-full of tiles is fixed (tiles r, r + R, ...): they are fetched before the predecessor
+      // kernel has finished.  The shared tile counter may only be touched after it has: the last CTA of
+      // the previous launch is the one that re-arms it.
+      const int PRE = max(1, NS / KSUB);
+      for (int j = 0; j < PRE && ok; ++j)
+        if (r + j * a.R < T) issue(r + j * a.R);
+      pdl_wait();
+      const int dyn0 = PRE * a.R;
+      int next_tile = dyn0 + atomicAdd(tileq, 1);
+      while (ok && next_tile < T) {
+        const int tile = next_tile;
+        next_tile = dyn0 + atomicAdd(tileq, 1);   // the next number is on its way while this tile's loads are issued
+        issue(tile);
       }
-      if (issued < total_it || *((volatile int*)&s_abort)) {
+      s_total = local;
+      if (!ok || *((volatile int*)&s_abort)) {
         // a wait ran out somewhere: let the copies already issued land before this CTA's memory goes away
-        for (int it = max(0, issued - NS); it < issued; ++it)
-          mbar_wait(bar_full + 8 * (it % NS), (uint32_t)(it / NS) & 1u, a.err);
+        for (int j = max(0, it - NS); j < it; ++j) mbar_wait(bar_full + 8 * (j % NS), (uint32_t)(j / NS) & 1u, a.err);
       }
     }
     pdl_wait();
@@ -513,14 +549,27 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // swizzle stores logical chunk c of row g at physical chunk c ^ (g & 7)
     const uint32_t wchunk0 = (uint32_t)(((2 * t) ^ g) << 4), wchunk1 = (uint32_t)(((2 * t + 1) ^ g) << 4);
     int round = 0;
-    for (int tile = grp; tile < ntiles && alive; tile += NG, ++round) {
+    for (int L = grp; alive; L += NG, ++round) {
+      // wait until local tile L has been issued, or until the producer has run out of tiles
+      if (s_issued <= L) {
+        const unsigned long long t0 = gtimer();
+        bool done = false;
+        while (s_issued <= L) {
+          const int tot = s_total;
+          if (tot >= 0 && L >= tot) { done = true; break; }
+          __nanosleep(32);
+          if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); s_abort = 1; done = true; break; }
+        }
+        if (done) break;
+      }
+      const int tile = tile_ids[L & 63];
       float acc[NT][4][4];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[nt][c][0] = acc[nt][c][1] = acc[nt][c][2] = acc[nt][c][3] = 0.f;
       for (int ks = rank; ks < KSUB; ks += G) {
-        const int it = tile * KSUB + ks, slot = it % NS, use = it / NS;
+        const int it = L * KSUB + ks, slot = it % NS, use = it / NS;
         if (use > 0 && consumed[slot] < use) {
           const unsigned long long t0 = gtimer();
           while (consumed[slot] < use) {
@@ -580,12 +629,12 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         for (int e = rank * 32 + lane; e < NT * 128; e += G * 32) {
           float sum = 0.f;
           for (int w = 0; w < G; ++w) sum += gbase[w * (NT * 128) + e];
-          const int col = e >> 4, n = row_begin + tile * 16 + (e & 15);
+          const int col = e >> 4, n = tile * 16 + (e & 15);
           if (col < a.M && n < a.N) a.part[((size_t)s * SPS_MAX_ROWS + col) * a.N + n] = sum;
         }
       } else {
         if (!alive) break;
-        const int n0 = row_begin + tile * 16 + g, n1 = n0 + 8;
+        const int n0 = tile * 16 + g, n1 = n0 + 8;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           const int col = nt * 8 + 2 * t;
@@ -602,18 +651,18 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
     }
   }
-  // ---- arrival.  The S CTAs that split D for this row range meet on a counter; once all partials are
-  // visible each of them finishes 1/S of the range's rows, so the reduction is S-way parallel and short.
-  // All CTAs of the grid are resident together (the grid never exceeds one CTA per SM), so the wait
-  // ends as soon as the slowest of the S is done; it is bounded all the same.
+  // ---- arrival.  All CTAs of the grid meet on a counter; once every partial result is visible each CTA
+  // finishes 1/C of the layer's rows, so the split-K reduction is C-way parallel and short.  The grid
+  // never exceeds one CTA per SM, so all of them are resident together and the wait ends as soon as the
+  // slowest is done; it is bounded all the same.
   __threadfence();
   __syncthreads();
   if (tid == 0) {
     int ok = 1;
-    if (a.S > 1) {
-      atomicAdd(&a.counters[r], 1);
+    if (C > 1) {
+      atomicAdd(&a.counters[0], 1);
       const unsigned long long t0 = gtimer();
-      while (*((volatile int*)&a.counters[r]) < a.S) {
+      while (*((volatile int*)&a.counters[0]) < C) {
         __nanosleep(100);
         if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); ok = 0; break; }
       }
@@ -624,18 +673,20 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   if (!s_flag) return;
   __threadfence();
   {
-    // slice s of the range, cut on multiples of 4 rows
-    const int quads = (nrows + 3) >> 2;
-    const int q0 = (int)(((long long)s * quads) / a.S), q1 = (int)(((long long)(s + 1) * quads) / a.S);
-    const int b0 = min(q0 * 4, nrows), b1 = min(q1 * 4, nrows);
-    lin_epilogue_slice(a, r * a.S + s, row_begin + b0, b1 - b0, reinterpret_cast<float*>(smem2 + LIN2_HDR_BYTES));
+    // slice `cta` of the rows, cut on multiples of 4
+    const int quads = (a.N + 3) >> 2;
+    const int q0 = (int)(((long long)cta * quads) / C), q1 = (int)(((long long)(cta + 1) * quads) / C);
+    const int b0 = min(q0 * 4, a.N), b1 = min(q1 * 4, a.N);
+    lin_epilogue_slice(a, cta, b0, b1 - b0, reinterpret_cast<float*>(smem2 + LIN2_HDR_BYTES),
+                       (int)((xbytes + (uint32_t)NS * STAGE) / sizeof(float)), reinterpret_cast<float*>(smem2 + 576));
   }
-  if (a.S > 1) {
-    // departure: the last CTA to leave re-arms the counters for the next launch
-    __syncthreads();
-    if (tid == 0 && atomicAdd(&a.counters[LIN_MAX_R + r], 1) == a.S - 1) {
-      a.counters[r] = 0;
-      a.counters[LIN_MAX_R + r] = 0;
+  // departure: the last CTA to leave re-arms the counters and the tile queues for the next launch
+  __syncthreads();
+  if (tid == 0) {
+    if (C == 1 || atomicAdd(&a.counters[1], 1) == C - 1) {
+      a.counters[0] = 0;
+      a.counters[1] = 0;
+      for (int i = 0; i < a.S; ++i) a.counters[2 + i] = 0;
     }
   }
 }
@@ -734,7 +785,13 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     return e ? atoi(e) : 2;
   }();
   p.variant = variant;
-  if (variant == 2) {
+  {
+    // more k-splits than the TMA kernel has tile queues (D = 128 x a large prime): register-streaming kernel
+    int ks = 128;
+    for (int k = 128; k <= ((p.NT == 1) ? 2048 : 1024) && k <= D; k += 128) if (D % k == 0) ks = k;
+    if (D / ks > LIN_MAX_S) p.variant = 1;
+  }
+  if (p.variant == 2) {
     // bulk-copy variant: KS = largest multiple of 128 dividing D up to the slab budget
     static const int ks_env = [] { const char* e = getenv("SPS_LIN_KSMAX"); return e ? atoi(e) : 0; }();
     int ks_max = (p.NT == 1) ? 2048 : 1024;
