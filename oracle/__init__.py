@@ -193,6 +193,8 @@ class Model:
         tok = _i32(tokens)
         pos = _i32(positions)
         M = tok.shape[0]
+        if pos.shape[0] != M:
+            raise ValueError("tokens and positions differ in length")
         out = np.zeros((M, self.V), dtype=np.float32) if want_logits else None
         lib().orc_model_forward(self._h, _p(tok), _p(pos), M, _p(out))
         return out
@@ -249,6 +251,8 @@ class Transformer(Model):
 
     def forward64(self, tokens, positions):
         tok, pos = _i32(tokens), _i32(positions)
+        if pos.shape[0] != tok.shape[0]:
+            raise ValueError("tokens and positions differ in length")
         out = np.zeros((tok.shape[0], self.V), dtype=np.float64)
         lib().orc_model_forward64(self._h, _p(tok), _p(pos), tok.shape[0], _p(out))
         return out

@@ -75,8 +75,8 @@ cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st) {
 // kernel waits for its predecessor: old cache rows do not depend on it.  The rows of this pass (rotary
 // applied, rounded to the storage type, appended to the cache) are patched into the tile from shared
 // memory, so the tile never depends on reading back what this CTA just wrote.  Per tile: scores with
-// one thread per (position, row group), running max / sum per row (online softmax), then P.V with one
-// thread per (dim, position group).  Loops over rows are the only unrolled ones: the code stays small
+// one warp per position (lanes split the dims), running max / sum per row (online softmax), then P.V
+// with one thread per (pair of dims, position group).  Loops over rows are the only unrolled ones: the code stays small
 // enough for the instruction cache, which is what a kernel that runs for microseconds lives or dies by.
 // ------------------------------------------------------------------------------------------------
 #define ATTN_THREADS 512
@@ -128,11 +128,9 @@ __device__ __forceinline__ int row_position(const AttnArgs& a, int b, int i) {
 template <int DH, typename CT, int MR>
 __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   constexpr int TP = ATTN_TILE_BYTES / (DH * (int)sizeof(CT));   // positions per tile
-  constexpr int SG = ATTN_THREADS / TP;                          // row groups in the score phase (1, 2 or 4)
-  constexpr int RPG = (MR + SG - 1) / SG;                        // rows per score thread
-  constexpr int PG = ATTN_THREADS / DH;                          // position groups in the P.V phase (2 or 4)
-  constexpr int VEC = 16 / (int)sizeof(CT);                      // elements per 128-bit chunk
-  constexpr int NCH = DH / VEC;                                  // chunks per row
+  constexpr int DPL = DH / 32;                                   // dims per lane in the score phase (4 or 2)
+  constexpr int PG = ATTN_THREADS / (DH / 2);                    // position groups in the P.V phase (8 or 16)
+  constexpr int LOG_MR = MR == 2 ? 1 : (MR == 8 ? 3 : 4);
   extern __shared__ __align__(128) unsigned char asm_[];
   CT* Ks = reinterpret_cast<CT*>(asm_);                          // [TP][DH]
   CT* Vs = Ks + TP * DH;                                         // [TP][DH]
@@ -225,10 +223,11 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   }
   for (int idx = tid; idx < (MR - Mb) * DH; idx += ATTN_THREADS) q_s[Mb * DH + idx] = 0.f;
 
-  float o[MR];   // P.V accumulators: this thread's dim, its position group
+  float o[MR][2];   // P.V accumulators: this thread's pair of dims, its position group
 #pragma unroll
-  for (int i = 0; i < MR; ++i) o[i] = 0.f;
-  const int dim = tid % DH, pg = tid / DH;
+  for (int i = 0; i < MR; ++i) o[i][0] = o[i][1] = 0.f;
+  const int dp = tid % (DH / 2), pg = tid / (DH / 2);
+  float qreg[MR][DPL];   // this lane's dims of every query row (score phase)
   bool ok = true;
   int phase = 0;
   for (int t0 = 0; t0 < n_ctx; t0 += TP, phase ^= 1) {
@@ -241,53 +240,44 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
       const int j = pos_s[i] - t0;
       if (j >= 0 && j < TP) { Ks[j * DH + e] = knew[idx]; Vs[j * DH + e] = vnew[idx]; }
     }
+    if (t0 == 0) {
+#pragma unroll
+      for (int i = 0; i < MR; ++i)
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) qreg[i][e] = q_s[i * DH + lane * DPL + e];
+    }
     __syncthreads();
-    // ---- scores: thread = (position j, row group sg); chunks are visited in a per-position rotated
-    // order so that neighbouring positions hit different banks
-    {
-      const int j = tid % TP, sg = tid / TP;
-      if (j < tn) {
-        float acc[RPG];
+    // ---- scores: a warp takes one position at a time, its lanes split the head's dims (the key row is
+    // read as one contiguous 32-lane access); the MR partial dot products are summed across lanes with
+    // a folding butterfly that halves the values a lane carries at every step.
+    for (int j = warp; j < tn; j += ATTN_WARPS) {
+      float kf[DPL];
+      const CT* kr = Ks + j * DH + lane * DPL;
 #pragma unroll
-        for (int r = 0; r < RPG; ++r) acc[r] = 0.f;
-        const CT* kr = Ks + j * DH;
-#pragma unroll 2
-        for (int c = 0; c < NCH; ++c) {
-          const int cc = (c + j) % NCH;
-          const uint4 raw = *reinterpret_cast<const uint4*>(kr + cc * VEC);
-          float kv[VEC];
-          if (sizeof(CT) == 2) {
-            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+      for (int e = 0; e < DPL; ++e) kf[e] = ct_to_f<CT>(kr[e]);
+      float v[MR];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              kv[2 * e] = __uint_as_float(w[e] << 16);
-              kv[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-            }
-          } else {
-            kv[0] = __uint_as_float(raw.x); kv[1] = __uint_as_float(raw.y);
-            kv[2] = __uint_as_float(raw.z); kv[3] = __uint_as_float(raw.w);
-          }
+      for (int i = 0; i < MR; ++i) {
+        float t = 0.f;
 #pragma unroll
-          for (int r = 0; r < RPG; ++r) {
-            const int i = sg * RPG + r;
-            if (i < MR) {
-              const float* qp = q_s + i * DH + cc * VEC;
-              const float4 qa = *reinterpret_cast<const float4*>(qp);
-              float t = kv[0] * qa.x + kv[1] * qa.y + kv[2] * qa.z + kv[3] * qa.w;
-              if (VEC == 8) {
-                const float4 qb = *reinterpret_cast<const float4*>(qp + 4);
-                t += kv[VEC - 4] * qb.x + kv[VEC - 3] * qb.y + kv[VEC - 2] * qb.z + kv[VEC - 1] * qb.w;
-              }
-              acc[r] += t;
-            }
-          }
-        }
+        for (int e = 0; e < DPL; ++e) t += kf[e] * qreg[i][e];
+        v[i] = t;
+      }
+      int off = 16;
 #pragma unroll
-        for (int r = 0; r < RPG; ++r) {
-          const int i = sg * RPG + r;
-          if (i < Mb) sc[i * TP + j] = (t0 + j <= pos_s[i]) ? acc[r] : -INFINITY;
+      for (int w = MR / 2; w >= 1; w >>= 1, off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int k = 0; k < w; ++k) {
+          const float send = upper ? v[k] : v[k + w];
+          const float keep = upper ? v[k + w] : v[k];
+          v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
         }
       }
+#pragma unroll
+      for (int o2 = 16 >> LOG_MR; o2 >= 1; o2 >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], o2);
+      const int i = lane >> (5 - LOG_MR);   // the row whose sum this lane ended up with
+      if ((lane & ((32 >> LOG_MR) - 1)) == 0 && i < Mb) sc[i * TP + j] = (t0 + j <= pos_s[i]) ? v[0] : -INFINITY;
     }
     __syncthreads();
     // ---- online softmax: warp per row
@@ -313,20 +303,27 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
       }
     }
     __syncthreads();
-    // ---- o = alpha * o + sum_j p_j v_j: thread = (dim, position group)
+    // ---- o = alpha * o + sum_j p_j v_j: thread = (pair of dims, position group)
 #pragma unroll
-    for (int i = 0; i < MR; ++i) if (i < Mb) o[i] *= row_a[i];
-#pragma unroll 2
+    for (int i = 0; i < MR; ++i) if (i < Mb) { o[i][0] *= row_a[i]; o[i][1] *= row_a[i]; }
+#pragma unroll 4
     for (int j = pg; j < tn; j += PG) {
-      const float v = ct_to_f<CT>(Vs[j * DH + dim]);
+      const float v0 = ct_to_f<CT>(Vs[j * DH + 2 * dp]), v1 = ct_to_f<CT>(Vs[j * DH + 2 * dp + 1]);
 #pragma unroll
-      for (int i = 0; i < MR; ++i) if (i < Mb) o[i] += sc[i * TP + j] * v;
+      for (int i = 0; i < MR; ++i) {
+        if (i < Mb) {
+          const float p = sc[i * TP + j];
+          o[i][0] += p * v0;
+          o[i][1] += p * v1;
+        }
+      }
     }
     __syncthreads();   // the tile buffers and sc are free again
     if (tid == 0 && t0 + TP < n_ctx) issue_tile(t0 + TP, t0 + TP);
   }
 #pragma unroll
-  for (int i = 0; i < MR; ++i) if (i < Mb) red[(pg * MR + i) * DH + dim] = o[i];
+  for (int i = 0; i < MR; ++i)
+    if (i < Mb) { red[(pg * MR + i) * DH + 2 * dp] = o[i][0]; red[(pg * MR + i) * DH + 2 * dp + 1] = o[i][1]; }
   __syncthreads();
   for (int idx = tid; idx < Mb * DH; idx += ATTN_THREADS) {
     const int i = idx / DH, e = idx - i * DH;
@@ -340,7 +337,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
 template <int DH, typename CT, int MR>
 static size_t attn_smem_t() {
   constexpr int TP = ATTN_TILE_BYTES / (DH * (int)sizeof(CT));
-  constexpr int PG = ATTN_THREADS / DH;
+  constexpr int PG = ATTN_THREADS / (DH / 2);
   return 2 * (size_t)ATTN_TILE_BYTES + 2 * (size_t)MR * DH * sizeof(CT) + sizeof(float) * ((size_t)MR * DH + (size_t)MR * TP + (size_t)PG * MR * DH + 3 * MR) +
          sizeof(int) * MR + 16;
 }
