@@ -1,0 +1,54 @@
+"""Parity at the bench's full layer shapes: the 70B-shaped target (d 8192, FFN 32768, 64 heads, V 32000) and
+the 4B-shaped draft (d 6144, FFN 24576, 48 heads) with a reduced layer count, so that every kernel runs
+in exactly the launch configuration `bench.py` times (same grids, k-splits and tile queues), and the
+oracle -- fed the very weights read back from the device, one layer at a time -- finishes in seconds.
+Tolerance: bf16 models, logits within 5e-2 abs (the benchmark spec); observed error is ~1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2302_01318_b200 as sps
+import sps_synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def oracle_logits(cfg, w_dev, tokens, positions_ctx, rows):
+    """prefix tokens at positions 0..len-1 go through the oracle layer by layer together with `rows`"""
+    seq = np.concatenate([tokens, rows]).astype(np.int32)
+    pos = np.arange(len(seq), dtype=np.int32)
+    m = oracle.Transformer(cfg, None, len(seq) + 1)
+    emb = sps_synth.to_numpy(w_dev["tok_embed"][torch.from_numpy(seq.astype(np.int64)).to(DEV)])
+    m.begin_rows(emb, pos)
+    for l, lw in enumerate(w_dev["layers"]):
+        m.layer(l, {k: sps_synth.to_numpy(v) for k, v in lw.items()})
+    out = m.end(sps_synth.to_numpy(w_dev["final_norm"]), sps_synth.to_numpy(w_dev["unembed"]))
+    return out[len(tokens):]
+
+
+def test_scoring_pass_at_70b_layer_shapes():
+    c = sps_synth.CONFIGS["70b"]
+    tc, dc = dict(c["target"], n_layers=2), dict(c["draft"], n_layers=1)
+    wt = sps_synth.make_weights(tc, tag="target", device=DEV)
+    wd = sps_synth.make_weights(dc, tag="draft", device=DEV, share_embed_from=wt)
+    h = sps.Handle(tc, wt, dc, wd, max_seq=64, max_K=4)
+    V = tc["vocab"]
+    prompt = sps_synth.make_prompt(0, 20, V)
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(1, 4, V)])
+    h.sps_prefill(prompt)
+    out = torch.zeros((5, V), device=DEV)
+    worst = {}
+    for which, cfg, w in ((0, tc, wt), (1, dc, wd)):
+        h.sps_score(which, rows, out)
+        got = out.cpu().numpy().astype(np.float64)
+        want = oracle_logits(cfg, w, prompt[:-1], None, rows)
+        worst[which] = float(np.abs(got - want).max())
+        assert np.isfinite(got).all()
+        assert worst[which] < 5e-2, worst
+    print("worst logit error target / draft:", worst)
+    # the whole loop runs at these shapes and keeps its invariants
+    toks, st = h.sps_generate(prompt, 12, 4, 1.0, 3)
+    assert ((toks >= 0) & (toks < V)).all() and st["loops"] == sum(st["hist_emitted"]) and st["emitted"] - st["overshoot"] == 12
+    h.close()
