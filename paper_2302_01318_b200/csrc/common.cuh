@@ -157,7 +157,6 @@ struct LinArgs {
   int PR;                 // rows per shared-memory pass (multiple of 32)      [register-streaming variant]
   int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
   int* err;               // sticky error word: set to 3 if a bounded wait ran out
-  int dbg;                // experiments only: bit 0 = consumers skip the arithmetic
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };

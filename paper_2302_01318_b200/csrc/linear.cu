@@ -113,54 +113,68 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
   if (tid == 0) a.counters[r] = 0;
 }
 
-// Epilogue of the TMA variant.  Every CTA of a split finishes one slice of the range's rows once all
-// S partial results are in: output elements (m, n) go to threads in m-major order (neighbouring
-// threads, neighbouring n), and a thread fetches all the partials it needs before it adds them in
-// split order -- the loads are independent, the latency is paid once.  sq_s: shared scratch (sq_cap
-// floats; the slice is walked in chunks that fit) for the squares of a residual update, summed per row
-// m in index order afterwards; ssq_s: 16 shared floats that carry the per-row sums across chunks.
+// Epilogue of the TMA variant.  Every CTA of the grid finishes one slice of the layer's output columns
+// once all S partial results are in.  Output elements (m, n..n+3) go to threads in m-major order
+// (neighbouring threads, neighbouring n), and a thread has all the partials it needs in flight before it
+// adds them in split order: a slice costs one trip to L2.  sq_s: shared scratch (sq_cap floats; the
+// slice is walked in chunks that fit) for the squares of a residual update, summed per row m in index
+// order afterwards; ssq_s: 16 shared floats that carry the per-row sums across chunks.
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
 __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, int rows_all, float* sq_s, int sq_cap,
                                    float* ssq_s) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   const int S = a.S, N = a.N;
   const bool resid = a.epi == EPI_RESIDUAL;
-  int chunk_rows = sq_cap / a.M;
-  if (chunk_rows > rows_all) chunk_rows = rows_all;
-  if (chunk_rows < 1) chunk_rows = 1;
   if (resid) {
     if (tid < SPS_MAX_ROWS) ssq_s[tid] = 0.f;
     __syncthreads();
   }
-  for (int c0 = 0; c0 < rows_all; c0 += chunk_rows) {
-    const int rows = min(chunk_rows, rows_all - c0), n_begin = n_first + c0, total = rows * a.M;
-    if (S <= 4) {
-      for (int e0 = tid; e0 < total; e0 += 4 * nthr) {
-        float v[4][4], old[4];
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int e = e0 + b * nthr;
-          const int m = e < total ? e / rows : 0, n = n_begin + (e < total ? e - m * rows : 0);
+  const bool vec = (((N | n_first | rows_all) & 3) == 0) && ((a.ldy & 3) == 0) &&
+                   ((((size_t)a.Y | (size_t)a.part) & 15) == 0);
+  const int unit = vec ? 4 : 1;                       // columns per work item
+  const int items_all = rows_all / unit;
+  int chunk_items = sq_cap / a.M;
+  if (chunk_items > items_all) chunk_items = items_all;
+  if (chunk_items < 1) chunk_items = 1;
+  for (int c0 = 0; c0 < items_all; c0 += chunk_items) {
+    const int items = min(chunk_items, items_all - c0), n_begin = n_first + c0 * unit, total = items * a.M;
+    if (vec) {
+      for (int e = tid; e < total; e += nthr) {
+        const int m = e / items, n = n_begin + 4 * (e - m * items);
+        float* dst = a.Y + (long long)m * a.ldy + n;
+        const float* src = a.part + (size_t)m * N + n;
+        const size_t sstride = (size_t)SPS_MAX_ROWS * N;
+        float4 old = make_float4(0.f, 0.f, 0.f, 0.f), y;
+        if (resid) old = __ldcg(reinterpret_cast<const float4*>(dst));
+        if (S <= 4) {
+          float4 v[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            v[b][j] = (e < total && j < S) ? __ldcg(a.part + ((size_t)j * SPS_MAX_ROWS + m) * N + n) : 0.f;
-          old[b] = (e < total && resid) ? a.Y[(long long)m * a.ldy + n] : 0.f;
-        }
+            v[j] = j < S ? __ldcg(reinterpret_cast<const float4*>(src + j * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          y = f4_add(f4_add(f4_add(v[0], v[1]), v[2]), v[3]);
+        } else {
+          y = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int s0 = 0; s0 < S; s0 += 8) {
+            float4 v[8];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int e = e0 + b * nthr;
-          if (e < total) {
-            const int m = e / rows, n = n_begin + (e - m * rows);
-            float y = ((v[b][0] + v[b][1]) + v[b][2]) + v[b][3];
-            if (resid) { y += old[b]; sq_s[e] = y * y; }
-            a.Y[(long long)m * a.ldy + n] = y;
+            for (int j = 0; j < 8; ++j)
+              v[j] = s0 + j < S ? __ldcg(reinterpret_cast<const float4*>(src + (s0 + j) * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
           }
         }
+        if (resid) {
+          y = f4_add(y, old);
+          sq_s[e] = ((y.x * y.x + y.y * y.y) + y.z * y.z) + y.w * y.w;
+        }
+        *reinterpret_cast<float4*>(dst) = y;
       }
     } else {
       for (int e = tid; e < total; e += nthr) {
-        const int m = e / rows, n = n_begin + (e - m * rows);
+        const int m = e / items, n = n_begin + (e - m * items);
         float y = 0.f;
-        const float old = resid ? a.Y[(long long)m * a.ldy + n] : 0.f;
+        const float old = resid ? __ldcg(a.Y + (long long)m * a.ldy + n) : 0.f;
         for (int s0 = 0; s0 < S; s0 += 16) {
           float v[16];
 #pragma unroll
@@ -176,7 +190,7 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
       __syncthreads();
       for (int m = warp; m < a.M; m += nwarp) {   // row m always falls to the same warp: no race on ssq_s[m]
         float t = 0.f;
-        for (int i = lane; i < rows; i += 32) t += sq_s[m * rows + i];
+        for (int i = lane; i < items; i += 32) t += sq_s[m * items + i];
         t = warp_sum(t);
         if (lane == 0) ssq_s[m] += t;
       }
@@ -486,55 +500,66 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // Weights never change, so the producer is already streaming; X is the predecessor's output.
     pdl_wait();
     {
-      if (a.pro == PRO_RMSNORM) {
-        // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
-        for (int m = warp; m < a.M; m += NCW) {
-          const int srow = a.x_row0 + m * a.x_rowstep;
-          float t = 0.f;
-          for (int i = lane; i < a.ssq_in_n; i += 32) t += a.ssq_in[(size_t)i * SPS_MAX_ROWS + srow];
-          t = warp_sum(t);
-          if (lane == 0) s_scale[m] = rsqrtf(t / (float)D + a.eps);
-        }
-        asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
-      }
-      // a thread owns 8 consecutive k of every row: all rows' loads are issued before any is used
-      const int groups = KS >> 3;
-      for (int kg = tid; kg < groups; kg += NCW * 32) {
-        float4 v0[NT * 8], v1[NT * 8];
+      // A thread owns 4 consecutive k (one 16-byte load per row, neighbouring lanes neighbouring addresses)
+      // of up to two places of the k-range, eight rows at a time; all those loads are in flight before the
+      // partial sums of squares of the norm are fetched, so the slab costs one trip to L2, not two.
+      const int nchunk = KS >> 2;
+      float4 gg[2];
+      gg[0] = gg[1] = make_float4(1.f, 1.f, 1.f, 1.f);
 #pragma unroll
-        for (int m = 0; m < NT * 8; ++m) {
-          if (m < a.M) {
-            const float* src = a.X + (size_t)(a.x_row0 + m * a.x_rowstep) * a.ldx + k_base + kg * 8;
-            v0[m] = *reinterpret_cast<const float4*>(src);
-            v1[m] = *reinterpret_cast<const float4*>(src + 4);
-          }
-        }
-        float gg[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
-        if (a.pro == PRO_RMSNORM) {
-          const float4 g0 = *reinterpret_cast<const float4*>(a.gain + k_base + kg * 8);
-          const float4 g1 = *reinterpret_cast<const float4*>(a.gain + k_base + kg * 8 + 4);
-          gg[0] = g0.x; gg[1] = g0.y; gg[2] = g0.z; gg[3] = g0.w; gg[4] = g1.x; gg[5] = g1.y; gg[6] = g1.z; gg[7] = g1.w;
-        }
+      for (int h = 0; h < NT; ++h) {
+        float4 v[2][8];
 #pragma unroll
-        for (int m = 0; m < NT * 8; ++m) {
-          uint4 hi = make_uint4(0u, 0u, 0u, 0u), lo = hi;
-          if (m < a.M) {
-            float v[8] = {v0[m].x, v0[m].y, v0[m].z, v0[m].w, v1[m].x, v1[m].y, v1[m].z, v1[m].w};
-            if (a.pro == PRO_RMSNORM) {
-              const float scale = s_scale[m];
+        for (int i = 0; i < 2; ++i) {
+          const int c = tid + i * (NCW * 32);
+          if (c < nchunk) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = gg[i] * v[i] * scale;
-            } else if (a.pro == PRO_GELU) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = gelu_tanh(v[i]);
+            for (int mm = 0; mm < 8; ++mm) {
+              const int m = h * 8 + mm;
+              if (m < a.M)
+                v[i][mm] = *reinterpret_cast<const float4*>(a.X + (size_t)(a.x_row0 + m * a.x_rowstep) * a.ldx + k_base + 4 * c);
             }
-            split_pack(v[0], v[1], hi.x, lo.x);
-            split_pack(v[2], v[3], hi.y, lo.y);
-            split_pack(v[4], v[5], hi.z, lo.z);
-            split_pack(v[6], v[7], hi.w, lo.w);
           }
-          *reinterpret_cast<uint4*>(xs_hi_p + (size_t)m * XP + kg * 16) = hi;
-          *reinterpret_cast<uint4*>(xs_lo_p + (size_t)m * XP + kg * 16) = lo;
+        }
+        if (h == 0 && a.pro == PRO_RMSNORM) {
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int c = tid + i * (NCW * 32);
+            if (c < nchunk) gg[i] = *reinterpret_cast<const float4*>(a.gain + k_base + 4 * c);
+          }
+          // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
+          for (int m = warp; m < a.M; m += NCW) {
+            const int srow = a.x_row0 + m * a.x_rowstep;
+            float tt = 0.f;
+            for (int i = lane; i < a.ssq_in_n; i += 32) tt += a.ssq_in[(size_t)i * SPS_MAX_ROWS + srow];
+            tt = warp_sum(tt);
+            if (lane == 0) s_scale[m] = rsqrtf(tt / (float)D + a.eps);
+          }
+          asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int c = tid + i * (NCW * 32);
+          if (c < nchunk) {
+#pragma unroll
+            for (int mm = 0; mm < 8; ++mm) {
+              const int m = h * 8 + mm;
+              uint2 hi = make_uint2(0u, 0u), lo = hi;
+              if (m < a.M) {
+                float4 x = v[i][mm];
+                if (a.pro == PRO_RMSNORM) {
+                  const float scale = s_scale[m];
+                  x.x = gg[i].x * x.x * scale; x.y = gg[i].y * x.y * scale; x.z = gg[i].z * x.z * scale; x.w = gg[i].w * x.w * scale;
+                } else if (a.pro == PRO_GELU) {
+                  x.x = gelu_tanh(x.x); x.y = gelu_tanh(x.y); x.z = gelu_tanh(x.z); x.w = gelu_tanh(x.w);
+                }
+                split_pack(x.x, x.y, hi.x, lo.x);
+                split_pack(x.z, x.w, hi.y, lo.y);
+              }
+              *reinterpret_cast<uint2*>(xs_hi_p + (size_t)m * XP + c * 8) = hi;
+              *reinterpret_cast<uint2*>(xs_lo_p + (size_t)m * XP + c * 8) = lo;
+            }
+          }
         }
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
@@ -558,9 +583,9 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           const int tot = s_total;
           if (tot >= 0 && L >= tot) { done = true; break; }
           __nanosleep(32);
-          if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); s_abort = 1; done = true; break; }
+          if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); s_abort = 1; alive = false; break; }
         }
-        if (done) break;
+        if (done) break;   // every warp of the group sees the same numbers and leaves here together
       }
       const int tile = tile_ids[L & 63];
       float acc[NT][4][4];
@@ -568,7 +593,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[nt][c][0] = acc[nt][c][1] = acc[nt][c][2] = acc[nt][c][3] = 0.f;
-      for (int ks = rank; ks < KSUB; ks += G) {
+      for (int ks = rank; ks < KSUB && alive; ks += G) {
         const int it = L * KSUB + ks, slot = it % NS, use = it / NS;
         if (use > 0 && consumed[slot] < use) {
           const unsigned long long t0 = gtimer();
@@ -582,7 +607,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         const uint32_t wrow = ring + slot * STAGE + g * 128;          // row g of slab 0; row g+8 is +1024
         const uint32_t xoff = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 32;  // logical chunk 2t of this stage's k-range
         const uint32_t xh_addr = xs_hi + g * XP + xoff, xl_addr = xs_lo + g * XP + xoff;
-        const int slabs = (a.dbg & 1) ? 0 : (KST >> 6);
+        const int slabs = KST >> 6;
 #pragma unroll 2
         for (int q = 0; q < slabs; ++q) {
 #pragma unroll
@@ -655,23 +680,25 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   // finishes 1/C of the layer's rows, so the split-K reduction is C-way parallel and short.  The grid
   // never exceeds one CTA per SM, so all of them are resident together and the wait ends as soon as the
   // slowest is done; it is bounded all the same.
-  __threadfence();
   __syncthreads();
   if (tid == 0) {
-    int ok = 1;
-    if (C > 1) {
+    // one fence for the whole CTA: the barrier above orders every thread's stores before it
+    int ok = (*((volatile int*)&s_abort) == 0);
+    if (ok && C > 1) {
+      __threadfence();
       atomicAdd(&a.counters[0], 1);
       const unsigned long long t0 = gtimer();
       while (*((volatile int*)&a.counters[0]) < C) {
-        __nanosleep(100);
+        __nanosleep(64);
+        if (*((volatile int*)a.err) == 3) { ok = 0; break; }   // another CTA gave up: so do we
         if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); ok = 0; break; }
       }
+      __threadfence();
     }
     s_flag = ok;
   }
   __syncthreads();
   if (!s_flag) return;
-  __threadfence();
   {
     // slice `cta` of the rows, cut on multiples of 4
     const int quads = (a.N + 3) >> 2;
@@ -895,8 +922,6 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   LinArgs a = a_in;
   a.R = p.R; a.S = p.S; a.WC = p.WC; a.PR = p.PR; a.KS = p.KS; a.KST = p.KST; a.NS = p.NS; a.G = p.G;
   if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
-  static const int dbg_env = [] { const char* e = getenv("SPS_LIN_DBG"); return e ? atoi(e) : 0; }();
-  a.dbg = dbg_env;
   static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
   cudaError_t e;
   if (dtype == 0) {
