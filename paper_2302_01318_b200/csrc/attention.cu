@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a) {
   if (tid == 0) {
     float t = 0.f;
     for (int w = 0; w < 8; ++w) t += s_part[w];
-    a.ssq[row] = t;
+    a.ssq[SSQ_IDX(0, row)] = t;
   }
 }
 

@@ -143,13 +143,13 @@ struct LinArgs {
   int ldx, x_row0, x_rowstep;
   int pro;                // PRO_*
   const float* gain;      // [D] fp32 (PRO_RMSNORM)
-  const float* ssq_in;    // [ssq_in_n][16] partial sums of squares of each X row (PRO_RMSNORM)
+  const float* ssq_in;    // partial sums of squares of each X row (PRO_RMSNORM): SSQ_IDX(part, row), part < ssq_in_n
   int ssq_in_n;
   float eps;
   int epi;                // EPI_*
   float* Y;               // EPI_STORE: Y[m*ldy + n] = y.  EPI_RESIDUAL: Y[m*ldy + n] += y
   long long ldy;
-  float* ssq_out;         // EPI_RESIDUAL: [R][16] per-range sums over n of the updated Y[m][n]^2
+  float* ssq_out;         // EPI_RESIDUAL: SSQ_IDX(part, m) = one CTA's share of the sum over n of the updated Y[m][n]^2
   // scratch (owned by the handle / caller): split-K partials and arrival counters
   float* part;            // [S][SPS_MAX_ROWS][N]
   int* counters;          // [2 * LIN_MAX_R + 2], zero between launches (the kernel re-zeroes what it used)
@@ -157,6 +157,17 @@ struct LinArgs {
   int PR;                 // rows per shared-memory pass (multiple of 32)      [register-streaming variant]
   int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
   int* err;               // sticky error word: set to 3 if a bounded wait ran out
+  // Packed activations (bf16 TMA kernel only).  A layer may leave, beside Y, the next layer's input ready
+  // for the tensor cores: act(y) * gain split into a bf16 high part and a bf16 remainder.  A layer given
+  // such an input copies it into shared memory instead of converting X; with PRO_RMSNORM the gain is
+  // already in it and the row's 1/rms (from ssq_in) multiplies the output instead of the input.
+  const __nv_bfloat16* xp_hi;   // [*][ldx] packed input (row = x_row0 + m * x_rowstep), null = convert X
+  const __nv_bfloat16* xp_lo;
+  __nv_bfloat16* yp_hi;         // [M][ldyp] packed copy of the output, null = none
+  __nv_bfloat16* yp_lo;
+  long long ldyp;
+  const float* yp_gain;         // [N] multiplied in before packing, null = ones
+  int yp_act;                   // PRO_GELU: gelu before packing; PRO_NONE: none
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };
@@ -165,6 +176,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream
 size_t lin_part_floats(int N, int S_max);
 void sps_set_global_error(const char* msg);   // text returned by sps_last_error(NULL)
 #define LIN_MAX_R 512
+// partial sums of squares: the partials of one row are neighbours, so a warp fetches them with a few coalesced loads
+#define SSQ_IDX(part, row) ((size_t)(row) * LIN_MAX_R + (size_t)(part))
 #define LIN_CONSUMER_WARPS 8
 #define LIN_MAX_S 64
 
@@ -177,7 +190,7 @@ struct EmbedArgs {
   int dtype, d, V;
   int mode, t, K, c0, rows_per_seq, B;
   float* x;               // [rows][d] fp32 residual stream
-  float* ssq;             // [1][16]: one partial per row
+  float* ssq;             // SSQ_IDX(0, row): one partial per row
 };
 cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st);
 

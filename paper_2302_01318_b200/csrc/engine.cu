@@ -25,6 +25,7 @@ struct ModelDev {
   char* vcache = nullptr;
   size_t layer_bytes = 0;
   float2* rope = nullptr;  // [max_seq][dh/2]
+  bool packed = false;     // every linear layer of this model runs on the bf16 TMA kernel: activations travel packed
 };
 
 struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uint64_t seed; };
@@ -42,6 +43,7 @@ struct sps_handle {
   DevState hst{};          // host image of the device state block
   DevState* dst = nullptr;
   float *x = nullptr, *qkv = nullptr, *attn = nullptr, *up = nullptr, *ssqA = nullptr, *ssqB = nullptr;
+  __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
   int32_t* res = nullptr;    // device: [n_acc B][flags B][out_tok B*(maxK+1)][err 1]
@@ -144,6 +146,18 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
   return need;
 }
 
+// packed activations need every shape of the model, at every row count, on the TMA kernel
+bool model_can_pack(const ModelDev& m, int num_sm) {
+  const sps_model_cfg& c = m.cfg;
+  if (!m.present || c.dtype != 1) return false;
+  const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  for (int M : {1, SPS_MAX_ROWS})
+    for (auto& s : shapes)
+      if (lin_plan(c.dtype, M, s[0], s[1], num_sm).variant != 2) return false;
+  static const bool off = [] { const char* e = getenv("SPS_LIN_PACKED"); return e && atoi(e) == 0; }();   // tuning: 0 = convert in every layer
+  return !off;
+}
+
 struct PassSpec {
   int mode, t, K, c0, rows_per_seq;
   float* logits;        // null: skip the unembedding
@@ -172,6 +186,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.rows_per_mat = d; a.N = 3 * d; a.D = d; a.M = rows;
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
+      if (m.packed && l > 0) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }   // left there by the layer below
       a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = 3 * d;
       CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
     }
@@ -189,6 +204,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = d; a.M = rows;
       a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
+      if (m.packed) { a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_gain = (const float*)m.ffn_norm[l]; a.yp_act = PRO_NONE; }
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
       nB = pl.ssq_parts;
       CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
@@ -199,6 +215,10 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB; a.ssq_in_n = nB;
       a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
+      if (m.packed) {
+        a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo;
+        a.yp_hi = h->up_hi; a.yp_lo = h->up_lo; a.ldyp = dff; a.yp_gain = nullptr; a.yp_act = PRO_GELU;
+      }
       CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
     }
     {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
@@ -206,6 +226,11 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
       a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
+      if (m.packed) {
+        a.xp_hi = h->up_hi; a.xp_lo = h->up_lo;
+        a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_act = PRO_NONE;
+        a.yp_gain = (const float*)(l + 1 < c.n_layers ? m.attn_norm[l + 1] : m.final_norm);
+      }
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
       nA = pl.ssq_parts;
       CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
@@ -216,6 +241,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
     a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
     a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
+    if (m.packed) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }
     a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
     CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm), st)); h->launches++;
   }
@@ -408,6 +434,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   for (auto& ev : h->ev) if (cudaEventCreate(&ev) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "event creation failed"));
   if ((rc = load_model(h, h->tgt, cfg->target, target_w, cfg->max_seq, cfg->max_batch))) return bail(rc);
   if (draft_w && (rc = load_model(h, h->drf, cfg->draft, draft_w, cfg->max_seq, cfg->max_batch))) return bail(rc);
+  h->tgt.packed = model_can_pack(h->tgt, h->num_sm);
+  h->drf.packed = model_can_pack(h->drf, h->num_sm);
 
   const int V = cfg->target.vocab, maxK = cfg->max_K > 0 ? cfg->max_K : 1, MB = cfg->max_batch;
   int dmax = cfg->target.d_model, fmax = cfg->target.d_ff;
@@ -424,6 +452,10 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->qkv, sizeof(float) * SPS_MAX_ROWS * 3 * (size_t)dmax},
       {(void**)&h->attn, sizeof(float) * SPS_MAX_ROWS * (size_t)dmax},
       {(void**)&h->up, sizeof(float) * SPS_MAX_ROWS * (size_t)fmax},
+      {(void**)&h->xp_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->xp_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->up_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
+      {(void**)&h->up_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
       {(void**)&h->ssqA, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
       {(void**)&h->ssqB, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
       {(void**)&h->q_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
@@ -468,7 +500,7 @@ int sps_destroy(sps_handle* h) {
   for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
   free_model(h->tgt);
   free_model(h->drf);
-  void* bufs[] = {h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
+  void* bufs[] = {h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
                   h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);

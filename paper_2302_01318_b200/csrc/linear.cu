@@ -54,6 +54,13 @@ __device__ __forceinline__ float gelu_tanh(float v) {
   return 0.5f * v * (1.0f + tanhf(0.7978845608028654f * (v + 0.044715f * v * v * v)));
 }
 
+// the same function as v * sigmoid(2u), u = sqrt(2/pi) (v + 0.044715 v^3): one exponential and one division
+// (relative error about 1e-6: far below that of the bf16 weights it is multiplied with)
+__device__ __forceinline__ float gelu_fast(float v) {
+  const float u = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+  return __fdividef(v, 1.0f + __expf(-2.0f * u));
+}
+
 __device__ __forceinline__ const void* pick_mat(const LinArgs& a, int n, int& row_in_mat) {
   const int rpm = a.rows_per_mat;
   if (n < rpm) { row_in_mat = n; return a.W[0]; }
@@ -65,7 +72,7 @@ __device__ __forceinline__ const void* pick_mat(const LinArgs& a, int n, int& ro
 // sum of the partial sums of squares of one X row, in partial order
 __device__ __forceinline__ float ssq_total(const LinArgs& a, int srow) {
   float t = 0.f;
-  for (int i = 0; i < a.ssq_in_n; ++i) t += a.ssq_in[(size_t)i * SPS_MAX_ROWS + srow];
+  for (int i = 0; i < a.ssq_in_n; ++i) t += a.ssq_in[SSQ_IDX(i, srow)];
   return t;
 }
 
@@ -107,7 +114,7 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
     if (tid < a.M) {
       float t = 0.f;
       for (int w = 0; w < nwarp; ++w) t += s_red[w * SPS_MAX_ROWS + tid];
-      a.ssq_out[(size_t)r * SPS_MAX_ROWS + tid] = t;
+      a.ssq_out[SSQ_IDX(r, tid)] = t;
     }
   }
   if (tid == 0) a.counters[r] = 0;
@@ -122,7 +129,7 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
 __device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 
 __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, int rows_all, float* sq_s, int sq_cap,
-                                   float* ssq_s) {
+                                   float* ssq_s, const float* row_scale) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   const int S = a.S, N = a.N;
   const bool resid = a.epi == EPI_RESIDUAL;
@@ -131,7 +138,9 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
     __syncthreads();
   }
   const bool vec = (((N | n_first | rows_all) & 3) == 0) && ((a.ldy & 3) == 0) &&
-                   ((((size_t)a.Y | (size_t)a.part) & 15) == 0);
+                   ((((size_t)a.Y | (size_t)a.part) & 15) == 0) &&
+                   (!a.yp_hi || (((a.ldyp & 3) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 7) == 0) &&
+                                 (!a.yp_gain || (((size_t)a.yp_gain & 15) == 0))));
   const int unit = vec ? 4 : 1;                       // columns per work item
   const int items_all = rows_all / unit;
   int chunk_items = sq_cap / a.M;
@@ -164,11 +173,24 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
             for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
           }
         }
+        if (row_scale) { const float sc = row_scale[m]; y.x *= sc; y.y *= sc; y.z *= sc; y.w *= sc; }
         if (resid) {
           y = f4_add(y, old);
           sq_s[e] = ((y.x * y.x + y.y * y.y) + y.z * y.z) + y.w * y.w;
         }
         *reinterpret_cast<float4*>(dst) = y;
+        if (a.yp_hi) {
+          if (a.yp_act == PRO_GELU) { y.x = gelu_fast(y.x); y.y = gelu_fast(y.y); y.z = gelu_fast(y.z); y.w = gelu_fast(y.w); }
+          if (a.yp_gain) {
+            const float4 gn = __ldg(reinterpret_cast<const float4*>(a.yp_gain + n));
+            y.x *= gn.x; y.y *= gn.y; y.z *= gn.z; y.w *= gn.w;
+          }
+          uint2 hi, lo;
+          split_pack(y.x, y.y, hi.x, lo.x);
+          split_pack(y.z, y.w, hi.y, lo.y);
+          *reinterpret_cast<uint2*>(a.yp_hi + (long long)m * a.ldyp + n) = hi;
+          *reinterpret_cast<uint2*>(a.yp_lo + (long long)m * a.ldyp + n) = lo;
+        }
       }
     } else {
       for (int e = tid; e < total; e += nthr) {
@@ -182,8 +204,16 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
 #pragma unroll
           for (int j = 0; j < 16; ++j) y += v[j];
         }
+        if (row_scale) y *= row_scale[m];
         if (resid) { y += old; sq_s[e] = y * y; }
         a.Y[(long long)m * a.ldy + n] = y;
+        if (a.yp_hi) {
+          if (a.yp_act == PRO_GELU) y = gelu_fast(y);
+          if (a.yp_gain) y *= __ldg(a.yp_gain + n);
+          const __nv_bfloat16 h = __float2bfloat16_rn(y);
+          a.yp_hi[(long long)m * a.ldyp + n] = h;
+          a.yp_lo[(long long)m * a.ldyp + n] = __float2bfloat16_rn(y - __bfloat162float(h));
+        }
       }
     }
     if (resid) {
@@ -197,7 +227,7 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
       __syncthreads();
     }
   }
-  if (resid && tid < a.M) a.ssq_out[(size_t)part_idx * SPS_MAX_ROWS + tid] = ssq_s[tid];
+  if (resid && tid < a.M) a.ssq_out[SSQ_IDX(part_idx, tid)] = ssq_s[tid];
 }
 
 template <int NT>
@@ -397,6 +427,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy)
       : "memory");
 }
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
@@ -432,7 +467,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   const uint32_t XP = (uint32_t)KS * 2 + 16, STAGE = 16u * (uint32_t)KST * 2u;
   const uint32_t xbytes = ((2u * NT * 8u * XP + 1023u) / 1024u) * 1024u;
   const uint32_t sm0 = smem_u32(smem2);
-  const uint32_t bar_full = sm0, bar_empty = sm0 + 8 * NS;
+  const uint32_t bar_full = sm0, bar_empty = sm0 + 8 * NS, bar_x = sm0 + 960;   // bar_x: the packed X slab has landed
   // consumed[slot] = how many times the slot has been read out.  A consumer may look at a slot's
   // "full" barrier only once every earlier use of the slot is over: an mbarrier parity wait cannot
   // tell phase u from phase u-2, and consumer warps run several ring revolutions ahead.
@@ -443,6 +478,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); consumed[i] = 0; }
+    mbar_init(bar_x, 1);
     s_abort = 0;
     s_issued = 0;
     s_total = -1;
@@ -498,14 +534,62 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // ------------------------------------------------------------------ consumer warps
     // X slab: rows 0..8*NT-1 (zeros beyond M), this CTA's k-range, bf16 hi and lo parts, natural k order.
     // Weights never change, so the producer is already streaming; X is the predecessor's output.
+    bool alive = true;
+    if (a.xp_hi) {
+      // Packed input: the slab is a copy.  Rows beyond M are zeroed before the wait on the predecessor;
+      // after it one lane per row asks the copy engine for that row's high and low halves, and everyone
+      // waits for the bytes on one barrier.  With PRO_RMSNORM the rows' 1/rms is worked out meanwhile: the
+      // epilogue multiplies by it.
+      for (int m = a.M + warp; m < NT * 8; m += NCW)
+        for (uint32_t off = lane * 16; off < (uint32_t)KS * 2; off += 512) {
+          *reinterpret_cast<uint4*>(xs_hi_p + (size_t)m * XP + off) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(xs_lo_p + (size_t)m * XP + off) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      if (tid == 0) mbar_expect_tx(bar_x, (uint32_t)a.M * (uint32_t)KS * 4u);
+      pdl_wait();
+      asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
+      for (int m = warp; m < a.M; m += NCW) {
+        if (lane == 0) {
+          const size_t off = (size_t)(a.x_row0 + m * a.x_rowstep) * a.ldx + k_base;
+          bulk_load(xs_hi + m * XP, a.xp_hi + off, (uint32_t)KS * 2u, bar_x);
+          bulk_load(xs_lo + m * XP, a.xp_lo + off, (uint32_t)KS * 2u, bar_x);
+        }
+      }
+      if (a.pro == PRO_RMSNORM) {
+        for (int m = warp; m < a.M; m += NCW) {
+          const int srow = a.x_row0 + m * a.x_rowstep;
+          float pv[LIN_MAX_R / 32];
+#pragma unroll
+          for (int j = 0; j < LIN_MAX_R / 32; ++j) {
+            const int i = lane + 32 * j;
+            pv[j] = i < a.ssq_in_n ? a.ssq_in[SSQ_IDX(i, srow)] : 0.f;
+          }
+          float tt = 0.f;
+#pragma unroll
+          for (int j = 0; j < LIN_MAX_R / 32; ++j) tt += pv[j];
+          tt = warp_sum(tt);
+          if (lane == 0) s_scale[m] = rsqrtf(tt / (float)D + a.eps);
+        }
+      }
+      if (!mbar_wait(bar_x, 0u, a.err)) { alive = false; s_abort = 1; }
+    } else {
+    // A thread owns 4 consecutive k (one 16-byte load per row, neighbouring lanes neighbouring addresses)
+    // of up to two places of the k-range.  The gain of the norm is a weight: it comes from HBM, and is
+    // asked for before the wait on the predecessor.
+    const int nchunk = KS >> 2;
+    float4 gg[2];
+    gg[0] = gg[1] = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (a.pro == PRO_RMSNORM) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int c = tid + i * (NCW * 32);
+        if (c < nchunk) gg[i] = __ldg(reinterpret_cast<const float4*>(a.gain + k_base + 4 * c));
+      }
+    }
     pdl_wait();
     {
-      // A thread owns 4 consecutive k (one 16-byte load per row, neighbouring lanes neighbouring addresses)
-      // of up to two places of the k-range, eight rows at a time; all those loads are in flight before the
-      // partial sums of squares of the norm are fetched, so the slab costs one trip to L2, not two.
-      const int nchunk = KS >> 2;
-      float4 gg[2];
-      gg[0] = gg[1] = make_float4(1.f, 1.f, 1.f, 1.f);
+      // Eight rows at a time; all of a thread's loads are in flight before the partial sums of squares of
+      // the norm are fetched, so the slab costs one trip to L2, not two.
 #pragma unroll
       for (int h = 0; h < NT; ++h) {
         float4 v[2][8];
@@ -522,16 +606,19 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           }
         }
         if (h == 0 && a.pro == PRO_RMSNORM) {
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            const int c = tid + i * (NCW * 32);
-            if (c < nchunk) gg[i] = *reinterpret_cast<const float4*>(a.gain + k_base + 4 * c);
-          }
           // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
           for (int m = warp; m < a.M; m += NCW) {
             const int srow = a.x_row0 + m * a.x_rowstep;
+            // all of a lane's partials are asked for before any is added (up to LIN_MAX_R / 32 of them)
+            float pv[LIN_MAX_R / 32];
+#pragma unroll
+            for (int j = 0; j < LIN_MAX_R / 32; ++j) {
+              const int i = lane + 32 * j;
+              pv[j] = i < a.ssq_in_n ? a.ssq_in[SSQ_IDX(i, srow)] : 0.f;
+            }
             float tt = 0.f;
-            for (int i = lane; i < a.ssq_in_n; i += 32) tt += a.ssq_in[(size_t)i * SPS_MAX_ROWS + srow];
+#pragma unroll
+            for (int j = 0; j < LIN_MAX_R / 32; ++j) tt += pv[j];
             tt = warp_sum(tt);
             if (lane == 0) s_scale[m] = rsqrtf(tt / (float)D + a.eps);
           }
@@ -551,7 +638,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
                   const float scale = s_scale[m];
                   x.x = gg[i].x * x.x * scale; x.y = gg[i].y * x.y * scale; x.z = gg[i].z * x.z * scale; x.w = gg[i].w * x.w * scale;
                 } else if (a.pro == PRO_GELU) {
-                  x.x = gelu_tanh(x.x); x.y = gelu_tanh(x.y); x.z = gelu_tanh(x.z); x.w = gelu_tanh(x.w);
+                  x.x = gelu_fast(x.x); x.y = gelu_fast(x.y); x.z = gelu_fast(x.z); x.w = gelu_fast(x.w);
                 }
                 split_pack(x.x, x.y, hi.x, lo.x);
                 split_pack(x.z, x.w, hi.y, lo.y);
@@ -564,7 +651,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     }
-    bool alive = true;
+    }
     // Consumer warps work in groups of G: a tile goes to group (tile % NG) and its stage ks to warp
     // (ks % G) of the group, so that up to NCW warps chew on the ring at once; the G partial tiles meet
     // in a small shared scratch (double-buffered by tile parity, one group barrier per tile).
@@ -705,7 +792,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     const int q0 = (int)(((long long)cta * quads) / C), q1 = (int)(((long long)(cta + 1) * quads) / C);
     const int b0 = min(q0 * 4, a.N), b1 = min(q1 * 4, a.N);
     lin_epilogue_slice(a, cta, b0, b1 - b0, reinterpret_cast<float*>(smem2 + LIN2_HDR_BYTES),
-                       (int)((xbytes + (uint32_t)NS * STAGE) / sizeof(float)), reinterpret_cast<float*>(smem2 + 576));
+                       (int)((xbytes + (uint32_t)NS * STAGE) / sizeof(float)), reinterpret_cast<float*>(smem2 + 576),
+                       (a.xp_hi && a.pro == PRO_RMSNORM) ? s_scale : nullptr);
   }
   // departure: the last CTA to leave re-arms the counters and the tile queues for the next launch
   __syncthreads();
@@ -778,7 +866,7 @@ __global__ void __launch_bounds__(256) lin_f32_kernel(const LinArgs a) {
   if (tid < M) {
     float t = 0.f;
     for (int w = 0; w < 8; ++w) t += s_ssq[w][tid];
-    a.ssq_out[(size_t)r * SPS_MAX_ROWS + tid] = t;
+    a.ssq_out[SSQ_IDX(r, tid)] = t;
   }
 }
 
@@ -922,6 +1010,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   LinArgs a = a_in;
   a.R = p.R; a.S = p.S; a.WC = p.WC; a.PR = p.PR; a.KS = p.KS; a.KST = p.KST; a.NS = p.NS; a.G = p.G;
   if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
+  if ((a.xp_hi || a.yp_hi) && !(dtype == 1 && p.variant == 2)) return cudaErrorInvalidValue;   // packed activations: TMA kernel only
+  if ((a.xp_hi && !a.xp_lo) || (a.yp_hi && !a.yp_lo)) return cudaErrorInvalidValue;
   static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
   cudaError_t e;
   if (dtype == 0) {
