@@ -487,6 +487,13 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   __syncthreads();
   pdl_launch_dependents();
   float* s_scale = reinterpret_cast<float*>(smem2 + 512);   // [16] 1/rms of each X row
+  if (a.yp_gain && tid < 32) {
+    // the gain this CTA's epilogue slice will need is a weight in HBM: bring it into L2 now
+    const int quads = (a.N + 3) >> 2;
+    const int c0 = min((int)(((long long)cta * quads) / C) * 4, a.N), c1 = min((int)(((long long)(cta + 1) * quads) / C) * 4, a.N);
+    const int n = c0 + tid * 32;
+    if (n < c1) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.yp_gain + n));
+  }
 
   if (warp == NCW) {
     // ------------------------------------------------------------------ producer (one lane)
