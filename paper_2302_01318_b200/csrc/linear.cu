@@ -465,16 +465,19 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   __shared__ volatile int s_issued, s_total;
   volatile int* tile_ids = reinterpret_cast<volatile int*>(smem2 + 704);   // [64] ring: local tile -> tile number
   const uint32_t XP = (uint32_t)KS * 2 + 16, STAGE = 16u * (uint32_t)KST * 2u;
-  const uint32_t xbytes = ((2u * NT * 8u * XP + 1023u) / 1024u) * 1024u;
+  // The slab holds the M activation rows and, when M is short of the MMA's 8*NT columns, one row of zeros
+  // that all the missing columns read.
+  const uint32_t XR = (uint32_t)min(a.M + 1, NT * 8);
+  const uint32_t xbytes = ((2u * XR * XP + 1023u) / 1024u) * 1024u;
   const uint32_t sm0 = smem_u32(smem2);
   const uint32_t bar_full = sm0, bar_empty = sm0 + 8 * NS, bar_x = sm0 + 960;   // bar_x: the packed X slab has landed
   // consumed[slot] = how many times the slot has been read out.  A consumer may look at a slot's
   // "full" barrier only once every earlier use of the slot is over: an mbarrier parity wait cannot
   // tell phase u from phase u-2, and consumer warps run several ring revolutions ahead.
   volatile int* consumed = reinterpret_cast<volatile int*>(smem2 + 16 * NS);
-  const uint32_t xs_hi = sm0 + LIN2_HDR_BYTES, xs_lo = xs_hi + NT * 8 * XP, ring = sm0 + LIN2_HDR_BYTES + xbytes;
+  const uint32_t xs_hi = sm0 + LIN2_HDR_BYTES, xs_lo = xs_hi + XR * XP, ring = sm0 + LIN2_HDR_BYTES + xbytes;
   unsigned char* xs_hi_p = smem2 + LIN2_HDR_BYTES;
-  unsigned char* xs_lo_p = xs_hi_p + NT * 8 * XP;
+  unsigned char* xs_lo_p = xs_hi_p + XR * XP;
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); consumed[i] = 0; }
@@ -539,7 +542,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     pdl_wait();
   } else {
     // ------------------------------------------------------------------ consumer warps
-    // X slab: rows 0..8*NT-1 (zeros beyond M), this CTA's k-range, bf16 hi and lo parts, natural k order.
+    // X slab: the M activation rows (and the row of zeros), this CTA's k-range, bf16 hi and lo parts, natural k order.
     // Weights never change, so the producer is already streaming; X is the predecessor's output.
     bool alive = true;
     if (a.xp_hi) {
@@ -547,7 +550,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       // after it one lane per row asks the copy engine for that row's high and low halves, and everyone
       // waits for the bytes on one barrier.  With PRO_RMSNORM the rows' 1/rms is worked out meanwhile: the
       // epilogue multiplies by it.
-      for (int m = a.M + warp; m < NT * 8; m += NCW)
+      for (int m = a.M + warp; m < (int)XR; m += NCW)
         for (uint32_t off = lane * 16; off < (uint32_t)KS * 2; off += 512) {
           *reinterpret_cast<uint4*>(xs_hi_p + (size_t)m * XP + off) = make_uint4(0u, 0u, 0u, 0u);
           *reinterpret_cast<uint4*>(xs_lo_p + (size_t)m * XP + off) = make_uint4(0u, 0u, 0u, 0u);
@@ -639,6 +642,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
             for (int mm = 0; mm < 8; ++mm) {
               const int m = h * 8 + mm;
               uint2 hi = make_uint2(0u, 0u), lo = hi;
+              if (m >= (int)XR) continue;
               if (m < a.M) {
                 float4 x = v[i][mm];
                 if (a.pro == PRO_RMSNORM) {
@@ -700,7 +704,9 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         if (!mbar_wait(bar_full + 8 * slot, (uint32_t)use & 1u, a.err)) { alive = false; s_abort = 1; break; }
         const uint32_t wrow = ring + slot * STAGE + g * 128;          // row g of slab 0; row g+8 is +1024
         const uint32_t xoff = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 32;  // logical chunk 2t of this stage's k-range
-        const uint32_t xh_addr = xs_hi + g * XP + xoff, xl_addr = xs_lo + g * XP + xoff;
+        uint32_t xrow[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) xrow[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xoff;   // columns beyond M read the zero row
         const int slabs = KST >> 6;
 #pragma unroll 2
         for (int q = 0; q < slabs; ++q) {
@@ -710,8 +716,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
             const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-              const uint4 xh = lds128(xh_addr + nt * 8 * XP + q * 128 + hf * 16);
-              const uint4 xl = lds128(xl_addr + nt * 8 * XP + q * 128 + hf * 16);
+              const uint4 xh = lds128(xs_hi + xrow[nt] + q * 128 + hf * 16);
+              const uint4 xl = lds128(xs_lo + xrow[nt] + q * 128 + hf * 16);
               mma_bf16_16816(acc[nt][0], wa.x, wb.x, wa.y, wb.y, xh.x, xh.y);
               mma_bf16_16816(acc[nt][1], wa.x, wb.x, wa.y, wb.y, xl.x, xl.y);
               mma_bf16_16816(acc[nt][2], wa.z, wb.z, wa.w, wb.w, xh.z, xh.w);
@@ -930,7 +936,8 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     if (R > max_r) R = max_r;
     if (R > LIN_MAX_R) R = LIN_MAX_R;
     p.R = R;
-    size_t xbytes = (size_t)2 * p.NT * 8 * ((size_t)KS * 2 + 16);
+    const int xr = M + 1 < p.NT * 8 ? M + 1 : p.NT * 8;   // activation rows plus one row of zeros
+    size_t xbytes = (size_t)2 * xr * ((size_t)KS * 2 + 16);
     xbytes = ((xbytes + 1023) / 1024) * 1024;
     const size_t stage = (size_t)16 * (size_t)KST * 2;
     int NS = (int)((kSmemBudget + 8 * 1024 - 1024 - xbytes) / stage);
