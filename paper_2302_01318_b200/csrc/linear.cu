@@ -887,6 +887,8 @@ __global__ void __launch_bounds__(256) lin_f32_kernel(const LinArgs a) {
 // host side: how a shape is cut into CTAs
 // ------------------------------------------------------------------------------------------------
 static const size_t kSmemBudget = 200 * 1024;
+// TMA variant: everything a CTA may ask for (227 KB) less the kernel's 1 KB of static shared memory and a little slack
+static const size_t kSmemTma = 225 * 1024;
 
 bool sps_pdl_enabled() {
   static const bool on = [] { const char* e = getenv("SPS_PDL"); return !(e && atoi(e) == 0); }();
@@ -940,13 +942,13 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     size_t xbytes = (size_t)2 * xr * ((size_t)KS * 2 + 16);
     xbytes = ((xbytes + 1023) / 1024) * 1024;
     const size_t stage = (size_t)16 * (size_t)KST * 2;
-    int NS = (int)((kSmemBudget + 8 * 1024 - 1024 - xbytes) / stage);
+    int NS = (int)((kSmemTma - 1024 - xbytes) / stage);
     if (NS > 24) NS = 24;
     if (NS < 2) NS = 2;
     const int ksub = KS / KST;
     p.G = (ksub % 4 == 0) ? 4 : ((ksub % 2 == 0) ? 2 : 1);
     const size_t gscr = (size_t)2 * LIN_CONSUMER_WARPS * p.NT * 128 * sizeof(float);
-    NS = (int)((kSmemBudget + 8 * 1024 - 1024 - xbytes - gscr) / stage);
+    NS = (int)((kSmemTma - 1024 - xbytes - gscr) / stage);
     if (NS > 24) NS = 24;
     if (NS < 2) NS = 2;
     p.NS = NS;
