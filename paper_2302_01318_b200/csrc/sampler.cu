@@ -139,19 +139,41 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; }
   const float invT = 1.0f / T;
   const float* row = a.logits + (long long)b * a.ld;
-  float m = -INFINITY;
-  for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
-  m = block_max_f(m, s_part, &s_val);
   const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, a.t);
   int tok;
-  if (a.smem_weights) {
+  if (a.smem_weights && a.V <= 32 * SAMPLER_THREADS) {
+    // the row is read once: a thread keeps its (at most 32) logits in registers between the max and the exp
     extern __shared__ float ws[];
-    for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = expf((row[i] - m) * invT);
+    float l[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int i = threadIdx.x + j * SAMPLER_THREADS;
+      l[j] = i < a.V ? row[i] : -INFINITY;
+    }
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) m = fmaxf(m, l[j]);
+    m = block_max_f(m, s_part, &s_val);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const int i = threadIdx.x + j * SAMPLER_THREADS;
+      if (i < a.V) ws[skew(i)] = expf((l[j] - m) * invT);
+    }
     __syncthreads();
     tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
   } else {
-    auto w = [&](int i) { return expf((row[i] - m) * invT); };
-    tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
+    m = block_max_f(m, s_part, &s_val);
+    if (a.smem_weights) {
+      extern __shared__ float ws[];
+      for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = expf((row[i] - m) * invT);
+      __syncthreads();
+      tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
+    } else {
+      auto w = [&](int i) { return expf((row[i] - m) * invT); };
+      tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+    }
   }
   if (threadIdx.x == 0) a.out[(long long)b * a.out_ld] = tok;
 }
