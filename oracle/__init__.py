@@ -78,6 +78,12 @@ def lib():
         L.orc_sps_generate.argtypes = [vp, vp, i32, i32, i32, f64, u64, u32, u32, vp, vp, vp, vp]
         L.orc_sps_generate.restype = i32
         L.orc_sps_trials.argtypes = [vp, vp, vp, i32, i32, i32, f64, u64, u32, i64, i32, vp, vp, vp, vp]
+        L.orc_sps_trials_f.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, f64, u64, u32, i64, vp, vp, vp, vp]
+        L.orc_sps_set_sampling.argtypes = [vp, i32, f64]
+        L.orc_sample_row_f.argtypes = [vp, i32, f64, i32, f64, f64, vp]
+        L.orc_sample_row_f.restype = i32
+        L.orc_filtered.argtypes = [vp, i32, f64, i32, f64, vp, vp]
+        L.orc_accept_chain_f.argtypes = [vp, vp, vp, i32, i32, f64, i32, f64, u64, u32, u32, vp, vp, vp, vp]
         L.orc_num_threads.restype = i32
         L.orc_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp]
         _lib = L
@@ -135,15 +141,27 @@ def softmax(logits, T: float = 1.0):
     return out
 
 
-def sample_row(logits, T: float, u: float):
+def filtered(logits, T: float = 1.0, top_k: int = 0, top_p: float = 1.0):
+    """softmax(l / T) after top-k and nucleus filtering, renormalised; also whether the nucleus cut was a near tie."""
+    lg = _f32(logits)
+    out = np.zeros(lg.shape[-1], dtype=np.float64)
+    nc = C.c_int(0)
+    lib().orc_filtered(_p(lg), lg.shape[-1], float(T), int(top_k), float(top_p), _p(out), C.byref(nc))
+    return out, bool(nc.value)
+
+
+def sample_row(logits, T: float, u: float, top_k: int = 0, top_p: float = 1.0):
     lg = _f32(logits)
     nt = C.c_int(0)
-    tok = lib().orc_sample_row(_p(lg), lg.shape[-1], float(T), float(u), C.byref(nt))
+    if top_k == 0 and top_p >= 1.0:
+        tok = lib().orc_sample_row(_p(lg), lg.shape[-1], float(T), float(u), C.byref(nt))
+    else:
+        tok = lib().orc_sample_row_f(_p(lg), lg.shape[-1], float(T), int(top_k), float(top_p), float(u), C.byref(nt))
     return int(tok), bool(nt.value)
 
 
 def accept_chain(q_logits, p_logits, drafts, T: float, seed: int, b: int, s: int, want_beta: bool = False,
-                 wrong_rule: bool = False):
+                 wrong_rule: bool = False, top_k: int = 0, top_p: float = 1.0):
     """One loop's accept / resample / extra-token decision.  q_logits [K+1,V], p_logits [K,V]."""
     q = _f32(q_logits)
     K = q.shape[0] - 1
@@ -157,14 +175,18 @@ def accept_chain(q_logits, p_logits, drafts, T: float, seed: int, b: int, s: int
         lib().orc_accept_chain_wrong(_p(q), _p(p), _p(d), K, V, float(T), seed, b, s, _p(out), C.byref(na))
         return {"n_accepted": int(na.value), "tokens": out}
     beta = np.zeros(max(K, 1), dtype=np.float64) if want_beta else None
-    lib().orc_accept_chain(_p(q), _p(p), _p(d), K, V, float(T), seed, b, s, _p(out), C.byref(na), C.byref(fl), _p(beta))
+    if top_k == 0 and top_p >= 1.0:
+        lib().orc_accept_chain(_p(q), _p(p), _p(d), K, V, float(T), seed, b, s, _p(out), C.byref(na), C.byref(fl), _p(beta))
+    else:
+        lib().orc_accept_chain_f(_p(q), _p(p), _p(d), K, V, float(T), int(top_k), float(top_p), seed, b, s, _p(out),
+                                 C.byref(na), C.byref(fl), _p(beta))
     res = {"n_accepted": int(na.value), "tokens": out, "flags": int(fl.value)}
     if want_beta:
         res["beta"] = beta[:K]
     return res
 
 
-def accept_batch(q_logits, p_logits, drafts, T: float, seed: int, step: int):
+def accept_batch(q_logits, p_logits, drafts, T: float, seed: int, step: int, top_k: int = 0, top_p: float = 1.0):
     """accept_chain over a batch: q [B,K+1,V], p [B,K,V], drafts [B,K]; sequence index = row."""
     q = _f32(q_logits)
     B, K1, V = q.shape
@@ -175,7 +197,7 @@ def accept_batch(q_logits, p_logits, drafts, T: float, seed: int, step: int):
     toks = np.full((B, K + 1), -1, dtype=np.int32)
     flags = np.zeros(B, dtype=np.uint32)
     for b in range(B):
-        r = accept_chain(q[b], p[b], d[b], T, seed, b, step)
+        r = accept_chain(q[b], p[b], d[b], T, seed, b, step, top_k=top_k, top_p=top_p)
         n_acc[b] = r["n_accepted"]
         toks[b] = r["tokens"]
         flags[b] = r["flags"]
@@ -296,6 +318,10 @@ class Sps:
         self.V = target.V
         self._h = lib().orc_sps_create(target._h, draft._h if draft is not None else None)
 
+    def set_sampling(self, top_k: int = 0, top_p: float = 1.0):
+        """top-k / nucleus filtering of both models' distributions (0 / 1.0 = off)."""
+        lib().orc_sps_set_sampling(self._h, int(top_k), float(top_p))
+
     def reset(self, prompt):
         p = _i32(prompt)
         lib().orc_sps_reset(self._h, _p(p), p.shape[0])
@@ -337,13 +363,18 @@ class Sps:
 
 
 def trials(target: Model, draft: Model | None, prompt, n_new: int, K: int, T: float, seed: int, n_trials: int,
-           b0: int = 0, wrong_rule: bool = False):
+           b0: int = 0, wrong_rule: bool = False, top_k: int = 0, top_p: float = 1.0):
     """n_trials independent generations of n_new tokens (trial i uses sequence index b0+i)."""
     p = _i32(prompt)
     out = np.zeros((n_trials, n_new), dtype=np.int32)
     hist = np.zeros(K + 2, dtype=np.int64)
     first_acc = np.zeros(n_trials, dtype=np.int32)
     first_flags = np.zeros(n_trials, dtype=np.uint32)
-    lib().orc_sps_trials(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
-                         seed, b0, n_trials, int(wrong_rule), _p(out), _p(hist), _p(first_acc), _p(first_flags))
+    if top_k == 0 and top_p >= 1.0:
+        lib().orc_sps_trials(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
+                             seed, b0, n_trials, int(wrong_rule), _p(out), _p(hist), _p(first_acc), _p(first_flags))
+    else:
+        assert not wrong_rule
+        lib().orc_sps_trials_f(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
+                               int(top_k), float(top_p), seed, b0, n_trials, _p(out), _p(hist), _p(first_acc), _p(first_flags))
     return {"tokens": out, "hist_emitted": hist, "first_n_accepted": first_acc, "first_flags": first_flags}

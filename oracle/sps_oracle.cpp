@@ -114,6 +114,62 @@ static void softmax_T(const float* logits, int V, double T, std::vector<double>&
   for (int i = 0; i < V; ++i) prob[i] /= sum;
 }
 
+// Top-k and nucleus (top-p) filtering ("With standard sampling methods such as
+// nucleus, top-k sampling and adjusting temperature, we can modify the
+// probabilities accordingly before applying this rejection sampling scheme",
+// Modified Rejection Sampling).  The paper names the methods and gives no
+// formula; this build's reading, applied to the draft and the target alike:
+//   1. pr = softmax(l / T);
+//   2. top-k (k >= 1; 0 = off): keep every token whose logit is at least the
+//      k-th largest logit (tokens tied with the k-th are all kept);
+//   3. nucleus (0 < top_p < 1; 1 = off), on what step 2 kept, mass Z_k: walk the
+//      distinct logit values downwards adding the mass of each value's tokens;
+//      stop at the first value where the running mass reaches top_p * Z_k, keep
+//      that value and everything above it;
+//   4. zero the rest and renormalise.
+// Greedy decoding is top_k = 1.  *near_cut is set when the running mass passes
+// top_p * Z_k within 1e-5 * Z_k on either side of the cut, i.e. when sums taken
+// in another order or precision could legitimately cut one value earlier or later.
+struct Filt { int top_k = 0; double top_p = 1.0; };
+
+static void filtered_T(const float* logits, int V, double T, const Filt& f, std::vector<double>& prob, int* near_cut) {
+  softmax_T(logits, V, T, prob);
+  if (near_cut) *near_cut = 0;
+  const bool use_k = f.top_k >= 1 && f.top_k < V, use_p = f.top_p < 1.0;
+  if (!use_k && !use_p) return;
+  std::vector<int> order(V);
+  for (int i = 0; i < V; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return logits[a] > logits[b]; });
+  float cut = -INFINITY;            // keep logits >= cut
+  int n_k = V;                      // how many tokens step 2 keeps (a prefix of `order`)
+  if (use_k) {
+    const float lk = logits[order[f.top_k - 1]];
+    n_k = f.top_k;
+    while (n_k < V && logits[order[n_k]] == lk) ++n_k;
+    cut = lk;
+  }
+  if (use_p) {
+    double Zk = 0.0;
+    for (int j = 0; j < n_k; ++j) Zk += prob[order[j]];
+    const double target = f.top_p * Zk, band = 1e-5 * Zk;
+    double run = 0.0;
+    int j = 0;
+    while (j < n_k) {
+      const float v = logits[order[j]];
+      const double before = run;
+      while (j < n_k && logits[order[j]] == v) run += prob[order[j++]];
+      if (run >= target) {
+        if (v > cut) cut = v;
+        if (near_cut && ((run - target < band && j < n_k) || (before > 0.0 && target - before < band))) *near_cut = 1;
+        break;
+      }
+    }
+  }
+  double Z = 0.0;
+  for (int i = 0; i < V; ++i) { if (logits[i] < cut) prob[i] = 0.0; else Z += prob[i]; }
+  for (int i = 0; i < V; ++i) prob[i] /= Z;
+}
+
 // Inverse-CDF draw on unnormalised weights, in index order: the smallest i
 // whose inclusive running sum C_i exceeds u * C_{V-1}; if rounding leaves none,
 // the largest i with w_i > 0.  *near_tie is set when u * total lies within
@@ -155,6 +211,22 @@ extern "C" int orc_sample_row(const float* logits, int V, double T, double u, in
   softmax_T(logits, V, T, pr);
   return invcdf(pr.data(), V, u, near_tie);
 }
+// the same draw from the top-k / nucleus filtered distribution; *near_tie also covers a near cut
+extern "C" int orc_sample_row_f(const float* logits, int V, double T, int top_k, double top_p, double u, int* near_tie) {
+  std::vector<double> pr;
+  Filt f; f.top_k = top_k; f.top_p = top_p;
+  int nc = 0, nt = 0;
+  filtered_T(logits, V, T, f, pr, &nc);
+  const int tok = invcdf(pr.data(), V, u, &nt);
+  if (near_tie) *near_tie = (nc || nt) ? 1 : 0;
+  return tok;
+}
+extern "C" void orc_filtered(const float* logits, int V, double T, int top_k, double top_p, double* out, int* near_cut) {
+  std::vector<double> pr;
+  Filt f; f.top_k = top_k; f.top_p = top_p;
+  filtered_T(logits, V, T, f, pr, near_cut);
+  for (int i = 0; i < V; ++i) out[i] = pr[i];
+}
 
 extern "C" void orc_softmax(const float* logits, int V, double T, double* out) {
   std::vector<double> pr;
@@ -167,7 +239,8 @@ enum : uint32_t {
   ORC_BONUS = 2u,           // all K drafts accepted, extra token drawn from q_{K+1}
   ORC_FALLBACK = 4u,        // rejected although sum max(0, q-p) == 0: drawn from q_t
   ORC_NEAR_ACCEPT = 256u,   // |u_acc - min(1, q/p)| < 1e-4 at some tested position
-  ORC_NEAR_CDF = 512u       // the resample / extra-token draw fell in a CDF edge band
+  ORC_NEAR_CDF = 512u,      // the resample / extra-token draw fell in a CDF edge band
+  ORC_NEAR_CUT = 1024u      // a nucleus cut of a distribution this loop used was within its tie band
 };
 
 // Modified rejection sampling over one loop's K drafts (Algorithm 2, second
@@ -178,12 +251,18 @@ enum : uint32_t {
 // Writes the emitted tokens (n_accepted drafts then one resampled or extra
 // token) to out_tokens[0..n_accepted], -1 beyond; optional beta[K] receives
 // sum_x min(p_t(x), q_t(x)) (Theorem 1's acceptance probability).
-extern "C" void orc_accept_chain(const float* q_logits, const float* p_logits, const int32_t* drafts,
-                                 int K, int V, double T, uint64_t seed, uint32_t b, uint32_t s,
-                                 int32_t* out_tokens, int32_t* n_accepted, uint32_t* flags,
-                                 double* beta) {
+static void accept_chain_impl(const float* q_logits, const float* p_logits, const int32_t* drafts,
+                              int K, int V, double T, const Filt& filt, uint64_t seed, uint32_t b, uint32_t s,
+                              int32_t* out_tokens, int32_t* n_accepted, uint32_t* flags,
+                              double* beta) {
   std::vector<double> q, p, r(V);
   uint32_t fl = 0;
+  // q and p below are the distributions after temperature, top-k and nucleus
+  auto softmax_T = [&](const float* lg, int V_, double T_, std::vector<double>& out) {
+    int nc = 0;
+    filtered_T(lg, V_, T_, filt, out, &nc);
+    if (nc) fl |= ORC_NEAR_CUT;
+  };
   int a = 0;
   for (int i = 0; i <= K; ++i) out_tokens[i] = -1;
   if (beta) {
@@ -243,6 +322,20 @@ extern "C" void orc_accept_chain(const float* q_logits, const float* p_logits, c
   }
   *n_accepted = a;
   *flags = fl;
+}
+
+extern "C" void orc_accept_chain(const float* q_logits, const float* p_logits, const int32_t* drafts,
+                                 int K, int V, double T, uint64_t seed, uint32_t b, uint32_t s,
+                                 int32_t* out_tokens, int32_t* n_accepted, uint32_t* flags,
+                                 double* beta) {
+  accept_chain_impl(q_logits, p_logits, drafts, K, V, T, Filt(), seed, b, s, out_tokens, n_accepted, flags, beta);
+}
+extern "C" void orc_accept_chain_f(const float* q_logits, const float* p_logits, const int32_t* drafts,
+                                   int K, int V, double T, int top_k, double top_p, uint64_t seed, uint32_t b, uint32_t s,
+                                   int32_t* out_tokens, int32_t* n_accepted, uint32_t* flags,
+                                   double* beta) {
+  Filt f; f.top_k = top_k; f.top_p = top_p;
+  accept_chain_impl(q_logits, p_logits, drafts, K, V, T, f, seed, b, s, out_tokens, n_accepted, flags, beta);
 }
 
 // The same chain with the WRONG resampling rule (draw from q_t instead of the
@@ -541,6 +634,7 @@ struct OrcSps {
   // what the last loop saw (for element-wise comparison with another implementation)
   std::vector<float> last_q, last_p;
   std::vector<int32_t> last_drafts;
+  Filt filt;               // top-k / nucleus applied to both models' distributions
 };
 
 extern "C" OrcSps* orc_sps_create(OrcModel* target, OrcModel* draft) {
@@ -549,6 +643,7 @@ extern "C" OrcSps* orc_sps_create(OrcModel* target, OrcModel* draft) {
   return c;
 }
 extern "C" void orc_sps_destroy(OrcSps* c) { delete c; }
+extern "C" void orc_sps_set_sampling(OrcSps* c, int top_k, double top_p) { c->filt.top_k = top_k; c->filt.top_p = top_p; }
 
 // Start from a prompt x_0..x_{P-1}: both caches take positions 0..P-2, so that
 // the first loop feeds x_{P-1} (n = P).
@@ -599,7 +694,7 @@ extern "C" int orc_sps_loop(OrcSps* c, int K, double T, uint64_t seed, uint32_t 
     double u[3];
     orc_uniforms(seed, b, s, (uint32_t)t, u);
     int nt = 0;
-    d[t] = orc_sample_row(last, V, T, u[0], &nt);
+    d[t] = orc_sample_row_f(last, V, T, c->filt.top_k, c->filt.top_p, u[0], &nt);
     if (nt) dnt |= (1u << t);
   }
   // --- score: K+1 sets of target logits in one call over [x_{n-1}, d_0..d_{K-1}]
@@ -613,7 +708,7 @@ extern "C" int orc_sps_loop(OrcSps* c, int K, double T, uint64_t seed, uint32_t 
   // --- accept from left to right, resample or draw the extra token
   int a = 0;
   uint32_t fl = 0;
-  orc_accept_chain(c->last_q.data(), c->last_p.data(), d.data(), K, V, T, seed, b, s, out_tokens, &a, &fl, nullptr);
+  accept_chain_impl(c->last_q.data(), c->last_p.data(), d.data(), K, V, T, c->filt, seed, b, s, out_tokens, &a, &fl, nullptr);
   for (int i = 0; i <= a; ++i) c->x.push_back(out_tokens[i]);
   // --- caches: nothing is undone, only the valid lengths move
   c->tlen = n + a;
@@ -652,14 +747,15 @@ extern "C" int orc_sps_generate(OrcSps* c, const int32_t* prompt, int P, int n_n
 // trial i using sequence index b0 + i (so each trial has its own uniforms).
 // Meant for table models, where a forward costs nothing.  wrong_rule != 0
 // swaps in the negative-control chain.
-extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,
-                               double T, uint64_t seed, uint32_t b0, int64_t n_trials, int wrong_rule,
-                               int32_t* out_tokens /*[n_trials][n_new]*/, int64_t* emitted_hist /*[K+2]*/,
-                               int32_t* first_n_accepted /*[n_trials] or null*/,
-                               uint32_t* first_flags /*[n_trials] or null*/) {
+static void sps_trials_impl(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,
+                            double T, const Filt& filt, uint64_t seed, uint32_t b0, int64_t n_trials, int wrong_rule,
+                            int32_t* out_tokens /*[n_trials][n_new]*/, int64_t* emitted_hist /*[K+2]*/,
+                            int32_t* first_n_accepted /*[n_trials] or null*/,
+                            uint32_t* first_flags /*[n_trials] or null*/) {
   const int V = target->V;
   for (int i = 0; i < K + 2; ++i) emitted_hist[i] = 0;
   OrcSps* c = orc_sps_create(target, draft);
+  c->filt = filt;
   std::vector<int32_t> em(K + 1), d(K);
   for (int64_t tr = 0; tr < n_trials; ++tr) {
     const uint32_t b = b0 + (uint32_t)tr;
@@ -708,6 +804,21 @@ extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t*
     }
   }
   orc_sps_destroy(c);
+}
+
+extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,
+                               double T, uint64_t seed, uint32_t b0, int64_t n_trials, int wrong_rule,
+                               int32_t* out_tokens, int64_t* emitted_hist, int32_t* first_n_accepted, uint32_t* first_flags) {
+  sps_trials_impl(target, draft, prompt, P, n_new, K, T, Filt(), seed, b0, n_trials, wrong_rule, out_tokens, emitted_hist,
+                  first_n_accepted, first_flags);
+}
+// the same with top-k / nucleus filtering of both models (not with the negative-control chain)
+extern "C" void orc_sps_trials_f(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,
+                                 double T, int top_k, double top_p, uint64_t seed, uint32_t b0, int64_t n_trials,
+                                 int32_t* out_tokens, int64_t* emitted_hist, int32_t* first_n_accepted, uint32_t* first_flags) {
+  Filt f; f.top_k = top_k; f.top_p = top_p;
+  sps_trials_impl(target, draft, prompt, P, n_new, K, T, f, seed, b0, n_trials, 0, out_tokens, emitted_hist,
+                  first_n_accepted, first_flags);
 }
 
 // Y[m][n] = sum_k X[m][k] W[n][k]: the linear layer by its definition, in double.
