@@ -132,10 +132,25 @@ const char* sps_last_error(sps_handle* h);
  *   out_tokens  host  [n_new]
  *   out_stats   host, may be NULL
  * temperature > 0 scales both models' logits before the rejection scheme
- * ("adjusting temperature ... modify the probabilities accordingly").
- * SPS_ERANGE if prompt_len + n_new + K > max_seq. */
+ * ("adjusting temperature ... modify the probabilities accordingly");
+ * temperature == 0 is greedy decoding (top-k with k = 1 on both models, see
+ * sps_set_sampling).  SPS_ERANGE if prompt_len + n_new + K > max_seq. */
 int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K,
                  float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
+
+/* Top-k and nucleus filtering of BOTH models' distributions ahead of the
+ * rejection scheme ("With standard sampling methods such as nucleus, top-k
+ * sampling and adjusting temperature, we can modify the probabilities
+ * accordingly before applying this rejection sampling scheme", section
+ * Modified Rejection Sampling).  The paper gives no formula; this library's:
+ * after softmax(l / temperature), top_k >= 1 keeps every token whose logit is
+ * at least the k-th largest (tokens tied with it stay; 0 = off); then
+ * 0 < top_p < 1 keeps, of those, the tokens whose logit is at least v, v the
+ * largest logit value such that the tokens with logit >= v hold at least top_p
+ * of the mass top-k kept (1 = off); the rest weigh nothing and what is left is
+ * renormalised.  The setting stays on the handle for every later sps_generate*,
+ * sps_step; no device work.  SPS_EINVAL for top_k < 0 or top_p outside (0, 1]. */
+int sps_set_sampling(sps_handle* h, int32_t top_k, float top_p);
 
 /* Same for B sequences with equal prompt lengths, advanced in lock-step with
  * ragged progress; sequence b uses Philox sequence index b.
@@ -184,12 +199,22 @@ int sps_accept(const float* q_logits, const float* p_logits, const int32_t* draf
                int32_t V, float temperature, uint64_t seed, uint32_t step, void* stream, int32_t* out_n_accepted,
                int32_t* out_tokens, uint32_t* out_flags);
 
+/* sps_accept with both distributions filtered as sps_set_sampling describes
+ * (top_k 0 and top_p 1 = plain sps_accept; temperature 0 = greedy). */
+int sps_accept_filtered(const float* q_logits, const float* p_logits, const int32_t* draft_tokens, int32_t B, int32_t K,
+                        int32_t V, float temperature, int32_t top_k, float top_p, uint64_t seed, uint32_t step,
+                        void* stream, int32_t* out_n_accepted, int32_t* out_tokens, uint32_t* out_flags);
+
 /* One inverse-CDF draw per row from softmax(logits / temperature) with
  * u_draft of counter (t, step, b, 0): Algorithm 2's "sample draft
  * auto-regressively" for given logits.  logits device fp32 [B, V];
  * out_tokens device int32 [B]. */
 int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uint64_t seed, uint32_t step, uint32_t t,
                void* stream, int32_t* out_tokens);
+
+/* sps_sample from the filtered distribution (see sps_set_sampling). */
+int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float temperature, int32_t top_k, float top_p,
+                        uint64_t seed, uint32_t step, uint32_t t, void* stream, int32_t* out_tokens);
 
 /* The memory-bound linear layer alone ("dense matrix multiplies ... become
  * memory bound", Conditional Scoring): Y[M, N] = X[M, D] W[N, D]^T with fp32

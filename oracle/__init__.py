@@ -26,6 +26,7 @@ FLAG_BONUS = 2
 FLAG_FALLBACK = 4
 FLAG_NEAR_ACCEPT = 256
 FLAG_NEAR_CDF = 512
+FLAG_NEAR_CUT = 1024
 
 
 def build(force: bool = False) -> str:

@@ -82,6 +82,9 @@ def lib():
         L.sps_score.argtypes = [vp, i32, vp, i32, vp, C.POINTER(f32)]
         L.sps_accept.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp]
         L.sps_sample.argtypes = [vp, i32, i32, f32, u64, u32, u32, vp, vp]
+        L.sps_set_sampling.argtypes = [vp, i32, f32]
+        L.sps_accept_filtered.argtypes = [vp, vp, vp, i32, i32, i32, f32, i32, f32, u64, u32, vp, vp, vp, vp]
+        L.sps_sample_filtered.argtypes = [vp, i32, i32, f32, i32, f32, u64, u32, u32, vp, vp]
         L.sps_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
         L.sps_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sps_linear_workspace_bytes.restype = i64
@@ -169,6 +172,9 @@ class Handle:
         _check(lib().sps_generate_batch(self._h, _np_ptr(p), B, P, n_new, K, temperature, seed, _np_ptr(out), st), self._h)
         return out, [s.as_dict() for s in st]
 
+    def sps_set_sampling(self, top_k=0, top_p=1.0):
+        _check(lib().sps_set_sampling(self._h, int(top_k), float(top_p)), self._h)
+
     def sps_reset(self):
         _check(lib().sps_reset(self._h), self._h)
 
@@ -219,6 +225,23 @@ def sps_accept(q_logits, p_logits, draft_tokens, temperature, seed, step, out_n_
     _check(lib().sps_accept(q_logits.data_ptr(), p_logits.data_ptr() if K else None,
                             draft_tokens.data_ptr() if K else None, B, K, V, temperature, seed, step,
                             _stream_ptr(stream), out_n_accepted.data_ptr(), out_tokens.data_ptr(), out_flags.data_ptr()))
+
+
+def sps_accept_filtered(q_logits, p_logits, draft_tokens, temperature, top_k, top_p, seed, step, out_n_accepted, out_tokens,
+                        out_flags, stream=None):
+    """sps_accept with top-k / nucleus filtering of both distributions (temperature 0 = greedy)."""
+    B, K1, V = q_logits.shape
+    K = K1 - 1
+    _check(lib().sps_accept_filtered(q_logits.data_ptr(), p_logits.data_ptr() if K else None,
+                                     draft_tokens.data_ptr() if K else None, B, K, V, temperature, top_k, top_p, seed, step,
+                                     _stream_ptr(stream), out_n_accepted.data_ptr(), out_tokens.data_ptr(),
+                                     out_flags.data_ptr()))
+
+
+def sps_sample_filtered(logits, temperature, top_k, top_p, seed, step, t, out_tokens, stream=None):
+    B, V = logits.shape
+    _check(lib().sps_sample_filtered(logits.data_ptr(), B, V, temperature, top_k, top_p, seed, step, t, _stream_ptr(stream),
+                                     out_tokens.data_ptr()))
 
 
 def sps_sample(logits, temperature, seed, step, t, out_tokens, stream=None):

@@ -98,6 +98,8 @@ struct DevState {
   uint32_t step;      // loop index s, advanced on the device after each loop
   uint32_t pad0;
   uint64_t seed;
+  float top_p;        // nucleus mass kept (1 = off), both models
+  int32_t top_k;      // tokens kept (0 = off), both models
   int32_t B;          // live sequences
   int32_t max_seq;
   // per sequence
@@ -216,6 +218,7 @@ struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(log
   int32_t* out;            // out[b*out_ld]
   int out_ld;
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+  int top_k; float top_p;  // used when st == nullptr (0 / 1 = no filtering)
   int smem_weights;        // set by the launcher: weights are staged in shared memory
 };
 cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st);
@@ -232,6 +235,7 @@ struct AcceptArgs {
   int out_ld;
   uint32_t* flags;         // [B]
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
+  int top_k; float top_p;  // used when st == nullptr (0 / 1 = no filtering)
   int smem_weights;        // set by the launcher: weights are staged in shared memory
 };
 cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);

@@ -28,7 +28,7 @@ struct ModelDev {
   bool packed = false;     // every linear layer of this model runs on the bf16 TMA kernel: activations travel packed
 };
 
-struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uint64_t seed; };
+struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uint64_t seed; float top_p; int32_t top_k; };   // head of DevState
 
 }  // namespace
 
@@ -49,6 +49,8 @@ struct sps_handle {
   int32_t* res = nullptr;    // device: [n_acc B][flags B][out_tok B*(maxK+1)][err 1]
   int32_t* h_res = nullptr;  // pinned mirror
   HostParams* h_par = nullptr;  // pinned
+  int top_k = 0;                // sps_set_sampling: tokens kept (0 = off)
+  float top_p = 1.f;            //                   nucleus mass kept (1 = off)
   int32_t* h_rows = nullptr;    // pinned [2][16]
   size_t res_words = 0;
   int B = 0;
@@ -314,8 +316,13 @@ int launch_phase(sps_handle* h, std::map<int, cudaGraphExec_t>& cache, int K, in
 }
 
 int write_params(sps_handle* h, float T, uint64_t seed, uint32_t step) {
+  // temperature 0 = greedy decoding: the one-token limit of top-k, applied to both models
+  const bool greedy = T == 0.f;
+  if (greedy) T = 1.f;
   h->h_par->temperature = T; h->h_par->inv_temperature = 1.0f / T; h->h_par->step = step; h->h_par->pad0 = 0;
   h->h_par->seed = seed;
+  h->h_par->top_k = greedy ? 1 : h->top_k;
+  h->h_par->top_p = greedy ? 1.f : h->top_p;
   CU(h, cudaMemcpyAsync(h->dst, h->h_par, sizeof(HostParams), cudaMemcpyHostToDevice, h->stream));
   return SPS_OK;
 }
@@ -479,7 +486,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   if (cudaMallocHost(&h->h_res, 4 * h->res_words) != cudaSuccess || cudaMallocHost(&h->h_par, sizeof(HostParams)) != cudaSuccess ||
       cudaMallocHost(&h->h_rows, 4 * 2 * SPS_MAX_ROWS) != cudaSuccess)
     return bail(fail(h, SPS_ENOMEM, "pinned host allocation failed"));
-  s.temperature = 1.f; s.inv_temperature = 1.f; s.step = 0; s.seed = 0; s.B = 1; s.max_seq = cfg->max_seq; s.max_K = maxK;
+  s.temperature = 1.f; s.inv_temperature = 1.f; s.step = 0; s.seed = 0; s.top_p = 1.f; s.top_k = 0; s.B = 1; s.max_seq = cfg->max_seq; s.max_K = maxK;
   s.n_acc = h->res;
   s.flags = (uint32_t*)(h->res + MB);
   s.out_tok = h->res + 2 * MB;
@@ -540,7 +547,7 @@ int sps_step(sps_handle* h, int32_t K, float temperature, uint64_t seed, uint32_
              int32_t* out_n_emitted, uint32_t* out_flags) {
   if (!h || !out_tokens || !out_n_emitted) return fail(h, SPS_EINVAL, "null argument");
   if (!h->ready) return fail(h, SPS_ESTATE, "sps_step before sps_prefill");
-  if (!(temperature > 0.f)) return fail(h, SPS_EINVAL, "temperature must be > 0");
+  if (!(temperature >= 0.f)) return fail(h, SPS_EINVAL, "temperature must be >= 0 (0 = greedy)");
   CU(h, cudaSetDevice(h->cfg.device));
   int rc = check_K(h, K);
   if (rc) return rc;
@@ -576,7 +583,7 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
                          int32_t* out_tokens, sps_stats* out_stats) {
   if (!h || !prompts || !out_tokens) return fail(h, SPS_EINVAL, "null argument");
   if (n_new < 1) return fail(h, SPS_EINVAL, "n_new must be >= 1");
-  if (!(T > 0.f)) return fail(h, SPS_EINVAL, "temperature must be > 0");
+  if (!(T >= 0.f)) return fail(h, SPS_EINVAL, "temperature must be >= 0 (0 = greedy)");
   CU(h, cudaSetDevice(h->cfg.device));
   if (P < 1) return fail(h, SPS_EINVAL, "prompt_len must be >= 1");
   if ((long long)P + n_new + K > h->cfg.max_seq) return fail(h, SPS_ERANGE, "prompt_len + n_new + K exceeds max_seq");
@@ -687,18 +694,37 @@ int sps_verify(sps_handle* h, const int32_t* rows, int32_t K, float* out_logits,
   return sps_score(h, 0, rows, K + 1, out_logits, out_ms);
 }
 
+int sps_set_sampling(sps_handle* h, int32_t top_k, float top_p) {
+  if (!h) return fail(nullptr, SPS_EINVAL, "null handle");
+  if (top_k < 0) return fail(h, SPS_EINVAL, "top_k must be >= 0 (0 = off)");
+  if (!(top_p > 0.f && top_p <= 1.f)) return fail(h, SPS_EINVAL, "top_p must be in (0, 1] (1 = off)");
+  h->top_k = top_k;
+  h->top_p = top_p;
+  return SPS_OK;
+}
+
 int sps_accept(const float* q_logits, const float* p_logits, const int32_t* draft_tokens, int32_t B, int32_t K, int32_t V,
                float temperature, uint64_t seed, uint32_t step, void* stream, int32_t* out_n_accepted,
                int32_t* out_tokens, uint32_t* out_flags) {
+  if (!(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "temperature must be > 0");
+  return sps_accept_filtered(q_logits, p_logits, draft_tokens, B, K, V, temperature, 0, 1.f, seed, step, stream, out_n_accepted,
+                             out_tokens, out_flags);
+}
+
+int sps_accept_filtered(const float* q_logits, const float* p_logits, const int32_t* draft_tokens, int32_t B, int32_t K,
+                        int32_t V, float temperature, int32_t top_k, float top_p, uint64_t seed, uint32_t step, void* stream,
+                        int32_t* out_n_accepted, int32_t* out_tokens, uint32_t* out_flags) {
   if (!q_logits || !out_n_accepted || !out_tokens || !out_flags) return fail(nullptr, SPS_EINVAL, "null argument");
   if (K > 0 && (!p_logits || !draft_tokens)) return fail(nullptr, SPS_EINVAL, "K > 0 needs p_logits and draft_tokens");
   if (B < 1 || K < 0 || K > SPS_MAX_K || V < 1) return fail(nullptr, SPS_EINVAL, "B, K or V out of range");
-  if (!(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "temperature must be > 0");
+  if (!(temperature >= 0.f)) return fail(nullptr, SPS_EINVAL, "temperature must be >= 0 (0 = greedy)");
+  if (top_k < 0 || !(top_p > 0.f && top_p <= 1.f)) return fail(nullptr, SPS_EINVAL, "top_k must be >= 0 and top_p in (0, 1]");
+  if (temperature == 0.f) { temperature = 1.f; top_k = 1; top_p = 1.f; }
   AcceptArgs a{};
   a.st = nullptr; a.q_logits = q_logits; a.p_logits = p_logits ? p_logits : q_logits;
   a.drafts = draft_tokens ? draft_tokens : out_tokens; a.drafts_ld = K;
   a.B = B; a.K = K; a.V = V; a.n_acc = out_n_accepted; a.out_tok = out_tokens; a.out_ld = K + 1; a.flags = out_flags;
-  a.temperature = temperature; a.seed = seed; a.step = step;
+  a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p;
   cudaError_t e = accept_launch(a, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("accept launch: ") + cudaGetErrorString(e));
   return SPS_OK;
@@ -706,11 +732,19 @@ int sps_accept(const float* q_logits, const float* p_logits, const int32_t* draf
 
 int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uint64_t seed, uint32_t step, uint32_t t,
                void* stream, int32_t* out_tokens) {
+  if (!(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "B, V or temperature out of range");
+  return sps_sample_filtered(logits, B, V, temperature, 0, 1.f, seed, step, t, stream, out_tokens);
+}
+
+int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float temperature, int32_t top_k, float top_p, uint64_t seed,
+                        uint32_t step, uint32_t t, void* stream, int32_t* out_tokens) {
   if (!logits || !out_tokens) return fail(nullptr, SPS_EINVAL, "null argument");
-  if (B < 1 || V < 1 || !(temperature > 0.f)) return fail(nullptr, SPS_EINVAL, "B, V or temperature out of range");
+  if (B < 1 || V < 1 || !(temperature >= 0.f)) return fail(nullptr, SPS_EINVAL, "B, V or temperature out of range");
+  if (top_k < 0 || !(top_p > 0.f && top_p <= 1.f)) return fail(nullptr, SPS_EINVAL, "top_k must be >= 0 and top_p in (0, 1]");
+  if (temperature == 0.f) { temperature = 1.f; top_k = 1; top_p = 1.f; }
   SampleArgs a{};
   a.st = nullptr; a.logits = logits; a.ld = V; a.V = V; a.B = B; a.t = t; a.out = out_tokens; a.out_ld = 1;
-  a.temperature = temperature; a.seed = seed; a.step = step;
+  a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p;
   cudaError_t e = sample_launch(a, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("sample launch: ") + cudaGetErrorString(e));
   return SPS_OK;

@@ -123,11 +123,152 @@ __device__ inline float block_sum_f(float v, float* s_part, float* s_out) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Top-k and nucleus filtering ("standard sampling methods such as nucleus, top-k sampling and adjusting
+// temperature ... modify the probabilities accordingly before applying this rejection sampling scheme",
+// section Modified Rejection Sampling).  A row keeps every token whose logit is at least a cut:
+//   top-k   : the cut is the k-th largest logit (tokens tied with it stay);
+//   nucleus : over what top-k kept, mass Z_k, the largest logit value v such that the tokens with logit
+//             >= v hold at least top_p * Z_k.
+// Both are "the largest key whose upper tail reaches a target": a radix descent over the order-preserving
+// bit pattern of the logit, eight bits per pass, with a 256-bin histogram of the tail function (token
+// counts for top-k, weights for the nucleus).  No sort.  Weights enter the histogram as 40-bit fixed
+// point integers, so the sums do not depend on the order in which threads add them.
+// ------------------------------------------------------------------------------------------------
+struct CutSmem {
+  unsigned long long bin[256];
+  unsigned long long acc;
+  unsigned int sel;
+  unsigned int found;
+};
+
+__device__ __forceinline__ uint32_t order_key(float f) {   // unsigned order of keys == order of the floats
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float order_key_inv(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+__device__ __forceinline__ unsigned long long fixed40(float w) {   // w in [0, 1]
+  return __float2ull_rn(w * 1099511627776.0f);
+}
+
+// The largest key K* (among tokens with key >= dom_key) with F(K*) = sum over tokens of key >= K* of f
+// reaching `target`; f = 1 (SUM == false) or the token's fixed-point weight.  Returns F(K*) and whether
+// such a key exists.  All threads of the block call it; all get the same answer.
+template <bool SUM>
+__device__ bool tail_descent(const float* row, int V, float m, float invT, uint32_t dom_key, unsigned long long target,
+                             CutSmem& cs, uint32_t* key_out, unsigned long long* F_out) {
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t prefix = 0, mask = 0;
+  unsigned long long acc = 0, at_key = 0;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int d = tid; d < 256; d += nthr) cs.bin[d] = 0;
+    __syncthreads();
+    // a thread adds runs of equal digits locally: in the first passes nearly all tokens share one digit
+    int cur = -1;
+    unsigned long long loc = 0;
+    for (int i = tid; i < V; i += nthr) {
+      const float l = row[i];
+      const uint32_t k = order_key(l);
+      if ((k & mask) != prefix || k < dom_key) continue;
+      const int d = (int)((k >> shift) & 255u);
+      const unsigned long long f = SUM ? fixed40(expf((l - m) * invT)) : 1ull;
+      if (d != cur) {
+        if (cur >= 0) atomicAdd(&cs.bin[cur], loc);
+        cur = d;
+        loc = 0;
+      }
+      loc += f;
+    }
+    if (cur >= 0) atomicAdd(&cs.bin[cur], loc);
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns digits 255 - 8l .. 248 - 8l; the tail above them is a warp prefix sum
+      unsigned long long t = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) t += cs.bin[255 - 8 * lane - j];
+      unsigned long long incl = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const unsigned long long above = acc + (incl - t);
+      const bool cross = above < target && above + t >= target;
+      const unsigned int who = __ballot_sync(0xffffffffu, cross);
+      if (lane == 0) cs.found = who != 0u;
+      if (cross) {
+        unsigned long long run = above;
+        for (int j = 0; j < 8; ++j) {
+          const int d = 255 - 8 * lane - j;
+          if (run + cs.bin[d] >= target) { cs.sel = (unsigned int)d; cs.acc = run; break; }
+          run += cs.bin[d];
+        }
+      }
+    }
+    __syncthreads();
+    if (!cs.found) return false;   // the whole domain holds less than the target (callers make sure it does not)
+    prefix |= cs.sel << shift;
+    mask |= 255u << shift;
+    acc = cs.acc;
+    at_key = cs.bin[cs.sel];
+    __syncthreads();
+  }
+  *key_out = prefix;
+  *F_out = acc + at_key;
+  return true;
+}
+
+// sum over tokens with key >= dom_key of the fixed-point weight
+__device__ unsigned long long tail_mass(const float* row, int V, float m, float invT, uint32_t dom_key, CutSmem& cs) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  if (tid == 0) cs.acc = 0;
+  __syncthreads();
+  unsigned long long loc = 0;
+  for (int i = tid; i < V; i += nthr) {
+    const float l = row[i];
+    if (order_key(l) >= dom_key) loc += fixed40(expf((l - m) * invT));
+  }
+  loc += __shfl_xor_sync(0xffffffffu, loc, 16);
+  loc += __shfl_xor_sync(0xffffffffu, loc, 8);
+  loc += __shfl_xor_sync(0xffffffffu, loc, 4);
+  loc += __shfl_xor_sync(0xffffffffu, loc, 2);
+  loc += __shfl_xor_sync(0xffffffffu, loc, 1);
+  if ((tid & 31) == 0) atomicAdd(&cs.acc, loc);
+  __syncthreads();
+  const unsigned long long z = cs.acc;
+  __syncthreads();
+  return z;
+}
+
+// The cut of one row and the mass it keeps (sum of exp((l - m) / T) over kept tokens).  m = the row's maximum.
+__device__ void row_cut(const float* row, int V, float m, float invT, int top_k, float top_p, CutSmem& cs,
+                        float* cut_out, float* mass_out) {
+  uint32_t key = 0;   // keep everything
+  unsigned long long F = 0;
+  if (top_k >= 1 && top_k < V) {
+    if (!tail_descent<false>(row, V, m, invT, 0u, (unsigned long long)top_k, cs, &key, &F)) key = 0;
+  }
+  unsigned long long Z = tail_mass(row, V, m, invT, key, cs);
+  if (top_p < 1.0f) {
+    unsigned long long target = (unsigned long long)((double)top_p * (double)Z);
+    if (target < 1ull) target = 1ull;
+    uint32_t kp;
+    unsigned long long Fp;
+    if (target <= Z && tail_descent<true>(row, V, m, invT, key, target, cs, &kp, &Fp)) { key = kp; Z = Fp; }
+  }
+  *cut_out = key == 0u ? -INFINITY : order_key_inv(key);
+  *mass_out = (float)((double)Z * (1.0 / 1099511627776.0));
+}
+
+// ------------------------------------------------------------------------------------------------
 // x ~ softmax(logits / T) by inverse CDF with u_draft(b, s, t)  (Algorithm 2: "sample draft
 // auto-regressively"; with t = 0 and u_res it is Algorithm 1's sample).
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   __shared__ ScanSmem sm;
+  __shared__ CutSmem cs;
   __shared__ float s_part[SAMPLER_WARPS];
   __shared__ float s_val;
   const int b = blockIdx.x;
@@ -136,12 +277,30 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   float T = a.temperature;
   uint64_t seed = a.seed;
   uint32_t step = a.step;
-  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; }
+  int top_k = a.top_k;
+  float top_p = a.top_p;
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; }
   const float invT = 1.0f / T;
   const float* row = a.logits + (long long)b * a.ld;
   const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, a.t);
   int tok;
-  if (a.smem_weights && a.V <= 32 * SAMPLER_THREADS) {
+  if ((top_k >= 1 && top_k < a.V) || top_p < 1.0f) {
+    // filtered draw: tokens under the cut weigh nothing
+    float m = -INFINITY;
+    for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
+    m = block_max_f(m, s_part, &s_val);
+    float cut, mass;
+    row_cut(row, a.V, m, invT, top_k, top_p, cs, &cut, &mass);
+    auto w = [&](int i) { const float l = row[i]; return l >= cut ? expf((l - m) * invT) : 0.f; };
+    if (a.smem_weights) {
+      extern __shared__ float ws[];
+      for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = w(i);
+      __syncthreads();
+      tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
+    } else {
+      tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+    }
+  } else if (a.smem_weights && a.V <= 32 * SAMPLER_THREADS) {
     // the row is read once: a thread keeps its (at most 32) logits in registers between the max and the exp
     extern __shared__ float ws[];
     float l[32];
@@ -212,8 +371,9 @@ cudaError_t sample_launch(const SampleArgs& a_in, cudaStream_t st) {
 __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   __shared__ ScanSmem sm;
   __shared__ float s_red[SAMPLER_WARPS][ACC_MAX_ROWS + 1];
-  __shared__ float s_max[ACC_MAX_ROWS], s_sum[ACC_MAX_ROWS];
+  __shared__ float s_max[ACC_MAX_ROWS], s_sum[ACC_MAX_ROWS], s_cut[ACC_MAX_ROWS];
   __shared__ int s_stop;
+  __shared__ CutSmem cs;
   extern __shared__ float ws[];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, V = a.V, R = 2 * K + 1;
@@ -222,7 +382,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   float T = a.temperature;
   uint64_t seed = a.seed;
   uint32_t step = a.step;
-  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; }
+  int top_k = a.top_k;
+  float top_p = a.top_p;
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; }
+  const bool filt = (top_k >= 1 && top_k < V) || top_p < 1.0f;
   const float invT = 1.0f / T;
   const float* qrow = a.q_logits + (long long)b * (K + 1) * V;
   const float* prow = a.p_logits + (long long)b * K * V;
@@ -257,26 +420,51 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     float s = 0.f;
     for (int w = 0; w < SAMPLER_WARPS; ++w) s += s_red[w][tid];
     s_sum[tid] = s;
+    s_cut[tid] = -INFINITY;
   }
   __syncthreads();
+  // with top-k / nucleus filtering a row's cut and kept mass replace its plain sum; rows are cut when the
+  // chain reaches them (block-wide work), so a loop that stops early does not pay for the later rows
+  auto cut_row = [&](int r) {
+    float cut, mass;
+    row_cut(rowptr(r), V, s_max[r], invT, top_k, top_p, cs, &cut, &mass);
+    if (tid == 0) { s_cut[r] = cut; s_sum[r] = mass; }
+    __syncthreads();
+  };
 
   // ---- phase 2: accept chain, left to right
   const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
-  if (tid == 0) {
-    int stop = K;
-    for (int t = 0; t < K; ++t) {
-      int d = drafts[t];
-      if (d < 0 || d >= V) { d = 0; if (a.st) atomicExch(a.st->err, 1); }
-      const float qd = expf((qrow[(long long)t * V + d] - s_max[t]) * invT) / s_sum[t];
-      const float pd = expf((prow[(long long)t * V + d] - s_max[K + 1 + t]) * invT) / s_sum[K + 1 + t];
-      // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
-      const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
-      const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)t);
-      if (!(u.u_acc < ratio)) { stop = t; break; }
+  auto accept_at = [&](int t) {   // thread 0: does draft t pass?
+    int d = drafts[t];
+    if (d < 0 || d >= V) { d = 0; if (a.st) atomicExch(a.st->err, 1); }
+    const float lq = qrow[(long long)t * V + d], lp = prow[(long long)t * V + d];
+    const float qd = lq >= s_cut[t] ? expf((lq - s_max[t]) * invT) / s_sum[t] : 0.f;
+    const float pd = lp >= s_cut[K + 1 + t] ? expf((lp - s_max[K + 1 + t]) * invT) / s_sum[K + 1 + t] : 0.f;
+    // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
+    const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
+    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)t);
+    return u.u_acc < ratio;
+  };
+  if (!filt) {
+    if (tid == 0) {
+      int stop = K;
+      for (int t = 0; t < K; ++t)
+        if (!accept_at(t)) { stop = t; break; }
+      s_stop = stop;
     }
-    s_stop = stop;
+    __syncthreads();
+  } else {
+    if (tid == 0) s_stop = K;
+    __syncthreads();
+    for (int t = 0; t < K; ++t) {
+      cut_row(t);
+      cut_row(K + 1 + t);
+      if (tid == 0 && !accept_at(t)) s_stop = t;
+      __syncthreads();
+      if (s_stop != K) break;
+    }
+    if (s_stop == K) cut_row(K);
   }
-  __syncthreads();
   const int stop = s_stop;
   uint32_t fl = 0;
   int tok;
@@ -287,10 +475,14 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     const float mq = s_max[stop], mp = s_max[K + 1 + stop];
     const float iq = 1.0f / s_sum[stop], ip = 1.0f / s_sum[K + 1 + stop];
     const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)stop);
+    const float cq = s_cut[stop], cp = s_cut[K + 1 + stop];
     auto wres = [&](int i) {
-      return fmaxf(0.f, expf((ql[i] - mq) * invT) * iq - expf((pl[i] - mp) * invT) * ip);
+      const float lq = ql[i], lp = pl[i];
+      const float qv = lq >= cq ? expf((lq - mq) * invT) * iq : 0.f;
+      const float pv = lp >= cp ? expf((lp - mp) * invT) * ip : 0.f;
+      return fmaxf(0.f, qv - pv);
     };
-    auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
+    auto wq = [&](int i) { const float lq = ql[i]; return lq >= cq ? expf((lq - mq) * invT) : 0.f; };
     float total;
     if (a.smem_weights) {
       for (int i = tid; i < V; i += SAMPLER_THREADS) ws[skew(i)] = wres(i);
@@ -307,9 +499,9 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   } else {
     // ---- every draft accepted: extra token from the (K+1)-th target distribution
     const float* ql = qrow + (long long)K * V;
-    const float mq = s_max[K];
+    const float mq = s_max[K], cq = s_cut[K];
     const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)K);
-    auto wq = [&](int i) { return expf((ql[i] - mq) * invT); };
+    auto wq = [&](int i) { const float lq = ql[i]; return lq >= cq ? expf((lq - mq) * invT) : 0.f; };
     if (a.smem_weights) {
       for (int i = tid; i < V; i += SAMPLER_THREADS) ws[skew(i)] = wq(i);
       __syncthreads();

@@ -1,0 +1,137 @@
+"""GPU parity of top-k / nucleus / greedy filtering (sps_sample_filtered, sps_accept_filtered, sps_set_sampling)
+with the CPU oracle.
+
+Tolerance: tokens, accept counts and flags are bit-exact except where the oracle flags a near tie: the accept
+test within 1e-4, an inverse-CDF draw within 2e-6 * total of an interval edge, or a nucleus cut whose running
+mass passes top_p * Z_k within 1e-5 * Z_k; those are counted and must stay rare.  Top-k alone depends on
+comparisons of the logits only and has no tie band of its own."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2302_01318_b200 as sps
+import sps_synth
+from test_gpu_sampler import DEV, t32
+
+pytestmark = pytest.mark.gpu
+NEAR = oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF | oracle.FLAG_NEAR_CUT
+
+SETTINGS = [(1, 1.0), (5, 1.0), (40, 1.0), (0, 0.8), (0, 0.95), (0, 0.3), (50, 0.9), (3, 0.5)]
+
+
+@pytest.mark.parametrize("V", [2, 17, 1000, 32000, 40000])
+@pytest.mark.parametrize("top_k,top_p", SETTINGS)
+def test_filtered_sample_matches_oracle(V, top_k, top_p):
+    rng = np.random.default_rng(V + top_k)
+    B, T = 32, 0.8
+    lg = (rng.normal(size=(B, V)) * 3).astype(np.float32)
+    out = torch.zeros(B, dtype=torch.int32, device=DEV)
+    sps.sps_sample_filtered(t32(lg), T, top_k, top_p, 5, 1, 0, out)
+    got = out.cpu().numpy()
+    near = 0
+    for b in range(B):
+        u = oracle.uniforms(5, b, 1, 0)[0]
+        tok, nt = oracle.sample_row(lg[b], T, u, top_k=top_k, top_p=top_p)
+        pr, _ = oracle.filtered(lg[b], T, top_k, top_p)
+        if got[b] != tok:
+            assert nt, (b, got[b], tok)
+            near += 1
+        else:
+            assert pr[got[b]] > 0
+    assert near <= 2
+
+
+def test_filtered_sample_with_ties_and_extreme_logits():
+    V = 4096
+    lg = np.zeros((4, V), dtype=np.float32)
+    lg[1, ::7] = 2.0                      # 586 tied maxima
+    lg[2] = -np.arange(V) * 0.01           # strictly decreasing
+    lg[3, :] = -1e30
+    lg[3, 100] = 5.0
+    lg[3, 200] = 5.0
+    for top_k, top_p in [(1, 1.0), (10, 1.0), (0, 0.5), (600, 0.9)]:
+        out = torch.zeros(4, dtype=torch.int32, device=DEV)
+        sps.sps_sample_filtered(t32(lg), 1.0, top_k, top_p, 9, 0, 3, out)
+        got = out.cpu().numpy()
+        for b in range(4):
+            u = oracle.uniforms(9, b, 0, 3)[0]
+            tok, nt = oracle.sample_row(lg[b], 1.0, u, top_k=top_k, top_p=top_p)
+            assert got[b] == tok or nt, (top_k, top_p, b, got[b], tok)
+
+
+def run_accept_f(q, p, d, T, top_k, top_p, seed, step):
+    B, K1, V = q.shape
+    K = K1 - 1
+    n_acc = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+    toks = torch.full((B, K + 1), -7, dtype=torch.int32, device=DEV)
+    flags = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+    sps.sps_accept_filtered(t32(q), t32(p), t32(d), T, top_k, top_p, seed, step, n_acc, toks, flags)
+    torch.cuda.synchronize()
+    return n_acc.cpu().numpy(), toks.cpu().numpy(), flags.cpu().numpy()
+
+
+@pytest.mark.parametrize("top_k,top_p", SETTINGS)
+@pytest.mark.parametrize("V,K", [(1000, 4), (32000, 4), (32000, 1)])
+def test_filtered_accept_matches_oracle(V, K, top_k, top_p):
+    B, T, seed, step = 24, 0.9, 13, 2
+    q, p, _ = sps_synth.sampler_batch(B, K, V, seed=V + K + top_k, sigma=2.0)
+    # drafts as the algorithm would draw them: from the filtered draft law
+    d = np.zeros((B, K), dtype=np.int32)
+    for b in range(B):
+        for t in range(K):
+            d[b, t], _ = oracle.sample_row(p[b, t], T, oracle.uniforms(seed, b, step, t)[0], top_k=top_k, top_p=top_p)
+    na, tk, fl = run_accept_f(q, p, d, T, top_k, top_p, seed, step)
+    ona, otk, ofl = oracle.accept_batch(q, p, d, T, seed, step, top_k=top_k, top_p=top_p)
+    near = 0
+    for b in range(B):
+        same = na[b] == ona[b] and (tk[b] == otk[b]).all() and fl[b] == (ofl[b] & 7)
+        if not same:
+            assert ofl[b] & NEAR, (b, na[b], ona[b], tk[b], otk[b], fl[b], ofl[b])
+            near += 1
+        a = na[b]
+        assert 0 <= a <= K and (tk[b, :a] == d[b, :a]).all() and 0 <= tk[b, a] < V and (tk[b, a + 1:] == -1).all()
+        qf, _ = oracle.filtered(q[b, a], T, top_k, top_p)
+        if not (ofl[b] & NEAR):
+            assert qf[tk[b, a]] > 0          # whatever is emitted has mass under the filtered target
+    assert near <= 2, near
+
+
+def test_greedy_accept_is_deterministic_and_follows_argmax():
+    B, K, V = 16, 4, 32000
+    q, p, _ = sps_synth.sampler_batch(B, K, V, seed=3, sigma=2.0)
+    d = np.argmax(p, axis=-1).astype(np.int32)          # greedy drafts
+    d[::2, 1] = np.argmax(q[::2, 1], axis=-1)           # some of them agree with the target
+    for seed in (1, 2):
+        na, tk, fl = run_accept_f(q, p, d, 0.0, 0, 1.0, seed, 0)
+        for b in range(B):
+            agree = [int(d[b, t] == np.argmax(q[b, t])) for t in range(K)]
+            want = K if all(agree) else agree.index(0)
+            assert na[b] == want
+            assert tk[b, want] == np.argmax(q[b, want])
+
+
+@pytest.mark.parametrize("top_k,top_p,T", [(4, 1.0, 1.0), (0, 0.8, 1.0), (8, 0.9, 0.8), (0, 1.0, 0.0)])
+def test_generate_with_filters_matches_oracle_tokens(top_k, top_p, T):
+    """Whole loop on the fp32 parity configuration: tokens equal the oracle's outside flagged near ties."""
+    from gpu_util import make_pair
+    h, ot, od, c = make_pair("tiny")
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(0, 24, V)
+    h.sps_set_sampling(top_k, top_p)
+    osps = oracle.Sps(ot, od)
+    if T == 0.0:
+        osps.set_sampling(1, 1.0)       # greedy is the one-token limit of top-k
+        oT = 1.0
+    else:
+        osps.set_sampling(top_k, top_p)
+        oT = T
+    for K in (0, 3):
+        got, st = h.sps_generate(prompt, 24, K, T, 11)
+        want = osps.generate(prompt, 24, K, oT, 11)
+        if (got != want["tokens"]).any():
+            assert want["flags"] & NEAR, (K, got, want["tokens"])
+        if T == 0.0:
+            again, _ = h.sps_generate(prompt, 24, K, T, 12345)     # greedy output does not depend on the seed
+            assert (again == got).all()
+    h.close()
