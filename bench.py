@@ -213,10 +213,10 @@ def run_ours(args):
     # independent replicas: rank r generates the global sequences r, r + world, ... (no collective on the data path)
     seeds = replicas.shard_sequences((args.warmup + args.steps + 8) * world, rank, world)
 
-    def gen(i, k):
+    def gen(i, k, temp=None):
         prompt = sps_synth.make_prompt(seeds[i], P, V)
         t0 = time.perf_counter()
-        out, st = h.sps_generate(prompt, n_new, k, T, seeds[i])
+        out, st = h.sps_generate(prompt, n_new, k, T if temp is None else temp, seeds[i])
         return out, st, time.perf_counter() - t0
 
     def barrier():
@@ -326,6 +326,19 @@ def run_ours(args):
                                         "tokens_per_loop": sum(s["emitted"] for s in al) / al_loops,
                                         "accept_rate": sum(s["accepted"] for s in al) / (al_loops * K) if K else None,
                                         "speedup_vs_ar": al_tps / ar_tps if ar_tps else None}}
+        # the decoding settings the paper's speed table uses, on the same pair: nucleus 0.8 and greedy
+        # (top-k / nucleus / greedy filtering of both models ahead of the rejection scheme)
+        for name, top_k, top_p, temp in (("aligned_nucleus_0.8", 0, 0.8, T), ("aligned_greedy", 0, 1.0, 0.0)):
+            h.sps_set_sampling(top_k, top_p)
+            gen(0, K, temp)
+            fs = [gen(args.warmup + i, K, temp)[1] for i in range(args.aligned_steps)]
+            f_ms, f_loops = sum(s["ms_decode"] for s in fs), sum(s["loops"] for s in fs)
+            line["variants"][name] = {"value": args.aligned_steps * n_new / (f_ms / 1e3), "unit": UNIT,
+                                      "tokens_per_loop": sum(s["emitted"] for s in fs) / f_loops,
+                                      "accept_rate": sum(s["accepted"] for s in fs) / (f_loops * K) if K else None,
+                                      "ms_draft_per_step": sum(s["ms_draft"] for s in fs) / (f_loops * max(K, 1)),
+                                      "ms_accept_per_loop": sum(s["ms_accept"] for s in fs) / f_loops}
+        h.sps_set_sampling(0, 1.0)
     h.close()
     if rank == 0:
         print(json.dumps(line))
