@@ -129,16 +129,19 @@ __device__ inline float block_sum_f(float v, float* s_part, float* s_out) {
 //   top-k   : the cut is the k-th largest logit (tokens tied with it stay);
 //   nucleus : over what top-k kept, mass Z_k, the largest logit value v such that the tokens with logit
 //             >= v hold at least top_p * Z_k.
-// Both are "the largest key whose upper tail reaches a target": a radix descent over the order-preserving
-// bit pattern of the logit, eight bits per pass, with a 256-bin histogram of the tail function (token
-// counts for top-k, weights for the nucleus).  No sort.  Weights enter the histogram as 40-bit fixed
-// point integers, so the sums do not depend on the order in which threads add them.
+// Both are "the largest key whose upper tail reaches a target", the key being the order-preserving bit
+// pattern of the fp32 logit and the tail a token count (top-k) or a weight mass (nucleus).  The key is
+// built from its top bit down, two bits per step: the block evaluates the tail at the three candidate
+// keys and keeps the largest that still reaches the target.  No sort, no atomics: a thread holds the keys
+// of its 32 tokens (tid, tid + 1024, ...) in registers, the weights sit in shared memory, and every sum
+// runs in a fixed order (thread, warp butterfly, butterfly over the warps), so results are reproducible.
+// (A radix descent with shared-memory histograms was 5-10 times slower: the digits of real logits fall in
+// a handful of bins and the adds to them serialise.)
 // ------------------------------------------------------------------------------------------------
+#define CUT_ELEMS 32   // tokens per thread held in registers: rows up to 32 * 1024 tokens
 struct CutSmem {
-  unsigned long long bin[256];
-  unsigned long long acc;
-  unsigned int sel;
-  unsigned int found;
+  float f[2][3][SAMPLER_WARPS];
+  int i[2][3][SAMPLER_WARPS];
 };
 
 __device__ __forceinline__ uint32_t order_key(float f) {   // unsigned order of keys == order of the floats
@@ -148,118 +151,138 @@ __device__ __forceinline__ uint32_t order_key(float f) {   // unsigned order of 
 __device__ __forceinline__ float order_key_inv(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
-__device__ __forceinline__ unsigned long long fixed40(float w) {   // w in [0, 1]
-  return __float2ull_rn(w * 1099511627776.0f);
-}
 
-// The largest key K* (among tokens with key >= dom_key) with F(K*) = sum over tokens of key >= K* of f
-// reaching `target`; f = 1 (SUM == false) or the token's fixed-point weight.  Returns F(K*) and whether
-// such a key exists.  All threads of the block call it; all get the same answer.
-template <bool SUM>
-__device__ bool tail_descent(const float* row, int V, float m, float invT, uint32_t dom_key, unsigned long long target,
-                             CutSmem& cs, uint32_t* key_out, unsigned long long* F_out) {
-  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-  uint32_t prefix = 0, mask = 0;
-  unsigned long long acc = 0, at_key = 0;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    for (int d = tid; d < 256; d += nthr) cs.bin[d] = 0;
-    __syncthreads();
-    // a thread adds runs of equal digits locally: in the first passes nearly all tokens share one digit
-    int cur = -1;
-    unsigned long long loc = 0;
-    for (int i = tid; i < V; i += nthr) {
-      const float l = row[i];
-      const uint32_t k = order_key(l);
-      if ((k & mask) != prefix || k < dom_key) continue;
-      const int d = (int)((k >> shift) & 255u);
-      const unsigned long long f = SUM ? fixed40(expf((l - m) * invT)) : 1ull;
-      if (d != cur) {
-        if (cur >= 0) atomicAdd(&cs.bin[cur], loc);
-        cur = d;
-        loc = 0;
-      }
-      loc += f;
-    }
-    if (cur >= 0) atomicAdd(&cs.bin[cur], loc);
-    __syncthreads();
-    if (warp == 0) {
-      // lane l owns digits 255 - 8l .. 248 - 8l; the tail above them is a warp prefix sum
-      unsigned long long t = 0;
+// sums of three per-thread values over the block, the same bits in every thread; `slot` alternates
+// between consecutive calls so that one barrier per call is enough
+__device__ __forceinline__ void block_total3(float (&v)[3], CutSmem& cs, int slot) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) t += cs.bin[255 - 8 * lane - j];
-      unsigned long long incl = t;
+  for (int c = 0; c < 3; ++c) {
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      const unsigned long long above = acc + (incl - t);
-      const bool cross = above < target && above + t >= target;
-      const unsigned int who = __ballot_sync(0xffffffffu, cross);
-      if (lane == 0) cs.found = who != 0u;
-      if (cross) {
-        unsigned long long run = above;
-        for (int j = 0; j < 8; ++j) {
-          const int d = 255 - 8 * lane - j;
-          if (run + cs.bin[d] >= target) { cs.sel = (unsigned int)d; cs.acc = run; break; }
-          run += cs.bin[d];
-        }
+    for (int o = 16; o > 0; o >>= 1) v[c] += __shfl_xor_sync(0xffffffffu, v[c], o);
+    if (lane == 0) cs.f[slot][c][warp] = v[c];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < 3; ++c) {
+    float t = cs.f[slot][c][lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    v[c] = t;
+  }
+}
+__device__ __forceinline__ void block_total3(int (&v)[3], CutSmem& cs, int slot) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int c = 0; c < 3; ++c) {
+    v[c] = __reduce_add_sync(0xffffffffu, v[c]);
+    if (lane == 0) cs.i[slot][c][warp] = v[c];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int c = 0; c < 3; ++c) v[c] = __reduce_add_sync(0xffffffffu, cs.i[slot][c][lane]);
+}
+
+// The cut of one row and the mass it keeps.
+// FAST: V <= CUT_ELEMS * SAMPLER_THREADS and ws holds the row's weights exp((l - m) / T) in shared memory
+// (skewed layout, written and visible to the block).  Otherwise keys and weights are recomputed from the
+// logits in every step (large vocabularies; slow but the same arithmetic).
+template <bool FAST>
+__device__ void row_cut_impl(const float* row, const float* ws, int V, float m, float invT, int top_k, float top_p,
+                             CutSmem& cs, float* cut_out, float* mass_out) {
+  const int tid = threadIdx.x;
+  uint32_t kr[CUT_ELEMS];   // FAST: a thread's keys; 0 = no token here, or a token already cut away
+  if (FAST) {
+#pragma unroll
+    for (int j = 0; j < CUT_ELEMS; ++j) {
+      const int i = tid + j * SAMPLER_THREADS;
+      kr[j] = i < V ? order_key(row[i]) : 0u;
+    }
+  }
+  const int wbase = tid + (tid >> 5);                      // skew(tid + 1024 j) = wbase + 1056 j
+  uint32_t floor_key = 0;                                   // slow path: tokens under it are cut away
+  // visit every token of this thread: body(key, weight)
+  auto each = [&](auto body) {
+    if (FAST) {
+#pragma unroll
+      for (int j = 0; j < CUT_ELEMS; ++j)   // no token, no load: the buffer only covers V entries
+        body(kr[j], kr[j] ? ws[wbase + j * (SAMPLER_THREADS + SAMPLER_WARPS)] : 0.f);
+    } else {
+      for (int i = tid; i < V; i += SAMPLER_THREADS) {
+        const float l = row[i];
+        const uint32_t k = order_key(l);
+        body(k >= floor_key ? k : 0u, expf((l - m) * invT));
       }
     }
-    __syncthreads();
-    if (!cs.found) return false;   // the whole domain holds less than the target (callers make sure it does not)
-    prefix |= cs.sel << shift;
-    mask |= 255u << shift;
-    acc = cs.acc;
-    at_key = cs.bin[cs.sel];
-    __syncthreads();
-  }
-  *key_out = prefix;
-  *F_out = acc + at_key;
-  return true;
-}
-
-// sum over tokens with key >= dom_key of the fixed-point weight
-__device__ unsigned long long tail_mass(const float* row, int V, float m, float invT, uint32_t dom_key, CutSmem& cs) {
-  const int tid = threadIdx.x, nthr = blockDim.x;
-  if (tid == 0) cs.acc = 0;
-  __syncthreads();
-  unsigned long long loc = 0;
-  for (int i = tid; i < V; i += nthr) {
-    const float l = row[i];
-    if (order_key(l) >= dom_key) loc += fixed40(expf((l - m) * invT));
-  }
-  loc += __shfl_xor_sync(0xffffffffu, loc, 16);
-  loc += __shfl_xor_sync(0xffffffffu, loc, 8);
-  loc += __shfl_xor_sync(0xffffffffu, loc, 4);
-  loc += __shfl_xor_sync(0xffffffffu, loc, 2);
-  loc += __shfl_xor_sync(0xffffffffu, loc, 1);
-  if ((tid & 31) == 0) atomicAdd(&cs.acc, loc);
-  __syncthreads();
-  const unsigned long long z = cs.acc;
-  __syncthreads();
-  return z;
-}
-
-// The cut of one row and the mass it keeps (sum of exp((l - m) / T) over kept tokens).  m = the row's maximum.
-__device__ void row_cut(const float* row, int V, float m, float invT, int top_k, float top_p, CutSmem& cs,
-                        float* cut_out, float* mass_out) {
-  uint32_t key = 0;   // keep everything
-  unsigned long long F = 0;
+  };
+  uint32_t key = 0;
+  int slot = 0;
   if (top_k >= 1 && top_k < V) {
-    if (!tail_descent<false>(row, V, m, invT, 0u, (unsigned long long)top_k, cs, &key, &F)) key = 0;
+#pragma unroll 1
+    for (int b = 30; b >= 0; b -= 2) {
+      int cnt[3] = {0, 0, 0};
+      const uint32_t c1 = key | (1u << b), c2 = key | (2u << b), c3 = key | (3u << b);
+      each([&](uint32_t k, float) {
+        cnt[0] += k >= c1;
+        cnt[1] += k >= c2;
+        cnt[2] += k >= c3;
+      });
+      block_total3(cnt, cs, slot);
+      slot ^= 1;
+      key = cnt[2] >= top_k ? c3 : (cnt[1] >= top_k ? c2 : (cnt[0] >= top_k ? c1 : key));
+    }
+    if (FAST) {
+#pragma unroll
+      for (int j = 0; j < CUT_ELEMS; ++j)
+        if (kr[j] < key) kr[j] = 0u;
+    }
+    floor_key = key;
   }
-  unsigned long long Z = tail_mass(row, V, m, invT, key, cs);
+  // mass of what is left
+  float z[3] = {0.f, 0.f, 0.f};
+  each([&](uint32_t k, float w) { if (k) z[0] += w; });
+  block_total3(z, cs, slot);
+  slot ^= 1;
+  float Z = z[0];
   if (top_p < 1.0f) {
-    unsigned long long target = (unsigned long long)((double)top_p * (double)Z);
-    if (target < 1ull) target = 1ull;
-    uint32_t kp;
-    unsigned long long Fp;
-    if (target <= Z && tail_descent<true>(row, V, m, invT, key, target, cs, &kp, &Fp)) { key = kp; Z = Fp; }
+    const float target = top_p * Z;
+    uint32_t kp = 0;
+#pragma unroll 1
+    for (int b = 30; b >= 0; b -= 2) {
+      float sm3[3] = {0.f, 0.f, 0.f};
+      const uint32_t c1 = kp | (1u << b), c2 = kp | (2u << b), c3 = kp | (3u << b);
+      each([&](uint32_t k, float w) {
+        if (k >= c1) sm3[0] += w;
+        if (k >= c2) sm3[1] += w;
+        if (k >= c3) sm3[2] += w;
+      });
+      block_total3(sm3, cs, slot);
+      slot ^= 1;
+      kp = sm3[2] >= target ? c3 : (sm3[1] >= target ? c2 : (sm3[0] >= target ? c1 : kp));
+    }
+    if (kp > key) {
+      key = kp;
+      float zz[3] = {0.f, 0.f, 0.f};
+      each([&](uint32_t k, float w) { if (k >= key) zz[0] += w; });
+      block_total3(zz, cs, slot);
+      Z = zz[0];
+    }
   }
+  __syncthreads();   // the scratch may be reused at once by the caller's next cut
   *cut_out = key == 0u ? -INFINITY : order_key_inv(key);
-  *mass_out = (float)((double)Z * (1.0 / 1099511627776.0));
+  *mass_out = Z;
+}
+
+// Cuts row `row` (maximum m).  With have_ws the weights are staged in ws first (the caller's shared buffer).
+__device__ void row_cut(const float* row, float* ws, bool have_ws, int V, float m, float invT, int top_k, float top_p,
+                        CutSmem& cs, float* cut_out, float* mass_out) {
+  if (have_ws && V <= CUT_ELEMS * SAMPLER_THREADS) {
+    for (int i = threadIdx.x; i < V; i += SAMPLER_THREADS) ws[i + (i >> 5)] = expf((row[i] - m) * invT);
+    __syncthreads();
+    row_cut_impl<true>(row, ws, V, m, invT, top_k, top_p, cs, cut_out, mass_out);
+  } else {
+    row_cut_impl<false>(row, ws, V, m, invT, top_k, top_p, cs, cut_out, mass_out);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -289,11 +312,11 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
     float m = -INFINITY;
     for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
     m = block_max_f(m, s_part, &s_val);
+    extern __shared__ float ws[];
     float cut, mass;
-    row_cut(row, a.V, m, invT, top_k, top_p, cs, &cut, &mass);
+    row_cut(row, ws, a.smem_weights != 0, a.V, m, invT, top_k, top_p, cs, &cut, &mass);
     auto w = [&](int i) { const float l = row[i]; return l >= cut ? expf((l - m) * invT) : 0.f; };
     if (a.smem_weights) {
-      extern __shared__ float ws[];
       for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = w(i);
       __syncthreads();
       tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
@@ -427,7 +450,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   // chain reaches them (block-wide work), so a loop that stops early does not pay for the later rows
   auto cut_row = [&](int r) {
     float cut, mass;
-    row_cut(rowptr(r), V, s_max[r], invT, top_k, top_p, cs, &cut, &mass);
+    row_cut(rowptr(r), ws, a.smem_weights != 0, V, s_max[r], invT, top_k, top_p, cs, &cut, &mass);
     if (tid == 0) { s_cut[r] = cut; s_sum[r] = mass; }
     __syncthreads();
   };

@@ -207,7 +207,13 @@ def test_error_paths():
         h.sps_generate(prompt, 8, 5, 1.0, 0)             # K > max_K
     assert e.value.code == sps.SPS_EINVAL
     with pytest.raises(sps.SpsError) as e:
-        h.sps_generate(prompt, 8, 4, 0.0, 0)
+        h.sps_generate(prompt, 8, 4, -1.0, 0)            # temperature 0 is greedy decoding, below 0 is an error
+    assert e.value.code == sps.SPS_EINVAL
+    with pytest.raises(sps.SpsError) as e:
+        h.sps_set_sampling(-1, 1.0)
+    assert e.value.code == sps.SPS_EINVAL
+    with pytest.raises(sps.SpsError) as e:
+        h.sps_set_sampling(0, 0.0)
     assert e.value.code == sps.SPS_EINVAL
     h.sps_reset()
     with pytest.raises(sps.SpsError) as e:
