@@ -46,6 +46,19 @@ def test_linear_bf16_small(M, N, D):
     assert np.abs(got - want).max() <= tol(W.float(), X, D)
 
 
+@pytest.mark.parametrize("M", [1, 5, 16])
+def test_linear_bf16_width_with_a_large_prime_factor(M):
+    """D = 128 * 67 only splits into 67 ranges of 128: more than the TMA kernel's tile queues, so the
+    register-streaming kernel takes it."""
+    N, D = 300, 128 * 67
+    g = torch.Generator().manual_seed(M)
+    W = (torch.randn((N, D), generator=g) * 0.05).to(torch.bfloat16)
+    X = torch.randn((M, D), generator=g)
+    got = run_linear(W.to(DEV), X.to(DEV))
+    want = oracle.linear(sps_synth.to_numpy(W), X.numpy())
+    assert np.abs(got - want).max() <= tol(W.float(), X, D)
+
+
 @pytest.mark.parametrize("M", [1, 5, 9])
 @pytest.mark.parametrize("N,D", [(1024, 256), (130, 128), (515, 1024)])
 def test_linear_fp32(M, N, D):
