@@ -170,10 +170,12 @@ struct LinArgs {
   long long ldyp;
   const float* yp_gain;         // [N] multiplied in before packing, null = ones
   int yp_act;                   // PRO_GELU: gelu before packing; PRO_NONE: none
+  int split_epi;                // set by the launcher: the split-K epilogue runs as a kernel of its own
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };
 LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
+int lin_launch_count(const LinPlan& p);   // kernels one lin_launch enqueues
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
 size_t lin_part_floats(int N, int S_max);
 void sps_set_global_error(const char* msg);   // text returned by sps_last_error(NULL)
@@ -182,6 +184,7 @@ void sps_set_global_error(const char* msg);   // text returned by sps_last_error
 #define SSQ_IDX(part, row) ((size_t)(row) * LIN_MAX_R + (size_t)(part))
 #define LIN_CONSUMER_WARPS 8
 #define LIN_MAX_S 64
+#define LIN_SCALE_SLOT 768   // counters[768..783] as floats: the rows' 1/rms handed from the layer kernel to its epilogue kernel
 
 // ------------------------------------------------------------------------------------------------
 // Rows / embedding, attention, samplers

@@ -190,7 +190,8 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
       if (m.packed && l > 0) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }   // left there by the layer below
       a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = 3 * d;
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
+      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
     }
     {
       AttnArgs aa{};
@@ -209,7 +210,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       if (m.packed) { a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_gain = (const float*)m.ffn_norm[l]; a.yp_act = PRO_NONE; }
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
       nB = pl.ssq_parts;
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
     }
     {  // up = Wup rmsnorm(x, g_ffn)
       LinArgs a = base;
@@ -221,7 +222,8 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
         a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo;
         a.yp_hi = h->up_hi; a.yp_lo = h->up_lo; a.ldyp = dff; a.yp_gain = nullptr; a.yp_act = PRO_GELU;
       }
-      CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, rows, a.N, a.D, h->num_sm), st)); h->launches++;
+      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
     }
     {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
       LinArgs a = base;
@@ -235,7 +237,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       }
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
       nA = pl.ssq_parts;
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches++;
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
     }
   }
   if (ps.logits) {
@@ -245,7 +247,8 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
     if (m.packed) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }
     a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
-    CU(h, lin_launch(c.dtype, a, lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm), st)); h->launches++;
+    const LinPlan pl = lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm);
+    CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
   }
   return SPS_OK;
 }

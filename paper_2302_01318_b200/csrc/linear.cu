@@ -776,6 +776,22 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
     }
   }
+  if (a.split_epi) {
+    // The split-K epilogue is a kernel of its own (lin_epilogue_kernel): this CTA is done once its partial
+    // results are written, and its SM is free for the next layer's CTA, which starts streaming weights
+    // while the slower CTAs of this grid are still at work.  The last CTA to leave re-arms the tile queues.
+    __syncthreads();
+    if (tid == 0) {
+      if (a.xp_hi && a.pro == PRO_RMSNORM && cta == 0)
+        for (int m = 0; m < a.M; ++m) reinterpret_cast<float*>(a.counters + LIN_SCALE_SLOT)[m] = s_scale[m];
+      if (C == 1 || atomicAdd(&a.counters[1], 1) == C - 1) {
+        a.counters[0] = 0;
+        a.counters[1] = 0;
+        for (int i = 0; i < a.S; ++i) a.counters[2 + i] = 0;
+      }
+    }
+    return;
+  }
   // ---- arrival.  All CTAs of the grid meet on a counter; once every partial result is visible each CTA
   // finishes 1/C of the layer's rows, so the split-K reduction is C-way parallel and short.  The grid
   // never exceeds one CTA per SM, so all of them are resident together and the wait ends as soon as the
@@ -817,6 +833,30 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       for (int i = 0; i < a.S; ++i) a.counters[2 + i] = 0;
     }
   }
+}
+
+// ---- the split-K epilogue of the TMA kernel as a kernel of its own.  Its CTAs are small enough to sit
+// beside the layer kernel's on the same SMs: they wait for that grid to complete (the hardware's grid-wide
+// meeting), then each finishes its slice of the output columns.
+__global__ void __launch_bounds__(256) lin_epilogue_kernel(const LinArgs a, int C) {
+  __shared__ float sq_s[1024];
+  __shared__ float ssq_s[SPS_MAX_ROWS];
+  __shared__ float row_scale[SPS_MAX_ROWS];
+  const int cta = blockIdx.x, tid = threadIdx.x;
+  pdl_launch_dependents();
+  const int quads = (a.N + 3) >> 2;
+  const int q0 = (int)(((long long)cta * quads) / C), q1 = (int)(((long long)(cta + 1) * quads) / C);
+  const int b0 = min(q0 * 4, a.N), b1 = min(q1 * 4, a.N);
+  if (a.yp_gain && tid < 32) {
+    // the gain of the packed output is a weight in HBM: ask for this slice before the wait
+    const int n = b0 + tid * 32;
+    if (n < b1) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.yp_gain + n));
+  }
+  pdl_wait();
+  const bool scaled = a.xp_hi && a.pro == PRO_RMSNORM;
+  if (scaled && tid < a.M) row_scale[tid] = __ldcg(reinterpret_cast<const float*>(a.counters + LIN_SCALE_SLOT) + tid);
+  __syncthreads();
+  lin_epilogue_slice(a, cta, b0, b1 - b0, sq_s, 1024, ssq_s, scaled ? row_scale : nullptr);
 }
 
 // ---- fp32 weights: one warp per output row, X (after the prologue) in shared memory ---------------
@@ -889,6 +929,12 @@ __global__ void __launch_bounds__(256) lin_f32_kernel(const LinArgs a) {
 static const size_t kSmemBudget = 200 * 1024;
 // TMA variant: everything a CTA may ask for (227 KB) less the kernel's 1 KB of static shared memory and a little slack
 static const size_t kSmemTma = 225 * 1024;
+
+static bool lin_split_epilogue() {
+  static const bool on = [] { const char* e = getenv("SPS_LIN_SPLIT_EPI"); return !(e && atoi(e) == 0); }();
+  return on;
+}
+int lin_launch_count(const LinPlan& p) { return (p.variant == 2 && p.KS > 0 && lin_split_epilogue()) ? 2 : 1; }
 
 bool sps_pdl_enabled() {
   static const bool on = [] { const char* e = getenv("SPS_PDL"); return !(e && atoi(e) == 0); }();
@@ -1046,6 +1092,7 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     const int nmat = a.N / a.rows_per_mat > 0 ? (a.N + a.rows_per_mat - 1) / a.rows_per_mat : 1;
     for (int i = 0; i < 3; ++i)
       if ((e = weight_tensor_map(a.W[i < nmat ? i : 0], a.rows_per_mat, a.D, p.KST, &ta.tm[i])) != cudaSuccess) return e;
+    ta.a.split_epi = lin_split_epilogue() ? 1 : 0;
     if (p.NT == 1) {
       if ((e = ensure_smem(lin_bf16_tma_kernel<1>, p.smem, c_t1)) != cudaSuccess) return e;
       e = launch_k(lin_bf16_tma_kernel<1>, grid, dim3(threads), p.smem, st, ta);
@@ -1053,6 +1100,7 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
       if ((e = ensure_smem(lin_bf16_tma_kernel<2>, p.smem, c_t2)) != cudaSuccess) return e;
       e = launch_k(lin_bf16_tma_kernel<2>, grid, dim3(threads), p.smem, st, ta);
     }
+    if (e == cudaSuccess && ta.a.split_epi) e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
   } else {
     dim3 grid(p.R, p.S);
     if (p.NT == 1) {
