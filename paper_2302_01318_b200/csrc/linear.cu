@@ -838,7 +838,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 // ---- the split-K epilogue of the TMA kernel as a kernel of its own.  Its CTAs are small enough to sit
 // beside the layer kernel's on the same SMs: they wait for that grid to complete (the hardware's grid-wide
 // meeting), then each finishes its slice of the output columns.
-__global__ void __launch_bounds__(256) lin_epilogue_kernel(const LinArgs a, int C) {
+__global__ void __launch_bounds__(256, 5) lin_epilogue_kernel(const LinArgs a, int C) {   // <= 48 registers: it has to fit beside the layer kernel
   __shared__ float sq_s[1024];
   __shared__ float ssq_s[SPS_MAX_ROWS];
   __shared__ float row_scale[SPS_MAX_ROWS];
@@ -1100,7 +1100,17 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
       if ((e = ensure_smem(lin_bf16_tma_kernel<2>, p.smem, c_t2)) != cudaSuccess) return e;
       e = launch_k(lin_bf16_tma_kernel<2>, grid, dim3(threads), p.smem, st, ta);
     }
-    if (e == cudaSuccess && ta.a.split_epi) e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
+    if (e == cudaSuccess && ta.a.split_epi) {
+      // The epilogue CTAs must fit beside the layer kernel's on the same SM: that needs the same split between
+      // L1 and shared memory, i.e. the largest shared-memory carve-out, although they use only 5 KB of it.
+      static bool carve_set = false;
+      if (!carve_set) {
+        e = cudaFuncSetAttribute(lin_epilogue_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        carve_set = true;
+      }
+      e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
+    }
   } else {
     dim3 grid(p.R, p.S);
     if (p.NT == 1) {
