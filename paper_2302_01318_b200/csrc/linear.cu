@@ -671,6 +671,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
     // lane (g, t) reads logical 16-byte chunks 2t and 2t+1 of every 128-byte (64 k) row segment; the
     // swizzle stores logical chunk c of row g at physical chunk c ^ (g & 7)
     const uint32_t wchunk0 = (uint32_t)(((2 * t) ^ g) << 4), wchunk1 = (uint32_t)(((2 * t + 1) ^ g) << 4);
+    const bool pk = NT == 1 && a.M <= 4;   // both halves of the activations fit the eight columns of one MMA
     int round = 0;
     for (int L = grp; alive; L += NG, ++round) {
       // wait until local tile L has been issued, or until the producer has run out of tiles
@@ -708,6 +709,23 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) xrow[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xoff;   // columns beyond M read the zero row
         const int slabs = KST >> 6;
+        if (pk) {
+          // Up to four activation rows: one MMA carries both halves -- columns 0..3 the high parts of rows
+          // 0..3, columns 4..7 their low parts (lane group g reads one source row) -- so a k-step costs half
+          // the MMAs and half the activation loads; the two halves of a column meet in a shuffle at the end.
+          const uint32_t xsrc = (g < 4 ? xs_hi : xs_lo) + (uint32_t)min(g & 3, a.M) * XP + xoff;
+#pragma unroll 2
+          for (int q = 0; q < slabs; ++q) {
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              const uint32_t wc = hf ? wchunk1 : wchunk0;
+              const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
+              const uint4 x = lds128(xsrc + q * 128 + hf * 16);
+              mma_bf16_16816(acc[0][0], wa.x, wb.x, wa.y, wb.y, x.x, x.y);
+              mma_bf16_16816(acc[0][2], wa.z, wb.z, wa.w, wb.w, x.z, x.w);
+            }
+          }
+        } else
 #pragma unroll 2
         for (int q = 0; q < slabs; ++q) {
 #pragma unroll
@@ -737,6 +755,11 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[nt][i] = (acc[nt][0][i] + acc[nt][1][i]) + (acc[nt][2][i] + acc[nt][3][i]);
+      if (pk) {
+        // column c (lanes t = 0, 1) += column c + 4 (lanes t = 2, 3): high-part sum + low-part sum
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[0][i] += __shfl_xor_sync(0xffffffffu, c[0][i], 2);
+      }
       if (G > 1) {
         // element e = col * 16 + row of the 16 x (8*NT) tile
         float* mine = gscr + ((size_t)(round & 1) * NCW + warp) * (NT * 128);
