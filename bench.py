@@ -340,11 +340,52 @@ def run_ours(args):
                                       "ms_accept_per_loop": sum(s["ms_accept"] for s in fs) / f_loops}
         h.sps_set_sampling(0, 1.0)
     h.close()
+    if rank == 0 and world == 1 and not args.no_sampler:
+        line["sampler"] = sampler_bench(dev, peak)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def sampler_bench(dev, peak_gbs):
+    """The fused accept / resample / extra-token kernel alone (vocab 32000, K = 4, target logits N(0, 9), draft =
+    target + N(0, 1)): device time per launch against the time its reads, V * (2K + 1) * 4 bytes per sequence, take
+    at the measured HBM rate.  One CTA per sequence: at batch 1 the kernel is a latency chain on one SM, not a
+    bandwidth problem, and its 1.15 MB of logits were just written by the two models (L2-resident, as here)."""
+    import torch
+    import paper_2302_01318_b200 as sps
+    out = []
+    K, V = 4, 32000
+    for B in (1, 8, 64):
+        ncopy = max(2, int(160e6 // (B * (2 * K + 1) * V * 4)) + 1) if B >= 8 else 2   # B >= 8: rotate past the L2
+        bufs = []
+        for i in range(ncopy):
+            q, p, d = sps_synth.sampler_batch(B, K, V, seed=i, sigma=1.0)
+            bufs.append([torch.from_numpy(x).to(dev) for x in (q, p, d)])
+        na = torch.zeros(B, dtype=torch.int32, device=dev)
+        tk = torch.zeros((B, K + 1), dtype=torch.int32, device=dev)
+        fl = torch.zeros(B, dtype=torch.int32, device=dev)
+        def run(i):
+            q, p, d = bufs[i % ncopy]
+            sps.sps_accept(q, p, d, 1.0, 7, i, na, tk, fl)
+        for i in range(5):
+            run(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 40
+        e0.record()
+        for i in range(n):
+            run(5 + i)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        nbytes = B * (2 * K + 1) * V * 4
+        bound_us = nbytes / (peak_gbs * 1e9) * 1e6
+        out.append({"B": B, "K": K, "V": V, "us": us, "read_bytes": nbytes, "bound_us": bound_us, "frac": bound_us / us,
+                    "mean_accepted": float(na.float().mean().item())})
+    return out
 
 
 def main():
@@ -359,6 +400,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--aligned-steps", type=int, default=2)
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
+    ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per launch of the dominant kernel; default: bytes_per_launch x the ratio measured in profiles/")
     args = ap.parse_args()
