@@ -208,7 +208,7 @@ def run_ours(args):
     P, n_new, T = c["prompt_len"], c["n_new"], 1.0
     V = c["target"]["vocab"]
     max_seq = ((P + n_new + max(K, 8) + 63) // 64) * 64
-    h = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=max_seq, max_batch=1, max_K=max(K, 1), device=local)
+    h = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=max_seq, max_batch=1, max_K=max(K, 8), device=local)
     from paper_2302_01318_b200 import replicas
     # independent replicas: rank r generates the global sequences r, r + world, ... (no collective on the data path)
     seeds = replicas.shard_sequences((args.warmup + args.steps + 8) * world, rank, world)
@@ -339,6 +339,16 @@ def run_ours(args):
                                       "ms_draft_per_step": sum(s["ms_draft"] for s in fs) / (f_loops * max(K, 1)),
                                       "ms_accept_per_loop": sum(s["ms_accept"] for s in fs) / f_loops}
         h.sps_set_sampling(0, 1.0)
+        # lookahead sweep on the damped pair (the paper's K trade-off figure): one generation per K
+        if args.k_sweep:
+            sweep = []
+            for k in (1, 2, 3, 4, 6, 8):
+                gen(0, k)
+                st = gen(args.warmup, k)[1]
+                sweep.append({"K": k, "value": n_new / (st["ms_decode"] / 1e3), "tokens_per_loop": st["emitted"] / st["loops"],
+                              "accepted_per_loop": st["accepted"] / st["loops"], "ms_verify_per_loop": st["ms_verify"] / st["loops"],
+                              "ms_draft_per_step": st["ms_draft"] / (st["loops"] * k)})
+            line["variants"]["k_sweep"] = sweep
     h.close()
     if rank == 0 and world == 1 and not args.no_sampler:
         line["sampler"] = sampler_bench(dev, peak)
@@ -400,6 +410,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--aligned-steps", type=int, default=2)
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
+    ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per launch of the dominant kernel; default: bytes_per_launch x the ratio measured in profiles/")
