@@ -1,20 +1,19 @@
 // The memory-bound linear layer of the draft steps (M = 1..2) and of the scoring pass (M = K+1):
 //   Y[M,N] = f(X)[M,D] W[N,D]^T,  W streamed once from HBM in its caller-owned row-major layout.
 //
-// bf16 path.  The weights are the 16-row "A" operand of mma.m16n8k16 and the (at most 16) activation
-// rows are the narrow "B" side, so the tensor cores only keep the FMA work off the critical path.
-// A warp owns a 128-wide slice of the reduction dimension for a whole range of output rows: its slice
-// of X is split into bf16 hi + lo parts once (fp32-grade accuracy with bf16 MMAs) and stays in
-// registers, while weight rows stream through registers with 128-bit loads, one 16-row tile of
-// look-ahead.  A dot product does not care about the order of k, so each lane feeds the 8 consecutive
-// bf16 it loaded straight into two MMAs and X uses the same permutation: no shared-memory staging
-// or transposes of the weights at all.
-// Partial sums meet in three fixed-order steps: the warps of a CTA through shared memory, the CTAs
-// that split D through an L2-resident scratch buffer (the last CTA to arrive sums them in split
-// order, not arrival order), and -- for the residual epilogue -- the per-range sums of squares that
-// the next RMSNorm needs.  No floating-point atomics: results are bit-reproducible.
-//
-// fp32 path (token-exact parity configuration): one warp per output row, plain FMAs.
+// Three kernels share one protocol (prologue: RMSNorm apply / GeLU / packed input; epilogue: store or
+// residual add with the sums of squares the next norm needs):
+//   lin_bf16_tma_kernel  bf16 weights, the product path: a TMA-fed shared-memory ring, mma.m16n8k16 with
+//                        the weights as the 16-row A operand, activations split into bf16 high + low
+//                        parts (fp32-grade accuracy), run-time tile queues, split-K partials reduced by
+//                        lin_epilogue_kernel.  Described at the kernel.
+//   lin_bf16_kernel      bf16 weights streamed through registers with 128-bit loads (one 16-row tile of
+//                        look-ahead per warp; each lane feeds the 8 consecutive bf16 it loaded straight
+//                        into two MMAs, X uses the same k permutation).  4.9 TB/s: kept as the fallback for
+//                        widths the TMA kernel cannot split.
+//   lin_f32_kernel       fp32 weights (the token-exact parity configuration): one warp per output row.
+// Partial sums always meet in a fixed order (warps of a CTA, then the k-splits in split order, then the
+// per-CTA sums of squares in CTA order): no floating-point atomics, results are bit-reproducible.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
@@ -368,17 +367,19 @@ __global__ void __launch_bounds__(NT == 1 ? 512 : 384, 1) lin_bf16_kernel(const 
 
 
 // ================================================================================================
-// TMA variant (the default for bf16).  CTA (r, s) owns a range of 16-row output tiles and the k-range
-// [s*KS, (s+1)*KS).  One producer lane feeds a ring of NS stages with tiled TMA loads
-// (cp.async.bulk.tensor, one instruction per stage: 16 weight rows x KST k), completion counted on an
-// mbarrier; the weight matrix is described to the copy engine as [D/64][rows][64] with the 128-byte
-// swizzle, so a stage lands as KST/64 slabs of 16 rows x 128 bytes whose 16-byte chunks are XOR-ed with
-// the row index.  Consumer warps take tiles in turn; a warp walks its tile's KS/KST stages, reading A
-// fragments with 128-bit shared loads (lane t reads logical chunks 2t and 2t+1 of each 128-byte row, which
-// the swizzle spreads over all banks) and the hi / lo B fragments of X from a slab prepared once per CTA
-// in the same k order.  A tile belongs to one warp from start to end: no cross-warp reduction and no
-// CTA-wide barrier in the main loop.  Every wait is bounded: when one runs out the warp records error 3
-// and stops, and the producer lets the copies already issued land before the CTA leaves.
+// TMA variant (the default for bf16).  CTA (r, s) works on the k-range [s*KS, (s+1)*KS); the R CTAs of a
+// k-range draw 16-row output tiles from a shared counter at run time.  One producer lane feeds a ring of NS
+// stages with tiled TMA loads (cp.async.bulk.tensor, one instruction per stage: 16 weight rows x KST k),
+// completion counted on an mbarrier; the weight matrix is described to the copy engine as
+// [D/64][rows][64] with the 128-byte swizzle, so a stage lands as KST/64 slabs of 16 rows x 128 bytes
+// whose 16-byte chunks are XOR-ed with the row index.  Consumer warps work in groups of G, one tile per
+// group and one stage per warp at a time, reading A fragments with 128-bit shared loads (lane t reads
+// logical chunks 2t and 2t+1 of each 128-byte row, which the swizzle spreads over all banks) and the
+// hi / lo B fragments of X from a slab in the same k order -- converted here from fp32, or copied in
+// ready-made when the producing layer left it packed.  The G partial tiles meet in a small shared
+// scratch; there is no CTA-wide barrier in the main loop.  A CTA ends when its partial sums are written:
+// lin_epilogue_kernel adds the k-splits up.  Every wait is bounded: when one runs out the warp records
+// error 3 and stops, and the producer lets the copies already issued land before the CTA leaves.
 // ================================================================================================
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
