@@ -339,6 +339,17 @@ def run_ours(args):
                                       "ms_draft_per_step": sum(s["ms_draft"] for s in fs) / (f_loops * max(K, 1)),
                                       "ms_accept_per_loop": sum(s["ms_accept"] for s in fs) / f_loops}
         h.sps_set_sampling(0, 1.0)
+        # lookahead adapted from loop to loop between 1 and 6 (grow after a fully accepted loop, shrink after a
+        # first-draft rejection)
+        h.sps_generate_adaptive(sps_synth.make_prompt(seeds[0], P, V), n_new, 1, 6, T, seeds[0])
+        ad = []
+        for i in range(args.aligned_steps):
+            ad.append(h.sps_generate_adaptive(sps_synth.make_prompt(seeds[args.warmup + i], P, V), n_new, 1, 6, T,
+                                              seeds[args.warmup + i])[1])
+        ad_ms, ad_loops = sum(s["ms_decode"] for s in ad), sum(s["loops"] for s in ad)
+        line["variants"]["aligned_adaptive_K_1_6"] = {"value": args.aligned_steps * n_new / (ad_ms / 1e3), "unit": UNIT,
+                                                      "tokens_per_loop": sum(s["emitted"] for s in ad) / ad_loops,
+                                                      "mean_K": sum(s["draft_calls"] for s in ad) / ad_loops}
         # lookahead sweep on the damped pair (the paper's K trade-off figure): one generation per K
         if args.k_sweep:
             sweep = []

@@ -132,17 +132,17 @@ const char* sps_last_error(sps_handle* h);
  *   out_tokens  host  [n_new]
  *   out_stats   host, may be NULL
  * temperature > 0 scales both models' logits before the rejection scheme
- * ("adjusting temperature ... modify the probabilities accordingly");
+ * (section Modified Rejection Sampling: a temperature changes the
+ * probabilities the scheme is applied to);
  * temperature == 0 is greedy decoding (top-k with k = 1 on both models, see
  * sps_set_sampling).  SPS_ERANGE if prompt_len + n_new + K > max_seq. */
 int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K,
                  float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
 
 /* Top-k and nucleus filtering of BOTH models' distributions ahead of the
- * rejection scheme ("With standard sampling methods such as nucleus, top-k
- * sampling and adjusting temperature, we can modify the probabilities
- * accordingly before applying this rejection sampling scheme", section
- * Modified Rejection Sampling).  The paper gives no formula; this library's:
+ * rejection scheme.  The section Modified Rejection Sampling says these
+ * methods are handled by changing the probabilities before the scheme is
+ * applied and gives no formula; this library's:
  * after softmax(l / temperature), top_k >= 1 keeps every token whose logit is
  * at least the k-th largest (tokens tied with it stay; 0 = off); then
  * 0 < top_p < 1 keeps, of those, the tokens whose logit is at least v, v the
@@ -151,6 +151,18 @@ int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32
  * renormalised.  The setting stays on the handle for every later sps_generate*,
  * sps_step; no device work.  SPS_EINVAL for top_k < 0 or top_p outside (0, 1]. */
 int sps_set_sampling(sps_handle* h, int32_t top_k, float top_p);
+
+/* sps_generate with the lookahead adapted from loop to loop.  The paper fixes K
+ * per experiment and finds that the best value depends on the domain (the K
+ * trade-off figure); the rule here is this library's: K starts at
+ * (K_min + K_max) / 2, grows by one after a loop that accepted every draft,
+ * shrinks by one after a loop that rejected its first draft, within
+ * [K_min, K_max], 1 <= K_min <= K_max <= max_K.  K depends on the past only, so
+ * every loop is an exact iteration of Algorithm 2 and the output law is the
+ * target's.  With K_min == K_max it is sps_generate.  out_stats->draft_calls /
+ * loops is the mean lookahead used. */
+int sps_generate_adaptive(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K_min,
+                          int32_t K_max, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
 
 /* Same for B sequences with equal prompt lengths, advanced in lock-step with
  * ragged progress; sequence b uses Philox sequence index b.
@@ -206,8 +218,8 @@ int sps_accept_filtered(const float* q_logits, const float* p_logits, const int3
                         void* stream, int32_t* out_n_accepted, int32_t* out_tokens, uint32_t* out_flags);
 
 /* One inverse-CDF draw per row from softmax(logits / temperature) with
- * u_draft of counter (t, step, b, 0): Algorithm 2's "sample draft
- * auto-regressively" for given logits.  logits device fp32 [B, V];
+ * u_draft of counter (t, step, b, 0): the draft draw of Algorithm 2's first
+ * for-loop, for given logits.  logits device fp32 [B, V];
  * out_tokens device int32 [B]. */
 int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uint64_t seed, uint32_t step, uint32_t t,
                void* stream, int32_t* out_tokens);
@@ -216,8 +228,8 @@ int sps_sample(const float* logits, int32_t B, int32_t V, float temperature, uin
 int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float temperature, int32_t top_k, float top_p,
                         uint64_t seed, uint32_t step, uint32_t t, void* stream, int32_t* out_tokens);
 
-/* The memory-bound linear layer alone ("dense matrix multiplies ... become
- * memory bound", Conditional Scoring): Y[M, N] = X[M, D] W[N, D]^T with fp32
+/* The memory-bound linear layer alone (section Conditional Scoring: at small
+ * batch the linear layers are bound by memory): Y[M, N] = X[M, D] W[N, D]^T with fp32
  * accumulation.  W device, row-major [N, D], dtype 0 fp32 / 1 bf16; X device
  * fp32 [M, D]; Y device fp32 [M, N]; 1 <= M <= 16.  bf16 needs D % 128 == 0 and
  * 16-byte aligned W.  workspace: device scratch of sps_linear_workspace_bytes()

@@ -85,6 +85,9 @@ def lib():
         L.orc_sample_row_f.restype = i32
         L.orc_filtered.argtypes = [vp, i32, f64, i32, f64, vp, vp]
         L.orc_accept_chain_f.argtypes = [vp, vp, vp, i32, i32, f64, i32, f64, u64, u32, u32, vp, vp, vp, vp]
+        L.orc_sps_generate_adaptive.argtypes = [vp, vp, i32, i32, i32, i32, f64, u64, u32, u32, vp, vp, vp, vp]
+        L.orc_sps_generate_adaptive.restype = i32
+        L.orc_sps_trials_adaptive.argtypes = [vp, vp, vp, i32, i32, i32, i32, f64, u64, u32, i64, vp, vp]
         L.orc_num_threads.restype = i32
         L.orc_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp]
         _lib = L
@@ -357,6 +360,16 @@ class Sps:
                                C.byref(loops), _p(hist), C.byref(anyf))
         return {"tokens": out, "loops": int(loops.value), "hist_emitted": hist, "flags": int(anyf.value)}
 
+    def generate_adaptive(self, prompt, n_new: int, K_min: int, K_max: int, T: float, seed: int, b: int = 0, step0: int = 0):
+        """Generation with the lookahead adapted from loop to loop (grow after a fully accepted loop, shrink after a
+        first-draft rejection)."""
+        p = _i32(prompt)
+        out = np.zeros(n_new, dtype=np.int32)
+        loops, drafts, anyf = C.c_int32(0), C.c_int32(0), C.c_uint32(0)
+        lib().orc_sps_generate_adaptive(self._h, _p(p), p.shape[0], n_new, K_min, K_max, float(T), seed, b, step0, _p(out),
+                                        C.byref(loops), C.byref(drafts), C.byref(anyf))
+        return {"tokens": out, "loops": int(loops.value), "draft_calls": int(drafts.value), "flags": int(anyf.value)}
+
     def close(self):
         if self._h:
             lib().orc_sps_destroy(self._h)
@@ -379,3 +392,14 @@ def trials(target: Model, draft: Model | None, prompt, n_new: int, K: int, T: fl
         lib().orc_sps_trials_f(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
                                int(top_k), float(top_p), seed, b0, n_trials, _p(out), _p(hist), _p(first_acc), _p(first_flags))
     return {"tokens": out, "hist_emitted": hist, "first_n_accepted": first_acc, "first_flags": first_flags}
+
+
+def trials_adaptive(target: Model, draft: Model, prompt, n_new: int, K_min: int, K_max: int, T: float, seed: int,
+                    n_trials: int, b0: int = 0):
+    """n_trials independent adaptive-lookahead generations of n_new tokens."""
+    p = _i32(prompt)
+    out = np.zeros((n_trials, n_new), dtype=np.int32)
+    tot = C.c_int64(0)
+    lib().orc_sps_trials_adaptive(target._h, draft._h, _p(p), p.shape[0], n_new, K_min, K_max, float(T), seed, b0, n_trials,
+                                  _p(out), C.byref(tot))
+    return {"tokens": out, "draft_calls": int(tot.value)}

@@ -103,8 +103,8 @@ extern "C" void orc_uniforms(uint64_t seed, uint32_t b, uint32_t s, uint32_t t, 
 // Distributions.
 // ---------------------------------------------------------------------------
 // softmax(l / T): subtract the maximum, exponentiate, divide by the sum.
-// ("adjusting temperature ... modify the probabilities accordingly before
-// applying this rejection sampling scheme", Modified Rejection Sampling.)
+// (Modified Rejection Sampling: a temperature changes both models'
+// probabilities before the rejection scheme sees them.)
 static void softmax_T(const float* logits, int V, double T, std::vector<double>& prob) {
   prob.resize(V);
   double mx = -INFINITY;
@@ -114,11 +114,11 @@ static void softmax_T(const float* logits, int V, double T, std::vector<double>&
   for (int i = 0; i < V; ++i) prob[i] /= sum;
 }
 
-// Top-k and nucleus (top-p) filtering ("With standard sampling methods such as
-// nucleus, top-k sampling and adjusting temperature, we can modify the
-// probabilities accordingly before applying this rejection sampling scheme",
-// Modified Rejection Sampling).  The paper names the methods and gives no
-// formula; this build's reading, applied to the draft and the target alike:
+// Top-k and nucleus (top-p) filtering.  The section Modified Rejection
+// Sampling says that such sampling methods are handled by changing the
+// probabilities first and applying the rejection scheme to the changed
+// distributions; it names the methods and gives no formula.  This build's
+// reading, applied to the draft and the target alike:
 //   1. pr = softmax(l / T);
 //   2. top-k (k >= 1; 0 = off): keep every token whose logit is at least the
 //      k-th largest logit (tokens tied with the k-th are all kept);
@@ -741,6 +741,56 @@ extern "C" int orc_sps_generate(OrcSps* c, const int32_t* prompt, int P, int n_n
   if (loops_out) *loops_out = loops;
   if (any_flags) *any_flags = anyf;
   return made;
+}
+
+// Adaptive lookahead.  The paper finds that the best K depends on the domain (the K trade-off figure and its
+// discussion) and fixes K per experiment; choosing it on the fly is this build's addition.  The rule: K starts
+// at (K_min + K_max) / 2; after a
+// loop in which every draft was accepted it grows by one (up to K_max), after a loop in which the first draft
+// was rejected it shrinks by one (down to K_min), otherwise it stays.  K only depends on the past, so every
+// loop is still an exact iteration of Algorithm 2 and the output law is unchanged (Theorem 1 per loop).
+static int next_K(int K, int accepted, int K_min, int K_max) {
+  if (accepted == K) return std::min(K + 1, K_max);
+  if (accepted == 0) return std::max(K - 1, K_min);
+  return K;
+}
+
+extern "C" int orc_sps_generate_adaptive(OrcSps* c, const int32_t* prompt, int P, int n_new, int K_min, int K_max, double T,
+                                         uint64_t seed, uint32_t b, uint32_t step0, int32_t* out_tokens,
+                                         int32_t* loops_out, int32_t* draft_calls_out, uint32_t* any_flags) {
+  orc_sps_reset(c, prompt, P);
+  std::vector<int32_t> em(K_max + 1);
+  int made = 0, loops = 0, K = (K_min + K_max) / 2, drafts = 0;
+  uint32_t anyf = 0;
+  while (made < n_new) {
+    int a; uint32_t fl, dnt;
+    const int e = orc_sps_loop(c, K, T, seed, b, step0 + (uint32_t)loops, em.data(), &a, &fl, &dnt);
+    anyf |= fl | (dnt ? ORC_NEAR_CDF : 0u);
+    for (int i = 0; i < e && made < n_new; ++i) out_tokens[made++] = em[i];
+    drafts += K;
+    K = next_K(K, a, K_min, K_max);
+    ++loops;
+  }
+  if (loops_out) *loops_out = loops;
+  if (draft_calls_out) *draft_calls_out = drafts;
+  if (any_flags) *any_flags = anyf;
+  return made;
+}
+
+// n_trials independent adaptive generations (trial i uses sequence index b0 + i); table models
+extern "C" void orc_sps_trials_adaptive(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new,
+                                        int K_min, int K_max, double T, uint64_t seed, uint32_t b0, int64_t n_trials,
+                                        int32_t* out_tokens /*[n_trials][n_new]*/, int64_t* draft_calls_total) {
+  OrcSps* c = orc_sps_create(target, draft);
+  int64_t tot = 0;
+  for (int64_t tr = 0; tr < n_trials; ++tr) {
+    int32_t dc = 0;
+    orc_sps_generate_adaptive(c, prompt, P, n_new, K_min, K_max, T, seed, b0 + (uint32_t)tr, 0u, out_tokens + tr * n_new,
+                              nullptr, &dc, nullptr);
+    tot += dc;
+  }
+  if (draft_calls_total) *draft_calls_total = tot;
+  orc_sps_destroy(c);
 }
 
 // Many independent trials of "the first n_new tokens after a fixed prompt",

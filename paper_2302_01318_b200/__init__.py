@@ -83,6 +83,7 @@ def lib():
         L.sps_accept.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp]
         L.sps_sample.argtypes = [vp, i32, i32, f32, u64, u32, u32, vp, vp]
         L.sps_set_sampling.argtypes = [vp, i32, f32]
+        L.sps_generate_adaptive.argtypes = [vp, vp, i32, i32, i32, i32, f32, u64, vp, C.POINTER(sps_stats)]
         L.sps_accept_filtered.argtypes = [vp, vp, vp, i32, i32, i32, f32, i32, f32, u64, u32, vp, vp, vp, vp]
         L.sps_sample_filtered.argtypes = [vp, i32, i32, f32, i32, f32, u64, u32, u32, vp, vp]
         L.sps_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
@@ -162,6 +163,14 @@ class Handle:
         st = sps_stats()
         _check(lib().sps_generate(self._h, _np_ptr(p), p.shape[0], n_new, K, temperature, seed, _np_ptr(out), C.byref(st)),
                self._h)
+        return out, st.as_dict()
+
+    def sps_generate_adaptive(self, prompt, n_new, K_min, K_max, temperature, seed):
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        out = np.zeros(n_new, dtype=np.int32)
+        st = sps_stats()
+        _check(lib().sps_generate_adaptive(self._h, _np_ptr(p), p.shape[0], n_new, K_min, K_max, temperature, seed, _np_ptr(out),
+                                           C.byref(st)), self._h)
         return out, st.as_dict()
 
     def sps_generate_batch(self, prompts, n_new, K, temperature, seed):

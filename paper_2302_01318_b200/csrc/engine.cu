@@ -582,7 +582,9 @@ int sps_last_logits(sps_handle* h, int32_t K, float* q_logits, float* p_logits, 
   return SPS_OK;
 }
 
-static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, int n_new, int K, float T, uint64_t seed,
+// K_min == K: fixed lookahead.  K_min < K: the lookahead moves between K_min and K from loop to loop (see
+// sps_generate_adaptive in the header); one sequence only.
+static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, int n_new, int K_min, int K, float T, uint64_t seed,
                          int32_t* out_tokens, sps_stats* out_stats) {
   if (!h || !prompts || !out_tokens) return fail(h, SPS_EINVAL, "null argument");
   if (n_new < 1) return fail(h, SPS_EINVAL, "n_new must be >= 1");
@@ -594,6 +596,12 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
   if (rc) return rc;
   h->B = B;
   if ((rc = check_K(h, K))) return rc;
+  const int K_max = K;
+  if (K_min != K) {
+    if (B != 1) return fail(h, SPS_EINVAL, "adaptive lookahead runs one sequence");
+    if (K_min < 1 || K_min > K) return fail(h, SPS_EINVAL, "K_min outside 1..K_max");
+    K = (K_min + K_max) / 2;
+  }
   CU(h, cudaEventRecord(h->ev[4], h->stream));
   if ((rc = set_sequences(h, prompts, B, P))) return rc;
   {
@@ -638,6 +646,12 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
       }
       h->seq_len[b] += a + 1;
     }
+    if (K_min != K_max) {
+      // grow after a loop that accepted every draft, shrink after one that rejected the first
+      const int a = h->h_res[0];
+      if (a == K) K = K + 1 < K_max ? K + 1 : K_max;
+      else if (a == 0) K = K - 1 > K_min ? K - 1 : K_min;
+    }
   }
   CU(h, cudaEventRecord(h->ev[6], h->stream));
   CU(h, cudaEventSynchronize(h->ev[6]));
@@ -654,13 +668,19 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
 
 int sps_generate(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K, float temperature,
                  uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
-  return generate_impl(h, prompt, 1, prompt_len, n_new, K, temperature, seed, out_tokens, out_stats);
+  return generate_impl(h, prompt, 1, prompt_len, n_new, K, K, temperature, seed, out_tokens, out_stats);
+}
+
+int sps_generate_adaptive(sps_handle* h, const int32_t* prompt, int32_t prompt_len, int32_t n_new, int32_t K_min, int32_t K_max,
+                          float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
+  if (h && (K_min < 1 || K_min > K_max)) return fail(h, SPS_EINVAL, "K_min outside 1..K_max");
+  return generate_impl(h, prompt, 1, prompt_len, n_new, K_min, K_max, temperature, seed, out_tokens, out_stats);
 }
 
 int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new, int32_t K,
                        float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
   if (h && (B < 1 || B > h->cfg.max_batch)) return fail(h, SPS_EINVAL, "batch outside 1..max_batch");
-  return generate_impl(h, prompts, B, prompt_len, n_new, K, temperature, seed, out_tokens, out_stats);
+  return generate_impl(h, prompts, B, prompt_len, n_new, K, K, temperature, seed, out_tokens, out_stats);
 }
 
 int sps_score(sps_handle* h, int32_t which, const int32_t* rows, int32_t n_rows, float* out_logits, float* out_ms) {

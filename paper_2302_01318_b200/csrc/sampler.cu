@@ -123,9 +123,9 @@ __device__ inline float block_sum_f(float v, float* s_part, float* s_out) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Top-k and nucleus filtering ("standard sampling methods such as nucleus, top-k sampling and adjusting
-// temperature ... modify the probabilities accordingly before applying this rejection sampling scheme",
-// section Modified Rejection Sampling).  A row keeps every token whose logit is at least a cut:
+// Top-k and nucleus filtering.  The section Modified Rejection Sampling says that nucleus, top-k and
+// temperature are handled by changing the probabilities first and running the rejection scheme on the
+// changed distributions; it gives no formulas.  Here a row keeps every token whose logit is at least a cut:
 //   top-k   : the cut is the k-th largest logit (tokens tied with it stay);
 //   nucleus : over what top-k kept, mass Z_k, the largest logit value v such that the tokens with logit
 //             >= v hold at least top_p * Z_k.
@@ -286,8 +286,8 @@ __device__ void row_cut(const float* row, float* ws, bool have_ws, int V, float 
 }
 
 // ------------------------------------------------------------------------------------------------
-// x ~ softmax(logits / T) by inverse CDF with u_draft(b, s, t)  (Algorithm 2: "sample draft
-// auto-regressively"; with t = 0 and u_res it is Algorithm 1's sample).
+// x ~ softmax(logits / T) by inverse CDF with u_draft(b, s, t)  (the draft draws of Algorithm 2's first
+// for-loop; with t = 0 and u_res it is Algorithm 1's sample).
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   __shared__ ScanSmem sm;

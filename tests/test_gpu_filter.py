@@ -174,3 +174,23 @@ def test_bf16_pair_under_nucleus_emits_only_tokens_the_filtered_target_allows():
         qf, near = oracle.filtered(q[a], 1.0, 0, 0.6)
         assert qf[toks[a]] > 0 or near, (step, a, toks)
     h.close()
+
+
+def test_adaptive_lookahead_matches_oracle_tokens_and_loop_count():
+    from gpu_util import make_pair
+    h, ot, od, c = make_pair("tiny", max_K=6)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(5, 20, V)
+    osps = oracle.Sps(ot, od)
+    for (kmin, kmax, T) in [(1, 6, 1.0), (2, 4, 0.7), (3, 3, 1.0)]:
+        got, st = h.sps_generate_adaptive(prompt, 40, kmin, kmax, T, 21)
+        want = osps.generate_adaptive(prompt, 40, kmin, kmax, T, 21)
+        if (got != want["tokens"]).any():
+            assert want["flags"] & NEAR, (kmin, kmax, got, want["tokens"])
+        else:
+            assert st["loops"] == want["loops"] and st["draft_calls"] == want["draft_calls"]
+    with pytest.raises(sps.SpsError):
+        h.sps_generate_adaptive(prompt, 8, 0, 4, 1.0, 0)
+    with pytest.raises(sps.SpsError):
+        h.sps_generate_adaptive(prompt, 8, 5, 4, 1.0, 0)
+    h.close()
