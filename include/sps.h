@@ -236,7 +236,15 @@ int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float tempera
  * bytes for the same (dtype, M, N, D), zero-filled once before its first use
  * (the kernel leaves it ready for the next call).
  * out_ms: host, device time of the kernel, may be NULL; when given the call
- * waits for the kernel and returns SPS_ETIMEOUT if a bounded wait inside it ran out. */
+ * waits for the kernel and returns SPS_ETIMEOUT if a bounded wait inside it ran out.
+ * sps_linear_scaled also takes dtype 2: W device int8 [N, D] (signed bytes) with
+ * row_scale device fp32 [N], Y[m, n] = row_scale[n] * sum_k X[m, k] W[n, k] -- the
+ * weight-only quantisation the paper's closing remark on quantisation refers to
+ * (it composes with speculative sampling because the transformer body is not
+ * touched): half the bytes per weight.  row_scale must be NULL for dtypes 0, 1.
+ * The same workspace size function serves all three. */
+int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, const float* X, int32_t M, int32_t N, int32_t D,
+                      float* Y, void* workspace, void* stream, float* out_ms);
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
                void* workspace, void* stream, float* out_ms);
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D);

@@ -87,6 +87,7 @@ def lib():
         L.sps_accept_filtered.argtypes = [vp, vp, vp, i32, i32, i32, f32, i32, f32, u64, u32, vp, vp, vp, vp]
         L.sps_sample_filtered.argtypes = [vp, i32, i32, f32, i32, f32, u64, u32, u32, vp, vp]
         L.sps_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
+        L.sps_linear_scaled.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
         L.sps_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sps_linear_workspace_bytes.restype = i64
         L.sps_philox.argtypes = [vp, vp, i32, vp, vp]
@@ -271,6 +272,16 @@ def sps_linear(W, X, Y, workspace, stream=None, timed=False):
     ms = C.c_float(0)
     _check(lib().sps_linear(W.data_ptr(), dtype, X.data_ptr(), M, N, D, Y.data_ptr(), workspace.data_ptr(),
                             _stream_ptr(stream), C.byref(ms) if timed else None))
+    return ms.value
+
+
+def sps_linear_scaled(W, row_scale, X, Y, workspace, stream=None, timed=False):
+    """Y[m,n] = row_scale[n] * sum_k X[m,k] W[n,k] with W CUDA int8 [N,D], row_scale CUDA fp32 [N]."""
+    N, D = W.shape
+    M = X.shape[0]
+    ms = C.c_float(0)
+    _check(lib().sps_linear_scaled(W.data_ptr(), 2, row_scale.data_ptr(), X.data_ptr(), M, N, D, Y.data_ptr(),
+                                   workspace.data_ptr(), _stream_ptr(stream), C.byref(ms) if timed else None))
     return ms.value
 
 

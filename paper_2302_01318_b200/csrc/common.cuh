@@ -171,6 +171,10 @@ struct LinArgs {
   const float* yp_gain;         // [N] multiplied in before packing, null = ones
   int yp_act;                   // PRO_GELU: gelu before packing; PRO_NONE: none
   int split_epi;                // set by the launcher: the split-K epilogue runs as a kernel of its own
+  // int8 weights (dtype 2): W holds signed bytes, row n of matrix i is scaled by wscale[i][n] (fp32, applied to
+  // the output); the activations' halves are then fp16, not bf16 -- in the slab and in the packed arrays.
+  const float* wscale[3];
+  int q8;                       // set by the launcher
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };

@@ -780,20 +780,29 @@ static int cur_num_sm() {
 }
 
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
-  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return -1;
+  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || dtype < 0 || dtype > 2) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
   return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256);
 }
 
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace,
                void* stream, float* out_ms) {
+  if (dtype != 0 && dtype != 1) return fail(nullptr, SPS_EINVAL, "dtype must be 0 or 1");
+  return sps_linear_scaled(W, dtype, nullptr, X, M, N, D, Y, workspace, stream, out_ms);
+}
+
+int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, const float* X, int32_t M, int32_t N, int32_t D,
+                      float* Y, void* workspace, void* stream, float* out_ms) {
   if (!W || !X || !Y || !workspace) return fail(nullptr, SPS_EINVAL, "null argument");
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1) return fail(nullptr, SPS_EINVAL, "M, N or D out of range");
-  if (dtype == 1 && D % 128) return fail(nullptr, SPS_EINVAL, "bf16 needs D to be a multiple of 128");
+  if (dtype >= 1 && D % 128) return fail(nullptr, SPS_EINVAL, "bf16 / int8 need D to be a multiple of 128");
   if (dtype == 0 && (size_t)M * D * 4 > 200 * 1024) return fail(nullptr, SPS_EINVAL, "fp32: M * D too large");
-  if (dtype != 0 && dtype != 1) return fail(nullptr, SPS_EINVAL, "dtype must be 0 or 1");
+  if (dtype < 0 || dtype > 2) return fail(nullptr, SPS_EINVAL, "dtype must be 0, 1 or 2");
+  if ((dtype == 2) != (row_scale != nullptr)) return fail(nullptr, SPS_EINVAL, "row scales go with int8 weights (dtype 2) and only with them");
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
+  if (p.variant < 0) return fail(nullptr, SPS_EINVAL, "int8: D splits into more ranges than the kernel has queues");
   LinArgs a{};
+  a.wscale[0] = row_scale;
   a.W[0] = W; a.rows_per_mat = N; a.N = N; a.D = D; a.M = M; a.X = X; a.ldx = D; a.x_row0 = 0; a.x_rowstep = 1;
   a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
   char* ws = (char*)workspace;

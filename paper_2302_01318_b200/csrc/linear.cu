@@ -16,6 +16,7 @@
 // per-CTA sums of squares in CTA order): no floating-point atomics, results are bit-reproducible.
 #include <cuda.h>
 #include <cudaTypedefs.h>
+#include <cuda_fp16.h>
 
 #include <cstdio>
 #include <cstdlib>
@@ -47,6 +48,53 @@ __device__ __forceinline__ void split_pack(float v0, float v1, uint32_t& hi, uin
   const __nv_bfloat16 l1 = __float2bfloat16_rn(v1 - __bfloat162float(h1));
   hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
   lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+
+// the same split into fp16 halves (int8-weight layers multiply in fp16: an int8 converts to fp16 in one step)
+__device__ __forceinline__ void split_pack_h(float v0, float v1, uint32_t& hi, uint32_t& lo) {
+  const __half h0 = __float2half_rn(v0), h1 = __float2half_rn(v1);
+  const __half l0 = __float2half_rn(v0 - __half2float(h0)), l1 = __float2half_rn(v1 - __half2float(h1));
+  hi = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+  lo = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+}
+template <bool H>
+__device__ __forceinline__ void split_pack_t(float v0, float v1, uint32_t& hi, uint32_t& lo) {
+  if (H) split_pack_h(v0, v1, hi, lo);
+  else split_pack(v0, v1, hi, lo);
+}
+
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Four signed bytes -> two fp16 pairs, exactly: flip the sign bits (byte + 128), drop each byte into the
+// mantissa of 1024.0 (0x64xx = 1024 + byte) and subtract 1152.
+__device__ __forceinline__ void s8x4_to_f16x2x2(uint32_t w, uint32_t& p01, uint32_t& p23) {
+  const uint32_t u = w ^ 0x80808080u;
+  const uint32_t l = __byte_perm(u, 0x64646464u, 0x4140), h = __byte_perm(u, 0x64646464u, 0x4342);
+  const __half2 bias = __halves2half2(__ushort_as_half(0x6480), __ushort_as_half(0x6480));
+  __half2 lf = __hsub2(*reinterpret_cast<const __half2*>(&l), bias), hf = __hsub2(*reinterpret_cast<const __half2*>(&h), bias);
+  p01 = *reinterpret_cast<uint32_t*>(&lf);
+  p23 = *reinterpret_cast<uint32_t*>(&hf);
+}
+
+// 16 weight rows x 16 k of int8 (wa: row g, wb: row g + 8, 16 bytes each) against the lane's 16 k of one
+// activation half (x0: k 0..7, x1: k 8..15 as fp16 pairs): four MMAs, alternating between two accumulators.
+__device__ __forceinline__ void q8_mma4(float (&c0)[4], float (&c1)[4], const uint4& wa, const uint4& wb, const uint4& x0,
+                                        const uint4& x1) {
+  uint32_t a01, a23, b01, b23;
+  s8x4_to_f16x2x2(wa.x, a01, a23); s8x4_to_f16x2x2(wb.x, b01, b23);
+  mma_f16_16816(c0, a01, b01, a23, b23, x0.x, x0.y);
+  s8x4_to_f16x2x2(wa.y, a01, a23); s8x4_to_f16x2x2(wb.y, b01, b23);
+  mma_f16_16816(c1, a01, b01, a23, b23, x0.z, x0.w);
+  s8x4_to_f16x2x2(wa.z, a01, a23); s8x4_to_f16x2x2(wb.z, b01, b23);
+  mma_f16_16816(c0, a01, b01, a23, b23, x1.x, x1.y);
+  s8x4_to_f16x2x2(wa.w, a01, a23); s8x4_to_f16x2x2(wb.w, b01, b23);
+  mma_f16_16816(c1, a01, b01, a23, b23, x1.z, x1.w);
 }
 
 __device__ __forceinline__ float gelu_tanh(float v) {
@@ -136,7 +184,8 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
     if (tid < SPS_MAX_ROWS) ssq_s[tid] = 0.f;
     __syncthreads();
   }
-  const bool vec = (((N | n_first | rows_all) & 3) == 0) && ((a.ldy & 3) == 0) &&
+  const bool vec = (((N | n_first | rows_all | a.rows_per_mat) & 3) == 0) && ((a.ldy & 3) == 0) &&
+                   (!a.wscale[0] || (((size_t)a.wscale[0] | (size_t)a.wscale[1] | (size_t)a.wscale[2]) & 15) == 0) &&
                    ((((size_t)a.Y | (size_t)a.part) & 15) == 0) &&
                    (!a.yp_hi || (((a.ldyp & 3) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 7) == 0) &&
                                  (!a.yp_gain || (((size_t)a.yp_gain & 15) == 0))));
@@ -172,6 +221,11 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
             for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
           }
         }
+        if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: rows_per_mat % 4 == 0)
+          const int mat = n / a.rows_per_mat;
+          const float4 ws = __ldg(reinterpret_cast<const float4*>(a.wscale[mat] + (n - mat * a.rows_per_mat)));
+          y.x *= ws.x; y.y *= ws.y; y.z *= ws.z; y.w *= ws.w;
+        }
         if (row_scale) { const float sc = row_scale[m]; y.x *= sc; y.y *= sc; y.z *= sc; y.w *= sc; }
         if (resid) {
           y = f4_add(y, old);
@@ -185,8 +239,8 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
             y.x *= gn.x; y.y *= gn.y; y.z *= gn.z; y.w *= gn.w;
           }
           uint2 hi, lo;
-          split_pack(y.x, y.y, hi.x, lo.x);
-          split_pack(y.z, y.w, hi.y, lo.y);
+          if (a.q8) { split_pack_h(y.x, y.y, hi.x, lo.x); split_pack_h(y.z, y.w, hi.y, lo.y); }
+          else { split_pack(y.x, y.y, hi.x, lo.x); split_pack(y.z, y.w, hi.y, lo.y); }
           *reinterpret_cast<uint2*>(a.yp_hi + (long long)m * a.ldyp + n) = hi;
           *reinterpret_cast<uint2*>(a.yp_lo + (long long)m * a.ldyp + n) = lo;
         }
@@ -203,15 +257,22 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
 #pragma unroll
           for (int j = 0; j < 16; ++j) y += v[j];
         }
+        if (a.wscale[0]) { const int mat = n / a.rows_per_mat; y *= __ldg(a.wscale[mat] + (n - mat * a.rows_per_mat)); }
         if (row_scale) y *= row_scale[m];
         if (resid) { y += old; sq_s[e] = y * y; }
         a.Y[(long long)m * a.ldy + n] = y;
         if (a.yp_hi) {
           if (a.yp_act == PRO_GELU) y = gelu_fast(y);
           if (a.yp_gain) y *= __ldg(a.yp_gain + n);
-          const __nv_bfloat16 h = __float2bfloat16_rn(y);
-          a.yp_hi[(long long)m * a.ldyp + n] = h;
-          a.yp_lo[(long long)m * a.ldyp + n] = __float2bfloat16_rn(y - __bfloat162float(h));
+          if (a.q8) {
+            const __half h = __float2half_rn(y);
+            reinterpret_cast<__half*>(a.yp_hi)[(long long)m * a.ldyp + n] = h;
+            reinterpret_cast<__half*>(a.yp_lo)[(long long)m * a.ldyp + n] = __float2half_rn(y - __half2float(h));
+          } else {
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            a.yp_hi[(long long)m * a.ldyp + n] = h;
+            a.yp_lo[(long long)m * a.ldyp + n] = __float2bfloat16_rn(y - __bfloat162float(h));
+          }
         }
       }
     }
@@ -446,7 +507,9 @@ struct LinTmaArgs {
   CUtensorMap tm[3];
 };
 
-template <int NT>
+// Q8: int8 weights (one byte per k, 128 k per 128-byte row segment), converted to fp16 in registers; the
+// activations' halves are fp16 too.  Otherwise bf16 weights and halves.
+template <int NT, bool Q8>
 __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma_kernel(const __grid_constant__ LinTmaArgs ta) {
   extern __shared__ __align__(1024) unsigned char smem2[];
   __shared__ int s_flag;
@@ -465,7 +528,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   int* tileq = a.counters + 2 + s;
   __shared__ volatile int s_issued, s_total;
   volatile int* tile_ids = reinterpret_cast<volatile int*>(smem2 + 704);   // [64] ring: local tile -> tile number
-  const uint32_t XP = (uint32_t)KS * 2 + 16, STAGE = 16u * (uint32_t)KST * 2u;
+  const uint32_t XP = (uint32_t)KS * 2 + 16, STAGE = 16u * (uint32_t)KST * (Q8 ? 1u : 2u);
+  constexpr int SEGK = Q8 ? 128 : 64;   // k per 128-byte row segment of the weights
   // The slab holds the M activation rows and, when M is short of the MMA's 8*NT columns, one row of zeros
   // that all the missing columns read.
   const uint32_t XR = (uint32_t)min(a.M + 1, NT * 8);
@@ -514,7 +578,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           const int slot = it % NS, use = it / NS;
           if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; return; }
           mbar_expect_tx(bar_full + 8 * slot, STAGE);
-          tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, row0 - mat * a.rows_per_mat, (k_base + ks * KST) >> 6,
+          tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, row0 - mat * a.rows_per_mat, (k_base + ks * KST) / SEGK,
                       bar_full + 8 * slot, policy);
         }
         ++local;
@@ -652,8 +716,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
                 } else if (a.pro == PRO_GELU) {
                   x.x = gelu_fast(x.x); x.y = gelu_fast(x.y); x.z = gelu_fast(x.z); x.w = gelu_fast(x.w);
                 }
-                split_pack(x.x, x.y, hi.x, lo.x);
-                split_pack(x.z, x.w, hi.y, lo.y);
+                split_pack_t<Q8>(x.x, x.y, hi.x, lo.x);
+                split_pack_t<Q8>(x.z, x.w, hi.y, lo.y);
               }
               *reinterpret_cast<uint2*>(xs_hi_p + (size_t)m * XP + c * 8) = hi;
               *reinterpret_cast<uint2*>(xs_lo_p + (size_t)m * XP + c * 8) = lo;
@@ -709,8 +773,45 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         uint32_t xrow[NT];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) xrow[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xoff;   // columns beyond M read the zero row
-        const int slabs = KST >> 6;
-        if (pk) {
+        const int slabs = KST / SEGK;
+        if (Q8) {
+          // int8 weights: a lane's two 16-byte chunks of a segment are 2 x 16 k; its activations for them are
+          // 2 x 32 bytes of the slab row (chunk c of the segment <-> bytes c*32 of the row's 256)
+          const uint32_t xq = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 64;
+          if (pk) {
+            const uint32_t xsrc = (g < 4 ? xs_hi : xs_lo) + (uint32_t)min(g & 3, a.M) * XP + xq;
+#pragma unroll 2
+            for (int q = 0; q < slabs; ++q) {
+#pragma unroll
+              for (int hf = 0; hf < 2; ++hf) {
+                const uint32_t wc = hf ? wchunk1 : wchunk0;
+                const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
+                const uint4 x0 = lds128(xsrc + q * 256 + hf * 32), x1 = lds128(xsrc + q * 256 + hf * 32 + 16);
+                q8_mma4(acc[0][0], acc[0][2], wa, wb, x0, x1);
+              }
+            }
+          } else {
+            uint32_t xr8[NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) xr8[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xq;
+#pragma unroll 2
+            for (int q = 0; q < slabs; ++q) {
+#pragma unroll
+              for (int hf = 0; hf < 2; ++hf) {
+                const uint32_t wc = hf ? wchunk1 : wchunk0;
+                const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                  const uint32_t xo = xr8[nt] + q * 256 + hf * 32;
+                  const uint4 h0 = lds128(xs_hi + xo), h1 = lds128(xs_hi + xo + 16);
+                  q8_mma4(acc[nt][0], acc[nt][2], wa, wb, h0, h1);
+                  const uint4 l0 = lds128(xs_lo + xo), l1 = lds128(xs_lo + xo + 16);
+                  q8_mma4(acc[nt][1], acc[nt][3], wa, wb, l0, l1);
+                }
+              }
+            }
+          }
+        } else if (pk) {
           // Up to four activation rows: one MMA carries both halves -- columns 0..3 the high parts of rows
           // 0..3, columns 4..7 their low parts (lane group g reads one source row) -- so a k-step costs half
           // the MMAs and half the activation loads; the two halves of a column meet in a shuffle at the end.
@@ -990,6 +1091,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     int ks = 128;
     for (int k = 128; k <= ((p.NT == 1) ? 2048 : 1024) && k <= D; k += 128) if (D % k == 0) ks = k;
     if (D / ks > LIN_MAX_S) p.variant = 1;
+    if (dtype == 2) p.variant = (D / ks > LIN_MAX_S) ? -1 : 2;   // int8 weights: TMA kernel or nothing
   }
   if (p.variant == 2) {
     // bulk-copy variant: KS = largest multiple of 128 dividing D up to the slab budget
@@ -1001,6 +1103,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     static const int kst_env = [] { const char* e = getenv("SPS_LIN_KST"); return e ? atoi(e) : 1024; }();
     int KST = 128;
     for (int k : {256, 512, 1024}) if (KS % k == 0 && k <= kst_env) KST = k;
+    if (dtype == 2) KST = KS;   // int8: a tile is one stage (16 rows x KS bytes <= 32 KB)
     p.KS = KS; p.KST = KST; p.S = D / KS; p.WC = LIN_CONSUMER_WARPS + 1; p.PR = 0;
     int R = num_sm / p.S;
     if (R < 1) R = 1;
@@ -1011,7 +1114,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     const int xr = M + 1 < p.NT * 8 ? M + 1 : p.NT * 8;   // activation rows plus one row of zeros
     size_t xbytes = (size_t)2 * xr * ((size_t)KS * 2 + 16);
     xbytes = ((xbytes + 1023) / 1024) * 1024;
-    const size_t stage = (size_t)16 * (size_t)KST * 2;
+    const size_t stage = (size_t)16 * (size_t)KST * (dtype == 2 ? 1 : 2);
     int NS = (int)((kSmemTma - 1024 - xbytes) / stage);
     if (NS > 24) NS = 24;
     if (NS < 2) NS = 2;
@@ -1061,10 +1164,10 @@ static cudaError_t ensure_smem(Kern k, size_t bytes, size_t& cached) {
 
 // A weight matrix [rows][D] bf16 as the copy engine sees it: dims {64 k, rows, D/64} with byte strides
 // {2, D*2, 128}, box {64, 16, KST/64}, 128-byte swizzle.  Descriptors are cached per (pointer, shape).
-static cudaError_t weight_tensor_map(const void* W, int rows, int D, int KST, CUtensorMap* out) {
+static cudaError_t weight_tensor_map(const void* W, int rows, int D, int KST, bool q8, CUtensorMap* out) {
   static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
   static std::mutex mu;
-  static std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;
+  static std::map<std::tuple<const void*, int, int, int, int>, CUtensorMap> cache;
   std::lock_guard<std::mutex> lock(mu);
   if (!encode) {
     void* fn = nullptr;
@@ -1074,15 +1177,17 @@ static cudaError_t weight_tensor_map(const void* W, int rows, int D, int KST, CU
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
   }
-  const auto key = std::make_tuple(W, rows, D, KST);
+  const auto key = std::make_tuple(W, rows, D, KST, q8 ? 1 : 0);
   auto it = cache.find(key);
   if (it != cache.end()) { *out = it->second; return cudaSuccess; }
-  const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(D / 64)};
-  const cuuint64_t gstride[2] = {(cuuint64_t)D * 2, 128};
-  const cuuint32_t box[3] = {64, 16, (cuuint32_t)(KST / 64)};
+  // a row segment is 128 bytes either way: 64 bf16 or 128 int8
+  const int segk = q8 ? 128 : 64;
+  const cuuint64_t gdim[3] = {(cuuint64_t)segk, (cuuint64_t)rows, (cuuint64_t)(D / segk)};
+  const cuuint64_t gstride[2] = {(cuuint64_t)D * (q8 ? 1 : 2), 128};
+  const cuuint32_t box[3] = {(cuuint32_t)segk, 16, (cuuint32_t)(KST / segk)};
   const cuuint32_t estr[3] = {1, 1, 1};
   CUtensorMap tm;
-  const CUresult cr = encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(W), gdim, gstride, box, estr,
+  const CUresult cr = encode(&tm, q8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(W), gdim, gstride, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -1096,7 +1201,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   LinArgs a = a_in;
   a.R = p.R; a.S = p.S; a.WC = p.WC; a.PR = p.PR; a.KS = p.KS; a.KST = p.KST; a.NS = p.NS; a.G = p.G;
   if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
-  if ((a.xp_hi || a.yp_hi) && !(dtype == 1 && p.variant == 2)) return cudaErrorInvalidValue;   // packed activations: TMA kernel only
+  if ((a.xp_hi || a.yp_hi) && !(dtype >= 1 && p.variant == 2)) return cudaErrorInvalidValue;   // packed activations: TMA kernel only
+  if (dtype == 2 && (p.variant != 2 || !a.wscale[0] || (a.D % 128))) return cudaErrorInvalidValue;   // int8 weights: TMA kernel, scales given
   if ((a.xp_hi && !a.xp_lo) || (a.yp_hi && !a.yp_lo)) return cudaErrorInvalidValue;
   static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
   cudaError_t e;
@@ -1115,14 +1221,22 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     ta.a = a;
     const int nmat = a.N / a.rows_per_mat > 0 ? (a.N + a.rows_per_mat - 1) / a.rows_per_mat : 1;
     for (int i = 0; i < 3; ++i)
-      if ((e = weight_tensor_map(a.W[i < nmat ? i : 0], a.rows_per_mat, a.D, p.KST, &ta.tm[i])) != cudaSuccess) return e;
+      if ((e = weight_tensor_map(a.W[i < nmat ? i : 0], a.rows_per_mat, a.D, p.KST, dtype == 2, &ta.tm[i])) != cudaSuccess) return e;
     ta.a.split_epi = lin_split_epilogue() ? 1 : 0;
-    if (p.NT == 1) {
-      if ((e = ensure_smem(lin_bf16_tma_kernel<1>, p.smem, c_t1)) != cudaSuccess) return e;
-      e = launch_k(lin_bf16_tma_kernel<1>, grid, dim3(threads), p.smem, st, ta);
+    ta.a.q8 = dtype == 2 ? 1 : 0;
+    static size_t c_q1 = 48 * 1024, c_q2 = 48 * 1024;
+    if (dtype == 2 && p.NT == 1) {
+      if ((e = ensure_smem(lin_bf16_tma_kernel<1, true>, p.smem, c_q1)) != cudaSuccess) return e;
+      e = launch_k(lin_bf16_tma_kernel<1, true>, grid, dim3(threads), p.smem, st, ta);
+    } else if (dtype == 2) {
+      if ((e = ensure_smem(lin_bf16_tma_kernel<2, true>, p.smem, c_q2)) != cudaSuccess) return e;
+      e = launch_k(lin_bf16_tma_kernel<2, true>, grid, dim3(threads), p.smem, st, ta);
+    } else if (p.NT == 1) {
+      if ((e = ensure_smem(lin_bf16_tma_kernel<1, false>, p.smem, c_t1)) != cudaSuccess) return e;
+      e = launch_k(lin_bf16_tma_kernel<1, false>, grid, dim3(threads), p.smem, st, ta);
     } else {
-      if ((e = ensure_smem(lin_bf16_tma_kernel<2>, p.smem, c_t2)) != cudaSuccess) return e;
-      e = launch_k(lin_bf16_tma_kernel<2>, grid, dim3(threads), p.smem, st, ta);
+      if ((e = ensure_smem(lin_bf16_tma_kernel<2, false>, p.smem, c_t2)) != cudaSuccess) return e;
+      e = launch_k(lin_bf16_tma_kernel<2, false>, grid, dim3(threads), p.smem, st, ta);
     }
     if (e == cudaSuccess && ta.a.split_epi) {
       // The epilogue CTAs must fit beside the layer kernel's on the same SM: that needs the same split between

@@ -59,6 +59,28 @@ def test_linear_bf16_width_with_a_large_prime_factor(M):
     assert np.abs(got - want).max() <= tol(W.float(), X, D)
 
 
+@pytest.mark.parametrize("M", [1, 2, 4, 5, 8, 9, 16])
+@pytest.mark.parametrize("N,D", [(1000, 256), (77, 128), (4096, 2048), (1536, 6144), (300, 8192)])
+def test_linear_int8_weights(M, N, D):
+    """Weight-only int8: Y = scale[n] * X W^T against the oracle on the dequantised matrix (scale * q is exact in
+    double; the kernel multiplies exact fp16 copies of the bytes and applies the scale to the sum)."""
+    g = torch.Generator().manual_seed(N + D + M)
+    q = torch.randint(-128, 128, (N, D), generator=g, dtype=torch.int32).to(torch.int8)
+    q[0, :8] = torch.tensor([-128, 127, 0, -1, 1, 64, -64, 100], dtype=torch.int8)      # the corners of the range
+    scale = (torch.rand(N, generator=g) * 0.01 + 0.001).float()
+    X = torch.randn((M, D), generator=g)
+    ws = torch.zeros(sps.sps_linear_workspace_bytes(2, M, N, D), dtype=torch.uint8, device=DEV)
+    Y = torch.full((M, N), float("nan"), device=DEV)
+    sps.sps_linear_scaled(q.to(DEV), scale.to(DEV), X.to(DEV), Y, ws)
+    Y2 = torch.full((M, N), float("nan"), device=DEV)
+    sps.sps_linear_scaled(q.to(DEV), scale.to(DEV), X.to(DEV), Y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2)
+    Wd = (q.double() * scale.double()[:, None]).float()           # exact: 8-bit integer times an fp32 scale fits fp32
+    want = oracle.linear(Wd.numpy(), X.numpy())
+    assert np.abs(Y.cpu().numpy() - want).max() <= tol(Wd, X, D)
+
+
 @pytest.mark.parametrize("M", [1, 5, 9])
 @pytest.mark.parametrize("N,D", [(1024, 256), (130, 128), (515, 1024)])
 def test_linear_fp32(M, N, D):
