@@ -60,7 +60,13 @@ typedef struct sps_handle sps_handle;
  * (The paper's Hyperparams table fixes d_model / heads / layers only.)
  * dtype: 0 = fp32, 1 = bf16; it is the storage type of the weight matrices,
  * the embeddings and the KV cache.  Norm gains are always fp32.
- * bf16 models need d_model and d_ff to be multiples of 128; d_head is 64 or 128. */
+ * dtype 2 = weight-only int8: the linear layers' matrices (wq .. w_down and the
+ * unembedding) are signed bytes with one fp32 scale per output row,
+ * w[n][k] = scale[n] * byte[n][k] (sps_weights' *_scale members); the token
+ * embedding and the KV cache stay bf16.  (The paper notes that quantisation
+ * composes with speculative sampling, since the method does not touch the
+ * transformer body; half the bytes per weight halve the floor of every pass.)
+ * bf16 / int8 models need d_model and d_ff to be multiples of 128; d_head is 64 or 128. */
 typedef struct {
   int32_t n_layers, d_model, n_heads, d_head, d_ff, vocab;
   int32_t dtype;
@@ -93,10 +99,18 @@ typedef struct {
   const void* const* wo;
   const void* const* w_up;      /* each [d_ff, d_model]  */
   const void* const* w_down;    /* each [d_model, d_ff]  */
+  /* dtype 2 only (NULL otherwise): fp32 row scales, 16-byte aligned, one per output row of the matrix */
+  const float* unembed_scale;        /* [vocab]               */
+  const float* const* wq_scale;      /* each [d_model]        */
+  const float* const* wk_scale;
+  const float* const* wv_scale;
+  const float* const* wo_scale;
+  const float* const* w_up_scale;    /* each [d_ff]           */
+  const float* const* w_down_scale;  /* each [d_model]        */
 } sps_weights;
 
-/* What a generation did ("we log the amount of tokens generated for each
- * speculative loop", Results). */
+/* What a generation did (the Results section counts the tokens each
+ * speculative loop produced; so does this). */
 typedef struct {
   int32_t loops;         /* target calls                                             */
   int32_t draft_calls;   /* draft forward passes                                     */
@@ -114,8 +128,8 @@ typedef struct {
   int32_t kernel_launches; /* kernels the loops launched (graph nodes counted per replay) */
 } sps_stats;
 
-/* Build a handle for a (target, draft) pair.  Algorithm 2's preamble: "given
- * lookahead K ..., target model q, draft model p".  draft_w may be NULL, then
+/* Build a handle for a (target, draft) pair: the target model q and the draft
+ * model p of Algorithm 2's preamble.  draft_w may be NULL, then
  * only K = 0 (Algorithm 1) is available.  Allocates the KV caches
  * [layer][sequence][head][position][d_head] in the model dtype, work buffers
  * and rotary tables on cfg->device.  *out receives the handle. */

@@ -88,6 +88,7 @@ def lib():
         L.orc_sps_generate_adaptive.argtypes = [vp, vp, i32, i32, i32, i32, f64, u64, u32, u32, vp, vp, vp, vp]
         L.orc_sps_generate_adaptive.restype = i32
         L.orc_sps_trials_adaptive.argtypes = [vp, vp, vp, i32, i32, i32, i32, f64, u64, u32, i64, vp, vp]
+        L.orc_tf_set_cache_dtype.argtypes = [vp, i32]
         L.orc_num_threads.restype = i32
         L.orc_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp]
         _lib = L
@@ -249,7 +250,7 @@ class Transformer(Model):
     weights: dict(tok_embed, unembed, final_norm, layers=[dict(LAYER_KEYS)]) of numpy arrays,
     fp32 for dtype 0; uint16 bf16 bit patterns (norm gains stay fp32) for dtype 1."""
 
-    def __init__(self, cfg: dict, weights: dict | None, max_seq: int):
+    def __init__(self, cfg: dict, weights: dict | None, max_seq: int, cache_dtype: int | None = None):
         self.cfg = dict(cfg)
         h = lib().orc_tf_create(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["d_head"], cfg["d_ff"],
                                 cfg["vocab"], cfg["dtype"], float(cfg.get("rms_eps", 1e-5)),
@@ -257,6 +258,8 @@ class Transformer(Model):
         if not h:
             raise ValueError("bad transformer config")
         super().__init__(h)
+        if cache_dtype is not None:     # e.g. fp32 (dequantised) weights with a bf16 KV cache
+            lib().orc_tf_set_cache_dtype(h, int(cache_dtype))
         if weights is not None:
             self.set_weights(weights)
 

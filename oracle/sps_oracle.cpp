@@ -446,6 +446,7 @@ static inline float round_storage(double x, int dtype) {
 
 struct Transformer : OrcModel {
   int L = 0, d = 0, H = 0, dh = 0, dff = 0, dtype = 0, max_seq = 0;
+  int cache_dtype = 0;   // storage type of cached keys / values; differs from the weights' for int8-weight models
   double eps = 1e-5, rope_base = 10000.0;
   const void *tok_embed = nullptr, *unembed = nullptr, *final_norm = nullptr;
   std::vector<TfLayer> layers;
@@ -515,8 +516,8 @@ struct Transformer : OrcModel {
         }
       }
       for (int j = 0; j < d; ++j) {
-        kcl[(size_t)p * d + j] = round_storage(kv[j], dtype);
-        vcl[(size_t)p * d + j] = round_storage(vv[j], dtype);
+        kcl[(size_t)p * d + j] = round_storage(kv[j], cache_dtype);
+        vcl[(size_t)p * d + j] = round_storage(vv[j], cache_dtype);
       }
       const double scale = 1.0 / std::sqrt((double)dh);
       for (int hd = 0; hd < H; ++hd) {
@@ -566,12 +567,13 @@ extern "C" OrcModel* orc_tf_create(int n_layers, int d_model, int n_heads, int d
   if (n_heads * d_head != d_model || (d_head & 1)) return nullptr;
   Transformer* t = new Transformer();
   t->L = n_layers; t->d = d_model; t->H = n_heads; t->dh = d_head; t->dff = d_ff; t->V = vocab;
-  t->dtype = dtype; t->eps = rms_eps; t->rope_base = rope_base; t->max_seq = max_seq;
+  t->dtype = dtype; t->cache_dtype = dtype; t->eps = rms_eps; t->rope_base = rope_base; t->max_seq = max_seq;
   t->layers.resize(n_layers);
   t->kc.assign((size_t)n_layers * max_seq * d_model, 0.f);
   t->vc.assign((size_t)n_layers * max_seq * d_model, 0.f);
   return t;
 }
+extern "C" void orc_tf_set_cache_dtype(OrcModel* m, int cache_dtype) { static_cast<Transformer*>(m)->cache_dtype = cache_dtype; }
 extern "C" void orc_tf_set_globals(OrcModel* m, const void* tok_embed, const void* unembed, const void* final_norm) {
   Transformer* t = static_cast<Transformer*>(m);
   t->tok_embed = tok_embed; t->unembed = unembed; t->final_norm = final_norm;

@@ -18,6 +18,7 @@ SPS_MAX_K = 15
 FLAG_RESAMPLED, FLAG_BONUS, FLAG_FALLBACK = 1, 2, 4
 CFG_NO_GRAPH = 1
 LAYER_KEYS = ("attn_norm", "ffn_norm", "wq", "wk", "wv", "wo", "w_up", "w_down")
+SCALED_KEYS = ("wq", "wk", "wv", "wo", "w_up", "w_down")   # matrices that carry row scales when weights are int8
 
 
 class SpsError(RuntimeError):
@@ -39,7 +40,8 @@ class sps_cfg(C.Structure):
 
 class sps_weights(C.Structure):
     _fields_ = [("tok_embed", C.c_void_p), ("unembed", C.c_void_p), ("final_norm", C.c_void_p)] + \
-               [(k, C.POINTER(C.c_void_p)) for k in LAYER_KEYS]
+               [(k, C.POINTER(C.c_void_p)) for k in LAYER_KEYS] + [("unembed_scale", C.c_void_p)] + \
+               [(k + "_scale", C.POINTER(C.c_void_p)) for k in SCALED_KEYS]
 
 
 class sps_stats(C.Structure):
@@ -120,6 +122,12 @@ def _weights(w: dict, keep: list) -> sps_weights:
         arr = (C.c_void_p * max(n, 1))(*[lw[k].data_ptr() for lw in w["layers"]])
         keep.append(arr)
         setattr(sw, k, C.cast(arr, C.POINTER(C.c_void_p)))
+    if "unembed_scale" in w:      # int8 weights (dtype 2): fp32 row scales beside every matrix
+        sw.unembed_scale = w["unembed_scale"].data_ptr()
+        for k in SCALED_KEYS:
+            arr = (C.c_void_p * max(n, 1))(*[lw[k + "_scale"].data_ptr() for lw in w["layers"]])
+            keep.append(arr)
+            setattr(sw, k + "_scale", C.cast(arr, C.POINTER(C.c_void_p)))
     return sw
 
 

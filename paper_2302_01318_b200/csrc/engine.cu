@@ -25,6 +25,8 @@ struct ModelDev {
   char* vcache = nullptr;
   size_t layer_bytes = 0;
   float2* rope = nullptr;  // [max_seq][dh/2]
+  const float* unembed_scale = nullptr;   // int8 weights: row scales
+  std::vector<const float*> wq_s, wk_s, wv_s, wo_s, w_up_s, w_down_s;
   bool packed = false;     // every linear layer of this model runs on the bf16 TMA kernel: activations travel packed
 };
 
@@ -78,14 +80,15 @@ int fail(sps_handle* h, int code, const std::string& msg) {
       return fail(h, SPS_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e__));       \
   } while (0)
 
-size_t esize(int dtype) { return dtype == 0 ? 4 : 2; }
+size_t esize(int dtype) { return dtype == 0 ? 4 : 2; }   // embeddings and KV cache: fp32, or bf16 (also for int8-weight models)
+inline int act_dtype(int dtype) { return dtype == 0 ? 0 : 1; }   // what the embedding / attention kernels see
 
 int check_model_cfg(const sps_model_cfg& c, std::string& why) {
   if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.d_ff <= 0 || c.vocab <= 0) { why = "non-positive model dimension"; return 0; }
   if (c.n_heads * c.d_head != c.d_model) { why = "n_heads * d_head must equal d_model"; return 0; }
   if (c.d_head != 64 && c.d_head != 128) { why = "d_head must be 64 or 128"; return 0; }
-  if (c.dtype != 0 && c.dtype != 1) { why = "dtype must be 0 (fp32) or 1 (bf16)"; return 0; }
-  if (c.dtype == 1 && (c.d_model % 128 || c.d_ff % 128)) { why = "bf16 models need d_model and d_ff multiples of 128"; return 0; }
+  if (c.dtype < 0 || c.dtype > 2) { why = "dtype must be 0 (fp32), 1 (bf16) or 2 (int8 weights)"; return 0; }
+  if (c.dtype >= 1 && (c.d_model % 128 || c.d_ff % 128)) { why = "bf16 / int8 models need d_model and d_ff multiples of 128"; return 0; }
   if (c.dtype == 0 && ((size_t)SPS_MAX_ROWS * (size_t)(c.d_ff > c.d_model ? c.d_ff : c.d_model) * 4 > 200 * 1024)) { why = "fp32 model too wide for the fp32 kernel"; return 0; }
   if (c.d_model % 4 || c.d_ff % 4) { why = "d_model and d_ff must be multiples of 4"; return 0; }
   return 1;
@@ -105,6 +108,24 @@ int load_model(sps_handle* h, ModelDev& m, const sps_model_cfg& c, const sps_wei
       if (!srcs[i][l]) return fail(h, SPS_EINVAL, "null layer weight pointer");
       if (((uintptr_t)srcs[i][l]) & 15) return fail(h, SPS_EINVAL, "weight pointers must be 16-byte aligned");
       (*dsts[i])[l] = srcs[i][l];
+    }
+  }
+  if (c.dtype == 2) {
+    const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+    for (int M : {1, SPS_MAX_ROWS})
+      for (auto& sh : shapes)
+        if (lin_plan(2, M, sh[0], sh[1], h->num_sm).variant != 2) return fail(h, SPS_EINVAL, "int8 weights: a layer width splits into more k-ranges than the kernel supports");
+    m.unembed_scale = w->unembed_scale;
+    if (!m.unembed_scale || ((uintptr_t)m.unembed_scale & 15)) return fail(h, SPS_EINVAL, "int8 weights need 16-byte aligned row scales");
+    const float* const* ssrc[6] = {w->wq_scale, w->wk_scale, w->wv_scale, w->wo_scale, w->w_up_scale, w->w_down_scale};
+    std::vector<const float*>* sdst[6] = {&m.wq_s, &m.wk_s, &m.wv_s, &m.wo_s, &m.w_up_s, &m.w_down_s};
+    for (int i = 0; i < 6; ++i) {
+      if (c.n_layers > 0 && !ssrc[i]) return fail(h, SPS_EINVAL, "int8 weights need row scales for every matrix");
+      sdst[i]->assign(c.n_layers, nullptr);
+      for (int l = 0; l < c.n_layers; ++l) {
+        if (!ssrc[i][l] || ((uintptr_t)ssrc[i][l] & 15)) return fail(h, SPS_EINVAL, "int8 weights need 16-byte aligned row scales");
+        (*sdst[i])[l] = ssrc[i][l];
+      }
     }
   }
   m.layer_bytes = (size_t)max_batch * c.n_heads * (size_t)max_seq * c.d_head * esize(c.dtype);
@@ -151,7 +172,7 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
 // packed activations need every shape of the model, at every row count, on the TMA kernel
 bool model_can_pack(const ModelDev& m, int num_sm) {
   const sps_model_cfg& c = m.cfg;
-  if (!m.present || c.dtype != 1) return false;
+  if (!m.present || c.dtype < 1) return false;
   const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
   for (int M : {1, SPS_MAX_ROWS})
     for (auto& s : shapes)
@@ -173,7 +194,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff;
   cudaStream_t st = h->stream;
   EmbedArgs ea{};
-  ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = c.dtype; ea.d = d; ea.V = c.vocab;
+  ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
   ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
   ea.x = h->x; ea.ssq = h->ssqA;
   CU(h, embed_launch(ea, st)); h->launches++;
@@ -185,6 +206,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     {  // q, k, v = Wq h, Wk h, Wv h with h = rmsnorm(x, g_attn), one launch over the three matrices
       LinArgs a = base;
       a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
+      if (c.dtype == 2) { a.wscale[0] = m.wq_s[l]; a.wscale[1] = m.wk_s[l]; a.wscale[2] = m.wv_s[l]; }
       a.rows_per_mat = d; a.N = 3 * d; a.D = d; a.M = rows;
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
@@ -197,7 +219,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       AttnArgs aa{};
       aa.st = h->dst; aa.qkv = h->qkv; aa.out = h->attn;
       aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
-      aa.rope = m.rope; aa.dtype = c.dtype; aa.H = c.n_heads; aa.dh = c.d_head; aa.d = d;
+      aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.dh = c.d_head; aa.d = d;
       aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
       aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
       CU(h, attn_launch(aa, st)); h->launches++;
@@ -205,6 +227,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     {  // x += Wo o ; also sum(x^2) for the FFN norm
       LinArgs a = base;
       a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = d; a.M = rows;
+      if (c.dtype == 2) a.wscale[0] = m.wo_s[l];
       a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
       if (m.packed) { a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_gain = (const float*)m.ffn_norm[l]; a.yp_act = PRO_NONE; }
@@ -215,6 +238,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     {  // up = Wup rmsnorm(x, g_ffn)
       LinArgs a = base;
       a.W[0] = m.w_up[l]; a.rows_per_mat = dff; a.N = dff; a.D = d; a.M = rows;
+      if (c.dtype == 2) a.wscale[0] = m.w_up_s[l];
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB; a.ssq_in_n = nB;
       a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
@@ -228,6 +252,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
       LinArgs a = base;
       a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
+      if (c.dtype == 2) a.wscale[0] = m.w_down_s[l];
       a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
       a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
       if (m.packed) {
@@ -243,6 +268,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   if (ps.logits) {
     LinArgs a = base;
     a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
+    if (c.dtype == 2) a.wscale[0] = m.unembed_scale;
     a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
     a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
     if (m.packed) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }

@@ -536,7 +536,10 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   const uint32_t xbytes = ((2u * XR * XP + 1023u) / 1024u) * 1024u;
   const uint32_t sm0 = smem_u32(smem2);
   const uint32_t bar_full = sm0, bar_empty = sm0 + 8 * NS, bar_x = sm0 + 960;   // bar_x: the packed X slab has landed
-  // consumed[slot] = how many times the slot has been read out.  A consumer may look at a slot's
+  // GS warps share one stage when a tile has fewer stages than its group has warps (int8 weights: one stage
+  // per tile, two warps take alternate 128-byte slabs of it); otherwise a warp owns whole stages.
+  const int GS = (KSUB >= a.G) ? 1 : a.G / KSUB;
+  // consumed[slot] = how many warps have finished reading the slot, over all its uses (GS per use).  A consumer may look at a slot's
   // "full" barrier only once every earlier use of the slot is over: an mbarrier parity wait cannot
   // tell phase u from phase u-2, and consumer warps run several ring revolutions ahead.
   volatile int* consumed = reinterpret_cast<volatile int*>(smem2 + 16 * NS);
@@ -545,7 +548,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
   unsigned char* xs_lo_p = xs_hi_p + XR * XP;
 
   if (tid == 0) {
-    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); consumed[i] = 0; }
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, (uint32_t)GS); consumed[i] = 0; }
     mbar_init(bar_x, 1);
     s_abort = 0;
     s_issued = 0;
@@ -757,11 +760,11 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[nt][c][0] = acc[nt][c][1] = acc[nt][c][2] = acc[nt][c][3] = 0.f;
-      for (int ks = rank; ks < KSUB && alive; ks += G) {
+      for (int ks = rank / GS; ks < KSUB && alive; ks += G / GS) {
         const int it = L * KSUB + ks, slot = it % NS, use = it / NS;
-        if (use > 0 && consumed[slot] < use) {
+        if (use > 0 && consumed[slot] < use * GS) {
           const unsigned long long t0 = gtimer();
-          while (consumed[slot] < use) {
+          while (consumed[slot] < use * GS) {
             __nanosleep(64);
             if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); alive = false; break; }
           }
@@ -773,7 +776,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         uint32_t xrow[NT];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) xrow[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xoff;   // columns beyond M read the zero row
-        const int slabs = KST / SEGK;
+        const int slabs = KST / SEGK, qfirst = rank % GS;
         if (Q8) {
           // int8 weights: a lane's two 16-byte chunks of a segment are 2 x 16 k; its activations for them are
           // 2 x 32 bytes of the slab row (chunk c of the segment <-> bytes c*32 of the row's 256)
@@ -781,7 +784,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           if (pk) {
             const uint32_t xsrc = (g < 4 ? xs_hi : xs_lo) + (uint32_t)min(g & 3, a.M) * XP + xq;
 #pragma unroll 2
-            for (int q = 0; q < slabs; ++q) {
+            for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
               for (int hf = 0; hf < 2; ++hf) {
                 const uint32_t wc = hf ? wchunk1 : wchunk0;
@@ -795,7 +798,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) xr8[nt] = (uint32_t)min(nt * 8 + g, a.M) * XP + xq;
 #pragma unroll 2
-            for (int q = 0; q < slabs; ++q) {
+            for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
               for (int hf = 0; hf < 2; ++hf) {
                 const uint32_t wc = hf ? wchunk1 : wchunk0;
@@ -817,7 +820,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           // the MMAs and half the activation loads; the two halves of a column meet in a shuffle at the end.
           const uint32_t xsrc = (g < 4 ? xs_hi : xs_lo) + (uint32_t)min(g & 3, a.M) * XP + xoff;
 #pragma unroll 2
-          for (int q = 0; q < slabs; ++q) {
+          for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
               const uint32_t wc = hf ? wchunk1 : wchunk0;
@@ -829,7 +832,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           }
         } else
 #pragma unroll 2
-        for (int q = 0; q < slabs; ++q) {
+        for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
             const uint32_t wc = hf ? wchunk1 : wchunk0;
@@ -848,7 +851,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         __syncwarp();
         if (lane == 0) {
           mbar_arrive(bar_empty + 8 * slot);
-          consumed[slot] = use + 1;
+          atomicAdd(const_cast<int*>(consumed) + slot, 1);
         }
       }
       // a group leaves its barrier together: abort is group-wide (checked after the barrier)
@@ -1103,7 +1106,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     static const int kst_env = [] { const char* e = getenv("SPS_LIN_KST"); return e ? atoi(e) : 1024; }();
     int KST = 128;
     for (int k : {256, 512, 1024}) if (KS % k == 0 && k <= kst_env) KST = k;
-    if (dtype == 2) KST = KS;   // int8: a tile is one stage (16 rows x KS bytes <= 32 KB)
+    if (dtype == 2) KST = KS;   // int8: a tile is one stage (16 rows x KS bytes <= 32 KB; 16 KB stages stream 20 % slower)
     p.KS = KS; p.KST = KST; p.S = D / KS; p.WC = LIN_CONSUMER_WARPS + 1; p.PR = 0;
     int R = num_sm / p.S;
     if (R < 1) R = 1;
@@ -1120,6 +1123,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     if (NS < 2) NS = 2;
     const int ksub = KS / KST;
     p.G = (ksub % 4 == 0) ? 4 : ((ksub % 2 == 0) ? 2 : 1);
+    if (dtype == 2) p.G = 2;   // int8: the two warps of a group share the tile's single stage
     const size_t gscr = (size_t)2 * LIN_CONSUMER_WARPS * p.NT * 128 * sizeof(float);
     NS = (int)((kSmemTma - 1024 - xbytes - gscr) / stage);
     if (NS > 24) NS = 24;

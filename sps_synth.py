@@ -29,6 +29,11 @@ CONFIGS = {
     # tiny shapes with bf16 storage: exercises the bf16 kernels at oracle-friendly size
     "tiny_bf16": dict(target=_cfg(2, 256, 2, 128, 1024, 1024, 1), draft=_cfg(1, 128, 1, 128, 512, 1024, 1),
                       prompt_len=16, n_new=64, K=4, T=1.0),
+    # the same shapes with int8 linear weights (dtype 2): bf16 matrices quantised per output row
+    "tiny_q8": dict(target=_cfg(2, 256, 2, 128, 1024, 1024, 2), draft=_cfg(1, 128, 1, 128, 512, 1024, 2),
+                    prompt_len=16, n_new=64, K=4, T=1.0),
+    "70b_q8": dict(target=_cfg(80, 8192, 64, 128, 32768, 32000, 2), draft=_cfg(8, 6144, 48, 128, 24576, 32000, 2),
+                   prompt_len=128, n_new=128, K=4, T=1.0),
     "mid": dict(target=_cfg(24, 2048, 16, 128, 8192, 32000, 1), draft=_cfg(6, 1024, 8, 128, 4096, 32000, 1),
                 prompt_len=128, n_new=256, K=4, T=1.0),
     # Hyperparams table: target 8192 / 64 heads / 80 layers, draft 6144 / 48 heads / 8 layers
@@ -60,6 +65,7 @@ def _normal(shape, std, seed, device, dtype):
 
 def make_weights(cfg, seed=0, tag="target", device="cpu", std=0.02, share_embed_from=None, body_gain=1.0):
     """Every matrix and embedding i.i.d. N(0, std^2); norm gains 1.  Returns torch tensors on `device`.
+    For dtype 2 the bf16 matrices are drawn the same way and then quantised (quantize_weights).
 
     share_embed_from: weights of a wider model whose first d_model columns of tok_embed / unembed are
     reused (the 70B-shaped pair shares its (un)embedding so that acceptance is non-zero).
@@ -69,7 +75,10 @@ def make_weights(cfg, seed=0, tag="target", device="cpu", std=0.02, share_embed_
     w = {}
     for name in ("tok_embed", "unembed"):
         if share_embed_from is not None:
-            w[name] = share_embed_from[name][:, : cfg["d_model"]].contiguous()
+            src = share_embed_from[name][:, : cfg["d_model"]]
+            if src.dtype == torch.int8:      # an int8 source: back to bf16 first, quantised again below
+                src = (src.float() * share_embed_from[name + "_scale"][:, None]).to(tdt)
+            w[name] = src.contiguous()
         else:
             w[name] = _normal(_shape(cfg, name), std, _tensor_seed(seed, tag, -1, name), device, tdt)
     w["final_norm"] = torch.ones(cfg["d_model"], device=device, dtype=torch.float32)
@@ -83,7 +92,7 @@ def make_weights(cfg, seed=0, tag="target", device="cpu", std=0.02, share_embed_
                 t.mul_(body_gain)
             lw[name] = t
         w["layers"].append(lw)
-    return w
+    return quantize_weights(w) if cfg["dtype"] == 2 else w
 
 
 def to_numpy(t: torch.Tensor) -> np.ndarray:
@@ -101,14 +110,54 @@ def weights_to_numpy(w):
 
 
 def weights_to(w, device):
-    out = {k: w[k].to(device) for k in ("tok_embed", "unembed", "final_norm")}
+    out = {k: v.to(device) for k, v in w.items() if k != "layers"}
     out["layers"] = [{k: v.to(device) for k, v in lw.items()} for lw in w["layers"]]
+    return out
+
+
+def quantize_rows(W):
+    """Weight-only int8, one scale per output row: scale = max|w| / 127, byte = round(w / scale).  Returns
+    (int8 [N, D], fp32 [N]).  Pure data preparation: what a matrix multiplied by these means is defined by the
+    oracle on the dequantised matrix and by the library's kernels, each on its own."""
+    Wf = W.float()
+    scale = (Wf.abs().amax(dim=1).clamp_min(1e-12) / 127.0).float()
+    q = torch.clamp(torch.round(Wf / scale[:, None]), -127, 127).to(torch.int8)
+    return q, scale
+
+
+def quantize_weights(w):
+    """bf16 weights -> the dtype-2 layout: int8 linear matrices and unembedding with `<name>_scale`, bf16 token
+    embedding, fp32 gains.  Matrices are converted one at a time (the 70B shape does not fit twice)."""
+    out = {"tok_embed": w["tok_embed"], "final_norm": w["final_norm"]}
+    out["unembed"], out["unembed_scale"] = quantize_rows(w["unembed"])
+    out["layers"] = []
+    for lw in w["layers"]:
+        q = {"attn_norm": lw["attn_norm"], "ffn_norm": lw["ffn_norm"]}
+        for k in LAYER_MATS:
+            q[k], q[k + "_scale"] = quantize_rows(lw[k])
+            lw[k] = None
+        out["layers"].append(q)
+    return out
+
+
+def dequantized_numpy(wq):
+    """What the oracle reads for a dtype-2 model: fp32 matrices scale * byte (exact in fp32), the bf16 token
+    embedding widened to fp32.  Use with an fp32-weights oracle whose KV cache is bf16."""
+    def deq(q, s):
+        return (q.double().cpu() * s.double().cpu()[:, None]).float().numpy()
+    out = {"tok_embed": wq["tok_embed"].float().cpu().numpy(), "final_norm": wq["final_norm"].cpu().numpy(),
+           "unembed": deq(wq["unembed"], wq["unembed_scale"]), "layers": []}
+    for lw in wq["layers"]:
+        d = {"attn_norm": lw["attn_norm"].cpu().numpy(), "ffn_norm": lw["ffn_norm"].cpu().numpy()}
+        for k in LAYER_MATS:
+            d[k] = deq(lw[k], lw[k + "_scale"])
+        out["layers"].append(d)
     return out
 
 
 def weight_bytes(cfg):
     """Bytes one forward pass must stream: all layer matrices + unembedding (+ gains, negligible)."""
-    es = 4 if cfg["dtype"] == 0 else 2
+    es = {0: 4, 1: 2, 2: 1}[cfg["dtype"]]
     d, f, v = cfg["d_model"], cfg["d_ff"], cfg["vocab"]
     return cfg["n_layers"] * (4 * d * d + 2 * d * f) * es + v * d * es
 

@@ -11,6 +11,14 @@ def have_gpu():
     return torch.cuda.is_available()
 
 
+def oracle_model(cfg, w, max_seq):
+    """The oracle over the same weights; an int8-weight model is the fp32 model of its dequantised matrices with
+    the keys and values cached in bf16."""
+    if cfg["dtype"] == 2:
+        return oracle.Transformer(dict(cfg, dtype=0), sps_synth.dequantized_numpy(w), max_seq, cache_dtype=1)
+    return oracle.Transformer(cfg, sps_synth.weights_to_numpy(w), max_seq)
+
+
 def make_pair(name, max_seq=160, max_batch=1, max_K=4, flags=0, seed=0, draft_equals_target=False, std=0.02):
     """(library handle, oracle target, oracle draft, config) over the very same weights."""
     c = sps_synth.CONFIGS[name]
@@ -19,8 +27,7 @@ def make_pair(name, max_seq=160, max_batch=1, max_K=4, flags=0, seed=0, draft_eq
         wd, dcfg = wt, c["target"]
     else:
         wd, dcfg = sps_synth.make_weights(c["draft"], seed=seed, tag="draft", std=std), c["draft"]
-    ot = oracle.Transformer(c["target"], sps_synth.weights_to_numpy(wt), max_seq)
-    od = oracle.Transformer(dcfg, sps_synth.weights_to_numpy(wd), max_seq)
+    ot, od = oracle_model(c["target"], wt, max_seq), oracle_model(dcfg, wd, max_seq)
     gt = sps_synth.weights_to(wt, "cuda")
     gd = gt if draft_equals_target else sps_synth.weights_to(wd, "cuda")
     h = sps.Handle(c["target"], gt, dcfg, gd, max_seq=max_seq, max_batch=max_batch, max_K=max_K, flags=flags)

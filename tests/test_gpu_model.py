@@ -15,10 +15,10 @@ from gpu_util import NEAR, make_pair
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-TOL = {"tiny": 1e-3, "tiny_bf16": 5e-2}
+TOL = {"tiny": 1e-3, "tiny_bf16": 5e-2, "tiny_q8": 5e-2}
 
 
-@pytest.mark.parametrize("name", ["tiny", "tiny_bf16"])
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16", "tiny_q8"])
 def test_scoring_pass_logits(name):
     h, ot, od, c = make_pair(name)
     V = c["target"]["vocab"]
@@ -155,6 +155,30 @@ def test_bf16_pair_logits_under_teacher_forcing():
     print(f"bf16: {loops} loops, {near} near ties, worst logit error {worst:.2e}")
     assert worst < 5e-2
     h.close()
+
+
+def test_int8_weight_pair_logits_under_teacher_forcing():
+    """int8 linear weights with row scales (weight-only quantisation): the oracle runs the fp32 model of the
+    dequantised matrices with a bf16 KV cache; activations on the GPU are fp16 halves, so the bf16 tolerance holds
+    with room to spare."""
+    h, ot, od, c = make_pair("tiny_q8")
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(1, 16, V)
+    loops, near, worst = teacher_forced(h, ot, od, prompt, 48, 4, 1.0, 3)
+    print(f"int8: {loops} loops, {near} near ties, worst logit error {worst:.2e}")
+    assert worst < 5e-2
+    a, st = h.sps_generate(prompt, 48, 4, 1.0, 5)
+    b, _ = h.sps_generate(prompt, 48, 4, 1.0, 5)
+    assert (a == b).all() and st["fallback"] == 0
+    h.close()
+
+
+def test_int8_weights_need_their_scales():
+    c = sps_synth.CONFIGS["tiny_q8"]
+    w = sps_synth.weights_to(sps_synth.make_weights(c["target"]), DEV)
+    bad = {k: v for k, v in w.items() if k != "unembed_scale"}
+    with pytest.raises(sps.SpsError):
+        sps.Handle(c["target"], bad, None, None, max_seq=64)
 
 
 def test_draft_equal_to_target_accepts_everything():

@@ -84,6 +84,33 @@ def test_forward_matches_matrix_restatement(name, tag):
     assert np.abs(got - want).max() < 1e-9 * max(1.0, np.abs(want).max())
 
 
+def test_int8_weight_model_is_the_dequantised_model_with_a_bf16_cache():
+    """The oracle of an int8-weight model: fp32 weights scale * byte, keys and values rounded to bf16 where they
+    are cached.  The matrix restatement takes the same two facts separately."""
+    cfg = sps_synth.CONFIGS["tiny_q8"]["target"]
+    wq = sps_synth.make_weights(cfg, seed=0, tag="target", std=0.08)
+    for lw in wq["layers"]:
+        for k in sps_synth.LAYER_MATS:
+            q, s = lw[k], lw[k + "_scale"]
+            assert q.dtype == torch.int8 and int(q.abs().max()) == 127 and s.shape == (q.shape[0],)
+            assert (q.abs().amax(dim=1) == 127).all()            # every row uses the full range
+    # quantisation error at most half a step per weight
+    ref = sps_synth.make_weights(dict(cfg, dtype=1), seed=0, tag="target", std=0.08)
+    q, s = wq["layers"][0]["w_up"], wq["layers"][0]["w_up_scale"]
+    err = (q.float() * s[:, None] - ref["layers"][0]["w_up"].float()).abs()
+    assert (err <= 0.5 * s[:, None] * (1 + 1e-3)).all()     # fp32 rounding of w / scale moves a half-way case
+    w = sps_synth.dequantized_numpy(wq)
+    toks = sps_synth.make_prompt(3, 12, cfg["vocab"])
+    m = oracle.Transformer(dict(cfg, dtype=0), w, max_seq=32, cache_dtype=1)
+    got = m.forward64(toks, np.arange(12))
+    want = matrix_forward(dict(cfg, dtype=1), w, toks)
+    assert np.abs(got - want).max() < 1e-9 * max(1.0, np.abs(want).max())
+    # the cache type matters (the check has power) and the default is the weights' type
+    plain = oracle.Transformer(dict(cfg, dtype=0), w, max_seq=32).forward64(toks, np.arange(12))
+    same = oracle.Transformer(dict(cfg, dtype=0), w, max_seq=32, cache_dtype=0).forward64(toks, np.arange(12))
+    assert np.array_equal(plain, same) and np.abs(plain - got).max() > 1e-6
+
+
 def test_parallel_scoring_equals_sequential_scoring():
     """K+1 rows in one call give the K+1 conditionals that single-row calls give (Conditional Scoring)."""
     cfg = TINY["target"]
