@@ -103,13 +103,14 @@ class ClockSampler:
 def build_models(cfgname, device):
     c = sps_synth.CONFIGS[cfgname]
     wt = sps_synth.make_weights(c["target"], seed=0, tag="target", device=device)
-    share = wt if cfgname == "70b" else None
+    share = wt if cfgname.startswith("70b") else None
     wd = sps_synth.make_weights(c["draft"], seed=0, tag="draft", device=device, share_embed_from=share)
     return c, wt, wd
 
 
 def kv_bytes_per_token(cfg):
-    return cfg["n_layers"] * 2 * cfg["d_model"] * (4 if cfg["dtype"] == 0 else 2)
+    dkv = cfg.get("n_kv_heads", cfg["n_heads"]) * cfg["d_head"]
+    return cfg["n_layers"] * 2 * dkv * (4 if cfg["dtype"] == 0 else 2)
 
 
 # ----------------------------------------------------------------------------------------------- CPU oracle legs
@@ -121,7 +122,10 @@ def oracle_sample_seconds(c, K, wt_layer, wd_layer, wt_unembed, wd_unembed, P):
     rng = np.random.default_rng(0)
     out = {}
     for tag, mc, lw, un, rows in (("target", tc, wt_layer, wt_unembed, K + 1), ("draft", dc, wd_layer, wd_unembed, 1)):
-        m = oracle.Transformer(dict(mc, n_layers=1), None, P + K + 2)
+        if mc["dtype"] == 2:     # int8 weights: the oracle runs the dequantised fp32 model with a bf16 cache
+            m = oracle.Transformer(dict(mc, n_layers=1, dtype=0), None, P + K + 2, cache_dtype=1)
+        else:
+            m = oracle.Transformer(dict(mc, n_layers=1), None, P + K + 2)
         emb = un[rng.integers(0, mc["vocab"], rows)]
         pos = np.arange(P - 1, P - 1 + rows, dtype=np.int32)
         m.begin_rows(np.ascontiguousarray(emb), pos)
@@ -144,7 +148,22 @@ def oracle_loop_seconds(c, K, s):
 
 
 def layer_numpy(lw):
+    """One layer as the oracle reads it; an int8 layer as its dequantised fp32 matrices."""
+    if "wq_scale" in lw:
+        out = {k: lw[k].cpu().numpy() for k in ("attn_norm", "ffn_norm")}
+        for k in sps_synth.LAYER_MATS:
+            out[k] = (lw[k].float() * lw[k + "_scale"][:, None]).cpu().numpy()
+        return out
     return {k: sps_synth.to_numpy(v) for k, v in lw.items()}
+
+
+def unembed_numpy(w):
+    if "unembed_scale" in w:
+        return (w["unembed"].float() * w["unembed_scale"][:, None]).cpu().numpy()
+    return sps_synth.to_numpy(w["unembed"])
+
+
+DTYPE_NAME = {0: "fp32", 1: "bf16", 2: "int8-weight (row scales, fp16 activations, bf16 KV cache)"}
 
 
 def run_reference(args):
@@ -160,7 +179,7 @@ def run_reference(args):
     one_t = sps_synth.make_weights(dict(tc, n_layers=1), seed=0, tag="target", device="cpu")
     one_d = sps_synth.make_weights(dict(dc, n_layers=1), seed=0, tag="draft", device="cpu")
     lt, ld = layer_numpy(one_t["layers"][0]), layer_numpy(one_d["layers"][0])
-    ut, ud = sps_synth.to_numpy(one_t["unembed"]), sps_synth.to_numpy(one_d["unembed"])
+    ut, ud = unembed_numpy(one_t), unembed_numpy(one_d)
     times = []
     for i in range(args.warmup + args.steps):
         s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
@@ -185,7 +204,7 @@ def workload_name(cfgname, K, P, n_new):
     c = sps_synth.CONFIGS[cfgname]
     t, d = c["target"], c["draft"]
     return (f"{cfgname}: target L{t['n_layers']}/d{t['d_model']}/ff{t['d_ff']}/V{t['vocab']}, draft L{d['n_layers']}/"
-            f"d{d['d_model']}/ff{d['d_ff']}, {'bf16' if t['dtype'] else 'fp32'} random-init N(0,0.02) "
+            f"d{d['d_model']}/ff{d['d_ff']}, {DTYPE_NAME[t['dtype']]} random-init N(0,0.02) "
             f"(shared (un)embedding), prompt {P}, generate {n_new}, K={K}, T=1.0, batch 1")
 
 
@@ -229,10 +248,12 @@ def run_ours(args):
     clk = ClockSampler(local)
     barrier()
     clk.start()
-    stats, walls = [], []
+    stats, walls, loop_ms, loop_tok = [], [], [], []
     for i in range(args.steps):
         _, st, w = gen(args.warmup + i, K)
         stats.append(st); walls.append(w)
+        ms, em, _ = h.sps_last_loop_trace()
+        loop_ms.append(ms); loop_tok.append(em)
     barrier()
     clocks = clk.stop()
     dec_s, tokens = replicas.job_time_and_tokens(sum(s["ms_decode"] for s in stats) / 1e3, args.steps * n_new, dist, dev)
@@ -261,10 +282,11 @@ def run_ours(args):
                 "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
                 # profiles/lin_bf16_tma_32000x8192_M5.md: dram read + write = 1.0096 x the algorithmic bytes of that launch;
                 # traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
-                "traffic": args.traffic if args.traffic is not None else 1.0096 * vbytes / n_lin_verify}
+                "traffic": args.traffic if args.traffic is not None else
+                (1.0096 * vbytes / n_lin_verify if c["target"]["dtype"] == 1 else None)}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dec_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if c["target"]["dtype"] else "f32", "data": "synthetic",
+            "dtype": {0: "f32", 1: "bf16", 2: "f16"}[c["target"]["dtype"]], "data": "synthetic",
             "config": {"workload": workload_name(cfgname, K, P, n_new), "l2": "weights streamed per pass exceed L2 by >1000x",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks,
@@ -279,6 +301,12 @@ def run_ours(args):
                      "ms_draft_per_step": ms_draft / loops / K if loops and K else None,
                      "ms_accept_per_loop": ms_accept / loops if loops else None,
                      "ms_prefill": stats[-1]["ms_prefill"]}}
+    # latency distribution over the timed loops: a loop delivers its tokens together, so a token's latency is its
+    # loop's device time divided by the tokens that loop emitted (each token weighted once)
+    lm, lt = np.concatenate(loop_ms), np.concatenate(loop_tok)
+    per_tok = np.repeat(lm / lt, lt)
+    pct = lambda a: {f"p{q}": float(np.percentile(a, q)) for q in (50, 90, 99)} | {"mean": float(a.mean()), "max": float(a.max())}
+    line["latency"] = {"unit": "ms", "loop": pct(lm), "per_token": pct(per_tok), "loops": int(lm.size)}
     if rank == 0 and world == 1:
         # the same library's autoregressive decode on the same models
         ar_tps = None
@@ -298,7 +326,7 @@ def run_ours(args):
             import oracle
             lt = layer_numpy(wt["layers"][0])
             ld = layer_numpy(wd["layers"][0])
-            ut, ud = sps_synth.to_numpy(wt["unembed"]), sps_synth.to_numpy(wd["unembed"])
+            ut, ud = unembed_numpy(wt), unembed_numpy(wd)
             s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
             loop_s = oracle_loop_seconds(c, K, s)
             tpl = emitted / loops if K > 0 else 1.0
@@ -307,15 +335,16 @@ def run_ours(args):
                                                f"target unembedding + 1 of {c['draft']['n_layers']} draft layers + draft "
                                                f"unembedding over 1 row (context {P}), scaled to one loop and divided into the "
                                                f"measured {tpl:.3f} tokens per loop"), "seconds": s}
-    if rank == 0 and world == 1 and args.aligned_steps > 0 and c["target"]["dtype"] == 1:
+    if rank == 0 and world == 1 and args.aligned_steps > 0 and c["target"]["dtype"] >= 1:
         # Same kernels, same shapes, but a pair whose draft agrees with its target about as often as the paper's
         # trained pair did: both bodies' output projections are damped in place (x gamma), so that the shared
         # (un)embedding dominates the logits.  A documented deviation from "all weights N(0, 0.02)", used only to
         # show tokens per loop in the paper's acceptance regime; kernel times do not depend on weight values.
+        sfx = "_scale" if c["target"]["dtype"] == 2 else ""      # int8 matrices are damped through their row scales
         for w in (wt, wd):
             for lw in w["layers"]:
-                lw["wo"].mul_(args.aligned_gamma)
-                lw["w_down"].mul_(args.aligned_gamma)
+                lw["wo" + sfx].mul_(args.aligned_gamma)
+                lw["w_down" + sfx].mul_(args.aligned_gamma)
         torch.cuda.synchronize()
         gen(0, K)
         al = [gen(args.warmup + i, K)[1] for i in range(args.aligned_steps)]

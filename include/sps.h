@@ -58,6 +58,13 @@ typedef struct sps_handle sps_handle;
  * n_heads * d_head == d_model, rotary positions on adjacent pairs over the
  * whole head, non-gated FFN with tanh-GeLU, no biases, untied (un)embedding.
  * (The paper's Hyperparams table fixes d_model / heads / layers only.)
+ * n_kv_heads: key / value heads; 0 or n_heads = one per query head.  A divisor
+ * of n_heads below it gives grouped-query attention, 1 multi-query attention
+ * (Related Work: multi-query attention shrinks the key / value cache;
+ * Conclusion: it combines with this method, which leaves the transformer
+ * body alone): query head h attends
+ * over key / value head h / (n_heads / n_kv_heads), wk and wv have
+ * n_kv_heads * d_head rows, and the cache holds that many numbers per position.
  * dtype: 0 = fp32, 1 = bf16; it is the storage type of the weight matrices,
  * the embeddings and the KV cache.  Norm gains are always fp32.
  * dtype 2 = weight-only int8: the linear layers' matrices (wq .. w_down and the
@@ -71,6 +78,7 @@ typedef struct {
   int32_t n_layers, d_model, n_heads, d_head, d_ff, vocab;
   int32_t dtype;
   float rms_eps, rope_base;
+  int32_t n_kv_heads;
 } sps_model_cfg;
 
 typedef struct {
@@ -94,7 +102,7 @@ typedef struct {
   const void* const* attn_norm; /* each [d_model] fp32   */
   const void* const* ffn_norm;  /* each [d_model] fp32   */
   const void* const* wq;        /* each [d_model, d_model] */
-  const void* const* wk;
+  const void* const* wk;        /* each [n_kv_heads * d_head, d_model] */
   const void* const* wv;
   const void* const* wo;
   const void* const* w_up;      /* each [d_ff, d_model]  */
@@ -102,7 +110,7 @@ typedef struct {
   /* dtype 2 only (NULL otherwise): fp32 row scales, 16-byte aligned, one per output row of the matrix */
   const float* unembed_scale;        /* [vocab]               */
   const float* const* wq_scale;      /* each [d_model]        */
-  const float* const* wk_scale;
+  const float* const* wk_scale;      /* each [n_kv_heads * d_head] */
   const float* const* wv_scale;
   const float* const* wo_scale;
   const float* const* w_up_scale;    /* each [d_ff]           */
@@ -183,6 +191,17 @@ int sps_generate_adaptive(sps_handle* h, const int32_t* prompt, int32_t prompt_l
  *   prompts host [B, prompt_len]; out_tokens host [B, n_new]; out_stats host [B] or NULL. */
 int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new,
                        int32_t K, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
+
+/* Per-loop record of the last sps_generate / sps_generate_adaptive /
+ * sps_generate_batch call, for latency percentiles (the Results section
+ * reports mean per-token latency; a loop delivers its tokens together, so the
+ * distribution of per-loop times is what a serving system sees).
+ *   loop_ms      host [cap], device time of loop i (draft + scoring + accept), may be NULL
+ *   loop_emitted host [cap], tokens loop i emitted for sequence 0 (before truncation to n_new), may be NULL
+ *   loop_K       host [cap], lookahead loop i ran with, may be NULL
+ *   *out_loops   loops the call ran (may exceed cap: only the first cap are copied)
+ * SPS_ESTATE before the first generation. */
+int sps_last_loop_trace(sps_handle* h, float* loop_ms, int32_t* loop_emitted, int32_t* loop_K, int32_t cap, int32_t* out_loops);
 
 /* Pieces of sps_generate, for tests that drive the loop themselves. */
 /* forget every sequence and both caches' lengths */

@@ -61,6 +61,8 @@ def lib():
         L.orc_tf_end.argtypes = [vp, vp, vp, vp, vp]
         L.orc_tf_hidden.argtypes = [vp, vp]
         L.orc_tf_kv.argtypes = [vp, i32, i32, vp, vp]
+        L.orc_tf_set_kv_heads.argtypes = [vp, i32]
+        L.orc_tf_set_kv_heads.restype = i32
         L.orc_model_forward.argtypes = [vp, vp, vp, i32, vp]
         L.orc_model_forward64.argtypes = [vp, vp, vp, i32, vp]
         L.orc_model_vocab.argtypes = [vp]
@@ -246,7 +248,7 @@ LAYER_KEYS = ("attn_norm", "ffn_norm", "wq", "wk", "wv", "wo", "w_up", "w_down")
 
 
 class Transformer(Model):
-    """cfg: dict(n_layers,d_model,n_heads,d_head,d_ff,vocab,dtype,rms_eps,rope_base);
+    """cfg: dict(n_layers,d_model,n_heads,d_head,d_ff,vocab,dtype,rms_eps,rope_base[,n_kv_heads]);
     weights: dict(tok_embed, unembed, final_norm, layers=[dict(LAYER_KEYS)]) of numpy arrays,
     fp32 for dtype 0; uint16 bf16 bit patterns (norm gains stay fp32) for dtype 1."""
 
@@ -258,6 +260,9 @@ class Transformer(Model):
         if not h:
             raise ValueError("bad transformer config")
         super().__init__(h)
+        if cfg.get("n_kv_heads", 0) not in (0, cfg["n_heads"]):      # multi-query / grouped-query attention
+            if lib().orc_tf_set_kv_heads(h, int(cfg["n_kv_heads"])) != 0:
+                raise ValueError("n_kv_heads must divide n_heads")
         if cache_dtype is not None:     # e.g. fp32 (dequantised) weights with a bf16 KV cache
             lib().orc_tf_set_cache_dtype(h, int(cache_dtype))
         if weights is not None:
@@ -310,7 +315,7 @@ class Transformer(Model):
         return out
 
     def kv(self, l: int, position: int):
-        d = self.cfg["d_model"]
+        d = (self.cfg.get("n_kv_heads", 0) or self.cfg["n_heads"]) * self.cfg["d_head"]
         k, v = np.zeros(d, dtype=np.float32), np.zeros(d, dtype=np.float32)
         lib().orc_tf_kv(self._h, l, position, _p(k), _p(v))
         return k, v

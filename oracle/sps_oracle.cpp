@@ -446,11 +446,12 @@ static inline float round_storage(double x, int dtype) {
 
 struct Transformer : OrcModel {
   int L = 0, d = 0, H = 0, dh = 0, dff = 0, dtype = 0, max_seq = 0;
+  int Hkv = 0;           // key / value heads; query head h reads key / value head h / (H / Hkv)  (Hkv = H: one each)
   int cache_dtype = 0;   // storage type of cached keys / values; differs from the weights' for int8-weight models
   double eps = 1e-5, rope_base = 10000.0;
   const void *tok_embed = nullptr, *unembed = nullptr, *final_norm = nullptr;
   std::vector<TfLayer> layers;
-  std::vector<float> kc, vc;  // [L][max_seq][d]
+  std::vector<float> kc, vc;  // [L][max_seq][Hkv * dh]
   // state of a layer-by-layer pass
   std::vector<double> x;      // [M][d]
   std::vector<int32_t> pos;
@@ -492,17 +493,18 @@ struct Transformer : OrcModel {
     for (size_t i = 0; i < (size_t)M * d; ++i) x[i] = load_w(emb_rows, i, dtype);
   }
   void layer(int l, const TfLayer& w) {
-    std::vector<double> h(d), qv(d), kv(d), vv(d), o(d), y(d), up(dff);
-    float* kcl = kc.data() + (size_t)l * max_seq * d;
-    float* vcl = vc.data() + (size_t)l * max_seq * d;
+    const int dkv = Hkv * dh, group = H / Hkv;
+    std::vector<double> h(d), qv(d), kv(dkv), vv(dkv), o(d), y(d), up(dff);
+    float* kcl = kc.data() + (size_t)l * max_seq * dkv;
+    float* vcl = vc.data() + (size_t)l * max_seq * dkv;
     // rows go in order, so row i sees the cache rows of rows <= i (in-block causality)
     for (int m = 0; m < M; ++m) {
       double* xm = x.data() + (size_t)m * d;
       const int p = pos[m];
       rmsnorm(xm, w.attn_norm, h.data());
       matvec(w.wq, h.data(), d, d, qv.data());
-      matvec(w.wk, h.data(), d, d, kv.data());
-      matvec(w.wv, h.data(), d, d, vv.data());
+      matvec(w.wk, h.data(), dkv, d, kv.data());
+      matvec(w.wv, h.data(), dkv, d, vv.data());
       for (int hd = 0; hd < H; ++hd) {
         for (int i = 0; i < dh / 2; ++i) {
           const double ang = (double)p * std::pow(rope_base, -2.0 * i / dh);
@@ -510,22 +512,24 @@ struct Transformer : OrcModel {
           double* a = qv.data() + hd * dh + 2 * i;
           double a0 = a[0], a1 = a[1];
           a[0] = a0 * c - a1 * s; a[1] = a0 * s + a1 * c;
+          if (hd >= Hkv) continue;
           double* bb = kv.data() + hd * dh + 2 * i;
           a0 = bb[0]; a1 = bb[1];
           bb[0] = a0 * c - a1 * s; bb[1] = a0 * s + a1 * c;
         }
       }
-      for (int j = 0; j < d; ++j) {
-        kcl[(size_t)p * d + j] = round_storage(kv[j], cache_dtype);
-        vcl[(size_t)p * d + j] = round_storage(vv[j], cache_dtype);
+      for (int j = 0; j < dkv; ++j) {
+        kcl[(size_t)p * dkv + j] = round_storage(kv[j], cache_dtype);
+        vcl[(size_t)p * dkv + j] = round_storage(vv[j], cache_dtype);
       }
       const double scale = 1.0 / std::sqrt((double)dh);
       for (int hd = 0; hd < H; ++hd) {
+        const int hk = hd / group;   // the key / value head this query head shares
         std::vector<double> sc(p + 1);
         double mx = -INFINITY;
         for (int j = 0; j <= p; ++j) {
           double acc = 0.0;
-          for (int i = 0; i < dh; ++i) acc += qv[hd * dh + i] * (double)kcl[(size_t)j * d + hd * dh + i];
+          for (int i = 0; i < dh; ++i) acc += qv[hd * dh + i] * (double)kcl[(size_t)j * dkv + hk * dh + i];
           sc[j] = acc * scale;
           mx = std::max(mx, sc[j]);
         }
@@ -533,7 +537,7 @@ struct Transformer : OrcModel {
         for (int j = 0; j <= p; ++j) { sc[j] = std::exp(sc[j] - mx); sum += sc[j]; }
         for (int i = 0; i < dh; ++i) {
           double acc = 0.0;
-          for (int j = 0; j <= p; ++j) acc += sc[j] * (double)vcl[(size_t)j * d + hd * dh + i];
+          for (int j = 0; j <= p; ++j) acc += sc[j] * (double)vcl[(size_t)j * dkv + hk * dh + i];
           o[hd * dh + i] = acc / sum;
         }
       }
@@ -566,12 +570,21 @@ extern "C" OrcModel* orc_tf_create(int n_layers, int d_model, int n_heads, int d
                                    int dtype, double rms_eps, double rope_base, int max_seq) {
   if (n_heads * d_head != d_model || (d_head & 1)) return nullptr;
   Transformer* t = new Transformer();
-  t->L = n_layers; t->d = d_model; t->H = n_heads; t->dh = d_head; t->dff = d_ff; t->V = vocab;
+  t->L = n_layers; t->d = d_model; t->H = n_heads; t->Hkv = n_heads; t->dh = d_head; t->dff = d_ff; t->V = vocab;
   t->dtype = dtype; t->cache_dtype = dtype; t->eps = rms_eps; t->rope_base = rope_base; t->max_seq = max_seq;
   t->layers.resize(n_layers);
   t->kc.assign((size_t)n_layers * max_seq * d_model, 0.f);
   t->vc.assign((size_t)n_layers * max_seq * d_model, 0.f);
   return t;
+}
+// fewer key / value heads than query heads (multi-query: 1; grouped: a divisor of n_heads); call before any pass
+extern "C" int orc_tf_set_kv_heads(OrcModel* m, int n_kv_heads) {
+  Transformer* t = static_cast<Transformer*>(m);
+  if (n_kv_heads < 1 || t->H % n_kv_heads) return -1;
+  t->Hkv = n_kv_heads;
+  t->kc.assign((size_t)t->L * t->max_seq * n_kv_heads * t->dh, 0.f);
+  t->vc.assign((size_t)t->L * t->max_seq * n_kv_heads * t->dh, 0.f);
+  return 0;
 }
 extern "C" void orc_tf_set_cache_dtype(OrcModel* m, int cache_dtype) { static_cast<Transformer*>(m)->cache_dtype = cache_dtype; }
 extern "C" void orc_tf_set_globals(OrcModel* m, const void* tok_embed, const void* unembed, const void* final_norm) {
@@ -603,11 +616,12 @@ extern "C" void orc_tf_hidden(OrcModel* m, double* out) {
   Transformer* t = static_cast<Transformer*>(m);
   std::memcpy(out, t->x.data(), sizeof(double) * t->x.size());
 }
-// cached keys / values of one layer at one position, [d] each
+// cached keys / values of one layer at one position, [n_kv_heads * d_head] each
 extern "C" void orc_tf_kv(OrcModel* m, int l, int position, float* k_out, float* v_out) {
   Transformer* t = static_cast<Transformer*>(m);
-  std::memcpy(k_out, t->kc.data() + ((size_t)l * t->max_seq + position) * t->d, sizeof(float) * t->d);
-  std::memcpy(v_out, t->vc.data() + ((size_t)l * t->max_seq + position) * t->d, sizeof(float) * t->d);
+  const size_t dkv = (size_t)t->Hkv * t->dh;
+  std::memcpy(k_out, t->kc.data() + ((size_t)l * t->max_seq + position) * dkv, sizeof(float) * dkv);
+  std::memcpy(v_out, t->vc.data() + ((size_t)l * t->max_seq + position) * dkv, sizeof(float) * dkv);
 }
 extern "C" void orc_model_forward(OrcModel* m, const int32_t* tokens, const int32_t* positions, int M,
                                   float* logits) {

@@ -30,7 +30,7 @@ class SpsError(RuntimeError):
 class sps_model_cfg(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32), ("d_head", C.c_int32),
                 ("d_ff", C.c_int32), ("vocab", C.c_int32), ("dtype", C.c_int32), ("rms_eps", C.c_float),
-                ("rope_base", C.c_float)]
+                ("rope_base", C.c_float), ("n_kv_heads", C.c_int32)]
 
 
 class sps_cfg(C.Structure):
@@ -80,6 +80,7 @@ def lib():
         L.sps_prefill.argtypes = [vp, vp, i32]
         L.sps_step.argtypes = [vp, i32, f32, u64, u32, vp, vp, vp]
         L.sps_last_logits.argtypes = [vp, i32, vp, vp, vp]
+        L.sps_last_loop_trace.argtypes = [vp, vp, vp, vp, i32, vp]
         L.sps_verify.argtypes = [vp, vp, i32, vp, C.POINTER(f32)]
         L.sps_score.argtypes = [vp, i32, vp, i32, vp, C.POINTER(f32)]
         L.sps_accept.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp]
@@ -111,7 +112,7 @@ def _np_ptr(a):
 
 def _model_cfg(c: dict) -> sps_model_cfg:
     return sps_model_cfg(c["n_layers"], c["d_model"], c["n_heads"], c["d_head"], c["d_ff"], c["vocab"], c["dtype"],
-                         c.get("rms_eps", 1e-5), c.get("rope_base", 10000.0))
+                         c.get("rms_eps", 1e-5), c.get("rope_base", 10000.0), c.get("n_kv_heads", 0))
 
 
 def _weights(w: dict, keep: list) -> sps_weights:
@@ -206,6 +207,14 @@ class Handle:
         fl = np.zeros(1, dtype=np.uint32)
         _check(lib().sps_step(self._h, K, temperature, seed, step, _np_ptr(out), _np_ptr(n), _np_ptr(fl)), self._h)
         return out, int(n[0]), int(fl[0])
+
+    def sps_last_loop_trace(self, cap=4096):
+        """(loop_ms, loop_emitted, loop_K) of the last generation, one entry per loop."""
+        ms, em, kk = np.zeros(cap, dtype=np.float32), np.zeros(cap, dtype=np.int32), np.zeros(cap, dtype=np.int32)
+        n = C.c_int32(0)
+        _check(lib().sps_last_loop_trace(self._h, _np_ptr(ms), _np_ptr(em), _np_ptr(kk), cap, C.byref(n)), self._h)
+        m = min(n.value, cap)
+        return ms[:m], em[:m], kk[:m]
 
     def sps_last_logits(self, K):
         q = np.zeros((K + 1, self.vocab), dtype=np.float32)

@@ -1,8 +1,10 @@
 // Row set-up + embedding, and decode attention over the KV cache for 1..16 query rows per sequence
 // with rotary positions and the cache append fused in.
 //
-// Cache layout (per layer): [sequence][head][position][d_head] in the model's storage type, so one
-// (sequence, head) CTA streams two contiguous spans.  Rejected drafts are never erased: a row only
+// Cache layout (per layer): [sequence][key / value head][position][d_head] in the model's storage type, so
+// one (sequence, head) CTA streams two contiguous spans.  With fewer key / value heads than query heads
+// (grouped-query / multi-query attention) the CTAs of a group read the same spans; each of them rotates
+// this pass's keys for itself and the group's first head alone appends them to the cache.  Rejected drafts are never erased: a row only
 // ever reads positions <= its own, and the next pass overwrites the stale ones ("rollback" is the
 // sequence length moving back, nothing else).
 #include "common.cuh"
@@ -147,8 +149,11 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
 
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Mb = a.rows_per_seq, row0 = b * Mb, d = a.d, max_seq = a.max_seq;
-  CT* kc = reinterpret_cast<CT*>(a.kcache) + ((size_t)b * a.H + h) * (size_t)max_seq * DH;
-  CT* vc = reinterpret_cast<CT*>(a.vcache) + ((size_t)b * a.H + h) * (size_t)max_seq * DH;
+  const int group = a.H / a.Hkv, hk = h / group;   // the key / value head this query head reads
+  const bool appends = (h - hk * group) == 0;       // one head of a group writes the cache
+  const int ldq = d + 2 * a.Hkv * DH;                // row stride of the q | k | v buffer
+  CT* kc = reinterpret_cast<CT*>(a.kcache) + ((size_t)b * a.Hkv + hk) * (size_t)max_seq * DH;
+  CT* vc = reinterpret_cast<CT*>(a.vcache) + ((size_t)b * a.Hkv + hk) * (size_t)max_seq * DH;
   const float scale = rsqrtf((float)DH);
   const uint32_t bar_addr = a_smem_u32(bar);
 
@@ -208,18 +213,22 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
     const int i = idx / (DH / 2), pr = idx - i * (DH / 2);
     const int pos = pos_s[i];
     const float2 cs = a.rope[(size_t)pos * (DH / 2) + pr];
-    const float* src = a.qkv + (size_t)(row0 + i) * 3 * d + h * DH + 2 * pr;
-    const float q0 = src[0], q1 = src[1];
-    const float k0 = src[d], k1 = src[d + 1];
-    const float v0 = src[2 * d], v1 = src[2 * d + 1];
+    const float* src = a.qkv + (size_t)(row0 + i) * ldq;
+    const float* ksrc = src + d + hk * DH + 2 * pr;
+    const float* vsrc = ksrc + a.Hkv * DH;
+    const float q0 = src[h * DH + 2 * pr], q1 = src[h * DH + 2 * pr + 1];
+    const float k0 = ksrc[0], k1 = ksrc[1];
+    const float v0 = vsrc[0], v1 = vsrc[1];
     q_s[i * DH + 2 * pr] = (q0 * cs.x - q1 * cs.y) * scale;
     q_s[i * DH + 2 * pr + 1] = (q0 * cs.y + q1 * cs.x) * scale;
     const CT ka = f_to_ct<CT>(k0 * cs.x - k1 * cs.y), kb = f_to_ct<CT>(k0 * cs.y + k1 * cs.x);
     const CT va = f_to_ct<CT>(v0), vb = f_to_ct<CT>(v1);
     knew[i * DH + 2 * pr] = ka; knew[i * DH + 2 * pr + 1] = kb;
     vnew[i * DH + 2 * pr] = va; vnew[i * DH + 2 * pr + 1] = vb;
-    kc[(size_t)pos * DH + 2 * pr] = ka; kc[(size_t)pos * DH + 2 * pr + 1] = kb;
-    vc[(size_t)pos * DH + 2 * pr] = va; vc[(size_t)pos * DH + 2 * pr + 1] = vb;
+    if (appends) {
+      kc[(size_t)pos * DH + 2 * pr] = ka; kc[(size_t)pos * DH + 2 * pr + 1] = kb;
+      vc[(size_t)pos * DH + 2 * pr] = va; vc[(size_t)pos * DH + 2 * pr + 1] = vb;
+    }
   }
   for (int idx = tid; idx < (MR - Mb) * DH; idx += ATTN_THREADS) q_s[Mb * DH + idx] = 0.f;
 
@@ -367,6 +376,7 @@ static cudaError_t attn_rows(const AttnArgs& a, cudaStream_t st) {
 }
 
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st) {
+  if (a.Hkv < 1 || a.H % a.Hkv) return cudaErrorInvalidValue;
   if (a.dh == 64 && a.dtype == 0) return attn_rows<64, float>(a, st);
   if (a.dh == 128 && a.dtype == 0) return attn_rows<128, float>(a, st);
   if (a.dh == 64 && a.dtype == 1) return attn_rows<64, __nv_bfloat16>(a, st);

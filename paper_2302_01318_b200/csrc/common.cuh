@@ -136,9 +136,10 @@ enum { PRO_NONE = 0, PRO_RMSNORM = 1, PRO_GELU = 2 };
 enum { EPI_STORE = 0, EPI_RESIDUAL = 1 };
 
 struct LinArgs {
-  const void* W[3];       // up to three stacked matrices (fused Q,K,V), each [rows_per_mat][D]
+  const void* W[3];       // up to three stacked matrices (fused Q,K,V): W[0] is [rows_per_mat][D], W[1], W[2] are [rows_tail][D]
   int rows_per_mat;
-  int N;                  // total output features = n_mats * rows_per_mat
+  int rows_tail;          // rows of the second and third matrix (0 = rows_per_mat; fewer for grouped key / value heads)
+  int N;                  // total output features = rows_per_mat + (n_mats - 1) * rows_tail
   int D;                  // input features
   int M;                  // activation rows, 1..16
   const float* X;         // [*, ldx] fp32; row of activation m is x_row0 + m * x_rowstep
@@ -205,12 +206,13 @@ cudaError_t embed_launch(const EmbedArgs& a, cudaStream_t st);
 
 struct AttnArgs {
   const DevState* st;
-  const float* qkv;       // [rows][3d]
+  const float* qkv;       // [rows][d + 2 * Hkv * dh]: queries, then keys, then values
   float* out;             // [rows][d]
-  void* kcache;           // this layer: [B][H][max_seq][dh]
+  void* kcache;           // this layer: [B][Hkv][max_seq][dh]
   void* vcache;
   const float2* rope;     // [max_seq][dh/2] (cos, sin)
   int dtype, H, dh, d, max_seq, rows_per_seq, B;
+  int Hkv;                // key / value heads: query head h uses head h / (H / Hkv)
   int mode, t, c0;        // which rows the pass feeds (PassMode), as in EmbedArgs
 };
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);

@@ -21,7 +21,7 @@ struct ModelDev {
   bool present = false;
   const void *tok_embed = nullptr, *unembed = nullptr, *final_norm = nullptr;
   std::vector<const void*> attn_norm, ffn_norm, wq, wk, wv, wo, w_up, w_down;
-  char* kcache = nullptr;  // [L][B][H][max_seq][dh] in the storage type
+  char* kcache = nullptr;  // [L][B][key / value heads][max_seq][dh] in the storage type
   char* vcache = nullptr;
   size_t layer_bytes = 0;
   float2* rope = nullptr;  // [max_seq][dh/2]
@@ -65,6 +65,9 @@ struct sps_handle {
   std::map<const void*, long long> graph_launches;
   std::string err;
   int last_K = -1;
+  std::vector<float> trace_ms;            // per-loop record of the last generation (sps_last_loop_trace)
+  std::vector<int32_t> trace_emit, trace_K;
+  bool traced = false;
 };
 
 namespace {
@@ -82,11 +85,14 @@ int fail(sps_handle* h, int code, const std::string& msg) {
 
 size_t esize(int dtype) { return dtype == 0 ? 4 : 2; }   // embeddings and KV cache: fp32, or bf16 (also for int8-weight models)
 inline int act_dtype(int dtype) { return dtype == 0 ? 0 : 1; }   // what the embedding / attention kernels see
+inline int kv_heads(const sps_model_cfg& c) { return c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads; }
+inline int kv_width(const sps_model_cfg& c) { return kv_heads(c) * c.d_head; }   // rows of wk / wv, numbers cached per position
 
 int check_model_cfg(const sps_model_cfg& c, std::string& why) {
   if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.d_ff <= 0 || c.vocab <= 0) { why = "non-positive model dimension"; return 0; }
   if (c.n_heads * c.d_head != c.d_model) { why = "n_heads * d_head must equal d_model"; return 0; }
   if (c.d_head != 64 && c.d_head != 128) { why = "d_head must be 64 or 128"; return 0; }
+  if (c.n_kv_heads < 0 || c.n_heads % kv_heads(c)) { why = "n_kv_heads must be 0 or a divisor of n_heads"; return 0; }
   if (c.dtype < 0 || c.dtype > 2) { why = "dtype must be 0 (fp32), 1 (bf16) or 2 (int8 weights)"; return 0; }
   if (c.dtype >= 1 && (c.d_model % 128 || c.d_ff % 128)) { why = "bf16 / int8 models need d_model and d_ff multiples of 128"; return 0; }
   if (c.dtype == 0 && ((size_t)SPS_MAX_ROWS * (size_t)(c.d_ff > c.d_model ? c.d_ff : c.d_model) * 4 > 200 * 1024)) { why = "fp32 model too wide for the fp32 kernel"; return 0; }
@@ -111,7 +117,7 @@ int load_model(sps_handle* h, ModelDev& m, const sps_model_cfg& c, const sps_wei
     }
   }
   if (c.dtype == 2) {
-    const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+    const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
     for (int M : {1, SPS_MAX_ROWS})
       for (auto& sh : shapes)
         if (lin_plan(2, M, sh[0], sh[1], h->num_sm).variant != 2) return fail(h, SPS_EINVAL, "int8 weights: a layer width splits into more k-ranges than the kernel supports");
@@ -128,7 +134,7 @@ int load_model(sps_handle* h, ModelDev& m, const sps_model_cfg& c, const sps_wei
       }
     }
   }
-  m.layer_bytes = (size_t)max_batch * c.n_heads * (size_t)max_seq * c.d_head * esize(c.dtype);
+  m.layer_bytes = (size_t)max_batch * kv_heads(c) * (size_t)max_seq * c.d_head * esize(c.dtype);
   const size_t total = m.layer_bytes * (size_t)(c.n_layers > 0 ? c.n_layers : 1);
   if (cudaMalloc(&m.kcache, total) != cudaSuccess || cudaMalloc(&m.vcache, total) != cudaSuccess)
     return fail(h, SPS_ENOMEM, "KV cache allocation failed");
@@ -159,7 +165,7 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
   if (!m.present) return 0;
   const sps_model_cfg& c = m.cfg;
   size_t need = 0;
-  const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
   for (int M : {1, SPS_MAX_ROWS})
     for (auto& s : shapes) {
       const LinPlan p = lin_plan(c.dtype, M, s[0], s[1], num_sm);
@@ -173,7 +179,7 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
 bool model_can_pack(const ModelDev& m, int num_sm) {
   const sps_model_cfg& c = m.cfg;
   if (!m.present || c.dtype < 1) return false;
-  const int shapes[5][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
   for (int M : {1, SPS_MAX_ROWS})
     for (auto& s : shapes)
       if (lin_plan(c.dtype, M, s[0], s[1], num_sm).variant != 2) return false;
@@ -207,11 +213,11 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       LinArgs a = base;
       a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
       if (c.dtype == 2) { a.wscale[0] = m.wq_s[l]; a.wscale[1] = m.wk_s[l]; a.wscale[2] = m.wv_s[l]; }
-      a.rows_per_mat = d; a.N = 3 * d; a.D = d; a.M = rows;
+      a.rows_per_mat = d; a.rows_tail = kv_width(c); a.N = d + 2 * kv_width(c); a.D = d; a.M = rows;
       a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
       a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
       if (m.packed && l > 0) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }   // left there by the layer below
-      a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = 3 * d;
+      a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = a.N;
       const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
       CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
     }
@@ -219,7 +225,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
       AttnArgs aa{};
       aa.st = h->dst; aa.qkv = h->qkv; aa.out = h->attn;
       aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
-      aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.dh = c.d_head; aa.d = d;
+      aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
       aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
       aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
       CU(h, attn_launch(aa, st)); h->launches++;
@@ -608,6 +614,19 @@ int sps_last_logits(sps_handle* h, int32_t K, float* q_logits, float* p_logits, 
   return SPS_OK;
 }
 
+int sps_last_loop_trace(sps_handle* h, float* loop_ms, int32_t* loop_emitted, int32_t* loop_K, int32_t cap, int32_t* out_loops) {
+  if (!h || !out_loops || cap < 0) return fail(h, SPS_EINVAL, "null argument");
+  if (!h->traced) return fail(h, SPS_ESTATE, "no generation has run on this handle");
+  const size_t n = h->trace_ms.size(), m = n < (size_t)cap ? n : (size_t)cap;
+  for (size_t i = 0; i < m; ++i) {
+    if (loop_ms) loop_ms[i] = h->trace_ms[i];
+    if (loop_emitted) loop_emitted[i] = h->trace_emit[i];
+    if (loop_K) loop_K[i] = h->trace_K[i];
+  }
+  *out_loops = (int32_t)n;
+  return SPS_OK;
+}
+
 // K_min == K: fixed lookahead.  K_min < K: the lookahead moves between K_min and K from loop to loop (see
 // sps_generate_adaptive in the header); one sequence only.
 static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, int n_new, int K_min, int K, float T, uint64_t seed,
@@ -648,6 +667,8 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
   float ms_draft = 0.f, ms_verify = 0.f, ms_accept = 0.f, ms_prefill = 0.f, ms_decode = 0.f;
   bool first = true;
   const long long launches0 = h->launches;
+  h->trace_ms.clear(); h->trace_emit.clear(); h->trace_K.clear();
+  h->traced = true;
   CU(h, cudaEventRecord(h->ev[5], h->stream));
   for (;;) {
     bool all = true;
@@ -660,6 +681,9 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
     cudaEventElapsedTime(&a12, h->ev[1], h->ev[2]);
     cudaEventElapsedTime(&a23, h->ev[2], h->ev[3]);
     ms_draft += a01; ms_verify += a12; ms_accept += a23;
+    h->trace_ms.push_back(a01 + a12 + a23);
+    h->trace_emit.push_back(h->h_res[0] + 1);
+    h->trace_K.push_back(K);
     for (int b = 0; b < B; ++b) {
       if (made[b] >= n_new) continue;
       const int a = h->h_res[b];

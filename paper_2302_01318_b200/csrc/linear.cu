@@ -108,13 +108,15 @@ __device__ __forceinline__ float gelu_fast(float v) {
   return __fdividef(v, 1.0f + __expf(-2.0f * u));
 }
 
-__device__ __forceinline__ const void* pick_mat(const LinArgs& a, int n, int& row_in_mat) {
-  const int rpm = a.rows_per_mat;
-  if (n < rpm) { row_in_mat = n; return a.W[0]; }
-  if (n < 2 * rpm) { row_in_mat = n - rpm; return a.W[1]; }
-  row_in_mat = n - 2 * rpm;
-  return a.W[2];
+// which of the stacked matrices output feature n belongs to, and its row there
+__device__ __forceinline__ int mat_of(const LinArgs& a, int n, int& row_in_mat) {
+  const int r0 = a.rows_per_mat, rt = a.rows_tail;
+  if (n < r0) { row_in_mat = n; return 0; }
+  if (n < r0 + rt) { row_in_mat = n - r0; return 1; }
+  row_in_mat = n - r0 - rt;
+  return 2;
 }
+__device__ __forceinline__ const void* pick_mat(const LinArgs& a, int n, int& row_in_mat) { return a.W[mat_of(a, n, row_in_mat)]; }
 
 // sum of the partial sums of squares of one X row, in partial order
 __device__ __forceinline__ float ssq_total(const LinArgs& a, int srow) {
@@ -184,7 +186,7 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
     if (tid < SPS_MAX_ROWS) ssq_s[tid] = 0.f;
     __syncthreads();
   }
-  const bool vec = (((N | n_first | rows_all | a.rows_per_mat) & 3) == 0) && ((a.ldy & 3) == 0) &&
+  const bool vec = (((N | n_first | rows_all | a.rows_per_mat | a.rows_tail) & 3) == 0) && ((a.ldy & 3) == 0) &&
                    (!a.wscale[0] || (((size_t)a.wscale[0] | (size_t)a.wscale[1] | (size_t)a.wscale[2]) & 15) == 0) &&
                    ((((size_t)a.Y | (size_t)a.part) & 15) == 0) &&
                    (!a.yp_hi || (((a.ldyp & 3) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 7) == 0) &&
@@ -221,9 +223,10 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
             for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
           }
         }
-        if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: rows_per_mat % 4 == 0)
-          const int mat = n / a.rows_per_mat;
-          const float4 ws = __ldg(reinterpret_cast<const float4*>(a.wscale[mat] + (n - mat * a.rows_per_mat)));
+        if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: every matrix has a multiple of 4 rows)
+          int rin;
+          const int mat = mat_of(a, n, rin);
+          const float4 ws = __ldg(reinterpret_cast<const float4*>(a.wscale[mat] + rin));
           y.x *= ws.x; y.y *= ws.y; y.z *= ws.z; y.w *= ws.w;
         }
         if (row_scale) { const float sc = row_scale[m]; y.x *= sc; y.y *= sc; y.z *= sc; y.w *= sc; }
@@ -257,7 +260,7 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
 #pragma unroll
           for (int j = 0; j < 16; ++j) y += v[j];
         }
-        if (a.wscale[0]) { const int mat = n / a.rows_per_mat; y *= __ldg(a.wscale[mat] + (n - mat * a.rows_per_mat)); }
+        if (a.wscale[0]) { int rin; const int mat = mat_of(a, n, rin); y *= __ldg(a.wscale[mat] + rin); }
         if (row_scale) y *= row_scale[m];
         if (resid) { y += old; sq_s[e] = y * y; }
         a.Y[(long long)m * a.ldy + n] = y;
@@ -576,12 +579,13 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       auto issue = [&](int tile) {
         tile_ids[local & 63] = tile;
         const int row0 = tile * 16;
-        const int mat = row0 / a.rows_per_mat;
+        int rin;
+        const int mat = mat_of(a, row0, rin);
         for (int ks = 0; ks < KSUB; ++ks, ++it) {
           const int slot = it % NS, use = it / NS;
           if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; return; }
           mbar_expect_tx(bar_full + 8 * slot, STAGE);
-          tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, row0 - mat * a.rows_per_mat, (k_base + ks * KST) / SEGK,
+          tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, rin, (k_base + ks * KST) / SEGK,
                       bar_full + 8 * slot, policy);
         }
         ++local;
@@ -1205,6 +1209,9 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   LinArgs a = a_in;
   a.R = p.R; a.S = p.S; a.WC = p.WC; a.PR = p.PR; a.KS = p.KS; a.KST = p.KST; a.NS = p.NS; a.G = p.G;
   if (!a.err) a.err = a.counters + 2 * LIN_MAX_R + 1;
+  if (a.rows_tail <= 0) a.rows_tail = a.rows_per_mat;
+  // stacked matrices: a 16-row weight tile (and a vector of 4 outputs) must lie inside one matrix
+  if (a.N > a.rows_per_mat && dtype >= 1 && ((a.rows_per_mat | a.rows_tail) % 16)) return cudaErrorInvalidValue;
   if ((a.xp_hi || a.yp_hi) && !(dtype >= 1 && p.variant == 2)) return cudaErrorInvalidValue;   // packed activations: TMA kernel only
   if (dtype == 2 && (p.variant != 2 || !a.wscale[0] || (a.D % 128))) return cudaErrorInvalidValue;   // int8 weights: TMA kernel, scales given
   if ((a.xp_hi && !a.xp_lo) || (a.yp_hi && !a.yp_lo)) return cudaErrorInvalidValue;
@@ -1223,9 +1230,11 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     const int threads = (LIN_CONSUMER_WARPS + 1) * 32;
     LinTmaArgs ta;
     ta.a = a;
-    const int nmat = a.N / a.rows_per_mat > 0 ? (a.N + a.rows_per_mat - 1) / a.rows_per_mat : 1;
-    for (int i = 0; i < 3; ++i)
-      if ((e = weight_tensor_map(a.W[i < nmat ? i : 0], a.rows_per_mat, a.D, p.KST, dtype == 2, &ta.tm[i])) != cudaSuccess) return e;
+    const int nmat = a.N > a.rows_per_mat ? 1 + (a.N - a.rows_per_mat + a.rows_tail - 1) / a.rows_tail : 1;
+    for (int i = 0; i < 3; ++i) {
+      const bool has = i < nmat;   // unused slots repeat the first matrix
+      if ((e = weight_tensor_map(a.W[has ? i : 0], has && i > 0 ? a.rows_tail : a.rows_per_mat, a.D, p.KST, dtype == 2, &ta.tm[i])) != cudaSuccess) return e;
+    }
     ta.a.split_epi = lin_split_epilogue() ? 1 : 0;
     ta.a.q8 = dtype == 2 ? 1 : 0;
     static size_t c_q1 = 48 * 1024, c_q2 = 48 * 1024;

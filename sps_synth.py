@@ -13,9 +13,10 @@ import numpy as np
 import torch
 
 
-def _cfg(n_layers, d_model, n_heads, d_head, d_ff, vocab, dtype):
+def _cfg(n_layers, d_model, n_heads, d_head, d_ff, vocab, dtype, n_kv_heads=0):
+    """n_kv_heads: key / value heads (0 = n_heads); fewer than n_heads = grouped-query, 1 = multi-query attention."""
     return dict(n_layers=n_layers, d_model=d_model, n_heads=n_heads, d_head=d_head, d_ff=d_ff, vocab=vocab,
-                dtype=dtype, rms_eps=1e-5, rope_base=10000.0)
+                dtype=dtype, rms_eps=1e-5, rope_base=10000.0, n_kv_heads=n_kv_heads or n_heads)
 
 
 # dtype: 0 = fp32 weights and KV cache, 1 = bf16 weights and KV cache
@@ -34,6 +35,15 @@ CONFIGS = {
                     prompt_len=16, n_new=64, K=4, T=1.0),
     "70b_q8": dict(target=_cfg(80, 8192, 64, 128, 32768, 32000, 2), draft=_cfg(8, 6144, 48, 128, 24576, 32000, 2),
                    prompt_len=128, n_new=128, K=4, T=1.0),
+    # fewer key / value heads than query heads: grouped (4 -> 2) target, multi-query (2 -> 1) draft, fp32
+    "tiny_gqa": dict(target=_cfg(2, 256, 4, 64, 1024, 1024, 0, 2), draft=_cfg(1, 128, 2, 64, 512, 1024, 0, 1),
+                     prompt_len=16, n_new=64, K=4, T=1.0),
+    # multi-query attention with bf16 storage (2 query heads share one key / value head)
+    "tiny_mqa_bf16": dict(target=_cfg(2, 256, 2, 128, 1024, 1024, 1, 1), draft=_cfg(1, 128, 1, 128, 512, 1024, 1, 1),
+                          prompt_len=16, n_new=64, K=4, T=1.0),
+    # the 70B-shaped pair with 8 key / value heads (the KV cache shrinks 8x and 6x)
+    "70b_gqa8": dict(target=_cfg(80, 8192, 64, 128, 32768, 32000, 1, 8), draft=_cfg(8, 6144, 48, 128, 24576, 32000, 1, 8),
+                     prompt_len=128, n_new=128, K=4, T=1.0),
     "mid": dict(target=_cfg(24, 2048, 16, 128, 8192, 32000, 1), draft=_cfg(6, 1024, 8, 128, 4096, 32000, 1),
                 prompt_len=128, n_new=256, K=4, T=1.0),
     # Hyperparams table: target 8192 / 64 heads / 80 layers, draft 6144 / 48 heads / 8 layers
@@ -46,7 +56,8 @@ LAYER_MATS = ("wq", "wk", "wv", "wo", "w_up", "w_down")
 
 def _shape(cfg, name):
     d, f, v = cfg["d_model"], cfg["d_ff"], cfg["vocab"]
-    return {"tok_embed": (v, d), "unembed": (v, d), "wq": (d, d), "wk": (d, d), "wv": (d, d), "wo": (d, d),
+    dkv = cfg.get("n_kv_heads", cfg["n_heads"]) * cfg["d_head"]
+    return {"tok_embed": (v, d), "unembed": (v, d), "wq": (d, d), "wk": (dkv, d), "wv": (dkv, d), "wo": (d, d),
             "w_up": (f, d), "w_down": (d, f)}[name]
 
 
@@ -159,7 +170,8 @@ def weight_bytes(cfg):
     """Bytes one forward pass must stream: all layer matrices + unembedding (+ gains, negligible)."""
     es = {0: 4, 1: 2, 2: 1}[cfg["dtype"]]
     d, f, v = cfg["d_model"], cfg["d_ff"], cfg["vocab"]
-    return cfg["n_layers"] * (4 * d * d + 2 * d * f) * es + v * d * es
+    dkv = cfg.get("n_kv_heads", cfg["n_heads"]) * cfg["d_head"]
+    return cfg["n_layers"] * (2 * d * d + 2 * dkv * d + 2 * d * f) * es + v * d * es
 
 
 def make_prompt(seed, length, vocab):

@@ -24,9 +24,9 @@ def test_every_declared_symbol_is_exported():
 
 
 def test_struct_sizes_match_header():
-    # int32 x7 + float x2 ; two of them + 4 int32 + pointer + uint32 (padded)
-    assert ctypes.sizeof(sps.sps_model_cfg) == 36
-    assert ctypes.sizeof(sps.sps_cfg) == 36 * 2 + 16 + 8 + 8
+    # int32 x7 + float x2 + int32 ; two of them + 4 int32 + pointer + uint32 (padded)
+    assert ctypes.sizeof(sps.sps_model_cfg) == 40
+    assert ctypes.sizeof(sps.sps_cfg) == 40 * 2 + 16 + 8 + 8
     assert ctypes.sizeof(sps.sps_weights) == (11 + 7) * 8      # 11 weight members + 7 row-scale members (int8 weights)
     assert ctypes.sizeof(sps.sps_stats) == 4 * (8 + 17 + 5 + 1)
 

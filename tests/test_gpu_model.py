@@ -15,10 +15,10 @@ from gpu_util import NEAR, make_pair
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-TOL = {"tiny": 1e-3, "tiny_bf16": 5e-2, "tiny_q8": 5e-2}
+TOL = {"tiny": 1e-3, "tiny_bf16": 5e-2, "tiny_q8": 5e-2, "tiny_gqa": 1e-3, "tiny_mqa_bf16": 5e-2}
 
 
-@pytest.mark.parametrize("name", ["tiny", "tiny_bf16", "tiny_q8"])
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16", "tiny_q8", "tiny_gqa", "tiny_mqa_bf16"])
 def test_scoring_pass_logits(name):
     h, ot, od, c = make_pair(name)
     V = c["target"]["vocab"]
@@ -33,7 +33,7 @@ def test_scoring_pass_logits(name):
         want = om.forward64(rows, np.arange(39, 44))
         err = np.abs(out.cpu().numpy() - want).max()
         assert err < TOL[name], err
-        if name == "tiny":
+        if name in ("tiny", "tiny_gqa"):
             assert err < 1e-4, err     # fp32 should land far inside the tolerance
     # parallel scoring == sequential scoring on the GPU too: rows fed one at a time give the same logits
     h.sps_reset()
@@ -122,6 +122,39 @@ def test_token_parity_tiny_fp32(K):
     h.close()
 
 
+@pytest.mark.parametrize("name", ["tiny_gqa", "tiny_mqa_bf16"])
+def test_grouped_key_value_heads(name):
+    """Fewer key / value heads than query heads (grouped-query target 4 -> 2 and multi-query draft 2 -> 1 in fp32,
+    multi-query 2 -> 1 in bf16): the whole loop against the oracle, token-exact on the fp32 pair outside near ties;
+    a batch of sequences equals the same sequences run alone (the cache is indexed per sequence and key / value head)."""
+    h, ot, od, c = make_pair(name, max_batch=3)
+    V = c["target"]["vocab"]
+    loops = near = 0
+    worst = 0.0
+    for seed in range(4):
+        prompt = sps_synth.make_prompt(seed, c["prompt_len"], V)
+        l, n, w = teacher_forced(h, ot, od, prompt, c["n_new"], 4, c["T"], seed)
+        loops += l; near += n; worst = max(worst, w)
+    print(f"{name}: {loops} loops, {near} near-tie mismatches, worst logit error {worst:.2e}")
+    assert worst < TOL[name]
+    if name == "tiny_gqa":
+        assert near <= max(2, loops // 50)
+    prompts = np.stack([sps_synth.make_prompt(10 + b, 16, V) for b in range(3)])
+    together, _ = h.sps_generate_batch(prompts, 24, 4, 1.0, 9)
+    again, _ = h.sps_generate_batch(prompts, 24, 4, 1.0, 9)
+    assert (again == together).all()
+    if name == "tiny_gqa":
+        osps, ok = oracle.Sps(ot, od), 0
+        for b in range(3):
+            want = osps.generate(prompts[b], 24, 4, 1.0, 9, b=b)
+            if (together[b] == want["tokens"]).all():
+                ok += 1
+            else:
+                assert want["flags"] & NEAR
+        assert ok >= 2
+    h.close()
+
+
 def test_generate_matches_oracle_generate():
     h, ot, od, c = make_pair("tiny")
     V = c["target"]["vocab"]
@@ -179,6 +212,30 @@ def test_int8_weights_need_their_scales():
     bad = {k: v for k, v in w.items() if k != "unembed_scale"}
     with pytest.raises(sps.SpsError):
         sps.Handle(c["target"], bad, None, None, max_seq=64)
+
+
+def test_loop_trace_matches_the_statistics():
+    h, _, _, c = make_pair("tiny", max_K=6)
+    with pytest.raises(sps.SpsError):
+        h.sps_last_loop_trace()                      # nothing generated yet
+    prompt = sps_synth.make_prompt(0, 16, c["target"]["vocab"])
+    _, st = h.sps_generate(prompt, 40, 4, 1.0, 1)
+    ms, em, kk = h.sps_last_loop_trace()
+    assert len(ms) == st["loops"] and int(em.sum()) == st["emitted"] and (kk == 4).all()
+    assert abs(float(ms.sum()) - (st["ms_draft"] + st["ms_verify"] + st["ms_accept"])) < 1e-2 and (ms > 0).all()
+    assert [int((em == j).sum()) for j in range(6)] == list(st["hist_emitted"][:6])
+    ms2, em2, _ = h.sps_last_loop_trace(cap=3)
+    assert len(ms2) == 3 and (em2 == em[:3]).all()
+    # adaptive lookahead: the recorded K follows the rule from the recorded acceptances
+    _, st = h.sps_generate_adaptive(prompt, 40, 1, 6, 1.0, 1)
+    ms, em, kk = h.sps_last_loop_trace()
+    K = 3
+    for i in range(len(kk)):
+        assert kk[i] == K
+        a = em[i] - 1
+        K = min(K + 1, 6) if a == K else (max(K - 1, 1) if a == 0 else K)
+    assert int(kk.sum()) == st["draft_calls"]
+    h.close()
 
 
 def test_draft_equal_to_target_accepts_everything():

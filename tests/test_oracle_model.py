@@ -40,6 +40,7 @@ def gelu_tanh(v):
 def matrix_forward(cfg, w, tokens):
     """Whole-sequence, matrix-form forward pass (positions 0..n-1), written independently of the oracle."""
     d, H, dh, eps = cfg["d_model"], cfg["n_heads"], cfg["d_head"], cfg["rms_eps"]
+    Hkv = cfg.get("n_kv_heads", H)
     n = len(tokens)
     x = as_f64(w["tok_embed"])[tokens]
     pos = np.arange(n)[:, None]
@@ -60,8 +61,10 @@ def matrix_forward(cfg, w, tokens):
     for lw in w["layers"]:
         h = norm(x, lw["attn_norm"])
         q = rope((h @ as_f64(lw["wq"]).T).reshape(n, H, dh))
-        k = round_storage(rope((h @ as_f64(lw["wk"]).T).reshape(n, H, dh)), cfg["dtype"])
-        v = round_storage((h @ as_f64(lw["wv"]).T).reshape(n, H, dh), cfg["dtype"])
+        k = round_storage(rope((h @ as_f64(lw["wk"]).T).reshape(n, Hkv, dh)), cfg["dtype"])
+        v = round_storage((h @ as_f64(lw["wv"]).T).reshape(n, Hkv, dh), cfg["dtype"])
+        # each key / value head serves H / Hkv consecutive query heads
+        k, v = np.repeat(k, H // Hkv, axis=1), np.repeat(v, H // Hkv, axis=1)
         sc = np.einsum("ihd,jhd->hij", q, k) / np.sqrt(dh)
         sc = np.where(mask[None], sc, -np.inf)
         pr = np.exp(sc - sc.max(-1, keepdims=True))
@@ -73,7 +76,8 @@ def matrix_forward(cfg, w, tokens):
     return norm(x, w["final_norm"]) @ as_f64(w["unembed"]).T
 
 
-@pytest.mark.parametrize("name,tag", [("tiny", "target"), ("tiny", "draft"), ("tiny_bf16", "target")])
+@pytest.mark.parametrize("name,tag", [("tiny", "target"), ("tiny", "draft"), ("tiny_bf16", "target"),
+                                      ("tiny_gqa", "target"), ("tiny_gqa", "draft"), ("tiny_mqa_bf16", "target")])
 def test_forward_matches_matrix_restatement(name, tag):
     cfg = sps_synth.CONFIGS[name][tag]
     w = np_weights(cfg, seed=0, tag=tag, std=0.08)   # larger std so attention is far from uniform
@@ -182,6 +186,37 @@ def test_special_cases_with_closed_forms():
     # (d) a norm gain of g scales that norm's output: with zero layers, final gain 2 doubles the logits
     w = dict(base, layers=[dict(zero)], final_norm=np.full(d, 2.0, dtype=np.float32))
     assert np.abs(run(w) - 2 * rms(E[toks]) @ U.T).max() < 1e-12
+
+
+@pytest.mark.parametrize("tag", ["target", "draft"])
+def test_grouped_heads_equal_full_heads_with_tied_key_value_matrices(tag):
+    """Grouped-query (or multi-query) attention is ordinary multi-head attention whose key and value projections
+    repeat one block of rows for all the query heads of a group."""
+    cfg = sps_synth.CONFIGS["tiny_gqa"][tag]
+    H, Hkv, dh, d = cfg["n_heads"], cfg["n_kv_heads"], cfg["d_head"], cfg["d_model"]
+    assert Hkv < H
+    w = np_weights(cfg, tag=tag, std=0.08)
+    full = dict(w, layers=[])
+    for lw in w["layers"]:
+        f = dict(lw)
+        for k in ("wk", "wv"):
+            assert lw[k].shape == (Hkv * dh, d)
+            f[k] = np.ascontiguousarray(np.repeat(lw[k].reshape(Hkv, dh, d), H // Hkv, axis=0).reshape(H * dh, d))
+        full["layers"].append(f)
+    toks = sps_synth.make_prompt(4, 10, cfg["vocab"])
+    a = oracle.Transformer(cfg, w, max_seq=16)
+    b = oracle.Transformer(dict(cfg, n_kv_heads=H), full, max_seq=16)
+    ga, gb = a.forward64(toks, np.arange(10)), b.forward64(toks, np.arange(10))
+    assert np.abs(ga - gb).max() < 1e-12 * max(1.0, np.abs(gb).max())
+    # the cache holds Hkv * d_head numbers per position, equal to the first block of each group in the full model
+    ka, va = a.kv(0, 3)
+    kb, vb = b.kv(0, 3)
+    assert ka.shape == (Hkv * dh,) and kb.shape == (H * dh,)
+    assert np.array_equal(kb.reshape(Hkv, H // Hkv, dh)[:, 0], ka.reshape(Hkv, dh))
+    assert np.array_equal(vb.reshape(Hkv, H // Hkv, dh)[:, 1 if H // Hkv > 1 else 0], va.reshape(Hkv, dh))
+    # a number of key / value heads that does not divide n_heads is refused
+    with pytest.raises(ValueError):
+        oracle.Transformer(dict(cfg, n_kv_heads=3), None, 8)
 
 
 def test_invariances():
