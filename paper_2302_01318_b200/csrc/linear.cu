@@ -785,15 +785,20 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           // int8 weights: a lane's two 16-byte chunks of a segment are 2 x 16 k; its activations for them are
           // 2 x 32 bytes of the slab row (chunk c of the segment <-> bytes c*32 of the row's 256)
           const uint32_t xq = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 64;
+          // A lane's 64 bytes of a slab row lie 64 bytes apart from its neighbour's: lanes t and t + 2 would hit the
+          // same banks.  Lanes t >= 2 therefore take their two 32-byte halves (and the matching weight chunks) in
+          // the opposite order, which puts the four lanes of a row on four different bank groups in every load.
+          const uint32_t swp = (uint32_t)(t >> 1);
+          const uint32_t wq0 = swp ? wchunk1 : wchunk0, wq1 = swp ? wchunk0 : wchunk1, xh0 = swp * 32, xh1 = 32 - swp * 32;
           if (pk) {
             const uint32_t xsrc = (g < 4 ? xs_hi : xs_lo) + (uint32_t)min(g & 3, a.M) * XP + xq;
 #pragma unroll 2
             for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
               for (int hf = 0; hf < 2; ++hf) {
-                const uint32_t wc = hf ? wchunk1 : wchunk0;
+                const uint32_t wc = hf ? wq1 : wq0, xo = hf ? xh1 : xh0;
                 const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
-                const uint4 x0 = lds128(xsrc + q * 256 + hf * 32), x1 = lds128(xsrc + q * 256 + hf * 32 + 16);
+                const uint4 x0 = lds128(xsrc + q * 256 + xo), x1 = lds128(xsrc + q * 256 + xo + 16);
                 q8_mma4(acc[0][0], acc[0][2], wa, wb, x0, x1);
               }
             }
@@ -805,11 +810,11 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
             for (int q = qfirst; q < slabs; q += GS) {
 #pragma unroll
               for (int hf = 0; hf < 2; ++hf) {
-                const uint32_t wc = hf ? wchunk1 : wchunk0;
+                const uint32_t wc = hf ? wq1 : wq0;
                 const uint4 wa = lds128(wrow + q * 2048 + wc), wb = lds128(wrow + q * 2048 + 1024 + wc);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
-                  const uint32_t xo = xr8[nt] + q * 256 + hf * 32;
+                  const uint32_t xo = xr8[nt] + q * 256 + (hf ? xh1 : xh0);
                   const uint4 h0 = lds128(xs_hi + xo), h1 = lds128(xs_hi + xo + 16);
                   q8_mma4(acc[nt][0], acc[nt][2], wa, wb, h0, h1);
                   const uint4 l0 = lds128(xs_lo + xo), l1 = lds128(xs_lo + xo + 16);
