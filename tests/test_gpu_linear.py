@@ -105,3 +105,25 @@ def test_linear_full_size_sampled_rows(N, D):
     want = oracle.linear(Wr, X.cpu().numpy())
     assert np.abs(got[:, rows] - want).max() <= tol(W[:64].float(), X, D)
     assert np.isfinite(got).all()
+
+
+@pytest.mark.parametrize("N,D", [(32768, 8192), (8192, 32768)])
+def test_linear_int8_full_size_sampled_rows(N, D):
+    """the 70B-shaped feed-forward matrices as int8 at full size (268 MB each), M = 5 as in the bench: sampled
+    output rows against the oracle's double dot products on the dequantised rows"""
+    g = torch.Generator(device=DEV).manual_seed(N + D)
+    q = torch.randint(-127, 128, (N, D), device=DEV, generator=g, dtype=torch.int32).to(torch.int8)
+    scale = (torch.rand(N, device=DEV, generator=g) * 1e-3 + 1e-4).float()
+    X = torch.randn((5, D), device=DEV, generator=g)
+    ws = torch.zeros(sps.sps_linear_workspace_bytes(2, 5, N, D), dtype=torch.uint8, device=DEV)
+    Y = torch.full((5, N), float("nan"), device=DEV)
+    sps.sps_linear_scaled(q, scale, X, Y, ws)
+    torch.cuda.synchronize()
+    got = Y.cpu().numpy()
+    rows = np.unique(np.concatenate([[0, 1, 15, 16, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 58)]))
+    idx = torch.from_numpy(rows).to(DEV)
+    Wd = (q[idx].double() * scale[idx].double()[:, None]).float().cpu()
+    want = oracle.linear(Wd.numpy(), X.cpu().numpy())
+    assert np.abs(got[:, rows] - want).max() <= tol(Wd, X.cpu(), D)
+    assert np.isfinite(got).all()
+
