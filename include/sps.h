@@ -282,6 +282,21 @@ int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t 
                void* workspace, void* stream, float* out_ms);
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D);
 
+/* The linear layer of the prompt pass (Algorithm 2 starts from a prompt of t
+ * tokens whose keys and values both models must hold before the first loop):
+ * the same product Y[M, N] = X[M, D] W[N, D]^T for up to 128 rows at once, so
+ * that the weights are read once for the whole prompt chunk.  bf16 weights
+ * only; W device row-major [N, D], 16-byte aligned; X device fp32 [M, D]; Y
+ * device fp32 [M, N]; 1 <= M <= 128; D a multiple of 64.  The activations enter
+ * the tensor cores as two bf16 halves (about 16 significant bits), products
+ * accumulate in fp32.  workspace: device scratch of
+ * sps_linear_wide_workspace_bytes(N, D) bytes, contents irrelevant.  The call
+ * waits for the result; out_ms (host, may be NULL) receives the device time.
+ * Returns SPS_ETIMEOUT if a bounded wait inside the kernel ran out. */
+int sps_linear_wide(const void* W, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace, void* stream,
+                    float* out_ms);
+int64_t sps_linear_wide_workspace_bytes(int32_t N, int32_t D);
+
 /* The same linear layer for callers that cannot allocate device memory (the
  * paper has no counterpart: this is a service of the library, not a step of
  * the method).  A host that runs inside a stream capture, or serves under a

@@ -91,6 +91,9 @@ def lib():
         L.sps_sample_filtered.argtypes = [vp, i32, i32, f32, i32, f32, u64, u32, u32, vp, vp]
         L.sps_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
         L.sps_linear_scaled.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
+        L.sps_linear_wide.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, C.POINTER(f32)]
+        L.sps_linear_wide_workspace_bytes.argtypes = [i32, i32]
+        L.sps_linear_wide_workspace_bytes.restype = i64
         L.sps_linear_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.sps_linear_workspace_bytes.restype = i64
         L.sps_philox.argtypes = [vp, vp, i32, vp, vp]
@@ -299,6 +302,20 @@ def sps_linear_scaled(W, row_scale, X, Y, workspace, stream=None, timed=False):
     ms = C.c_float(0)
     _check(lib().sps_linear_scaled(W.data_ptr(), 2, row_scale.data_ptr(), X.data_ptr(), M, N, D, Y.data_ptr(),
                                    workspace.data_ptr(), _stream_ptr(stream), C.byref(ms) if timed else None))
+    return ms.value
+
+
+def sps_linear_wide_workspace_bytes(N, D):
+    return int(lib().sps_linear_wide_workspace_bytes(N, D))
+
+
+def sps_linear_wide(W, X, Y, workspace, stream=None, timed=False):
+    """Y[M,N] = X[M,D] W[N,D]^T for up to 128 rows (the prompt pass): W CUDA bf16, X/Y CUDA fp32."""
+    N, D = W.shape
+    M = X.shape[0]
+    ms = C.c_float(0)
+    _check(lib().sps_linear_wide(W.data_ptr(), X.data_ptr(), M, N, D, Y.data_ptr(), workspace.data_ptr(),
+                                 _stream_ptr(stream), C.byref(ms) if timed else None))
     return ms.value
 
 

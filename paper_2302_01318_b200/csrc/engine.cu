@@ -45,6 +45,11 @@ struct sps_handle {
   DevState hst{};          // host image of the device state block
   DevState* dst = nullptr;
   float *x = nullptr, *qkv = nullptr, *attn = nullptr, *up = nullptr, *ssqA = nullptr, *ssqB = nullptr;
+  // the prompt pass over up to 128 rows at once (bf16 models, one sequence): residual stream, q|k|v, attention output,
+  // the GEMM operands' bf16 halves (normalised rows / GeLU outputs) and the k-splits' partial products
+  bool wide = false;
+  float *wx = nullptr, *wqkv = nullptr, *watt = nullptr, *wpart = nullptr;
+  void *wa_hi = nullptr, *wa_lo = nullptr, *wu_hi = nullptr, *wu_lo = nullptr;
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
@@ -402,11 +407,54 @@ int set_sequences(sps_handle* h, const int32_t* toks, int B, int n) {
 }
 
 // both caches ingest positions 0..n-2 of every live sequence
+// The prompt pass of a bf16 model, one sequence, in chunks of up to 128 rows: every linear layer is one GEMM on the
+// tcgen05 tensor cores (wide.cu), so a chunk reads the weights once; attention runs the decode kernel over 16 of the
+// chunk's rows at a time (earlier rows' keys come from the cache, which the chunk's earlier launches have filled).
+// No logits: the prompt's last token is fed by the first loop.
+int prefill_wide(sps_handle* h, ModelDev& m, int n) {
+  const sps_model_cfg& c = m.cfg;
+  const int d = c.d_model, dff = c.d_ff, dkv = kv_width(c), ldq = d + 2 * dkv;
+  cudaStream_t st = h->stream;
+  int* err = h->hst.err;
+  for (int c0 = 0; c0 < n - 1; c0 += WIDE_ROWS) {
+    const int rows = (n - 1 - c0) < WIDE_ROWS ? (n - 1 - c0) : WIDE_ROWS;
+    CU(h, wide_embed_launch(h->dst, m.tok_embed, h->wx, rows, d, c.vocab, c0, st)); h->launches++;
+    for (int l = 0; l < c.n_layers; ++l) {
+      CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
+      CU(h, wide_gemm_launch(m.wq[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+      CU(h, wide_gemm_launch(m.wk[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+      CU(h, wide_gemm_launch(m.wv[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d + dkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+      h->launches += 7;
+      for (int r0 = 0; r0 < rows; r0 += SPS_MAX_ROWS) {
+        AttnArgs aa{};
+        aa.st = h->dst; aa.qkv = h->wqkv + (size_t)r0 * ldq; aa.out = h->watt + (size_t)r0 * d;
+        aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
+        aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
+        aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = (rows - r0) < SPS_MAX_ROWS ? (rows - r0) : SPS_MAX_ROWS; aa.B = 1;
+        aa.mode = PASS_PREFILL; aa.t = 0; aa.c0 = c0 + r0;
+        CU(h, attn_launch(aa, st)); h->launches++;
+      }
+      CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
+      CU(h, wide_gemm_launch(m.wo[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+      CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
+      CU(h, wide_gemm_launch(m.w_up[l], h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st));
+      CU(h, wide_gemm_launch(m.w_down[l], h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+      h->launches += 8;
+    }
+  }
+  return SPS_OK;
+}
+
 int prefill_all(sps_handle* h, int n) {
   const int per = SPS_MAX_ROWS / h->B;
   for (int which = 0; which < 2; ++which) {
     ModelDev& m = which == 0 ? h->tgt : h->drf;
     if (!m.present) continue;
+    if (h->wide && h->B == 1 && m.cfg.dtype == 1 && n - 1 > SPS_MAX_ROWS) {
+      int rc = prefill_wide(h, m, n);
+      if (rc) return rc;
+      continue;
+    }
     for (int c0 = 0; c0 < n - 1; c0 += per) {
       PassSpec ps{};
       ps.mode = PASS_PREFILL; ps.c0 = c0; ps.rows_per_seq = (n - 1 - c0) < per ? (n - 1 - c0) : per;
@@ -487,6 +535,30 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   if (pf2 > part_floats) part_floats = pf2;
   if (part_floats == 0) part_floats = 1;
   h->res_words = (size_t)MB * 2 + (size_t)MB * (maxK + 1) + 1;
+  {
+    // buffers of the 128-row prompt pass, when a bf16 model is there to use it (SPS_WIDE_PREFILL=0 keeps the 16-row pass)
+    static const bool off = [] { const char* e = getenv("SPS_WIDE_PREFILL"); return e && atoi(e) == 0; }();
+    size_t wd = 0, wf = 0, wpart = 0;
+    for (const ModelDev* m : {&h->tgt, &h->drf}) {
+      if (!m->present || m->cfg.dtype != 1) continue;
+      const sps_model_cfg& c = m->cfg;
+      wd = std::max(wd, (size_t)c.d_model); wf = std::max(wf, (size_t)c.d_ff);
+      const int shapes[4][2] = {{c.d_model, c.d_model}, {kv_width(c), c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}};
+      for (auto& sh : shapes) wpart = std::max(wpart, wide_part_floats(sh[0], sh[1], h->num_sm));
+    }
+    if (wd > 0 && !off) {
+      struct WW { void** p; size_t bytes; };
+      const WW ww[] = {{(void**)&h->wx, sizeof(float) * WIDE_ROWS * wd},       {(void**)&h->wqkv, sizeof(float) * WIDE_ROWS * 3 * wd},
+                       {(void**)&h->watt, sizeof(float) * WIDE_ROWS * wd},     {(void**)&h->wpart, sizeof(float) * wpart},
+                       {&h->wa_hi, 2 * (size_t)WIDE_ROWS * wd},                {&h->wa_lo, 2 * (size_t)WIDE_ROWS * wd},
+                       {&h->wu_hi, 2 * (size_t)WIDE_ROWS * wf},                {&h->wu_lo, 2 * (size_t)WIDE_ROWS * wf}};
+      for (const WW& w : ww) {
+        if (cudaMalloc(w.p, w.bytes) != cudaSuccess) return bail(fail(h, SPS_ENOMEM, "device allocation failed"));
+        if (cudaMemsetAsync(*w.p, 0, w.bytes, h->stream) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "memset failed"));
+      }
+      h->wide = true;
+    }
+  }
   struct Want { void** p; size_t bytes; };
   DevState& s = h->hst;
   const Want wants[] = {
@@ -542,7 +614,7 @@ int sps_destroy(sps_handle* h) {
   for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
   free_model(h->tgt);
   free_model(h->drf);
-  void* bufs[] = {h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
+  void* bufs[] = {h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
                   h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);
@@ -833,6 +905,42 @@ int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t 
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || dtype < 0 || dtype > 2) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
   return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256);
+}
+
+int64_t sps_linear_wide_workspace_bytes(int32_t N, int32_t D) {
+  if (N < 1 || D < 64 || D % 64) return -1;
+  // error word + the activations' two bf16 halves (128 rows each) + the k-splits' partial products
+  return (int64_t)(256 + 2 * (size_t)WIDE_ROWS * D * 2 + sizeof(float) * wide_part_floats(N, D, cur_num_sm()));
+}
+
+int sps_linear_wide(const void* W, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace, void* stream,
+                    float* out_ms) {
+  if (!W || !X || !Y || !workspace) return fail(nullptr, SPS_EINVAL, "null argument");
+  if (M < 1 || M > WIDE_ROWS || N < 1 || D < 64 || D % 64) return fail(nullptr, SPS_EINVAL, "M must be 1..128, D a multiple of 64");
+  if (((uintptr_t)W | (uintptr_t)workspace) & 15) return fail(nullptr, SPS_EINVAL, "W and workspace must be 16-byte aligned");
+  char* ws = (char*)workspace;
+  int* err = (int*)ws;
+  void* hi = ws + 256;
+  void* lo = ws + 256 + (size_t)WIDE_ROWS * D * 2;
+  float* part = (float*)(ws + 256 + 2 * (size_t)WIDE_ROWS * D * 2);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaMemsetAsync(err, 0, 4, st);
+  if (out_ms) { cudaEventCreate(&e0); cudaEventCreate(&e1); cudaEventRecord(e0, st); }
+  if (e == cudaSuccess) e = wide_pack_launch(X, D, nullptr, 0.f, M, D, hi, lo, D, st);
+  if (e == cudaSuccess) e = wide_gemm_launch(W, hi, lo, M, N, D, part, WIDE_STORE, Y, N, nullptr, nullptr, 0, err, cur_num_sm(), st);
+  if (out_ms) {
+    cudaEventRecord(e1, st);
+    cudaEventSynchronize(e1);
+    cudaEventElapsedTime(out_ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+  }
+  if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("wide linear launch: ") + cudaGetErrorString(e));
+  int errw = 0;
+  if (cudaMemcpyAsync(&errw, err, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return fail(nullptr, SPS_ECUDA, std::string("wide linear: ") + cudaGetErrorString(cudaGetLastError()));
+  if (errw == 3) return fail(nullptr, SPS_ETIMEOUT, "a bounded device-side wait ran out in the wide linear kernel");
+  return SPS_OK;
 }
 
 int sps_linear(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y, void* workspace,

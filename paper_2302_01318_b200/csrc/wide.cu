@@ -1,0 +1,407 @@
+// The prompt pass as a real GEMM: up to 128 activation rows at once on the 5th-generation tensor cores.
+//
+// The decode kernels (linear.cu) stream every weight once per <= 16 rows, which is right for the loop
+// (1..K+1 rows) and wrong for the prompt: 127 prompt rows cost eight full sweeps over the weights.  Here
+// Y[128, N] = X[128, D] W[N, D]^T runs as tcgen05.mma (cta_group::1, M = 128, N = 256, K = 16, bf16
+// operands, fp32 accumulators in tensor memory), so the prompt costs one sweep:
+//
+//   * grid = (N / 256 weight-row tiles) x (S k-splits); one CTA keeps a 128 x 256 fp32 accumulator in
+//     256 columns of tensor memory;
+//   * warp 0 (one lane) is the copy producer: per 64-wide k-block one TMA box of W (256 rows x 128 B)
+//     and one each of the activations' high and low bf16 halves (128 rows x 128 B), 128-byte swizzle,
+//     into a 3-stage ring of 64 KB stages guarded by full / empty mbarriers;
+//   * warp 1 (one lane) issues the MMAs: 4 k-steps x (high, low) per k-block -- the two halves make the
+//     activations exact to ~16 bits as in the decode kernels -- and releases the stage with tcgen05.commit;
+//   * warps 2..5 read the accumulator back with tcgen05.ld once the last commit has landed (warp w owns
+//     tensor-memory lanes 32 (w % 4) ..) and write the CTA's partial tile; wide_epilogue_kernel adds the
+//     k-splits in a fixed order and applies the layer's epilogue (store / residual add / GeLU + split).
+//
+// Per weight byte the activations cost one byte of L2 traffic (128 rows x 2 halves x 2 B per 256 weight
+// rows), so the pass stays bound by the weight stream from HBM.  Every wait is bounded (2 s of
+// %globaltimer): on expiry the CTA records error 3, lets its copies land, frees its tensor memory and
+// returns.  No multicast, no clusters.
+#include "common.cuh"
+
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+namespace {
+
+constexpr int WIDE_M = 128;        // activation rows of one pass (tensor-memory lanes)
+constexpr int WIDE_BN = 256;       // weight rows per CTA (tensor-memory columns)
+constexpr int WIDE_BK = 64;        // k per stage: 128 bytes of bf16 = one swizzle row
+constexpr int WIDE_STAGES = 3;
+constexpr uint32_t WIDE_A_BYTES = WIDE_M * WIDE_BK * 2;     // 16 KB per half
+constexpr uint32_t WIDE_B_BYTES = WIDE_BN * WIDE_BK * 2;    // 32 KB
+constexpr uint32_t WIDE_STAGE_BYTES = 2 * WIDE_A_BYTES + WIDE_B_BYTES;
+constexpr size_t WIDE_SMEM = 1024 + (size_t)WIDE_STAGES * WIDE_STAGE_BYTES + 1024;   // header + ring + alignment slack
+
+__device__ __forceinline__ uint32_t w_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long w_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void w_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void w_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t w_mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// bounded wait: false (and error word 3) after 2 s
+__device__ __forceinline__ bool w_mbar_wait(uint32_t bar, uint32_t parity, int* err) {
+  if (w_mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = w_timer();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+      if (w_mbar_try(bar, parity)) return true;
+    if (w_timer() - t0 > 2000000000ull) {
+      atomicExch(err, 3);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void w_tma_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+// Shared-memory operand descriptor for a K-major tile whose rows are 128 bytes (64 bf16) under the
+// 128-byte swizzle: groups of 8 rows are 1024 bytes apart (stride offset), the leading offset is unused,
+// descriptor version 1, layout type 2 (128-byte swizzle).  Stepping 16 elements along k inside the
+// swizzle row adds 32 bytes to the start address.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)1 << 16;                       // leading byte offset (ignored for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset: 8 rows x 128 B
+  d |= (uint64_t)1 << 46;                       // descriptor version
+  d |= (uint64_t)2 << 61;                       // 128-byte swizzle
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N = 256, M = 128
+constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(WIDE_BN >> 3) << 17) | ((uint32_t)(WIDE_M >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(UMMA_IDESC), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier once every MMA issued so far by this thread has finished reading its operands
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+struct WideGemmArgs {
+  CUtensorMap tm_hi, tm_lo, tm_w;
+  float* part;        // [S][128][N] partial products of the k-splits
+  int M, N, D, S;     // live rows, weight rows, width, k-splits (D / 64 is a multiple of S)
+  int* err;
+};
+
+__global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant__ WideGemmArgs a) {
+  extern __shared__ unsigned char wsm_raw[];
+  // header: full[3], empty[3], accumulator-ready barrier, tensor-memory base, abort flag; ring 1024-aligned
+  const uint32_t raw = w_smem_u32(wsm_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* hdr = wsm_raw + (base - raw);
+  const uint32_t bar_full = base, bar_empty = base + 64, bar_acc = base + 128;
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(hdr + 192);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(hdr + 200);
+  const uint32_t ring = base + 1024;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x, s = blockIdx.y;
+  const int kb_all = a.D / WIDE_BK, kb_n = kb_all / a.S, kb0 = s * kb_n;
+
+  if (tid == 0) {
+    for (int i = 0; i < WIDE_STAGES; ++i) { w_mbar_init(bar_full + 8 * i, 1); w_mbar_init(bar_empty + 8 * i, 1); }
+    w_mbar_init(bar_acc, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    // 256 columns of tensor memory for the 128 x 256 fp32 accumulator (one CTA per SM: always available)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 192), "r"(WIDE_BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *s_tmem;
+  // the activations are the predecessor's output; nothing is fetched before it has finished
+  pdl_wait();
+  pdl_launch_dependents();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      int issued = 0;
+      for (int kb = 0; kb < kb_n && ok; ++kb, ++issued) {
+        const int st = kb % WIDE_STAGES, use = kb / WIDE_STAGES;
+        if (use > 0 && !w_mbar_wait(bar_empty + 8 * st, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; break; }
+        if (*s_abort) { ok = false; break; }
+        const uint32_t dst = ring + st * WIDE_STAGE_BYTES;
+        const int k = (kb0 + kb) * WIDE_BK;
+        w_mbar_expect_tx(bar_full + 8 * st, WIDE_STAGE_BYTES);
+        w_tma_2d(dst, &a.tm_hi, k, 0, bar_full + 8 * st);
+        w_tma_2d(dst + WIDE_A_BYTES, &a.tm_lo, k, 0, bar_full + 8 * st);
+        w_tma_2d(dst + 2 * WIDE_A_BYTES, &a.tm_w, k, tile * WIDE_BN, bar_full + 8 * st);
+      }
+      if (!ok) {
+        *s_abort = 1;
+        // let the copies already issued land before this CTA's shared memory goes away
+        for (int j = max(0, issued - WIDE_STAGES); j < issued; ++j)
+          w_mbar_wait(bar_full + 8 * (j % WIDE_STAGES), (uint32_t)(j / WIDE_STAGES) & 1u, a.err);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int kb = 0; kb < kb_n && ok; ++kb) {
+        const int st = kb % WIDE_STAGES, use = kb / WIDE_STAGES;
+        if (!w_mbar_wait(bar_full + 8 * st, (uint32_t)use & 1u, a.err) || *s_abort) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = ring + st * WIDE_STAGE_BYTES;
+        const uint64_t d_hi = umma_desc(sa), d_lo = umma_desc(sa + WIDE_A_BYTES), d_w = umma_desc(sa + 2 * WIDE_A_BYTES);
+#pragma unroll
+        for (int k = 0; k < WIDE_BK / 16; ++k) {
+          // 16 elements along k = 32 bytes = 2 units of the descriptor's address field
+          umma_bf16(tmem, d_hi + 2 * k, d_w + 2 * k, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_bf16(tmem, d_lo + 2 * k, d_w + 2 * k, 1u);
+        }
+        umma_commit(bar_empty + 8 * st);   // the stage is free once these MMAs have read it
+      }
+      if (ok) umma_commit(bar_acc);         // ... and the accumulator is complete once all of them are done
+      else *s_abort = 1;
+    }
+  } else {
+    // epilogue warps 2..5: tensor-memory lanes 32 q .. 32 q + 31 with q = warp % 4
+    const int q = warp & 3, row = q * 32 + lane;
+    bool ok = w_mbar_wait(bar_acc, 0u, a.err) && !*s_abort;
+    ok = __all_sync(0xffffffffu, ok);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+      float* dst = a.part + ((size_t)s * WIDE_M + row) * a.N + (size_t)tile * WIDE_BN;
+      const int ncols = min(WIDE_BN, a.N - tile * WIDE_BN);
+#pragma unroll 1
+      for (int c = 0; c < WIDE_BN; c += 32) {
+        float v[32];
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);   // the whole warp takes part in the load
+        if (row < a.M && c < ncols) {
+          if (c + 32 <= ncols && (a.N & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+          } else {
+            for (int i = 0; i < 32 && c + i < ncols; ++i) dst[c + i] = v[i];
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(WIDE_BN) : "memory");
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// Elementwise companions of the GEMM (all rows x features, memory-bound, a few microseconds each)
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+__device__ __forceinline__ void wide_split(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+  hi = __float2bfloat16_rn(v);
+  lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+__device__ __forceinline__ float wide_gelu(float v) {
+  return 0.5f * v * (1.0f + tanhf(0.7978845608028654f * (v + 0.044715f * v * v * v)));
+}
+
+// x[row] = E[token at position c0 + row] for the rows of one prompt chunk
+__global__ void __launch_bounds__(256) wide_embed_kernel(const DevState* st, const __nv_bfloat16* tok_embed, float* x, int d, int V, int c0) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int row = blockIdx.x;
+  int tok = st->tokens[c0 + row];   // sequence 0
+  if (tok < 0 || tok >= V) { tok = 0; if (threadIdx.x == 0) atomicExch(st->err, 1); }
+  const __nv_bfloat16* e = tok_embed + (size_t)tok * d;
+  for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)row * d + k] = __bfloat162float(e[k]);
+}
+
+// one CTA per row: (optionally) RMS-normalise with the gain, then split into bf16 high and low halves
+__global__ void __launch_bounds__(256) wide_pack_kernel(const float* x, int ldx, const float* gain, float eps, int d,
+                                                        __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp) {
+  __shared__ float s_part[8];
+  __shared__ float s_inv;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int row = blockIdx.x, tid = threadIdx.x;
+  const float* xr = x + (size_t)row * ldx;
+  float inv = 1.f;
+  if (gain) {
+    float local = 0.f;
+    for (int k = tid; k < d; k += 256) { const float v = xr[k]; local += v * v; }
+    local = warp_sum(local);
+    if ((tid & 31) == 0) s_part[tid >> 5] = local;
+    __syncthreads();
+    if (tid == 0) {
+      float t = 0.f;
+      for (int w = 0; w < 8; ++w) t += s_part[w];
+      s_inv = rsqrtf(t / (float)d + eps);
+    }
+    __syncthreads();
+    inv = s_inv;
+  }
+  for (int k = tid; k < d; k += 256) {
+    const float v = gain ? gain[k] * (xr[k] * inv) : xr[k];
+    __nv_bfloat16 h, l;
+    wide_split(v, h, l);
+    hi[(size_t)row * ldp + k] = h;
+    lo[(size_t)row * ldp + k] = l;
+  }
+}
+
+enum { WIDE_EPI_STORE = 0, WIDE_EPI_RESIDUAL = 1, WIDE_EPI_GELU_PACK = 2 };
+
+// y = sum over the k-splits in order, then: store / add to the residual stream / GeLU and split for the next GEMM
+__global__ void __launch_bounds__(256) wide_epilogue_kernel(const float* part, int S, int M, int N, int mode, float* y, long long ldy,
+                                                            __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const long long total = (long long)M * N;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+    const int row = (int)(i / N), n = (int)(i - (long long)row * N);
+    float t = 0.f;
+    for (int s = 0; s < S; ++s) t += part[((size_t)s * WIDE_M + row) * N + n];
+    if (mode == WIDE_EPI_STORE) y[row * ldy + n] = t;
+    else if (mode == WIDE_EPI_RESIDUAL) y[row * ldy + n] += t;
+    else {
+      __nv_bfloat16 h, l;
+      wide_split(wide_gelu(t), h, l);
+      hi[(size_t)row * ldp + n] = h;
+      lo[(size_t)row * ldp + n] = l;
+    }
+  }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 wide_encoder() {
+  static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return nullptr;
+    encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  return encode;
+}
+
+// bf16 [rows][D] row-major, boxes of 64 elements x box_rows rows under the 128-byte swizzle; rows beyond the
+// matrix read as zeros
+cudaError_t wide_map(const void* p, int rows, int D, int box_rows, CUtensorMap* out) {
+  static std::mutex mu;
+  static std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = wide_encoder();
+  if (!encode) return cudaErrorNotSupported;
+  std::lock_guard<std::mutex> lock(mu);
+  const auto key = std::make_tuple(p, rows, D, box_rows);
+  auto it = cache.find(key);
+  if (it != cache.end()) { *out = it->second; return cudaSuccess; }
+  const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)WIDE_BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  CUtensorMap tm;
+  const CUresult cr = encode(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(p), gdim, gstride, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  if (cache.size() > 100000) cache.clear();
+  cache[key] = tm;
+  *out = tm;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+int wide_splits(int N, int D, int num_sm) {
+  const int tiles = (N + WIDE_BN - 1) / WIDE_BN, kb = D / WIDE_BK;
+  int S = 1;
+  for (int s = 1; s <= kb && s * tiles <= (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK); ++s)
+    if (kb % s == 0) S = s;
+  return S;
+}
+size_t wide_part_floats(int N, int D, int num_sm) { return (size_t)wide_splits(N, D, num_sm) * WIDE_M * (size_t)N; }
+
+cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int c0, cudaStream_t s) {
+  return launch_k(wide_embed_kernel, dim3(rows), dim3(256), 0, s, st, reinterpret_cast<const __nv_bfloat16*>(tok_embed), x, d, V, c0);
+}
+cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s) {
+  return launch_k(wide_pack_kernel, dim3(rows), dim3(256), 0, s, x, ldx, gain, eps, d, reinterpret_cast<__nv_bfloat16*>(hi),
+                  reinterpret_cast<__nv_bfloat16*>(lo), ldp);
+}
+
+// Y = epilogue(sum_k-splits (hi + lo)[M, D] W[N, D]^T).  hi / lo: bf16 [128][D] (rows >= M are never read back);
+// part: wide_part_floats(N, D) floats.  mode WIDE_EPI_*: y / ldy for store and residual, yhi / ylo / ldp for GeLU + split.
+cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,
+                             long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st) {
+  if (M < 1 || M > WIDE_M || N < 1 || D < WIDE_BK || (D % WIDE_BK)) return cudaErrorInvalidValue;
+  WideGemmArgs a;
+  cudaError_t e;
+  if ((e = wide_map(hi, WIDE_M, D, WIDE_M, &a.tm_hi)) != cudaSuccess) return e;
+  if ((e = wide_map(lo, WIDE_M, D, WIDE_M, &a.tm_lo)) != cudaSuccess) return e;
+  if ((e = wide_map(W, N, D, WIDE_BN, &a.tm_w)) != cudaSuccess) return e;
+  a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits(N, D, num_sm); a.err = err;
+  static bool attr = false;
+  if (!attr) {
+    if ((e = cudaFuncSetAttribute(wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WIDE_SMEM)) != cudaSuccess) return e;
+    attr = true;
+  }
+  const int tiles = (N + WIDE_BN - 1) / WIDE_BN;
+  if ((e = launch_k(wide_gemm_kernel, dim3(tiles, a.S), dim3(192), WIDE_SMEM, st, a)) != cudaSuccess) return e;
+  const long long total = (long long)M * N;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK)) blocks = 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
+  return launch_k(wide_epilogue_kernel, dim3(blocks), dim3(256), 0, st, (const float*)part, a.S, M, N, mode, y, ldy,
+                  reinterpret_cast<__nv_bfloat16*>(yhi), reinterpret_cast<__nv_bfloat16*>(ylo), ldp);
+}

@@ -127,3 +127,28 @@ def test_linear_int8_full_size_sampled_rows(N, D):
     assert np.abs(got[:, rows] - want).max() <= tol(Wd, X.cpu(), D)
     assert np.isfinite(got).all()
 
+
+
+def run_linear_wide(W, X):
+    N, D = W.shape
+    ws = torch.empty(sps.sps_linear_wide_workspace_bytes(N, D), dtype=torch.uint8, device=DEV)
+    Y = torch.full((X.shape[0], N), float("nan"), device=DEV)
+    sps.sps_linear_wide(W, X, Y, ws)
+    torch.cuda.synchronize()
+    return Y.cpu().numpy()
+
+
+@pytest.mark.parametrize("M", [1, 5, 33, 127, 128])
+@pytest.mark.parametrize("N,D", [(256, 64), (300, 128), (1000, 256), (77, 1024), (4099, 2048)])
+def test_linear_wide_small(M, N, D):
+    """The prompt-pass GEMM (up to 128 rows on the tcgen05 tensor cores) against the oracle: ragged N (tiles of
+    256 weight rows), one to many k-blocks and k-splits, every row count class."""
+    g = torch.Generator().manual_seed(N + D + M)
+    W = (torch.randn((N, D), generator=g) * 0.05).to(torch.bfloat16)
+    X = torch.randn((M, D), generator=g)
+    got = run_linear_wide(W.to(DEV), X.to(DEV))
+    want = oracle.linear(sps_synth.to_numpy(W), X.numpy())
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= tol(W.float(), X, D)
+    # run to run the same bits (fixed k-split order)
+    assert np.array_equal(got, run_linear_wide(W.to(DEV), X.to(DEV)))
