@@ -152,3 +152,18 @@ def test_linear_wide_small(M, N, D):
     assert np.abs(got - want).max() <= tol(W.float(), X, D)
     # run to run the same bits (fixed k-split order)
     assert np.array_equal(got, run_linear_wide(W.to(DEV), X.to(DEV)))
+
+
+@pytest.mark.parametrize("N,D", [(32768, 8192), (8192, 32768)])
+def test_linear_wide_full_size_sampled_rows(N, D):
+    """the 70B-shaped feed-forward matrices at full size with the prompt's 127 rows: sampled output features of
+    every row against the oracle's double dot products"""
+    g = torch.Generator(device=DEV).manual_seed(N + D)
+    W = torch.empty((N, D), device=DEV, dtype=torch.bfloat16).normal_(0, 0.02, generator=g)
+    X = torch.randn((127, D), device=DEV, generator=g)
+    got = run_linear_wide(W, X)
+    rows = np.unique(np.concatenate([[0, 1, 255, 256, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 26)]))
+    Wr = sps_synth.to_numpy(W[torch.from_numpy(rows).to(DEV)])
+    want = oracle.linear(Wr, X.cpu().numpy())
+    assert np.abs(got[:, rows] - want).max() <= tol(W[:64].float(), X.cpu(), D)
+    assert np.isfinite(got).all()

@@ -214,6 +214,31 @@ def test_int8_weights_need_their_scales():
         sps.Handle(c["target"], bad, None, None, max_seq=64)
 
 
+@pytest.mark.parametrize("name", ["tiny_bf16", "tiny_mqa_bf16"])
+def test_long_prompt_through_the_wide_prompt_pass(name):
+    """A 200-token prompt goes through the 128-row prompt pass in two chunks (128 + 71 rows; the tensor-core GEMM,
+    attention 16 rows at a time over the cache the chunk is filling); the logits of the next five rows and a
+    generation's bookkeeping must agree with the oracle as for short prompts."""
+    h, ot, od, c = make_pair(name, max_seq=288)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(5, 200, V)
+    h.sps_prefill(prompt)
+    ot.forward(prompt[:-1], np.arange(199), want_logits=False)
+    od.forward(prompt[:-1], np.arange(199), want_logits=False)
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(6, 4, V)])
+    out = torch.zeros((5, V), device=DEV)
+    for which, om in ((0, ot), (1, od)):
+        h.sps_score(which, rows, out)
+        want = om.forward64(rows, np.arange(199, 204))
+        err = np.abs(out.cpu().numpy() - want).max()
+        print(f"{name} model {which}: logit error after a 199-row prompt pass {err:.2e}")
+        assert err < TOL[name], err
+    a, st = h.sps_generate(prompt, 32, 4, 1.0, 3)
+    b, _ = h.sps_generate(prompt, 32, 4, 1.0, 3)
+    assert (a == b).all() and st["emitted"] - st["overshoot"] == 32
+    h.close()
+
+
 def test_loop_trace_matches_the_statistics():
     h, _, _, c = make_pair("tiny", max_K=6)
     with pytest.raises(sps.SpsError):
