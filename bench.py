@@ -300,7 +300,13 @@ def run_ours(args):
                      "ms_verify_per_loop": ms_verify / loops if loops else None,
                      "ms_draft_per_step": ms_draft / loops / K if loops and K else None,
                      "ms_accept_per_loop": ms_accept / loops if loops else None,
-                     "ms_prefill": stats[-1]["ms_prefill"]}}
+                     "ms_prefill": stats[-1]["ms_prefill"]},
+            # the prompt pass: P - 1 rows through both models; bf16 models take it as tcgen05 GEMMs over 128-row chunks
+            # (two bf16 halves per activation: 4 flops per weight and row), so the weights are read once per chunk
+            "prefill": {"ms": stats[-1]["ms_prefill"], "rows": P - 1,
+                        "tflops": (4.0 * (P - 1) * (sps_synth.weight_bytes(c["target"]) - c["target"]["vocab"] * c["target"]["d_model"] * 2
+                                                   + sps_synth.weight_bytes(c["draft"]) - c["draft"]["vocab"] * c["draft"]["d_model"] * 2) / 2
+                                   / (stats[-1]["ms_prefill"] / 1e3) / 1e12) if c["target"]["dtype"] == 1 and stats[-1]["ms_prefill"] > 0 else None}}
     # latency distribution over the timed loops: a loop delivers its tokens together, so a token's latency is its
     # loop's device time divided by the tokens that loop emitted (each token weighted once)
     lm, lt = np.concatenate(loop_ms), np.concatenate(loop_tok)

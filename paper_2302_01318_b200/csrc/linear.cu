@@ -669,7 +669,15 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
     }
     pdl_wait();
-    {
+    // k-ranges beyond 2048 (int8 weights with one or two rows) take further rounds of the same two places
+    for (int cb = 0; cb < nchunk; cb += 2 * NCW * 32) {
+      if (cb > 0 && a.pro == PRO_RMSNORM) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int c = cb + tid + i * (NCW * 32);
+          if (c < nchunk) gg[i] = __ldg(reinterpret_cast<const float4*>(a.gain + k_base + 4 * c));
+        }
+      }
       // Eight rows at a time; all of a thread's loads are in flight before the partial sums of squares of
       // the norm are fetched, so the slab costs one trip to L2, not two.
 #pragma unroll
@@ -677,7 +685,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         float4 v[2][8];
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          const int c = tid + i * (NCW * 32);
+          const int c = cb + tid + i * (NCW * 32);
           if (c < nchunk) {
 #pragma unroll
             for (int mm = 0; mm < 8; ++mm) {
@@ -687,7 +695,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
             }
           }
         }
-        if (h == 0 && a.pro == PRO_RMSNORM) {
+        if (h == 0 && cb == 0 && a.pro == PRO_RMSNORM) {
           // 1/rms of each row: warp m adds that row's partial sums of squares (lanes stride, then a shuffle tree)
           for (int m = warp; m < a.M; m += NCW) {
             const int srow = a.x_row0 + m * a.x_rowstep;
@@ -708,7 +716,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          const int c = tid + i * (NCW * 32);
+          const int c = cb + tid + i * (NCW * 32);
           if (c < nchunk) {
 #pragma unroll
             for (int mm = 0; mm < 8; ++mm) {
@@ -1109,13 +1117,19 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     // bulk-copy variant: KS = largest multiple of 128 dividing D up to the slab budget
     static const int ks_env = [] { const char* e = getenv("SPS_LIN_KSMAX"); return e ? atoi(e) : 0; }();
     int ks_max = (p.NT == 1) ? 2048 : 1024;
+    // int8 rows are half as long in bytes: with one or two activation rows the slab leaves room for k-ranges of 4096,
+    // which restores 4 KB of contiguous bytes per weight row and tile (2 KB runs stream about 10 % slower)
+    const bool q8_long = dtype == 2 && M <= 2 && D % 4096 == 0 && !(ks_env > 0 && ks_env < 4096);
     if (ks_env > 0 && ks_env < ks_max) ks_max = ks_env;
     int KS = 128;
     for (int k = 128; k <= ks_max && k <= D; k += 128) if (D % k == 0) KS = k;
     static const int kst_env = [] { const char* e = getenv("SPS_LIN_KST"); return e ? atoi(e) : 1024; }();
     int KST = 128;
     for (int k : {256, 512, 1024}) if (KS % k == 0 && k <= kst_env) KST = k;
-    if (dtype == 2) KST = KS;   // int8: a tile is one stage (16 rows x KS bytes <= 32 KB; 16 KB stages stream 20 % slower)
+    // int8: a tile of up to 2048 k is one stage (16 rows x KS bytes <= 32 KB; 16 KB stages stream 20 % slower), a
+    // longer one two stages
+    if (q8_long) KS = 4096;
+    if (dtype == 2) KST = KS <= 2048 ? KS : KS / 2;
     p.KS = KS; p.KST = KST; p.S = D / KS; p.WC = LIN_CONSUMER_WARPS + 1; p.PR = 0;
     int R = num_sm / p.S;
     if (R < 1) R = 1;
@@ -1132,7 +1146,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     if (NS < 2) NS = 2;
     const int ksub = KS / KST;
     p.G = (ksub % 4 == 0) ? 4 : ((ksub % 2 == 0) ? 2 : 1);
-    if (dtype == 2) p.G = 2;   // int8: the two warps of a group share the tile's single stage
+    if (dtype == 2 && ksub == 1) p.G = 2;   // int8, one-stage tiles: the two warps of a group share the stage
     const size_t gscr = (size_t)2 * LIN_CONSUMER_WARPS * p.NT * 128 * sizeof(float);
     NS = (int)((kSmemTma - 1024 - xbytes - gscr) / stage);
     if (NS > 24) NS = 24;

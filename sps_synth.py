@@ -33,6 +33,9 @@ CONFIGS = {
     # the same shapes with int8 linear weights (dtype 2): bf16 matrices quantised per output row
     "tiny_q8": dict(target=_cfg(2, 256, 2, 128, 1024, 1024, 2), draft=_cfg(1, 128, 1, 128, 512, 1024, 2),
                     prompt_len=16, n_new=64, K=4, T=1.0),
+    # one int8 layer wide enough (d_model = d_ff = 4096) for the 4096-long k-ranges the int8 kernel uses at one or two rows
+    "q8_d4096": dict(target=_cfg(1, 4096, 32, 128, 4096, 512, 2), draft=_cfg(1, 4096, 32, 128, 4096, 512, 2),
+                     prompt_len=4, n_new=8, K=1, T=1.0),
     "70b_q8": dict(target=_cfg(80, 8192, 64, 128, 32768, 32000, 2), draft=_cfg(8, 6144, 48, 128, 24576, 32000, 2),
                    prompt_len=128, n_new=128, K=4, T=1.0),
     # fewer key / value heads than query heads: grouped (4 -> 2) target, multi-query (2 -> 1) draft, fp32

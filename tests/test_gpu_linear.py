@@ -60,7 +60,7 @@ def test_linear_bf16_width_with_a_large_prime_factor(M):
 
 
 @pytest.mark.parametrize("M", [1, 2, 4, 5, 8, 9, 16])
-@pytest.mark.parametrize("N,D", [(1000, 256), (77, 128), (4096, 2048), (1536, 6144), (300, 8192)])
+@pytest.mark.parametrize("N,D", [(1000, 256), (77, 128), (4096, 2048), (1536, 6144), (300, 8192), (520, 1536), (200, 640), (90, 12288)])
 def test_linear_int8_weights(M, N, D):
     """Weight-only int8: Y = scale[n] * X W^T against the oracle on the dequantised matrix (scale * q is exact in
     double; the kernel multiplies exact fp16 copies of the bytes and applies the scale to the sum)."""

@@ -206,6 +206,25 @@ def test_int8_weight_pair_logits_under_teacher_forcing():
     h.close()
 
 
+def test_int8_long_k_ranges_inside_a_model():
+    """d_model = d_ff = 4096: with one or two rows the int8 layers split k into ranges of 4096 (two stages per tile,
+    packed activations copied 8 KB per row); one and two rows against the oracle, then five rows (ranges of 2048)."""
+    h, ot, _, c = make_pair("q8_d4096", max_seq=32, draft_equals_target=True)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(2, 4, V)
+    h.sps_prefill(prompt)
+    ot.forward(prompt[:-1], np.arange(3), want_logits=False)
+    for n_rows in (1, 2, 5):
+        rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(3, 4, V)])[:n_rows]
+        out = torch.zeros((n_rows, V), device=DEV)
+        h.sps_score(0, rows, out)
+        want = ot.forward64(rows, np.arange(3, 3 + n_rows))
+        err = np.abs(out.cpu().numpy() - want).max()
+        print(f"int8 d=4096, {n_rows} rows: logit error {err:.2e}")
+        assert err < 5e-2, err
+    h.close()
+
+
 def test_int8_weights_need_their_scales():
     c = sps_synth.CONFIGS["tiny_q8"]
     w = sps_synth.weights_to(sps_synth.make_weights(c["target"]), DEV)
