@@ -84,7 +84,9 @@ typedef struct {
 typedef struct {
   sps_model_cfg target, draft;
   int32_t max_seq;   /* longest sequence (prompt + generated + K) a cache row exists for */
-  int32_t max_batch; /* sequences decoded together; max_batch * (max_K + 1) <= 16        */
+  int32_t max_batch; /* sequences decoded together, <= 8; max_batch * (max_K + 1) <= 16,
+                        or <= 128 when the target is bf16 (passes above 16 rows run
+                        their linear layers as tensor-core GEMMs)                        */
   int32_t max_K;     /* largest lookahead that will be asked for, <= SPS_MAX_K           */
   int32_t device;    /* CUDA device ordinal                                              */
   void* stream;      /* cudaStream_t to run on; NULL = the library creates its own       */

@@ -48,6 +48,7 @@ struct sps_handle {
   // the prompt pass over up to 128 rows at once (bf16 models, one sequence): residual stream, q|k|v, attention output,
   // the GEMM operands' bf16 halves (normalised rows / GeLU outputs) and the k-splits' partial products
   bool wide = false;
+  int max_rows = SPS_MAX_ROWS;   // rows one pass may carry: 16, or up to 128 when the target is bf16 (wide passes)
   float *wx = nullptr, *wqkv = nullptr, *watt = nullptr, *wpart = nullptr;
   void *wa_hi = nullptr, *wa_lo = nullptr, *wu_hi = nullptr, *wu_lo = nullptr;
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
@@ -200,9 +201,12 @@ struct PassSpec {
 };
 
 // one forward pass of a model over the rows `ps` describes, for the handle's B live sequences
+int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps);
+
 int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   const sps_model_cfg& c = m.cfg;
   const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff;
+  if (rows > SPS_MAX_ROWS) return run_pass_wide(h, m, ps);
   cudaStream_t st = h->stream;
   EmbedArgs ea{};
   ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
@@ -286,6 +290,48 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
     const LinPlan pl = lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm);
     CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+  }
+  return SPS_OK;
+}
+
+// A pass over 17..128 rows (several sequences' K + 1 rows): the same layers, every linear layer as one GEMM on the
+// tcgen05 tensor cores (wide.cu) instead of the 16-row weight-streaming kernel; attention as in run_pass, one CTA per
+// (head, sequence) over that sequence's rows.  bf16 models only.
+int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps) {
+  const sps_model_cfg& c = m.cfg;
+  const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff, dkv = kv_width(c), ldq = d + 2 * dkv;
+  if (!h->wide || c.dtype != 1 || rows > WIDE_ROWS) return fail(h, SPS_EINVAL, "more than 16 rows per pass need a bf16 model and at most 128 rows");
+  if (ps.logits && (ps.lrow0 != 0 || ps.lrowstep != 1 || ps.lrows != rows)) return fail(h, SPS_EINVAL, "a wide pass computes logits for all of its rows");
+  cudaStream_t st = h->stream;
+  int* err = h->hst.err;
+  EmbedArgs ea{};
+  ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
+  ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
+  ea.x = h->wx; ea.ssq = h->ssqA;
+  CU(h, embed_launch(ea, st)); h->launches++;
+  for (int l = 0; l < c.n_layers; ++l) {
+    CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
+    CU(h, wide_gemm_launch(m.wq[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+    CU(h, wide_gemm_launch(m.wk[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+    CU(h, wide_gemm_launch(m.wv[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d + dkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+    AttnArgs aa{};
+    aa.st = h->dst; aa.qkv = h->wqkv; aa.out = h->watt;
+    aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
+    aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
+    aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
+    aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
+    CU(h, attn_launch(aa, st));
+    CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
+    CU(h, wide_gemm_launch(m.wo[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+    CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
+    CU(h, wide_gemm_launch(m.w_up[l], h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st));
+    CU(h, wide_gemm_launch(m.w_down[l], h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+    h->launches += 16;
+  }
+  if (ps.logits) {
+    CU(h, wide_pack_launch(h->wx, d, (const float*)m.final_norm, c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
+    CU(h, wide_gemm_launch(m.unembed, h->wa_hi, h->wa_lo, rows, c.vocab, d, h->wpart, WIDE_STORE, ps.logits, ps.logits_ld, nullptr, nullptr, 0, err, h->num_sm, st));
+    h->launches += 3;
   }
   return SPS_OK;
 }
@@ -480,7 +526,8 @@ void add_loop_stats(sps_stats* s, int K, int a, uint32_t fl) {
 int check_K(sps_handle* h, int K) {
   if (K < 0 || K > h->cfg.max_K) return fail(h, SPS_EINVAL, "K outside 0..max_K");
   if (K > 0 && !h->drf.present) return fail(h, SPS_EINVAL, "K > 0 needs a draft model");
-  if (h->B * (K + 1) > SPS_MAX_ROWS) return fail(h, SPS_EINVAL, "batch * (K + 1) exceeds 16 rows");
+  if (h->B * (K + 1) > h->max_rows) return fail(h, SPS_EINVAL, "batch * (K + 1) exceeds the rows one pass may carry (16; 128 with a bf16 target)");
+  if (h->B * (K + 1) > SPS_MAX_ROWS && !(h->wide && h->tgt.cfg.dtype == 1)) return fail(h, SPS_EINVAL, "more than 16 rows per pass need a bf16 target");
   return SPS_OK;
 }
 
@@ -501,8 +548,9 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
     if (cfg->draft.vocab != cfg->target.vocab) return fail(nullptr, SPS_EINVAL, "draft and target vocabularies differ");
   }
   if (cfg->max_K < 0 || cfg->max_K > SPS_MAX_K) return fail(nullptr, SPS_EINVAL, "max_K outside 0..15");
-  if (cfg->max_batch < 1 || cfg->max_batch * (cfg->max_K + 1) > SPS_MAX_ROWS || cfg->max_batch * 2 > SPS_MAX_ROWS)
-    return fail(nullptr, SPS_EINVAL, "max_batch * (max_K + 1) must be <= 16");
+  const int want_rows = cfg->max_batch * (cfg->max_K + 1);
+  if (cfg->max_batch < 1 || cfg->max_batch * 2 > SPS_MAX_ROWS || want_rows > WIDE_ROWS || (want_rows > SPS_MAX_ROWS && cfg->target.dtype != 1))
+    return fail(nullptr, SPS_EINVAL, "max_batch * (max_K + 1) must be <= 16 (<= 128 with a bf16 target), max_batch <= 8");
   if (cfg->max_seq < 2) return fail(nullptr, SPS_EINVAL, "max_seq too small");
   {
     const int dh_max = (draft_w && cfg->draft.d_head > cfg->target.d_head) ? cfg->draft.d_head : cfg->target.d_head;
@@ -543,7 +591,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       if (!m->present || m->cfg.dtype != 1) continue;
       const sps_model_cfg& c = m->cfg;
       wd = std::max(wd, (size_t)c.d_model); wf = std::max(wf, (size_t)c.d_ff);
-      const int shapes[4][2] = {{c.d_model, c.d_model}, {kv_width(c), c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}};
+      const int shapes[5][2] = {{c.d_model, c.d_model}, {kv_width(c), c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
       for (auto& sh : shapes) wpart = std::max(wpart, wide_part_floats(sh[0], sh[1], h->num_sm));
     }
     if (wd > 0 && !off) {
@@ -558,7 +606,12 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       }
       h->wide = true;
     }
+    if (want_rows > SPS_MAX_ROWS) {
+      if (!h->wide) return bail(fail(h, SPS_EINVAL, "more than 16 rows per pass need the wide passes (SPS_WIDE_PREFILL=0 turns them off)"));
+      h->max_rows = want_rows;
+    }
   }
+  const size_t MR = (size_t)h->max_rows, PR = std::max((size_t)SPS_MAX_ROWS, (size_t)cfg->max_batch * (size_t)(cfg->max_K > 0 ? cfg->max_K : 1));
   struct Want { void** p; size_t bytes; };
   DevState& s = h->hst;
   const Want wants[] = {
@@ -570,10 +623,10 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->xp_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
       {(void**)&h->up_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
       {(void**)&h->up_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
-      {(void**)&h->ssqA, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
+      {(void**)&h->ssqA, sizeof(float) * LIN_MAX_R * MR},
       {(void**)&h->ssqB, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
-      {(void**)&h->q_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
-      {(void**)&h->p_logits, sizeof(float) * SPS_MAX_ROWS * (size_t)V},
+      {(void**)&h->q_logits, sizeof(float) * MR * (size_t)V},
+      {(void**)&h->p_logits, sizeof(float) * PR * (size_t)V},
       {(void**)&h->part, sizeof(float) * part_floats},
       {(void**)&h->counters, sizeof(int) * (2 * LIN_MAX_R + 2)},
       {(void**)&h->res, 4 * h->res_words},
@@ -582,8 +635,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&s.limit, 4 * (size_t)MB},
       {(void**)&s.tokens, 4 * (size_t)MB * cfg->max_seq},
       {(void**)&s.drafts, 4 * (size_t)MB * maxK},
-      {(void**)&s.row_tok, 4 * SPS_MAX_ROWS},
-      {(void**)&s.row_pos, 4 * SPS_MAX_ROWS},
+      {(void**)&s.row_tok, 4 * MR},
+      {(void**)&s.row_pos, 4 * MR},
       {(void**)&s.done_counter, 4},
   };
   for (const Want& w : wants) {

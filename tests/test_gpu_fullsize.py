@@ -16,20 +16,34 @@ DEV = "cuda"
 
 
 def oracle_logits(cfg, w_dev, tokens, positions_ctx, rows):
-    """prefix tokens at positions 0..len-1 go through the oracle layer by layer together with `rows`"""
+    """prefix tokens at positions 0..len-1 go through the oracle layer by layer together with `rows`; an int8 model is
+    the fp32 model of its dequantised matrices with a bf16 cache"""
     seq = np.concatenate([tokens, rows]).astype(np.int32)
     pos = np.arange(len(seq), dtype=np.int32)
-    m = oracle.Transformer(cfg, None, len(seq) + 1)
-    emb = sps_synth.to_numpy(w_dev["tok_embed"][torch.from_numpy(seq.astype(np.int64)).to(DEV)])
-    m.begin_rows(emb, pos)
-    for l, lw in enumerate(w_dev["layers"]):
-        m.layer(l, {k: sps_synth.to_numpy(v) for k, v in lw.items()})
-    out = m.end(sps_synth.to_numpy(w_dev["final_norm"]), sps_synth.to_numpy(w_dev["unembed"]))
+    q8 = cfg["dtype"] == 2
+    emb_t = w_dev["tok_embed"][torch.from_numpy(seq.astype(np.int64)).to(DEV)]
+    if q8:
+        m = oracle.Transformer(dict(cfg, dtype=0), None, len(seq) + 1, cache_dtype=1)
+        m.begin_rows(emb_t.float().cpu().numpy(), pos)
+        for l, lw in enumerate(w_dev["layers"]):
+            one = {k: lw[k].cpu().numpy() for k in ("attn_norm", "ffn_norm")}
+            for k in sps_synth.LAYER_MATS:
+                one[k] = (lw[k].float() * lw[k + "_scale"][:, None]).cpu().numpy()
+            m.layer(l, one)
+        un = (w_dev["unembed"].float() * w_dev["unembed_scale"][:, None]).cpu().numpy()
+        out = m.end(sps_synth.to_numpy(w_dev["final_norm"]), un)
+    else:
+        m = oracle.Transformer(cfg, None, len(seq) + 1)
+        m.begin_rows(sps_synth.to_numpy(emb_t), pos)
+        for l, lw in enumerate(w_dev["layers"]):
+            m.layer(l, {k: sps_synth.to_numpy(v) for k, v in lw.items()})
+        out = m.end(sps_synth.to_numpy(w_dev["final_norm"]), sps_synth.to_numpy(w_dev["unembed"]))
     return out[len(tokens):]
 
 
-def test_scoring_pass_at_70b_layer_shapes():
-    c = sps_synth.CONFIGS["70b"]
+@pytest.mark.parametrize("name", ["70b", "70b_q8", "70b_gqa8"])
+def test_scoring_pass_at_70b_layer_shapes(name):
+    c = sps_synth.CONFIGS[name]
     tc, dc = dict(c["target"], n_layers=2), dict(c["draft"], n_layers=1)
     wt = sps_synth.make_weights(tc, tag="target", device=DEV)
     wd = sps_synth.make_weights(dc, tag="draft", device=DEV, share_embed_from=wt)

@@ -258,6 +258,37 @@ def test_long_prompt_through_the_wide_prompt_pass(name):
     h.close()
 
 
+@pytest.mark.parametrize("B,K", [(4, 4), (8, 6), (8, 1)])
+def test_batches_above_16_rows_per_pass(B, K):
+    """Batch x (K + 1) above 16 rows (the K / batch sweep's corners): the scoring pass runs its linear layers as
+    tensor-core GEMMs over all the sequences' rows.  Every sequence must reproduce what the oracle generates for it
+    alone (Philox word c2 = its index), outside flagged near ties; (8, 1) is the 16-row case next to them."""
+    h, ot, od, c = make_pair("tiny_bf16", max_seq=96, max_batch=B, max_K=K)
+    V = c["target"]["vocab"]
+    prompts = np.stack([sps_synth.make_prompt(20 + b, 16, V) for b in range(B)])
+    got, st = h.sps_generate_batch(prompts, 24, K, 1.0, 5)
+    again, _ = h.sps_generate_batch(prompts, 24, K, 1.0, 5)
+    assert (got == again).all()
+    osps, ok = oracle.Sps(ot, od), 0
+    for b in range(B):
+        want = osps.generate(prompts[b], 24, K, 1.0, 5, b=b)
+        if (got[b] == want["tokens"]).all():
+            ok += 1
+            assert st[b]["loops"] == want["loops"]
+        else:
+            assert want["flags"] & NEAR, (b, got[b], want["tokens"])
+    print(f"batch {B} x K {K}: {ok} of {B} sequences token-identical to the oracle")
+    assert ok >= B - 2
+    h.close()
+
+
+def test_more_than_16_rows_need_a_bf16_target():
+    c = sps_synth.CONFIGS["tiny"]
+    w = sps_synth.weights_to(sps_synth.make_weights(c["target"]), DEV)
+    with pytest.raises(sps.SpsError):
+        sps.Handle(c["target"], w, None, None, max_seq=64, max_batch=4, max_K=4)
+
+
 def test_loop_trace_matches_the_statistics():
     h, _, _, c = make_pair("tiny", max_K=6)
     with pytest.raises(sps.SpsError):
