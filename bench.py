@@ -341,6 +341,21 @@ def run_ours(args):
                                                f"target unembedding + 1 of {c['draft']['n_layers']} draft layers + draft "
                                                f"unembedding over 1 row (context {P}), scaled to one loop and divided into the "
                                                f"measured {tpl:.3f} tokens per loop"), "seconds": s}
+    if rank == 0 and world == 1 and args.batch > 1 and c["target"]["dtype"] == 1:
+        # the K / batch sweep's corner: `batch` sequences decoded together, batch x (K + 1) rows per scoring pass
+        # (above 16 rows the linear layers run as tcgen05 GEMMs); aggregate tokens/s over the batch
+        Bn = args.batch
+        hb = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=max_seq, max_batch=Bn, max_K=K, device=local)
+        prompts = np.stack([sps_synth.make_prompt(1000 + b, P, V) for b in range(Bn)])
+        hb.sps_generate_batch(prompts, n_new, K, T, 1)
+        _, sb = hb.sps_generate_batch(prompts, n_new, K, T, 2)
+        b_ms, b_loops = sb[0]["ms_decode"], max(s["loops"] for s in sb)
+        line.setdefault("variants", {})[f"batch{Bn}_K{K}"] = {
+            "value": Bn * n_new / (b_ms / 1e3), "unit": UNIT, "rows_per_pass": Bn * (K + 1), "loops": b_loops,
+            "tokens_per_loop_per_sequence": sum(s["emitted"] for s in sb) / sum(s["loops"] for s in sb),
+            "ms_verify_per_loop": sb[0]["ms_verify"] / b_loops, "ms_draft_per_step": sb[0]["ms_draft"] / (b_loops * max(K, 1)),
+            "ms_prefill": sb[0]["ms_prefill"], "speedup_vs_batch1": Bn * n_new / (b_ms / 1e3) / value}
+        hb.close()
     if rank == 0 and world == 1 and args.aligned_steps > 0 and c["target"]["dtype"] >= 1:
         # Same kernels, same shapes, but a pair whose draft agrees with its target about as often as the paper's
         # trained pair did: both bodies' output projections are damped in place (x gamma), so that the shared
@@ -357,10 +372,11 @@ def run_ours(args):
         al_ms = sum(s["ms_decode"] for s in al)
         al_loops = sum(s["loops"] for s in al)
         al_tps = args.aligned_steps * n_new / (al_ms / 1e3)
-        line["variants"] = {"aligned": {"gamma": args.aligned_gamma, "value": al_tps, "unit": UNIT,
+        line.setdefault("variants", {})
+        line["variants"].update({"aligned": {"gamma": args.aligned_gamma, "value": al_tps, "unit": UNIT,
                                         "tokens_per_loop": sum(s["emitted"] for s in al) / al_loops,
                                         "accept_rate": sum(s["accepted"] for s in al) / (al_loops * K) if K else None,
-                                        "speedup_vs_ar": al_tps / ar_tps if ar_tps else None}}
+                                        "speedup_vs_ar": al_tps / ar_tps if ar_tps else None}})
         # the decoding settings the paper's speed table uses, on the same pair: nucleus 0.8 and greedy
         # (top-k / nucleus / greedy filtering of both models ahead of the rejection scheme)
         for name, top_k, top_p, temp in (("aligned_nucleus_0.8", 0, 0.8, T), ("aligned_greedy", 0, 1.0, 0.0)):
@@ -456,6 +472,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--aligned-steps", type=int, default=2)
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
+    ap.add_argument("--batch", type=int, default=8, help="also decode this many sequences together (0 / 1 = skip)")
     ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
     ap.add_argument("--traffic", type=float, default=None,

@@ -147,8 +147,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   int* pos_s = reinterpret_cast<int*>(row_a + MR);               // [MR]
   uint64_t* bar = reinterpret_cast<uint64_t*>(pos_s + MR);       // 8-byte aligned by construction
 
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int Mb = a.rows_per_seq, row0 = b * Mb, d = a.d, max_seq = a.max_seq;
+  const int h = blockIdx.x, b = a.seq0 + blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Mb = a.rows_per_seq, row0 = blockIdx.y * Mb, d = a.d, max_seq = a.max_seq;
   const int group = a.H / a.Hkv, hk = h / group;   // the key / value head this query head reads
   const bool appends = (h - hk * group) == 0;       // one head of a group writes the cache
   const int ldq = d + 2 * a.Hkv * DH;                // row stride of the q | k | v buffer

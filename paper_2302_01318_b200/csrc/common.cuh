@@ -213,6 +213,7 @@ struct AttnArgs {
   const float2* rope;     // [max_seq][dh/2] (cos, sin)
   int dtype, H, dh, d, max_seq, rows_per_seq, B;
   int Hkv;                // key / value heads: query head h uses head h / (H / Hkv)
+  int seq0;               // grid row y works on sequence seq0 + y (its cache and state) and on rows y * rows_per_seq .. of qkv / out
   int mode, t, c0;        // which rows the pass feeds (PassMode), as in EmbedArgs
 };
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
@@ -224,7 +225,7 @@ cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
 enum { WIDE_STORE = 0, WIDE_RESIDUAL = 1, WIDE_GELU_PACK = 2 };
 int wide_splits(int N, int D, int num_sm);
 size_t wide_part_floats(int N, int D, int num_sm);
-cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int c0, cudaStream_t s);
+cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int seq, int c0, cudaStream_t s);
 cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s);
 cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,
                              long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st);

@@ -453,18 +453,18 @@ int set_sequences(sps_handle* h, const int32_t* toks, int B, int n) {
 }
 
 // both caches ingest positions 0..n-2 of every live sequence
-// The prompt pass of a bf16 model, one sequence, in chunks of up to 128 rows: every linear layer is one GEMM on the
+// The prompt pass of a bf16 model for one sequence of the batch, in chunks of up to 128 rows: every linear layer is one GEMM on the
 // tcgen05 tensor cores (wide.cu), so a chunk reads the weights once; attention runs the decode kernel over 16 of the
 // chunk's rows at a time (earlier rows' keys come from the cache, which the chunk's earlier launches have filled).
 // No logits: the prompt's last token is fed by the first loop.
-int prefill_wide(sps_handle* h, ModelDev& m, int n) {
+int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
   const sps_model_cfg& c = m.cfg;
   const int d = c.d_model, dff = c.d_ff, dkv = kv_width(c), ldq = d + 2 * dkv;
   cudaStream_t st = h->stream;
   int* err = h->hst.err;
   for (int c0 = 0; c0 < n - 1; c0 += WIDE_ROWS) {
     const int rows = (n - 1 - c0) < WIDE_ROWS ? (n - 1 - c0) : WIDE_ROWS;
-    CU(h, wide_embed_launch(h->dst, m.tok_embed, h->wx, rows, d, c.vocab, c0, st)); h->launches++;
+    CU(h, wide_embed_launch(h->dst, m.tok_embed, h->wx, rows, d, c.vocab, seq, c0, st)); h->launches++;
     for (int l = 0; l < c.n_layers; ++l) {
       CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
       CU(h, wide_gemm_launch(m.wq[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
@@ -477,7 +477,7 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n) {
         aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
         aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
         aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = (rows - r0) < SPS_MAX_ROWS ? (rows - r0) : SPS_MAX_ROWS; aa.B = 1;
-        aa.mode = PASS_PREFILL; aa.t = 0; aa.c0 = c0 + r0;
+        aa.mode = PASS_PREFILL; aa.t = 0; aa.c0 = c0 + r0; aa.seq0 = seq;
         CU(h, attn_launch(aa, st)); h->launches++;
       }
       CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
@@ -496,9 +496,12 @@ int prefill_all(sps_handle* h, int n) {
   for (int which = 0; which < 2; ++which) {
     ModelDev& m = which == 0 ? h->tgt : h->drf;
     if (!m.present) continue;
-    if (h->wide && h->B == 1 && m.cfg.dtype == 1 && n - 1 > SPS_MAX_ROWS) {
-      int rc = prefill_wide(h, m, n);
-      if (rc) return rc;
+    if (h->wide && m.cfg.dtype == 1 && n - 1 > SPS_MAX_ROWS / h->B) {
+      // one sequence after the other, each in chunks of 128 rows
+      for (int b = 0; b < h->B; ++b) {
+        int rc = prefill_wide(h, m, n, b);
+        if (rc) return rc;
+      }
       continue;
     }
     for (int c0 = 0; c0 < n - 1; c0 += per) {

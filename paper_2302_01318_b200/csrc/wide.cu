@@ -34,11 +34,16 @@ namespace {
 constexpr int WIDE_M = 128;        // activation rows of one pass (tensor-memory lanes)
 constexpr int WIDE_BN = 256;       // weight rows per CTA (tensor-memory columns)
 constexpr int WIDE_BK = 64;        // k per stage: 128 bytes of bf16 = one swizzle row
-constexpr int WIDE_STAGES = 3;
-constexpr uint32_t WIDE_A_BYTES = WIDE_M * WIDE_BK * 2;     // 16 KB per half
 constexpr uint32_t WIDE_B_BYTES = WIDE_BN * WIDE_BK * 2;    // 32 KB
-constexpr uint32_t WIDE_STAGE_BYTES = 2 * WIDE_A_BYTES + WIDE_B_BYTES;
-constexpr size_t WIDE_SMEM = 1024 + (size_t)WIDE_STAGES * WIDE_STAGE_BYTES + 1024;   // header + ring + alignment slack
+// MR = rows the MMA carries: 128, or 64 for passes of up to 64 rows (half the tensor work, a fourth stage in the ring)
+template <int MR> struct WideCfg {
+  static constexpr int STAGES = MR == 64 ? 4 : 3;
+  static constexpr uint32_t A_BYTES = MR * WIDE_BK * 2;     // 16 KB (8 KB) per half
+  static constexpr uint32_t STAGE_BYTES = 2 * A_BYTES + WIDE_B_BYTES;
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 1024;   // header + ring + alignment slack
+  // kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N = 256, M = MR
+  static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(WIDE_BN >> 3) << 17) | ((uint32_t)(MR >> 4) << 24);
+};
 
 __device__ __forceinline__ uint32_t w_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ unsigned long long w_timer() {
@@ -95,14 +100,11 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                       // 128-byte swizzle
   return d;
 }
-// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N = 256, M = 128
-constexpr uint32_t UMMA_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(WIDE_BN >> 3) << 17) | ((uint32_t)(WIDE_M >> 4) << 24);
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
       " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(UMMA_IDESC), "r"(accumulate)
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // arrives on the barrier once every MMA issued so far by this thread has finished reading its operands
@@ -133,7 +135,10 @@ struct WideGemmArgs {
   int* err;
 };
 
+template <int MR>
 __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant__ WideGemmArgs a) {
+  constexpr int WIDE_STAGES = WideCfg<MR>::STAGES;
+  constexpr uint32_t WIDE_A_BYTES = WideCfg<MR>::A_BYTES, WIDE_STAGE_BYTES = WideCfg<MR>::STAGE_BYTES;
   extern __shared__ unsigned char wsm_raw[];
   // header: full[3], empty[3], accumulator-ready barrier, tensor-memory base, abort flag; ring 1024-aligned
   const uint32_t raw = w_smem_u32(wsm_raw);
@@ -162,9 +167,17 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *s_tmem;
-  // the activations are the predecessor's output; nothing is fetched before it has finished
-  pdl_wait();
+  // Weights do not depend on the predecessor kernel: the first ring-full of W boxes is on its way before the wait;
+  // the activations are the predecessor's output and follow after it.
+  const int pre = kb_n < WIDE_STAGES ? kb_n : WIDE_STAGES;
+  if (warp == 0 && lane == 0) {
+    for (int kb = 0; kb < pre; ++kb) {
+      w_mbar_expect_tx(bar_full + 8 * kb, WIDE_STAGE_BYTES);
+      w_tma_2d(ring + kb * WIDE_STAGE_BYTES + 2 * WIDE_A_BYTES, &a.tm_w, (kb0 + kb) * WIDE_BK, tile * WIDE_BN, bar_full + 8 * kb);
+    }
+  }
   pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -176,10 +189,10 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
         if (*s_abort) { ok = false; break; }
         const uint32_t dst = ring + st * WIDE_STAGE_BYTES;
         const int k = (kb0 + kb) * WIDE_BK;
-        w_mbar_expect_tx(bar_full + 8 * st, WIDE_STAGE_BYTES);
+        if (kb >= pre) w_mbar_expect_tx(bar_full + 8 * st, WIDE_STAGE_BYTES);
         w_tma_2d(dst, &a.tm_hi, k, 0, bar_full + 8 * st);
         w_tma_2d(dst + WIDE_A_BYTES, &a.tm_lo, k, 0, bar_full + 8 * st);
-        w_tma_2d(dst + 2 * WIDE_A_BYTES, &a.tm_w, k, tile * WIDE_BN, bar_full + 8 * st);
+        if (kb >= pre) w_tma_2d(dst + 2 * WIDE_A_BYTES, &a.tm_w, k, tile * WIDE_BN, bar_full + 8 * st);
       }
       if (!ok) {
         *s_abort = 1;
@@ -200,8 +213,8 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
 #pragma unroll
         for (int k = 0; k < WIDE_BK / 16; ++k) {
           // 16 elements along k = 32 bytes = 2 units of the descriptor's address field
-          umma_bf16(tmem, d_hi + 2 * k, d_w + 2 * k, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_bf16(tmem, d_lo + 2 * k, d_w + 2 * k, 1u);
+          umma_bf16(tmem, d_hi + 2 * k, d_w + 2 * k, WideCfg<MR>::IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_bf16(tmem, d_lo + 2 * k, d_w + 2 * k, WideCfg<MR>::IDESC, 1u);
         }
         umma_commit(bar_empty + 8 * st);   // the stage is free once these MMAs have read it
       }
@@ -209,8 +222,9 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
       else *s_abort = 1;
     }
   } else {
-    // epilogue warps 2..5: tensor-memory lanes 32 q .. 32 q + 31 with q = warp % 4
-    const int q = warp & 3, row = q * 32 + lane;
+    // epilogue warps 2..5: tensor-memory lanes 32 q .. 32 q + 31 with q = warp % 4.  A 128-row accumulator keeps row i
+    // in lane i; a 64-row one keeps 16 rows in the first 16 lanes of each of the four lane quarters.
+    const int q = warp & 3, row = MR == 128 ? q * 32 + lane : (lane < 16 ? q * 16 + lane : WIDE_M);
     bool ok = w_mbar_wait(bar_acc, 0u, a.err) && !*s_abort;
     ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -255,12 +269,13 @@ __device__ __forceinline__ float wide_gelu(float v) {
   return 0.5f * v * (1.0f + tanhf(0.7978845608028654f * (v + 0.044715f * v * v * v)));
 }
 
-// x[row] = E[token at position c0 + row] for the rows of one prompt chunk
-__global__ void __launch_bounds__(256) wide_embed_kernel(const DevState* st, const __nv_bfloat16* tok_embed, float* x, int d, int V, int c0) {
+// x[row] = E[token at position c0 + row of sequence seq] for the rows of one prompt chunk
+__global__ void __launch_bounds__(256) wide_embed_kernel(const DevState* st, const __nv_bfloat16* tok_embed, float* x, int d, int V, int seq,
+                                                         int c0) {
   pdl_wait();
   pdl_launch_dependents();
   const int row = blockIdx.x;
-  int tok = st->tokens[c0 + row];   // sequence 0
+  int tok = st->tokens[(long long)seq * st->max_seq + c0 + row];
   if (tok < 0 || tok >= V) { tok = 0; if (threadIdx.x == 0) atomicExch(st->err, 1); }
   const __nv_bfloat16* e = tok_embed + (size_t)tok * d;
   for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)row * d + k] = __bfloat162float(e[k]);
@@ -373,8 +388,8 @@ int wide_splits(int N, int D, int num_sm) {
 }
 size_t wide_part_floats(int N, int D, int num_sm) { return (size_t)wide_splits(N, D, num_sm) * WIDE_M * (size_t)N; }
 
-cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int c0, cudaStream_t s) {
-  return launch_k(wide_embed_kernel, dim3(rows), dim3(256), 0, s, st, reinterpret_cast<const __nv_bfloat16*>(tok_embed), x, d, V, c0);
+cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int seq, int c0, cudaStream_t s) {
+  return launch_k(wide_embed_kernel, dim3(rows), dim3(256), 0, s, st, reinterpret_cast<const __nv_bfloat16*>(tok_embed), x, d, V, seq, c0);
 }
 cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s) {
   return launch_k(wide_pack_kernel, dim3(rows), dim3(256), 0, s, x, ldx, gain, eps, d, reinterpret_cast<__nv_bfloat16*>(hi),
@@ -388,17 +403,21 @@ cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int 
   if (M < 1 || M > WIDE_M || N < 1 || D < WIDE_BK || (D % WIDE_BK)) return cudaErrorInvalidValue;
   WideGemmArgs a;
   cudaError_t e;
-  if ((e = wide_map(hi, WIDE_M, D, WIDE_M, &a.tm_hi)) != cudaSuccess) return e;
-  if ((e = wide_map(lo, WIDE_M, D, WIDE_M, &a.tm_lo)) != cudaSuccess) return e;
+  const int mr = M <= 64 ? 64 : WIDE_M;   // rows the MMA carries
+  if ((e = wide_map(hi, WIDE_M, D, mr, &a.tm_hi)) != cudaSuccess) return e;
+  if ((e = wide_map(lo, WIDE_M, D, mr, &a.tm_lo)) != cudaSuccess) return e;
   if ((e = wide_map(W, N, D, WIDE_BN, &a.tm_w)) != cudaSuccess) return e;
   a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits(N, D, num_sm); a.err = err;
   static bool attr = false;
   if (!attr) {
-    if ((e = cudaFuncSetAttribute(wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WIDE_SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(wide_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<64>::SMEM)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(wide_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<128>::SMEM)) != cudaSuccess) return e;
     attr = true;
   }
   const int tiles = (N + WIDE_BN - 1) / WIDE_BN;
-  if ((e = launch_k(wide_gemm_kernel, dim3(tiles, a.S), dim3(192), WIDE_SMEM, st, a)) != cudaSuccess) return e;
+  if (mr == 64) e = launch_k(wide_gemm_kernel<64>, dim3(tiles, a.S), dim3(192), WideCfg<64>::SMEM, st, a);
+  else e = launch_k(wide_gemm_kernel<128>, dim3(tiles, a.S), dim3(192), WideCfg<128>::SMEM, st, a);
+  if (e != cudaSuccess) return e;
   const long long total = (long long)M * N;
   int blocks = (int)((total + 255) / 256);
   if (blocks > 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK)) blocks = 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);

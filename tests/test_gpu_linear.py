@@ -138,7 +138,7 @@ def run_linear_wide(W, X):
     return Y.cpu().numpy()
 
 
-@pytest.mark.parametrize("M", [1, 5, 33, 127, 128])
+@pytest.mark.parametrize("M", [1, 5, 16, 17, 33, 48, 64, 65, 127, 128])
 @pytest.mark.parametrize("N,D", [(256, 64), (300, 128), (1000, 256), (77, 1024), (4099, 2048)])
 def test_linear_wide_small(M, N, D):
     """The prompt-pass GEMM (up to 128 rows on the tcgen05 tensor cores) against the oracle: ragged N (tiles of

@@ -265,7 +265,8 @@ def test_batches_above_16_rows_per_pass(B, K):
     alone (Philox word c2 = its index), outside flagged near ties; (8, 1) is the 16-row case next to them."""
     h, ot, od, c = make_pair("tiny_bf16", max_seq=96, max_batch=B, max_K=K)
     V = c["target"]["vocab"]
-    prompts = np.stack([sps_synth.make_prompt(20 + b, 16, V) for b in range(B)])
+    # 40-token prompts: each sequence's prompt goes through the 128-row prompt pass with its own cache rows
+    prompts = np.stack([sps_synth.make_prompt(20 + b, 40, V) for b in range(B)])
     got, st = h.sps_generate_batch(prompts, 24, K, 1.0, 5)
     again, _ = h.sps_generate_batch(prompts, 24, K, 1.0, 5)
     assert (got == again).all()
