@@ -225,6 +225,10 @@ cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
 enum { WIDE_STORE = 0, WIDE_RESIDUAL = 1, WIDE_GELU_PACK = 2 };
 int wide_splits(int N, int D, int num_sm);
 size_t wide_part_floats(int N, int D, int num_sm);
+size_t wide_part_bound(int N, int num_sm);
+cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int nmat, const void* hi, const void* lo, int M, int D,
+                                     float* part, int mode, float* y, long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm,
+                                     cudaStream_t st);
 cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int seq, int c0, cudaStream_t s);
 cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s);
 cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,

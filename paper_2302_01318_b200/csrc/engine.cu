@@ -311,9 +311,11 @@ int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   CU(h, embed_launch(ea, st)); h->launches++;
   for (int l = 0; l < c.n_layers; ++l) {
     CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
-    CU(h, wide_gemm_launch(m.wq[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
-    CU(h, wide_gemm_launch(m.wk[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
-    CU(h, wide_gemm_launch(m.wv[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d + dkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+    {
+      const void* qkv_w[3] = {m.wq[l], m.wk[l], m.wv[l]};
+      const int qkv_rows[3] = {d, dkv, dkv};
+      CU(h, wide_gemm_launch_stacked(qkv_w, qkv_rows, 3, h->wa_hi, h->wa_lo, rows, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+    }
     AttnArgs aa{};
     aa.st = h->dst; aa.qkv = h->wqkv; aa.out = h->watt;
     aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
@@ -326,7 +328,7 @@ int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
     CU(h, wide_gemm_launch(m.w_up[l], h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st));
     CU(h, wide_gemm_launch(m.w_down[l], h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
-    h->launches += 16;
+    h->launches += 12;
   }
   if (ps.logits) {
     CU(h, wide_pack_launch(h->wx, d, (const float*)m.final_norm, c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
@@ -467,10 +469,12 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
     CU(h, wide_embed_launch(h->dst, m.tok_embed, h->wx, rows, d, c.vocab, seq, c0, st)); h->launches++;
     for (int l = 0; l < c.n_layers; ++l) {
       CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
-      CU(h, wide_gemm_launch(m.wq[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
-      CU(h, wide_gemm_launch(m.wk[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
-      CU(h, wide_gemm_launch(m.wv[l], h->wa_hi, h->wa_lo, rows, dkv, d, h->wpart, WIDE_STORE, h->wqkv + d + dkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
-      h->launches += 7;
+      {
+        const void* qkv_w[3] = {m.wq[l], m.wk[l], m.wv[l]};
+        const int qkv_rows[3] = {d, dkv, dkv};
+        CU(h, wide_gemm_launch_stacked(qkv_w, qkv_rows, 3, h->wa_hi, h->wa_lo, rows, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+      }
+      h->launches += 3;
       for (int r0 = 0; r0 < rows; r0 += SPS_MAX_ROWS) {
         AttnArgs aa{};
         aa.st = h->dst; aa.qkv = h->wqkv + (size_t)r0 * ldq; aa.out = h->watt + (size_t)r0 * d;
@@ -594,8 +598,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       if (!m->present || m->cfg.dtype != 1) continue;
       const sps_model_cfg& c = m->cfg;
       wd = std::max(wd, (size_t)c.d_model); wf = std::max(wf, (size_t)c.d_ff);
-      const int shapes[5][2] = {{c.d_model, c.d_model}, {kv_width(c), c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
-      for (auto& sh : shapes) wpart = std::max(wpart, wide_part_floats(sh[0], sh[1], h->num_sm));
+      for (int n_out : {c.d_model + 2 * kv_width(c), c.d_ff, c.vocab}) wpart = std::max(wpart, wide_part_bound(n_out, h->num_sm));
     }
     if (wd > 0 && !off) {
       struct WW { void** p; size_t bytes; };

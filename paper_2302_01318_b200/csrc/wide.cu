@@ -129,9 +129,10 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 struct WideGemmArgs {
-  CUtensorMap tm_hi, tm_lo, tm_w;
+  CUtensorMap tm_hi, tm_lo, tm_w[3];   // up to three stacked weight matrices (q | k | v): output columns side by side
+  int rows_mat[3], tiles_mat[3];       // rows of each matrix and its tiles of 256 rows (0 for unused slots)
   float* part;        // [S][128][N] partial products of the k-splits
-  int M, N, D, S;     // live rows, weight rows, width, k-splits (D / 64 is a multiple of S)
+  int M, N, D, S;     // live rows, weight rows of all matrices together, width, k-splits (D / 64 is a multiple of S)
   int* err;
 };
 
@@ -151,6 +152,11 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, s = blockIdx.y;
   const int kb_all = a.D / WIDE_BK, kb_n = kb_all / a.S, kb0 = s * kb_n;
+  // which matrix this tile belongs to, its first row there, and its first column of the stacked output
+  int mat = 0, ltile = tile, col0 = 0;
+  while (mat < 2 && ltile >= a.tiles_mat[mat]) { ltile -= a.tiles_mat[mat]; col0 += a.rows_mat[mat]; ++mat; }
+  const int wrow0 = ltile * WIDE_BN;
+  const CUtensorMap* tm_w = &a.tm_w[mat];
 
   if (tid == 0) {
     for (int i = 0; i < WIDE_STAGES; ++i) { w_mbar_init(bar_full + 8 * i, 1); w_mbar_init(bar_empty + 8 * i, 1); }
@@ -173,7 +179,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
   if (warp == 0 && lane == 0) {
     for (int kb = 0; kb < pre; ++kb) {
       w_mbar_expect_tx(bar_full + 8 * kb, WIDE_STAGE_BYTES);
-      w_tma_2d(ring + kb * WIDE_STAGE_BYTES + 2 * WIDE_A_BYTES, &a.tm_w, (kb0 + kb) * WIDE_BK, tile * WIDE_BN, bar_full + 8 * kb);
+      w_tma_2d(ring + kb * WIDE_STAGE_BYTES + 2 * WIDE_A_BYTES, tm_w, (kb0 + kb) * WIDE_BK, wrow0, bar_full + 8 * kb);
     }
   }
   pdl_launch_dependents();
@@ -192,7 +198,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
         if (kb >= pre) w_mbar_expect_tx(bar_full + 8 * st, WIDE_STAGE_BYTES);
         w_tma_2d(dst, &a.tm_hi, k, 0, bar_full + 8 * st);
         w_tma_2d(dst + WIDE_A_BYTES, &a.tm_lo, k, 0, bar_full + 8 * st);
-        if (kb >= pre) w_tma_2d(dst + 2 * WIDE_A_BYTES, &a.tm_w, k, tile * WIDE_BN, bar_full + 8 * st);
+        if (kb >= pre) w_tma_2d(dst + 2 * WIDE_A_BYTES, tm_w, k, wrow0, bar_full + 8 * st);
       }
       if (!ok) {
         *s_abort = 1;
@@ -229,14 +235,14 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
     ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
-      float* dst = a.part + ((size_t)s * WIDE_M + row) * a.N + (size_t)tile * WIDE_BN;
-      const int ncols = min(WIDE_BN, a.N - tile * WIDE_BN);
+      float* dst = a.part + ((size_t)s * WIDE_M + row) * a.N + (size_t)(col0 + wrow0);
+      const int ncols = min(WIDE_BN, a.rows_mat[mat] - wrow0);
 #pragma unroll 1
       for (int c = 0; c < WIDE_BN; c += 32) {
         float v[32];
         tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);   // the whole warp takes part in the load
         if (row < a.M && c < ncols) {
-          if (c + 32 <= ncols && (a.N & 3) == 0) {
+          if (c + 32 <= ncols && ((a.N | col0) & 3) == 0) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
           } else {
@@ -379,6 +385,13 @@ cudaError_t wide_map(const void* p, int rows, int D, int box_rows, CUtensorMap* 
 
 }  // namespace
 
+static int wide_splits_tiles(int tiles, int D, int num_sm) {
+  const int kb = D / WIDE_BK;
+  int S = 1;
+  for (int s = 1; s <= kb && s * tiles <= (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK); ++s)
+    if (kb % s == 0) S = s;
+  return S;
+}
 int wide_splits(int N, int D, int num_sm) {
   const int tiles = (N + WIDE_BN - 1) / WIDE_BN, kb = D / WIDE_BK;
   int S = 1;
@@ -387,6 +400,11 @@ int wide_splits(int N, int D, int num_sm) {
   return S;
 }
 size_t wide_part_floats(int N, int D, int num_sm) { return (size_t)wide_splits(N, D, num_sm) * WIDE_M * (size_t)N; }
+// enough for any (stacked) shape of N output columns: S * tiles <= SMs bounds S * N by 256 * SMs when S > 1
+size_t wide_part_bound(int N, int num_sm) {
+  const size_t cap = (size_t)WIDE_BN * (size_t)(num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
+  return (size_t)WIDE_M * ((size_t)N + WIDE_BN > cap ? (size_t)N + WIDE_BN : cap);
+}
 
 cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int seq, int c0, cudaStream_t s) {
   return launch_k(wide_embed_kernel, dim3(rows), dim3(256), 0, s, st, reinterpret_cast<const __nv_bfloat16*>(tok_embed), x, d, V, seq, c0);
@@ -400,21 +418,38 @@ cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float e
 // part: wide_part_floats(N, D) floats.  mode WIDE_EPI_*: y / ldy for store and residual, yhi / ylo / ldp for GeLU + split.
 cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,
                              long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st) {
-  if (M < 1 || M > WIDE_M || N < 1 || D < WIDE_BK || (D % WIDE_BK)) return cudaErrorInvalidValue;
+  const void* Ws[3] = {W, nullptr, nullptr};
+  const int rows[3] = {N, 0, 0};
+  return wide_gemm_launch_stacked(Ws, rows, 1, hi, lo, M, D, part, mode, y, ldy, yhi, ylo, ldp, err, num_sm, st);
+}
+
+// the same over up to three matrices that share the activations (q | k | v): output columns are the matrices' rows side
+// by side; part must hold 128 * max(N, 256 * SMs) floats
+cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int nmat, const void* hi, const void* lo, int M, int D,
+                                     float* part, int mode, float* y, long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm,
+                                     cudaStream_t st) {
+  if (M < 1 || M > WIDE_M || nmat < 1 || nmat > 3 || D < WIDE_BK || (D % WIDE_BK)) return cudaErrorInvalidValue;
   WideGemmArgs a;
   cudaError_t e;
   const int mr = M <= 64 ? 64 : WIDE_M;   // rows the MMA carries
   if ((e = wide_map(hi, WIDE_M, D, mr, &a.tm_hi)) != cudaSuccess) return e;
   if ((e = wide_map(lo, WIDE_M, D, mr, &a.tm_lo)) != cudaSuccess) return e;
-  if ((e = wide_map(W, N, D, WIDE_BN, &a.tm_w)) != cudaSuccess) return e;
-  a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits(N, D, num_sm); a.err = err;
+  int N = 0, tiles = 0;
+  for (int i = 0; i < 3; ++i) {
+    const bool has = i < nmat;
+    if (has && (rows[i] < 1 || !Ws[i])) return cudaErrorInvalidValue;
+    a.rows_mat[i] = has ? rows[i] : 0;
+    a.tiles_mat[i] = has ? (rows[i] + WIDE_BN - 1) / WIDE_BN : 0;
+    if ((e = wide_map(Ws[has ? i : 0], rows[has ? i : 0], D, WIDE_BN, &a.tm_w[i])) != cudaSuccess) return e;
+    N += a.rows_mat[i]; tiles += a.tiles_mat[i];
+  }
+  a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits_tiles(tiles, D, num_sm); a.err = err;
   static bool attr = false;
   if (!attr) {
     if ((e = cudaFuncSetAttribute(wide_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<64>::SMEM)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(wide_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<128>::SMEM)) != cudaSuccess) return e;
     attr = true;
   }
-  const int tiles = (N + WIDE_BN - 1) / WIDE_BN;
   if (mr == 64) e = launch_k(wide_gemm_kernel<64>, dim3(tiles, a.S), dim3(192), WideCfg<64>::SMEM, st, a);
   else e = launch_k(wide_gemm_kernel<128>, dim3(tiles, a.S), dim3(192), WideCfg<128>::SMEM, st, a);
   if (e != cudaSuccess) return e;
