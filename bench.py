@@ -412,6 +412,8 @@ def run_ours(args):
                               "ms_draft_per_step": st["ms_draft"] / (st["loops"] * k)})
             line["variants"]["k_sweep"] = sweep
     h.close()
+    if rank == 0 and world == 1 and args.sweep and c["target"]["dtype"] == 1:
+        line["sweep"] = sweep_bench(sps, c, wt, wd, local, peak)
     if rank == 0 and world == 1 and not args.no_sampler:
         line["sampler"] = sampler_bench(dev, peak)
     if rank == 0:
@@ -419,6 +421,35 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def sweep_bench(sps, c, wt, wd, local, peak):
+    """The K / batch sweep on the pair at its natural acceptance: K in {1, 2, 3, 4, 6, 8} x temperature {0.5, 1} x batch
+    {1, 4, 8}, prompt 512, 256 new tokens; tokens/s over the batch, accepted drafts per target call, scoring-pass
+    latency and its weight bytes over time, against the same library's autoregressive decode at that batch."""
+    P, n_new, V = 512, 256, c["target"]["vocab"]
+    out = []
+    for Bn in (1, 4, 8):
+        hs = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=((P + n_new + 8 + 63) // 64) * 64, max_batch=Bn, max_K=8, device=local)
+        prompts = np.stack([sps_synth.make_prompt(2000 + b, P, V) for b in range(Bn)])
+        ar = {}
+        for T in (0.5, 1.0):
+            for K in (0, 1, 2, 3, 4, 6, 8):
+                hs.sps_generate_batch(prompts[:, :32], 8, K, T, 1)      # first use of (K, batch): eager run, then graph capture
+                _, st = hs.sps_generate_batch(prompts, n_new, K, T, 7)
+                ms, loops = st[0]["ms_decode"], max(s["loops"] for s in st)
+                tps = Bn * n_new / (ms / 1e3)
+                if K == 0:
+                    ar[T] = tps
+                    continue
+                ms_v = st[0]["ms_verify"] / loops
+                out.append({"batch": Bn, "T": T, "K": K, "value": tps, "vs_ar": tps / ar[T],
+                            "accepted_per_call": sum(s["accepted"] for s in st) / sum(s["loops"] for s in st),
+                            "ms_verify": ms_v, "verify_gbs": sps_synth.weight_bytes(c["target"]) / (ms_v / 1e3) / 1e9,
+                            "verify_frac": sps_synth.weight_bytes(c["target"]) / (ms_v / 1e3) / 1e9 / peak,
+                            "ms_draft_per_step": st[0]["ms_draft"] / (loops * K), "ar": ar[T]})
+        hs.close()
+    return out
 
 
 def sampler_bench(dev, peak_gbs):
@@ -473,6 +504,7 @@ def main():
     ap.add_argument("--aligned-steps", type=int, default=2)
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
     ap.add_argument("--batch", type=int, default=8, help="also decode this many sequences together (0 / 1 = skip)")
+    ap.add_argument("--sweep", action="store_true", help="also run the K x temperature x batch sweep (prompt 512, 256 tokens; minutes)")
     ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
     ap.add_argument("--traffic", type=float, default=None,
