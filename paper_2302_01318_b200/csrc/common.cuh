@@ -228,11 +228,13 @@ size_t wide_part_floats(int N, int D, int num_sm);
 size_t wide_part_bound(int N, int num_sm);
 cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int nmat, const void* hi, const void* lo, int M, int D,
                                      float* part, int mode, float* y, long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm,
-                                     cudaStream_t st);
+                                     cudaStream_t st, const float* const* scales = nullptr);
 cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* x, int rows, int d, int V, int seq, int c0, cudaStream_t s);
 cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s);
 cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,
-                             long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st);
+                             long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st,
+                             const float* scale = nullptr);
+cudaError_t wide_dequant_launch(const void* q, void* out, long long n, int num_sm, cudaStream_t st);
 size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh);
 
 struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(logits/T)

@@ -51,6 +51,7 @@ struct sps_handle {
   int max_rows = SPS_MAX_ROWS;   // rows one pass may carry: 16, or up to 128 when the target is bf16 (wide passes)
   float *wx = nullptr, *wqkv = nullptr, *watt = nullptr, *wpart = nullptr;
   void *wa_hi = nullptr, *wa_lo = nullptr, *wu_hi = nullptr, *wu_lo = nullptr;
+  void* wdq = nullptr;   // bf16 copy of the int8 matrix (or q | k | v) the prompt-pass GEMM is reading
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
@@ -464,15 +465,29 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
   const int d = c.d_model, dff = c.d_ff, dkv = kv_width(c), ldq = d + 2 * dkv;
   cudaStream_t st = h->stream;
   int* err = h->hst.err;
+  const bool q8 = c.dtype == 2;
+  // int8 weights: the GEMM reads a bf16 copy made just before it (bytes are exact in bf16); the row scales multiply the sums
+  cudaError_t dq_err = cudaSuccess;
+  auto Wb = [&](const void* w, size_t elems, size_t at) -> const void* {
+    if (!q8) return w;
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(h->wdq) + at;
+    const cudaError_t e = wide_dequant_launch(w, dst, (long long)elems, h->num_sm, st);
+    if (e != cudaSuccess) dq_err = e;
+    h->launches++;
+    return dst;
+  };
   for (int c0 = 0; c0 < n - 1; c0 += WIDE_ROWS) {
     const int rows = (n - 1 - c0) < WIDE_ROWS ? (n - 1 - c0) : WIDE_ROWS;
     CU(h, wide_embed_launch(h->dst, m.tok_embed, h->wx, rows, d, c.vocab, seq, c0, st)); h->launches++;
     for (int l = 0; l < c.n_layers; ++l) {
       CU(h, wide_pack_launch(h->wx, d, (const float*)m.attn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
       {
-        const void* qkv_w[3] = {m.wq[l], m.wk[l], m.wv[l]};
+        const void* qkv_w[3] = {Wb(m.wq[l], (size_t)d * d, 0), Wb(m.wk[l], (size_t)dkv * d, (size_t)d * d),
+                                Wb(m.wv[l], (size_t)dkv * d, (size_t)d * d + (size_t)dkv * d)};
         const int qkv_rows[3] = {d, dkv, dkv};
-        CU(h, wide_gemm_launch_stacked(qkv_w, qkv_rows, 3, h->wa_hi, h->wa_lo, rows, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st));
+        const float* qkv_s[3] = {q8 ? m.wq_s[l] : nullptr, q8 ? m.wk_s[l] : nullptr, q8 ? m.wv_s[l] : nullptr};
+        CU(h, wide_gemm_launch_stacked(qkv_w, qkv_rows, 3, h->wa_hi, h->wa_lo, rows, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st,
+                                       q8 ? qkv_s : nullptr));
       }
       h->launches += 3;
       for (int r0 = 0; r0 < rows; r0 += SPS_MAX_ROWS) {
@@ -485,11 +500,15 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
         CU(h, attn_launch(aa, st)); h->launches++;
       }
       CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
-      CU(h, wide_gemm_launch(m.wo[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+      CU(h, wide_gemm_launch(Wb(m.wo[l], (size_t)d * d, 0), h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st,
+                             q8 ? m.wo_s[l] : nullptr));
       CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
-      CU(h, wide_gemm_launch(m.w_up[l], h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st));
-      CU(h, wide_gemm_launch(m.w_down[l], h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
+      CU(h, wide_gemm_launch(Wb(m.w_up[l], (size_t)dff * d, 0), h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st,
+                             q8 ? m.w_up_s[l] : nullptr));
+      CU(h, wide_gemm_launch(Wb(m.w_down[l], (size_t)dff * d, 0), h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st,
+                             q8 ? m.w_down_s[l] : nullptr));
       h->launches += 8;
+      CU(h, dq_err);
     }
   }
   return SPS_OK;
@@ -500,7 +519,7 @@ int prefill_all(sps_handle* h, int n) {
   for (int which = 0; which < 2; ++which) {
     ModelDev& m = which == 0 ? h->tgt : h->drf;
     if (!m.present) continue;
-    if (h->wide && m.cfg.dtype == 1 && n - 1 > SPS_MAX_ROWS / h->B) {
+    if (h->wide && m.cfg.dtype >= 1 && n - 1 > SPS_MAX_ROWS / h->B) {
       // one sequence after the other, each in chunks of 128 rows
       for (int b = 0; b < h->B; ++b) {
         int rc = prefill_wide(h, m, n, b);
@@ -593,10 +612,11 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   {
     // buffers of the 128-row prompt pass, when a bf16 model is there to use it (SPS_WIDE_PREFILL=0 keeps the 16-row pass)
     static const bool off = [] { const char* e = getenv("SPS_WIDE_PREFILL"); return e && atoi(e) == 0; }();
-    size_t wd = 0, wf = 0, wpart = 0;
+    size_t wd = 0, wf = 0, wpart = 0, wdq = 0;
     for (const ModelDev* m : {&h->tgt, &h->drf}) {
-      if (!m->present || m->cfg.dtype != 1) continue;
+      if (!m->present || m->cfg.dtype < 1) continue;
       const sps_model_cfg& c = m->cfg;
+      if (c.dtype == 2) wdq = std::max(wdq, std::max((size_t)c.d_ff * c.d_model, (size_t)(c.d_model + 2 * kv_width(c)) * c.d_model));
       wd = std::max(wd, (size_t)c.d_model); wf = std::max(wf, (size_t)c.d_ff);
       for (int n_out : {c.d_model + 2 * kv_width(c), c.d_ff, c.vocab}) wpart = std::max(wpart, wide_part_bound(n_out, h->num_sm));
     }
@@ -605,7 +625,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       const WW ww[] = {{(void**)&h->wx, sizeof(float) * WIDE_ROWS * wd},       {(void**)&h->wqkv, sizeof(float) * WIDE_ROWS * 3 * wd},
                        {(void**)&h->watt, sizeof(float) * WIDE_ROWS * wd},     {(void**)&h->wpart, sizeof(float) * wpart},
                        {&h->wa_hi, 2 * (size_t)WIDE_ROWS * wd},                {&h->wa_lo, 2 * (size_t)WIDE_ROWS * wd},
-                       {&h->wu_hi, 2 * (size_t)WIDE_ROWS * wf},                {&h->wu_lo, 2 * (size_t)WIDE_ROWS * wf}};
+                       {&h->wu_hi, 2 * (size_t)WIDE_ROWS * wf},                {&h->wu_lo, 2 * (size_t)WIDE_ROWS * wf},
+                       {&h->wdq, 2 * (wdq > 0 ? wdq : 8)}};
       for (const WW& w : ww) {
         if (cudaMalloc(w.p, w.bytes) != cudaSuccess) return bail(fail(h, SPS_ENOMEM, "device allocation failed"));
         if (cudaMemsetAsync(*w.p, 0, w.bytes, h->stream) != cudaSuccess) return bail(fail(h, SPS_ECUDA, "memset failed"));
@@ -673,7 +694,7 @@ int sps_destroy(sps_handle* h) {
   for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
   free_model(h->tgt);
   free_model(h->drf);
-  void* bufs[] = {h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
+  void* bufs[] = {h->wdq, h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
                   h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);

@@ -133,6 +133,7 @@ struct WideGemmArgs {
   int rows_mat[3], tiles_mat[3];       // rows of each matrix and its tiles of 256 rows (0 for unused slots)
   float* part;        // [S][128][N] partial products of the k-splits
   int M, N, D, S;     // live rows, weight rows of all matrices together, width, k-splits (D / 64 is a multiple of S)
+  int w_is_output;    // the weights were written by the predecessor kernel (bf16 copy of int8 weights): no early fetch
   int* err;
 };
 
@@ -165,8 +166,10 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    // 256 columns of tensor memory for the 128 x 256 fp32 accumulator (one CTA per SM: always available)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 192), "r"(WIDE_BN) : "memory");
+    // all 512 columns of tensor memory: two 128 x 256 fp32 accumulators, one for the products of the activations'
+    // high halves and one for the low halves' (one CTA per SM: always available).  Kept apart, the small low-half
+    // products are not rounded against the large running sum at every step; the epilogue adds the two once.
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 192), "r"(2 * WIDE_BN) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -175,7 +178,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
   const uint32_t tmem = *s_tmem;
   // Weights do not depend on the predecessor kernel: the first ring-full of W boxes is on its way before the wait;
   // the activations are the predecessor's output and follow after it.
-  const int pre = kb_n < WIDE_STAGES ? kb_n : WIDE_STAGES;
+  const int pre = a.w_is_output ? 0 : (kb_n < WIDE_STAGES ? kb_n : WIDE_STAGES);
   if (warp == 0 && lane == 0) {
     for (int kb = 0; kb < pre; ++kb) {
       w_mbar_expect_tx(bar_full + 8 * kb, WIDE_STAGE_BYTES);
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
         for (int k = 0; k < WIDE_BK / 16; ++k) {
           // 16 elements along k = 32 bytes = 2 units of the descriptor's address field
           umma_bf16(tmem, d_hi + 2 * k, d_w + 2 * k, WideCfg<MR>::IDESC, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_bf16(tmem, d_lo + 2 * k, d_w + 2 * k, WideCfg<MR>::IDESC, 1u);
+          umma_bf16(tmem + WIDE_BN, d_lo + 2 * k, d_w + 2 * k, WideCfg<MR>::IDESC, (kb > 0 || k > 0) ? 1u : 0u);
         }
         umma_commit(bar_empty + 8 * st);   // the stage is free once these MMAs have read it
       }
@@ -239,8 +242,11 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
       const int ncols = min(WIDE_BN, a.rows_mat[mat] - wrow0);
 #pragma unroll 1
       for (int c = 0; c < WIDE_BN; c += 32) {
-        float v[32];
-        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);   // the whole warp takes part in the load
+        float v[32], vl[32];
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);   // the whole warp takes part in the loads
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(WIDE_BN + c), vl);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] += vl[i];
         if (row < a.M && c < ncols) {
           if (c + 32 <= ncols && ((a.N | col0) & 3) == 0) {
 #pragma unroll
@@ -256,7 +262,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(WIDE_BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * WIDE_BN) : "memory");
   }
 }
 
@@ -322,9 +328,31 @@ __global__ void __launch_bounds__(256) wide_pack_kernel(const float* x, int ldx,
 
 enum { WIDE_EPI_STORE = 0, WIDE_EPI_RESIDUAL = 1, WIDE_EPI_GELU_PACK = 2 };
 
+// int8 weights take this GEMM through a bf16 copy (signed bytes are exact in bf16); the rows' scales multiply the sums
+__global__ void __launch_bounds__(256) wide_dequant_kernel(const int8_t* q, __nv_bfloat16* out, long long n16) {
+  pdl_wait();
+  pdl_launch_dependents();
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n16; i += (long long)gridDim.x * 256) {
+    const int4 v = __ldg(reinterpret_cast<const int4*>(q) + i);
+    const int w[4] = {v.x, v.y, v.z, v.w};
+    __align__(16) __nv_bfloat16 o[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) o[4 * j + b] = __float2bfloat16_rn((float)(int8_t)((w[j] >> (8 * b)) & 0xff));
+    reinterpret_cast<uint4*>(out)[2 * i] = reinterpret_cast<const uint4*>(o)[0];
+    reinterpret_cast<uint4*>(out)[2 * i + 1] = reinterpret_cast<const uint4*>(o)[1];
+  }
+}
+
+struct WideScales {          // fp32 scale per output column, matrix by matrix (s[0] == nullptr: none)
+  const float* s[3];
+  int rows[3];
+};
+
 // y = sum over the k-splits in order, then: store / add to the residual stream / GeLU and split for the next GEMM
 __global__ void __launch_bounds__(256) wide_epilogue_kernel(const float* part, int S, int M, int N, int mode, float* y, long long ldy,
-                                                            __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp) {
+                                                            __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp, WideScales sc) {
   pdl_wait();
   pdl_launch_dependents();
   const long long total = (long long)M * N;
@@ -332,6 +360,11 @@ __global__ void __launch_bounds__(256) wide_epilogue_kernel(const float* part, i
     const int row = (int)(i / N), n = (int)(i - (long long)row * N);
     float t = 0.f;
     for (int s = 0; s < S; ++s) t += part[((size_t)s * WIDE_M + row) * N + n];
+    if (sc.s[0]) {
+      int m = 0, r = n;
+      while (m < 2 && r >= sc.rows[m]) { r -= sc.rows[m]; ++m; }
+      t *= __ldg(sc.s[m] + r);
+    }
     if (mode == WIDE_EPI_STORE) y[row * ldy + n] = t;
     else if (mode == WIDE_EPI_RESIDUAL) y[row * ldy + n] += t;
     else {
@@ -417,17 +450,28 @@ cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float e
 // Y = epilogue(sum_k-splits (hi + lo)[M, D] W[N, D]^T).  hi / lo: bf16 [128][D] (rows >= M are never read back);
 // part: wide_part_floats(N, D) floats.  mode WIDE_EPI_*: y / ldy for store and residual, yhi / ylo / ldp for GeLU + split.
 cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int M, int N, int D, float* part, int mode, float* y,
-                             long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st) {
+                             long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm, cudaStream_t st, const float* scale) {
   const void* Ws[3] = {W, nullptr, nullptr};
   const int rows[3] = {N, 0, 0};
-  return wide_gemm_launch_stacked(Ws, rows, 1, hi, lo, M, D, part, mode, y, ldy, yhi, ylo, ldp, err, num_sm, st);
+  const float* scs[3] = {scale, nullptr, nullptr};
+  return wide_gemm_launch_stacked(Ws, rows, 1, hi, lo, M, D, part, mode, y, ldy, yhi, ylo, ldp, err, num_sm, st, scale ? scs : nullptr);
+}
+
+// signed bytes -> bf16, n a multiple of 16, both pointers 16-byte aligned
+cudaError_t wide_dequant_launch(const void* q, void* out, long long n, int num_sm, cudaStream_t st) {
+  if (n % 16) return cudaErrorInvalidValue;
+  long long blocks = (n / 16 + 255) / 256;
+  const long long cap = 16LL * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
+  if (blocks > cap) blocks = cap;
+  return launch_k(wide_dequant_kernel, dim3((unsigned)blocks), dim3(256), 0, st, reinterpret_cast<const int8_t*>(q),
+                  reinterpret_cast<__nv_bfloat16*>(out), n / 16);
 }
 
 // the same over up to three matrices that share the activations (q | k | v): output columns are the matrices' rows side
 // by side; part must hold 128 * max(N, 256 * SMs) floats
 cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int nmat, const void* hi, const void* lo, int M, int D,
                                      float* part, int mode, float* y, long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, const float* const* scales) {
   if (M < 1 || M > WIDE_M || nmat < 1 || nmat > 3 || D < WIDE_BK || (D % WIDE_BK)) return cudaErrorInvalidValue;
   WideGemmArgs a;
   cudaError_t e;
@@ -444,6 +488,7 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
     N += a.rows_mat[i]; tiles += a.tiles_mat[i];
   }
   a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits_tiles(tiles, D, num_sm); a.err = err;
+  a.w_is_output = scales ? 1 : 0;
   static bool attr = false;
   if (!attr) {
     if ((e = cudaFuncSetAttribute(wide_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<64>::SMEM)) != cudaSuccess) return e;
@@ -456,6 +501,8 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   const long long total = (long long)M * N;
   int blocks = (int)((total + 255) / 256);
   if (blocks > 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK)) blocks = 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
+  WideScales sc{};
+  for (int i = 0; i < 3; ++i) { sc.s[i] = (scales && i < nmat) ? scales[i] : nullptr; sc.rows[i] = a.rows_mat[i]; }
   return launch_k(wide_epilogue_kernel, dim3(blocks), dim3(256), 0, st, (const float*)part, a.S, M, N, mode, y, ldy,
-                  reinterpret_cast<__nv_bfloat16*>(yhi), reinterpret_cast<__nv_bfloat16*>(ylo), ldp);
+                  reinterpret_cast<__nv_bfloat16*>(yhi), reinterpret_cast<__nv_bfloat16*>(ylo), ldp, sc);
 }

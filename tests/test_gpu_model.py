@@ -233,7 +233,7 @@ def test_int8_weights_need_their_scales():
         sps.Handle(c["target"], bad, None, None, max_seq=64)
 
 
-@pytest.mark.parametrize("name", ["tiny_bf16", "tiny_mqa_bf16"])
+@pytest.mark.parametrize("name", ["tiny_bf16", "tiny_mqa_bf16", "tiny_q8"])
 def test_long_prompt_through_the_wide_prompt_pass(name):
     """A 200-token prompt goes through the 128-row prompt pass in two chunks (128 + 71 rows; the tensor-core GEMM,
     attention 16 rows at a time over the cache the chunk is filling); the logits of the next five rows and a
