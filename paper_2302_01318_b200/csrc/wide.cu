@@ -293,36 +293,70 @@ __global__ void __launch_bounds__(256) wide_embed_kernel(const DevState* st, con
   for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)row * d + k] = __bfloat162float(e[k]);
 }
 
-// one CTA per row: (optionally) RMS-normalise with the gain, then split into bf16 high and low halves
-__global__ void __launch_bounds__(256) wide_pack_kernel(const float* x, int ldx, const float* gain, float eps, int d,
-                                                        __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp) {
-  __shared__ float s_part[8];
+__device__ __forceinline__ uint2 wide_split4(const float4& v, uint2& lo) {
+  __nv_bfloat16 h[4], l[4];
+  wide_split(v.x, h[0], l[0]); wide_split(v.y, h[1], l[1]); wide_split(v.z, h[2], l[2]); wide_split(v.w, h[3], l[3]);
+  uint2 hi;
+  hi.x = (uint32_t)__bfloat16_as_ushort(h[0]) | ((uint32_t)__bfloat16_as_ushort(h[1]) << 16);
+  hi.y = (uint32_t)__bfloat16_as_ushort(h[2]) | ((uint32_t)__bfloat16_as_ushort(h[3]) << 16);
+  lo.x = (uint32_t)__bfloat16_as_ushort(l[0]) | ((uint32_t)__bfloat16_as_ushort(l[1]) << 16);
+  lo.y = (uint32_t)__bfloat16_as_ushort(l[2]) | ((uint32_t)__bfloat16_as_ushort(l[3]) << 16);
+  return hi;
+}
+
+// one CTA of 1024 threads per row: (optionally) RMS-normalise with the gain, then split into bf16 high and low halves;
+// four features per thread and step when the widths allow (the second sweep over the row hits L1)
+__global__ void __launch_bounds__(1024) wide_pack_kernel(const float* x, int ldx, const float* gain, float eps, int d,
+                                                         __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp) {
+  __shared__ float s_part[32];
   __shared__ float s_inv;
   pdl_wait();
   pdl_launch_dependents();
-  const int row = blockIdx.x, tid = threadIdx.x;
+  const int row = blockIdx.x, tid = threadIdx.x, nth = blockDim.x;
   const float* xr = x + (size_t)row * ldx;
+  const bool vec = (((d | ldx | ldp) & 3) == 0) && ((((uintptr_t)x | (uintptr_t)hi | (uintptr_t)lo | (uintptr_t)gain) & 15) == 0);
   float inv = 1.f;
   if (gain) {
     float local = 0.f;
-    for (int k = tid; k < d; k += 256) { const float v = xr[k]; local += v * v; }
+    if (vec) {
+      for (int q = tid; q < (d >> 2); q += nth) {
+        const float4 v = reinterpret_cast<const float4*>(xr)[q];
+        local += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+      }
+    } else {
+      for (int k = tid; k < d; k += nth) { const float v = xr[k]; local += v * v; }
+    }
     local = warp_sum(local);
     if ((tid & 31) == 0) s_part[tid >> 5] = local;
     __syncthreads();
     if (tid == 0) {
       float t = 0.f;
-      for (int w = 0; w < 8; ++w) t += s_part[w];
+      for (int w = 0; w < (nth >> 5); ++w) t += s_part[w];
       s_inv = rsqrtf(t / (float)d + eps);
     }
     __syncthreads();
     inv = s_inv;
   }
-  for (int k = tid; k < d; k += 256) {
-    const float v = gain ? gain[k] * (xr[k] * inv) : xr[k];
-    __nv_bfloat16 h, l;
-    wide_split(v, h, l);
-    hi[(size_t)row * ldp + k] = h;
-    lo[(size_t)row * ldp + k] = l;
+  if (vec) {
+    for (int q = tid; q < (d >> 2); q += nth) {
+      float4 v = reinterpret_cast<const float4*>(xr)[q];
+      if (gain) {
+        const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + q);
+        v.x = g.x * (v.x * inv); v.y = g.y * (v.y * inv); v.z = g.z * (v.z * inv); v.w = g.w * (v.w * inv);
+      }
+      uint2 l;
+      const uint2 h = wide_split4(v, l);
+      reinterpret_cast<uint2*>(hi + (size_t)row * ldp)[q] = h;
+      reinterpret_cast<uint2*>(lo + (size_t)row * ldp)[q] = l;
+    }
+  } else {
+    for (int k = tid; k < d; k += nth) {
+      const float v = gain ? gain[k] * (xr[k] * inv) : xr[k];
+      __nv_bfloat16 h, l;
+      wide_split(v, h, l);
+      hi[(size_t)row * ldp + k] = h;
+      lo[(size_t)row * ldp + k] = l;
+    }
   }
 }
 
@@ -352,9 +386,42 @@ struct WideScales {          // fp32 scale per output column, matrix by matrix (
 
 // y = sum over the k-splits in order, then: store / add to the residual stream / GeLU and split for the next GEMM
 __global__ void __launch_bounds__(256) wide_epilogue_kernel(const float* part, int S, int M, int N, int mode, float* y, long long ldy,
-                                                            __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp, WideScales sc) {
+                                                            __nv_bfloat16* hi, __nv_bfloat16* lo, int ldp, WideScales sc, int vec) {
   pdl_wait();
   pdl_launch_dependents();
+  if (vec) {
+    // four columns per thread: they lie in one matrix (every matrix has a multiple of four rows)
+    const int N4 = N >> 2;
+    const long long total = (long long)M * N4;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+      const int row = (int)(i / N4), n = (int)(i - (long long)row * N4) << 2;
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < S; ++s) {
+        const float4 p = *reinterpret_cast<const float4*>(part + ((size_t)s * WIDE_M + row) * N + n);
+        t.x += p.x; t.y += p.y; t.z += p.z; t.w += p.w;
+      }
+      if (sc.s[0]) {
+        int m = 0, r = n;
+        while (m < 2 && r >= sc.rows[m]) { r -= sc.rows[m]; ++m; }
+        const float4 g = __ldg(reinterpret_cast<const float4*>(sc.s[m] + r));
+        t.x *= g.x; t.y *= g.y; t.z *= g.z; t.w *= g.w;
+      }
+      if (mode == WIDE_EPI_STORE) *reinterpret_cast<float4*>(y + row * ldy + n) = t;
+      else if (mode == WIDE_EPI_RESIDUAL) {
+        float4* yp = reinterpret_cast<float4*>(y + row * ldy + n);
+        float4 o = *yp;
+        o.x += t.x; o.y += t.y; o.z += t.z; o.w += t.w;
+        *yp = o;
+      } else {
+        t.x = wide_gelu(t.x); t.y = wide_gelu(t.y); t.z = wide_gelu(t.z); t.w = wide_gelu(t.w);
+        uint2 l;
+        const uint2 h = wide_split4(t, l);
+        *reinterpret_cast<uint2*>(hi + (size_t)row * ldp + n) = h;
+        *reinterpret_cast<uint2*>(lo + (size_t)row * ldp + n) = l;
+      }
+    }
+    return;
+  }
   const long long total = (long long)M * N;
   for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
     const int row = (int)(i / N), n = (int)(i - (long long)row * N);
@@ -443,7 +510,7 @@ cudaError_t wide_embed_launch(const DevState* st, const void* tok_embed, float* 
   return launch_k(wide_embed_kernel, dim3(rows), dim3(256), 0, s, st, reinterpret_cast<const __nv_bfloat16*>(tok_embed), x, d, V, seq, c0);
 }
 cudaError_t wide_pack_launch(const float* x, int ldx, const float* gain, float eps, int rows, int d, void* hi, void* lo, int ldp, cudaStream_t s) {
-  return launch_k(wide_pack_kernel, dim3(rows), dim3(256), 0, s, x, ldx, gain, eps, d, reinterpret_cast<__nv_bfloat16*>(hi),
+  return launch_k(wide_pack_kernel, dim3(rows), dim3(1024), 0, s, x, ldx, gain, eps, d, reinterpret_cast<__nv_bfloat16*>(hi),
                   reinterpret_cast<__nv_bfloat16*>(lo), ldp);
 }
 
@@ -498,11 +565,15 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   if (mr == 64) e = launch_k(wide_gemm_kernel<64>, dim3(tiles, a.S), dim3(192), WideCfg<64>::SMEM, st, a);
   else e = launch_k(wide_gemm_kernel<128>, dim3(tiles, a.S), dim3(192), WideCfg<128>::SMEM, st, a);
   if (e != cudaSuccess) return e;
-  const long long total = (long long)M * N;
+  // four columns per thread when every matrix, stride and pointer allows 16-byte accesses
+  int vec = ((N | a.rows_mat[0] | a.rows_mat[1] | a.rows_mat[2] | ldp) & 3) == 0 && (ldy & 3) == 0 &&
+            (((uintptr_t)part | (uintptr_t)y | (uintptr_t)yhi | (uintptr_t)ylo) & 15) == 0;
+  for (int i = 0; i < 3; ++i) if (scales && i < nmat && ((uintptr_t)scales[i] & 15)) vec = 0;
+  const long long total = (long long)M * (vec ? N / 4 : N);
   int blocks = (int)((total + 255) / 256);
   if (blocks > 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK)) blocks = 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
   WideScales sc{};
   for (int i = 0; i < 3; ++i) { sc.s[i] = (scales && i < nmat) ? scales[i] : nullptr; sc.rows[i] = a.rows_mat[i]; }
   return launch_k(wide_epilogue_kernel, dim3(blocks), dim3(256), 0, st, (const float*)part, a.S, M, N, mode, y, ldy,
-                  reinterpret_cast<__nv_bfloat16*>(yhi), reinterpret_cast<__nv_bfloat16*>(ylo), ldp, sc);
+                  reinterpret_cast<__nv_bfloat16*>(yhi), reinterpret_cast<__nv_bfloat16*>(ylo), ldp, sc, vec);
 }
