@@ -207,7 +207,11 @@ int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps);
 int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   const sps_model_cfg& c = m.cfg;
   const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff;
-  if (rows > SPS_MAX_ROWS) return run_pass_wide(h, m, ps);
+  // 9..16 rows: the tensor-core GEMM path also beats the 16-row weight-streaming variant (which is bound by shared-memory
+  // bandwidth) when the model can take it; SPS_WIDE_MIN_ROWS moves the switch (tuning only)
+  static const int wide_min = [] { const char* e = getenv("SPS_WIDE_MIN_ROWS"); return e ? atoi(e) : 9; }();
+  if (rows > SPS_MAX_ROWS || (rows >= wide_min && h->wide && c.dtype == 1 && (!ps.logits || (ps.lrow0 == 0 && ps.lrowstep == 1 && ps.lrows == rows))))
+    return run_pass_wide(h, m, ps);
   cudaStream_t st = h->stream;
   EmbedArgs ea{};
   ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
