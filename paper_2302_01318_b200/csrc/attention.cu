@@ -339,7 +339,14 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
     float t = 0.f;
 #pragma unroll
     for (int g = 0; g < PG; ++g) t += red[(g * MR + i) * DH + e];
-    a.out[(size_t)(row0 + i) * d + h * DH + e] = ok ? t / row_l[i] : 0.f;
+    const float val = ok ? t / row_l[i] : 0.f;
+    const size_t oi = (size_t)(row0 + i) * d + h * DH + e;
+    a.out[oi] = val;
+    if (a.out_hi) {
+      const __nv_bfloat16 vh = __float2bfloat16_rn(val);
+      reinterpret_cast<__nv_bfloat16*>(a.out_hi)[oi] = vh;
+      reinterpret_cast<__nv_bfloat16*>(a.out_lo)[oi] = __float2bfloat16_rn(val - __bfloat162float(vh));
+    }
   }
 }
 

@@ -208,6 +208,8 @@ struct AttnArgs {
   const DevState* st;
   const float* qkv;       // [rows][d + 2 * Hkv * dh]: queries, then keys, then values
   float* out;             // [rows][d]
+  void* out_hi;           // when non-null: the same values split into bf16 high and low halves, [rows][d] each
+  void* out_lo;           //   (the operand of a tensor-core GEMM that follows)
   void* kcache;           // this layer: [B][Hkv][max_seq][dh]
   void* vcache;
   const float2* rope;     // [max_seq][dh/2] (cos, sin)
@@ -226,6 +228,7 @@ enum { WIDE_STORE = 0, WIDE_RESIDUAL = 1, WIDE_GELU_PACK = 2 };
 int wide_splits(int N, int D, int num_sm);
 size_t wide_part_floats(int N, int D, int num_sm);
 size_t wide_part_bound(int N, int num_sm);
+int wide_gemm_launch_count(const int* rows, int nmat, int D, int num_sm);
 cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int nmat, const void* hi, const void* lo, int M, int D,
                                      float* part, int mode, float* y, long long ldy, void* yhi, void* ylo, int ldp, int* err, int num_sm,
                                      cudaStream_t st, const float* const* scales = nullptr);

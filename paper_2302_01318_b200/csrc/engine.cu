@@ -327,18 +327,23 @@ int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps) {
     aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
     aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
     aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
+    aa.out_hi = h->wa_hi; aa.out_lo = h->wa_lo;   // the next GEMM's operand, split into bf16 halves by the attention kernel
     CU(h, attn_launch(aa, st));
-    CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
     CU(h, wide_gemm_launch(m.wo[l], h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
     CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
     CU(h, wide_gemm_launch(m.w_up[l], h->wa_hi, h->wa_lo, rows, dff, d, h->wpart, WIDE_GELU_PACK, nullptr, 0, h->wu_hi, h->wu_lo, dff, err, h->num_sm, st));
     CU(h, wide_gemm_launch(m.w_down[l], h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st));
-    h->launches += 12;
+    {
+      const int qr[3] = {d, dkv, dkv}, r1[1] = {d}, r2[1] = {dff};
+      h->launches += 3 + wide_gemm_launch_count(qr, 3, d, h->num_sm) + wide_gemm_launch_count(r2, 1, d, h->num_sm) + wide_gemm_launch_count(r1, 1, d, h->num_sm) +
+                     wide_gemm_launch_count(r1, 1, dff, h->num_sm);
+    }
   }
   if (ps.logits) {
     CU(h, wide_pack_launch(h->wx, d, (const float*)m.final_norm, c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
     CU(h, wide_gemm_launch(m.unembed, h->wa_hi, h->wa_lo, rows, c.vocab, d, h->wpart, WIDE_STORE, ps.logits, ps.logits_ld, nullptr, nullptr, 0, err, h->num_sm, st));
-    h->launches += 3;
+    const int rv[1] = {c.vocab};
+    h->launches += 1 + wide_gemm_launch_count(rv, 1, d, h->num_sm);
   }
   return SPS_OK;
 }
@@ -493,7 +498,12 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
         CU(h, wide_gemm_launch_stacked(qkv_w, qkv_rows, 3, h->wa_hi, h->wa_lo, rows, d, h->wpart, WIDE_STORE, h->wqkv, ldq, nullptr, nullptr, 0, err, h->num_sm, st,
                                        q8 ? qkv_s : nullptr));
       }
-      h->launches += 3;
+      {
+        const int qr[3] = {d, dkv, dkv}, r1[1] = {d}, r2[1] = {dff};
+        // pack, q|k|v GEMM; pack, up GEMM; wo and down GEMMs (attention launches are counted where they are made)
+        h->launches += 2 + wide_gemm_launch_count(qr, 3, d, h->num_sm) + wide_gemm_launch_count(r2, 1, d, h->num_sm) + wide_gemm_launch_count(r1, 1, d, h->num_sm) +
+                       wide_gemm_launch_count(r1, 1, dff, h->num_sm);
+      }
       for (int r0 = 0; r0 < rows; r0 += SPS_MAX_ROWS) {
         AttnArgs aa{};
         aa.st = h->dst; aa.qkv = h->wqkv + (size_t)r0 * ldq; aa.out = h->watt + (size_t)r0 * d;
@@ -501,9 +511,11 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
         aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
         aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = (rows - r0) < SPS_MAX_ROWS ? (rows - r0) : SPS_MAX_ROWS; aa.B = 1;
         aa.mode = PASS_PREFILL; aa.t = 0; aa.c0 = c0 + r0; aa.seq0 = seq;
+        // the attention output is the next GEMM's operand: the kernel leaves it split into bf16 halves as well
+        aa.out_hi = reinterpret_cast<__nv_bfloat16*>(h->wa_hi) + (size_t)r0 * d;
+        aa.out_lo = reinterpret_cast<__nv_bfloat16*>(h->wa_lo) + (size_t)r0 * d;
         CU(h, attn_launch(aa, st)); h->launches++;
       }
-      CU(h, wide_pack_launch(h->watt, d, nullptr, 0.f, rows, d, h->wa_hi, h->wa_lo, d, st));
       CU(h, wide_gemm_launch(Wb(m.wo[l], (size_t)d * d, 0), h->wa_hi, h->wa_lo, rows, d, d, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st,
                              q8 ? m.wo_s[l] : nullptr));
       CU(h, wide_pack_launch(h->wx, d, (const float*)m.ffn_norm[l], c.rms_eps, rows, d, h->wa_hi, h->wa_lo, d, st));
@@ -511,7 +523,6 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
                              q8 ? m.w_up_s[l] : nullptr));
       CU(h, wide_gemm_launch(Wb(m.w_down[l], (size_t)dff * d, 0), h->wu_hi, h->wu_lo, rows, d, dff, h->wpart, WIDE_RESIDUAL, h->wx, d, nullptr, nullptr, 0, err, h->num_sm, st,
                              q8 ? m.w_down_s[l] : nullptr));
-      h->launches += 8;
       CU(h, dq_err);
     }
   }

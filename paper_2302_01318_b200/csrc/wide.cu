@@ -128,12 +128,34 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ float wide_gelu_dev(float v) {
+  return 0.5f * v * (1.0f + tanhf(0.7978845608028654f * (v + 0.044715f * v * v * v)));
+}
+__device__ __forceinline__ uint2 wide_split4_dev(const float4& v, uint2& lo) {
+  const float f[4] = {v.x, v.y, v.z, v.w};
+  uint32_t h[4], l[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat16 hb = __float2bfloat16_rn(f[i]);
+    h[i] = __bfloat16_as_ushort(hb);
+    l[i] = __bfloat16_as_ushort(__float2bfloat16_rn(f[i] - __bfloat162float(hb)));
+  }
+  lo = make_uint2(l[0] | (l[1] << 16), l[2] | (l[3] << 16));
+  return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+}
+
 struct WideGemmArgs {
   CUtensorMap tm_hi, tm_lo, tm_w[3];   // up to three stacked weight matrices (q | k | v): output columns side by side
   int rows_mat[3], tiles_mat[3];       // rows of each matrix and its tiles of 256 rows (0 for unused slots)
   float* part;        // [S][128][N] partial products of the k-splits
   int M, N, D, S;     // live rows, weight rows of all matrices together, width, k-splits (D / 64 is a multiple of S)
   int w_is_output;    // the weights were written by the predecessor kernel (bf16 copy of int8 weights): no early fetch
+  // one k-split: the epilogue warps finish the layer themselves (mode WIDE_EPI_*; scale: int8 row scales per matrix)
+  int fused, mode, vec, ldp;
+  float* y;
+  long long ldy;
+  __nv_bfloat16 *yhi, *ylo;
+  const float* scale[3];
   int* err;
 };
 
@@ -247,7 +269,50 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
         tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(WIDE_BN + c), vl);
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] += vl[i];
-        if (row < a.M && c < ncols) {
+        if (row < a.M && c < ncols && a.fused) {
+          // no other k-split: store / add to the residual stream / GeLU + split right here
+          const int lim = min(32, ncols - c), cn = col0 + wrow0 + c;
+          if (a.scale[0]) {
+            const float* sc = a.scale[mat] + wrow0 + c;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (i < lim) v[i] *= __ldg(sc + i);
+          }
+          if (a.mode == 2) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = wide_gelu_dev(v[i]);
+          }
+          const bool full = lim == 32 && a.vec;
+          if (a.mode == 0) {
+            float* yp = a.y + row * a.ldy + cn;
+            if (full) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(yp + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            } else {
+              for (int i = 0; i < lim; ++i) yp[i] = v[i];
+            }
+          } else if (a.mode == 1) {
+            float* yp = a.y + row * a.ldy + cn;
+            for (int i = 0; i < lim; ++i) yp[i] += v[i];
+          } else {
+            __nv_bfloat16* hp = a.yhi + (size_t)row * a.ldp + cn;
+            __nv_bfloat16* lp = a.ylo + (size_t)row * a.ldp + cn;
+            if (full) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) {
+                uint2 l;
+                const uint2 h = wide_split4_dev(make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]), l);
+                *reinterpret_cast<uint2*>(hp + i) = h;
+                *reinterpret_cast<uint2*>(lp + i) = l;
+              }
+            } else {
+              for (int i = 0; i < lim; ++i) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(v[i]);
+                hp[i] = h;
+                lp[i] = __float2bfloat16_rn(v[i] - __bfloat162float(h));
+              }
+            }
+          }
+        } else if (row < a.M && c < ncols) {
           if (c + 32 <= ncols && ((a.N | col0) & 3) == 0) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + c + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
@@ -499,6 +564,12 @@ int wide_splits(int N, int D, int num_sm) {
     if (kb % s == 0) S = s;
   return S;
 }
+// kernels one GEMM call launches: with a single k-split the epilogue is part of the GEMM kernel
+int wide_gemm_launch_count(const int* rows, int nmat, int D, int num_sm) {
+  int tiles = 0;
+  for (int i = 0; i < nmat; ++i) tiles += (rows[i] + WIDE_BN - 1) / WIDE_BN;
+  return wide_splits_tiles(tiles, D, num_sm) == 1 ? 1 : 2;
+}
 size_t wide_part_floats(int N, int D, int num_sm) { return (size_t)wide_splits(N, D, num_sm) * WIDE_M * (size_t)N; }
 // enough for any (stacked) shape of N output columns: S * tiles <= SMs bounds S * N by 256 * SMs when S > 1
 size_t wide_part_bound(int N, int num_sm) {
@@ -556,6 +627,13 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   }
   a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits_tiles(tiles, D, num_sm); a.err = err;
   a.w_is_output = scales ? 1 : 0;
+  // four columns per access when every matrix, stride and pointer allows 16-byte (8-byte for bf16) accesses
+  int vec = ((N | a.rows_mat[0] | a.rows_mat[1] | a.rows_mat[2] | ldp) & 3) == 0 && (ldy & 3) == 0 &&
+            (((uintptr_t)part | (uintptr_t)y | (uintptr_t)yhi | (uintptr_t)ylo) & 15) == 0;
+  for (int i = 0; i < 3; ++i) if (scales && i < nmat && ((uintptr_t)scales[i] & 15)) vec = 0;
+  a.fused = a.S == 1 ? 1 : 0; a.mode = mode; a.vec = vec; a.ldp = ldp; a.y = y; a.ldy = ldy;
+  a.yhi = reinterpret_cast<__nv_bfloat16*>(yhi); a.ylo = reinterpret_cast<__nv_bfloat16*>(ylo);
+  for (int i = 0; i < 3; ++i) a.scale[i] = (scales && i < nmat) ? scales[i] : nullptr;
   static bool attr = false;
   if (!attr) {
     if ((e = cudaFuncSetAttribute(wide_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<64>::SMEM)) != cudaSuccess) return e;
@@ -564,11 +642,7 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   }
   if (mr == 64) e = launch_k(wide_gemm_kernel<64>, dim3(tiles, a.S), dim3(192), WideCfg<64>::SMEM, st, a);
   else e = launch_k(wide_gemm_kernel<128>, dim3(tiles, a.S), dim3(192), WideCfg<128>::SMEM, st, a);
-  if (e != cudaSuccess) return e;
-  // four columns per thread when every matrix, stride and pointer allows 16-byte accesses
-  int vec = ((N | a.rows_mat[0] | a.rows_mat[1] | a.rows_mat[2] | ldp) & 3) == 0 && (ldy & 3) == 0 &&
-            (((uintptr_t)part | (uintptr_t)y | (uintptr_t)yhi | (uintptr_t)ylo) & 15) == 0;
-  for (int i = 0; i < 3; ++i) if (scales && i < nmat && ((uintptr_t)scales[i] & 15)) vec = 0;
+  if (e != cudaSuccess || a.fused) return e;
   const long long total = (long long)M * (vec ? N / 4 : N);
   int blocks = (int)((total + 255) / 256);
   if (blocks > 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK)) blocks = 8 * (num_sm > 0 ? num_sm : SPS_NUM_SM_FALLBACK);
