@@ -139,7 +139,7 @@ def run_linear_wide(W, X):
 
 
 @pytest.mark.parametrize("M", [1, 5, 16, 17, 33, 48, 64, 65, 127, 128])
-@pytest.mark.parametrize("N,D", [(256, 64), (300, 128), (1000, 256), (77, 1024), (4099, 2048)])
+@pytest.mark.parametrize("N,D", [(256, 64), (300, 128), (1000, 256), (77, 1024), (4099, 2048), (513, 192), (8, 448), (257, 6144)])
 def test_linear_wide_small(M, N, D):
     """The prompt-pass GEMM (up to 128 rows on the tcgen05 tensor cores) against the oracle: ragged N (tiles of
     256 weight rows), one to many k-blocks and k-splits, every row count class."""
