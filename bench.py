@@ -401,6 +401,18 @@ def run_ours(args):
         line["variants"]["aligned_adaptive_K_1_6"] = {"value": args.aligned_steps * n_new / (ad_ms / 1e3), "unit": UNIT,
                                                       "tokens_per_loop": sum(s["emitted"] for s in ad) / ad_loops,
                                                       "mean_K": sum(s["draft_calls"] for s in ad) / ad_loops}
+        # tokens per loop swept independently of the models: every draft accepted with a fixed probability (measurement
+        # mode; the tokens follow no law, the kernels run as always)
+        forced = []
+        for alpha in (0.5, 0.7, 0.8, 0.9):
+            h.sps_set_forced_acceptance(alpha)
+            gen(0, K)
+            st = gen(args.warmup, K)[1]
+            forced.append({"alpha": alpha, "value": n_new / (st["ms_decode"] / 1e3), "tokens_per_loop": st["emitted"] / st["loops"],
+                           "expected_tokens_per_loop": (1 - alpha ** (K + 1)) / (1 - alpha),
+                           "speedup_vs_ar": n_new / (st["ms_decode"] / 1e3) / ar_tps if ar_tps else None})
+        h.sps_set_forced_acceptance(0.0)
+        line["variants"]["forced_acceptance"] = forced
         # lookahead sweep on the damped pair (the paper's K trade-off figure): one generation per K
         if args.k_sweep:
             sweep = []

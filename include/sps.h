@@ -194,6 +194,16 @@ int sps_generate_adaptive(sps_handle* h, const int32_t* prompt, int32_t prompt_l
 int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new,
                        int32_t K, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
 
+/* Measurement mode (not part of the method): every draft is accepted with the
+ * fixed probability alpha instead of min(1, q/p), so that tokens per loop --
+ * (1 - alpha^(K+1)) / (1 - alpha) in expectation -- can be swept independently
+ * of how well a draft model happens to agree with its target (the Results
+ * section's speed-ups depend on that agreement; random-init models have
+ * little).  The emitted tokens then follow no particular law; every kernel
+ * runs exactly as otherwise.  alpha in (0, 1]; 0 switches the mode off (the
+ * default).  Applies to the generate / step calls of this handle. */
+int sps_set_forced_acceptance(sps_handle* h, float alpha);
+
 /* Per-loop record of the last sps_generate / sps_generate_adaptive /
  * sps_generate_batch call, for latency percentiles (the Results section
  * reports mean per-token latency; a loop delivers its tokens together, so the

@@ -81,6 +81,7 @@ def lib():
         L.sps_step.argtypes = [vp, i32, f32, u64, u32, vp, vp, vp]
         L.sps_last_logits.argtypes = [vp, i32, vp, vp, vp]
         L.sps_last_loop_trace.argtypes = [vp, vp, vp, vp, i32, vp]
+        L.sps_set_forced_acceptance.argtypes = [vp, f32]
         L.sps_verify.argtypes = [vp, vp, i32, vp, C.POINTER(f32)]
         L.sps_score.argtypes = [vp, i32, vp, i32, vp, C.POINTER(f32)]
         L.sps_accept.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, u32, vp, vp, vp, vp]
@@ -196,6 +197,10 @@ class Handle:
 
     def sps_set_sampling(self, top_k=0, top_p=1.0):
         _check(lib().sps_set_sampling(self._h, int(top_k), float(top_p)), self._h)
+
+    def sps_set_forced_acceptance(self, alpha):
+        """Measurement mode: accept every draft with probability alpha (0 = off)."""
+        _check(lib().sps_set_forced_acceptance(self._h, float(alpha)), self._h)
 
     def sps_reset(self):
         _check(lib().sps_reset(self._h), self._h)

@@ -96,7 +96,7 @@ struct DevState {
   float temperature;
   float inv_temperature;
   uint32_t step;      // loop index s, advanced on the device after each loop
-  uint32_t pad0;
+  uint32_t pad0;      // bits of the forced acceptance probability (0 = off): measurement mode, see sps_set_forced_acceptance
   uint64_t seed;
   float top_p;        // nucleus mass kept (1 = off), both models
   int32_t top_k;      // tokens kept (0 = off), both models

@@ -60,6 +60,7 @@ struct sps_handle {
   HostParams* h_par = nullptr;  // pinned
   int top_k = 0;                // sps_set_sampling: tokens kept (0 = off)
   float top_p = 1.f;            //                   nucleus mass kept (1 = off)
+  float forced_accept = 0.f;    // sps_set_forced_acceptance: fixed acceptance probability (0 = off; measurement only)
   int32_t* h_rows = nullptr;    // pinned [2][16]
   size_t res_words = 0;
   int B = 0;
@@ -417,7 +418,8 @@ int write_params(sps_handle* h, float T, uint64_t seed, uint32_t step) {
   // temperature 0 = greedy decoding: the one-token limit of top-k, applied to both models
   const bool greedy = T == 0.f;
   if (greedy) T = 1.f;
-  h->h_par->temperature = T; h->h_par->inv_temperature = 1.0f / T; h->h_par->step = step; h->h_par->pad0 = 0;
+  h->h_par->temperature = T; h->h_par->inv_temperature = 1.0f / T; h->h_par->step = step;
+  std::memcpy(&h->h_par->pad0, &h->forced_accept, 4);
   h->h_par->seed = seed;
   h->h_par->top_k = greedy ? 1 : h->top_k;
   h->h_par->top_p = greedy ? 1.f : h->top_p;
@@ -940,6 +942,13 @@ int sps_set_sampling(sps_handle* h, int32_t top_k, float top_p) {
   if (!(top_p > 0.f && top_p <= 1.f)) return fail(h, SPS_EINVAL, "top_p must be in (0, 1] (1 = off)");
   h->top_k = top_k;
   h->top_p = top_p;
+  return SPS_OK;
+}
+
+int sps_set_forced_acceptance(sps_handle* h, float alpha) {
+  if (!h) return fail(nullptr, SPS_EINVAL, "null handle");
+  if (!(alpha >= 0.f && alpha <= 1.f)) return fail(h, SPS_EINVAL, "alpha must be in [0, 1] (0 = off)");
+  h->forced_accept = alpha;
   return SPS_OK;
 }
 

@@ -457,6 +457,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
 
   // ---- phase 2: accept chain, left to right
   const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
+  const float forced = a.st ? __uint_as_float(a.st->pad0) : 0.f;
   auto accept_at = [&](int t) {   // thread 0: does draft t pass?
     int d = drafts[t];
     if (d < 0 || d >= V) { d = 0; if (a.st) atomicExch(a.st->err, 1); }
@@ -466,6 +467,9 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
     const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
     const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)t);
+    // measurement mode only: accept with a fixed probability whatever the models say (tokens per loop as a function
+    // of the acceptance rate alone); the emitted tokens then follow no particular law
+    if (forced > 0.f) return u.u_acc < forced;
     return u.u_acc < ratio;
   };
   if (!filt) {

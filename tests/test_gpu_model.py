@@ -290,6 +290,34 @@ def test_more_than_16_rows_need_a_bf16_target():
         sps.Handle(c["target"], w, None, None, max_seq=64, max_batch=4, max_K=4)
 
 
+def test_forced_acceptance_is_a_measurement_mode_only():
+    """With a forced acceptance probability every draft passes with that probability whatever the models say: alpha = 1
+    accepts all K drafts in every loop, alpha = 0.6 gives the geometric stop law, and switching it off restores the
+    oracle's tokens."""
+    h, ot, od, c = make_pair("tiny", max_K=4)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(0, 16, V)
+    want = oracle.Sps(ot, od).generate(prompt, 40, 4, 1.0, 3)
+    h.sps_set_forced_acceptance(1.0)
+    _, st = h.sps_generate(prompt, 40, 4, 1.0, 3)
+    assert st["hist_emitted"][5] == st["loops"] and st["accepted"] == 4 * st["loops"]
+    h.sps_set_forced_acceptance(0.6)
+    acc = loops = 0
+    hist = np.zeros(6)
+    for seed in range(12):
+        _, st = h.sps_generate(prompt, 60, 4, 1.0, seed)
+        acc += st["accepted"]; loops += st["loops"]; hist += np.array(st["hist_emitted"][:6])
+    expect = sum(0.6 ** j for j in range(1, 5))            # E[accepted] = alpha + alpha^2 + ... + alpha^K
+    assert abs(acc / loops - expect) < 5 * np.sqrt(1.2 / loops), (acc / loops, expect)
+    assert abs(hist[1] / loops - 0.4) < 5 * np.sqrt(0.24 / loops)          # stop at the first draft with 1 - alpha
+    with pytest.raises(sps.SpsError):
+        h.sps_set_forced_acceptance(1.5)
+    h.sps_set_forced_acceptance(0.0)
+    got, _ = h.sps_generate(prompt, 40, 4, 1.0, 3)
+    assert (got == want["tokens"]).all() or (want["flags"] & NEAR)
+    h.close()
+
+
 def test_loop_trace_matches_the_statistics():
     h, _, _, c = make_pair("tiny", max_K=6)
     with pytest.raises(sps.SpsError):
