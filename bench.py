@@ -238,6 +238,9 @@ def run_ours(args):
         out, st = h.sps_generate(prompt, n_new, k, T if temp is None else temp, seeds[i])
         return out, st, time.perf_counter() - t0
 
+    def sps_generate_seeded(hh, seed_, k):
+        return hh.sps_generate(sps_synth.make_prompt(seed_, P, V), n_new, k, T, seed_)[1]
+
     def barrier():
         if dist is not None:
             dist.barrier()
@@ -415,13 +418,21 @@ def run_ours(args):
         line["variants"]["forced_acceptance"] = forced
         # lookahead sweep on the damped pair (the paper's K trade-off figure): one generation per K
         if args.k_sweep:
+            # per K: `k_sweep_seeds` generations (different prompts and seeds); besides the rates, the time to n_new tokens
+            # with its spread -- a longer lookahead makes the time per generation more variable (the K trade-off figure)
             sweep = []
             for k in (1, 2, 3, 4, 6, 8):
                 gen(0, k)
-                st = gen(args.warmup, k)[1]
-                sweep.append({"K": k, "value": n_new / (st["ms_decode"] / 1e3), "tokens_per_loop": st["emitted"] / st["loops"],
-                              "accepted_per_loop": st["accepted"] / st["loops"], "ms_verify_per_loop": st["ms_verify"] / st["loops"],
-                              "ms_draft_per_step": st["ms_draft"] / (st["loops"] * k)})
+                sts = [sps_generate_seeded(h, 3000 + j, k) for j in range(args.k_sweep_seeds)]
+                t = np.array([s_["ms_decode"] for s_ in sts])
+                loops_k = sum(s_["loops"] for s_ in sts)
+                sweep.append({"K": k, "value": float(n_new * len(sts) / (t.sum() / 1e3)), "seeds": len(sts),
+                              "tokens_per_loop": sum(s_["emitted"] for s_ in sts) / loops_k,
+                              "accepted_per_loop": sum(s_["accepted"] for s_ in sts) / loops_k,
+                              "ms_verify_per_loop": sum(s_["ms_verify"] for s_ in sts) / loops_k,
+                              "ms_draft_per_step": sum(s_["ms_draft"] for s_ in sts) / (loops_k * k),
+                              "time_to_n_new_ms": {"mean": float(t.mean()), "std": float(t.std()), "p90": float(np.percentile(t, 90)),
+                                                   "min": float(t.min()), "max": float(t.max())}})
             line["variants"]["k_sweep"] = sweep
     h.close()
     if rank == 0 and world == 1 and args.sweep and c["target"]["dtype"] == 1:
@@ -517,6 +528,7 @@ def main():
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
     ap.add_argument("--batch", type=int, default=8, help="also decode this many sequences together (0 / 1 = skip)")
     ap.add_argument("--sweep", action="store_true", help="also run the K x temperature x batch sweep (prompt 512, 256 tokens; minutes)")
+    ap.add_argument("--k-sweep-seeds", type=int, default=8, help="generations per K in --k-sweep")
     ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
     ap.add_argument("--traffic", type=float, default=None,
