@@ -190,6 +190,18 @@ def test_bf16_pair_logits_under_teacher_forcing():
     h.close()
 
 
+def test_mid_pair_logits_under_teacher_forcing():
+    """The mid-size bf16 pair at its full depth (24-layer d 2048 target, 6-layer d 1024 draft, vocabulary 32000): a
+    few loops under teacher forcing, logits within the bf16 tolerance, token decisions equal outside flagged near ties."""
+    h, ot, od, c = make_pair("mid", max_seq=64)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(4, 12, V)
+    loops, near, worst = teacher_forced(h, ot, od, prompt, 10, 4, 1.0, 11)
+    print(f"mid: {loops} loops, {near} near ties, worst logit error {worst:.2e}")
+    assert worst < 5e-2
+    h.close()
+
+
 def test_int8_weight_pair_logits_under_teacher_forcing():
     """int8 linear weights with row scales (weight-only quantisation): the oracle runs the fp32 model of the
     dequantised matrices with a bf16 KV cache; activations on the GPU are fp16 halves, so the bf16 tolerance holds
