@@ -3,6 +3,8 @@ the 4B-shaped draft (d 6144, FFN 24576, 48 heads) with a reduced layer count, so
 in exactly the launch configuration `bench.py` times (same grids, k-splits and tile queues), and the
 oracle -- fed the very weights read back from the device, one layer at a time -- finishes in seconds.
 Tolerance: bf16 models, logits within 5e-2 abs (the benchmark spec); observed error is ~1e-3."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -65,4 +67,26 @@ def test_scoring_pass_at_70b_layer_shapes(name):
     # the whole loop runs at these shapes and keeps its invariants
     toks, st = h.sps_generate(prompt, 12, 4, 1.0, 3)
     assert ((toks >= 0) & (toks < V)).all() and st["loops"] == sum(st["hist_emitted"]) and st["emitted"] - st["overshoot"] == 12
+    h.close()
+
+
+@pytest.mark.skipif(os.environ.get("SPS_TEST_FULL_DEPTH") != "1",
+                    reason="minutes of CPU oracle time (80 layers of the 70B shape, one at a time); set SPS_TEST_FULL_DEPTH=1")
+def test_scoring_pass_at_full_depth():
+    """All 80 layers of the 70B-shaped target: a 10-token prompt, then one scoring pass over five rows, against the
+    oracle fed the same weights layer by layer.  The bf16 tolerance (5e-2 abs) must hold at full depth too."""
+    tc = sps_synth.CONFIGS["70b"]["target"]
+    wt = sps_synth.make_weights(tc, tag="target", device=DEV)
+    h = sps.Handle(tc, wt, None, None, max_seq=64, max_K=4)
+    V = tc["vocab"]
+    prompt = sps_synth.make_prompt(0, 10, V)
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(1, 4, V)])
+    h.sps_prefill(prompt)
+    out = torch.zeros((5, V), device=DEV)
+    h.sps_score(0, rows, out)
+    got = out.cpu().numpy().astype(np.float64)
+    want = oracle_logits(tc, wt, prompt[:-1], None, rows)
+    err = float(np.abs(got - want).max())
+    print(f"full depth (80 layers): worst logit error {err:.3e}, logits span [{want.min():.1f}, {want.max():.1f}]")
+    assert np.isfinite(got).all() and err < 5e-2, err
     h.close()
