@@ -1,25 +1,28 @@
-// The prompt pass as a real GEMM: up to 128 activation rows at once on the 5th-generation tensor cores.
+// Passes with many rows as a real GEMM: 9 .. 128 activation rows at once on the 5th-generation tensor cores.
 //
-// The decode kernels (linear.cu) stream every weight once per <= 16 rows, which is right for the loop
-// (1..K+1 rows) and wrong for the prompt: 127 prompt rows cost eight full sweeps over the weights.  Here
-// Y[128, N] = X[128, D] W[N, D]^T runs as tcgen05.mma (cta_group::1, M = 128, N = 256, K = 16, bf16
-// operands, fp32 accumulators in tensor memory), so the prompt costs one sweep:
+// The decode kernels (linear.cu) stream every weight once per <= 16 rows, which is right for the loop's usual
+// 1 .. K+1 rows and wrong for a prompt (127 prompt rows would cost eight full sweeps over the weights) or for
+// a batch of sequences.  Here Y[M, N] = X[M, D] W[N, D]^T runs as tcgen05.mma (cta_group::1, M = 128 -- or 64
+// when the pass has at most 64 rows --, N = 256, K = 16, bf16 operands, fp32 accumulators in tensor memory):
 //
-//   * grid = (N / 256 weight-row tiles) x (S k-splits); one CTA keeps a 128 x 256 fp32 accumulator in
-//     256 columns of tensor memory;
-//   * warp 0 (one lane) is the copy producer: per 64-wide k-block one TMA box of W (256 rows x 128 B)
-//     and one each of the activations' high and low bf16 halves (128 rows x 128 B), 128-byte swizzle,
-//     into a 3-stage ring of 64 KB stages guarded by full / empty mbarriers;
+//   * grid = (tiles of 256 weight rows, over up to three stacked matrices q | k | v) x (S k-splits);
+//   * warp 0 (one lane) is the copy producer: per 64-wide k-block one TMA box of W (256 rows x 128 B) and one
+//     each of the activations' high and low bf16 halves (128 or 64 rows x 128 B), 128-byte swizzle, into a ring
+//     of 3 (4) stages of 64 (48) KB guarded by full / empty mbarriers; the first ring-full of W boxes is
+//     asked for before the kernel waits for its predecessor (weights are constants);
 //   * warp 1 (one lane) issues the MMAs: 4 k-steps x (high, low) per k-block -- the two halves make the
-//     activations exact to ~16 bits as in the decode kernels -- and releases the stage with tcgen05.commit;
-//   * warps 2..5 read the accumulator back with tcgen05.ld once the last commit has landed (warp w owns
-//     tensor-memory lanes 32 (w % 4) ..) and write the CTA's partial tile; wide_epilogue_kernel adds the
-//     k-splits in a fixed order and applies the layer's epilogue (store / residual add / GeLU + split).
+//     activations exact to ~16 bits as in the decode kernels -- into two accumulators (all 512 columns of
+//     tensor memory: high-half products and low-half products are summed apart and added once at the end),
+//     and releases the stage with tcgen05.commit;
+//   * warps 2..5 read the accumulators back with tcgen05.ld once the last commit has landed (warp w owns
+//     tensor-memory lanes 32 (w % 4) ..).  With one k-split they finish the layer themselves (store / add
+//     to the residual stream / GeLU + split into bf16 halves, int8 row scales); otherwise they write the
+//     CTA's partial tile and wide_epilogue_kernel adds the k-splits in a fixed order and does the same.
 //
 // Per weight byte the activations cost one byte of L2 traffic (128 rows x 2 halves x 2 B per 256 weight
-// rows), so the pass stays bound by the weight stream from HBM.  Every wait is bounded (2 s of
-// %globaltimer): on expiry the CTA records error 3, lets its copies land, frees its tensor memory and
-// returns.  No multicast, no clusters.
+// rows), so the pass stays bound by the weight stream from HBM up to 64 rows and by the tensor pipe above.
+// Every wait is bounded (2 s of %globaltimer): on expiry the CTA records error 3, lets its copies land, frees
+// its tensor memory and returns.  No multicast, no clusters.
 #include "common.cuh"
 
 #include <cuda.h>
