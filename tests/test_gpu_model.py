@@ -330,6 +330,29 @@ def test_forced_acceptance_is_a_measurement_mode_only():
     h.close()
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16"])
+def test_long_context(name):
+    """A 1200-token context (the attention kernel walks it in tiles of 64 to 256 positions; the bf16 prompt goes
+    through ten 128-row chunks): logits of the next rows against the oracle, then a short generation."""
+    h, ot, od, c = make_pair(name, max_seq=1280)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(8, 1200, V)
+    h.sps_prefill(prompt)
+    ot.forward(prompt[:-1], np.arange(1199), want_logits=False)
+    od.forward(prompt[:-1], np.arange(1199), want_logits=False)
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(9, 4, V)])
+    out = torch.zeros((5, V), device=DEV)
+    for which, om in ((0, ot), (1, od)):
+        h.sps_score(which, rows, out)
+        want = om.forward64(rows, np.arange(1199, 1204))
+        err = np.abs(out.cpu().numpy() - want).max()
+        print(f"{name} model {which}: logit error at context 1200: {err:.2e}")
+        assert err < TOL[name], err
+    toks, st = h.sps_generate(prompt, 24, 4, 1.0, 1)
+    assert st["emitted"] - st["overshoot"] == 24 and ((toks >= 0) & (toks < V)).all()
+    h.close()
+
+
 def test_loop_trace_matches_the_statistics():
     h, _, _, c = make_pair("tiny", max_K=6)
     with pytest.raises(sps.SpsError):
