@@ -353,6 +353,30 @@ def test_long_context(name):
     h.close()
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_bf16"])
+def test_degenerate_sizes(name):
+    """The smallest and largest cases the loop has: a one-token prompt (no prompt pass at all), a single new token
+    (one loop, truncated), and the largest lookahead (K = 15: sixteen rows per scoring pass)."""
+    h, ot, od, c = make_pair(name, max_seq=96, max_K=15)
+    V = c["target"]["vocab"]
+    osps = oracle.Sps(ot, od)
+    cases = [(1, 20, 4), (16, 1, 4), (1, 1, 0), (16, 40, 15), (3, 17, 15)]      # (prompt length, n_new, K)
+    ok = 0
+    for P, n_new, K in cases:
+        prompt = sps_synth.make_prompt(P + K, P, V)
+        want = osps.generate(prompt, n_new, K, 1.0, 4)
+        got, st = h.sps_generate(prompt, n_new, K, 1.0, 4)
+        assert got.shape == (n_new,) and st["emitted"] - st["overshoot"] == n_new
+        assert sum(st["hist_emitted"][:K + 2]) == st["loops"] and st["draft_calls"] == K * st["loops"]
+        if (got == want["tokens"]).all():
+            ok += 1
+            assert st["loops"] == want["loops"]
+        else:
+            assert want["flags"] & NEAR, (P, n_new, K, got, want["tokens"])
+    assert ok >= len(cases) - 1
+    h.close()
+
+
 def test_loop_trace_matches_the_statistics():
     h, _, _, c = make_pair("tiny", max_K=6)
     with pytest.raises(sps.SpsError):
