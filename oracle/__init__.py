@@ -93,6 +93,9 @@ def lib():
         L.orc_tf_set_cache_dtype.argtypes = [vp, i32]
         L.orc_num_threads.restype = i32
         L.orc_linear.argtypes = [vp, i32, vp, i32, i32, i32, vp]
+        L.orc_set_threads.argtypes = [i32]
+        L.orc_invcdf.argtypes = [vp, i32, f64, vp]
+        L.orc_invcdf.restype = i32
         _lib = L
     return _lib
 
@@ -111,6 +114,19 @@ def _i32(a):
 
 def num_threads() -> int:
     return int(lib().orc_num_threads())
+
+
+def set_threads(n: int) -> None:
+    """Test hook: split large mat-vecs over n threads from now on (1 = none, 0 = the machine's count)."""
+    lib().orc_set_threads(int(n))
+
+
+def invcdf(weights, u: float):
+    """Inverse-CDF draw in index order on unnormalised float64 weights: (token, near_tie)."""
+    w = np.ascontiguousarray(weights, dtype=np.float64)
+    nt = C.c_int(0)
+    tok = lib().orc_invcdf(_p(w), w.shape[0], float(u), C.byref(nt))
+    return int(tok), bool(nt.value)
 
 
 def linear(W, X):

@@ -25,6 +25,9 @@
 //   transformer       : PARITY UNPINNED BY THE PAPER (it prints no architecture
 //                       values); pinned by cached == uncached forward, an
 //                       independent numpy restatement, and invariances.
+//   linear            : an independent float64 matrix product (fp32 and bf16 weights,
+//                       ragged shapes), also at sizes where the rows are split over
+//                       threads, where the result must equal the one-thread result bit for bit
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
@@ -35,7 +38,9 @@
 
 // Rows of a large mat-vec are split over plain std::threads (no OpenMP runtime: the host process
 // usually carries another one already).  Small problems run on the calling thread.
+static int g_threads_override = 0;   // test hook (orc_set_threads): > 0 replaces the machine's thread count
 static int hw_threads() {
+  if (g_threads_override > 0) return g_threads_override;
   static const int n = [] {
     unsigned h = std::thread::hardware_concurrency();
     int v = h ? (int)h : 1;
@@ -900,3 +905,10 @@ extern "C" void orc_linear(const void* W, int dtype, const float* X, int M, int 
 }
 
 extern "C" int orc_num_threads() { return hw_threads(); }
+// Test hook: n > 0 makes every later call split its rows over n threads (1 = the calling thread only), 0 goes
+// back to the machine's count.  The arithmetic of a row does not depend on which thread runs it, so results
+// must be identical for every n; a test checks exactly that.
+extern "C" void orc_set_threads(int n) { g_threads_override = n > 64 ? 64 : n; }
+// The inverse-CDF draw on given unnormalised weights (the "Sample" of Algorithms 1 and 2 under this build's
+// reading), exposed so that its two degenerate exits can be pinned directly.
+extern "C" int orc_invcdf(const double* w, int V, double u, int* near_tie) { return invcdf(w, V, u, near_tie); }

@@ -314,3 +314,55 @@ def test_sample_row_inverse_cdf_definition():
     lg = (rng.normal(size=64) * 3).astype(np.float32)
     for u in np.linspace(0.01, 0.99, 25):
         assert oracle.sample_row(lg, 1.0, u)[0] == oracle.sample_row(lg + 8.0, 1.0, u)[0]
+
+
+def test_inverse_cdf_degenerate_exits():
+    """The two exits of the inverse-CDF draw that rounding alone can reach, constructed on purpose: no running
+    sum exceeds u * total (u = 1: beyond the generator's grid, which ends at 1 - 2^-24) -> the largest index of
+    positive weight; weights that are all zero -> the last index.  Both are flagged as near ties."""
+    # u = 1: the running sum never exceeds the total; trailing zero weights are skipped
+    assert oracle.invcdf([0.2, 0.5, 0.3, 0.0, 0.0], 1.0) == (2, True)
+    assert oracle.invcdf([0.0, 4.0, 0.0], 1.0) == (1, True)
+    # through the public draw: a logit of -inf weighs exactly zero
+    lg = np.array([0.3, 1.0, -np.inf], dtype=np.float32)
+    assert oracle.sample_row(lg, 1.0, 1.0) == (1, True)
+    # nothing has weight: the last index, flagged
+    assert oracle.invcdf(np.zeros(6), 0.4) == (5, True)
+    # the ordinary exit, on unnormalised weights, against a cumulative sum written here
+    rng = np.random.default_rng(8)
+    for V in (1, 2, 9, 300):
+        w = rng.random(V) * rng.integers(0, 2, size=V)          # some exact zeros
+        if w.sum() == 0:
+            w[V // 2] = 1.0
+        c = np.cumsum(w)
+        for u in (0.0, 0.1, 0.5, 0.77, 1 - 2.0 ** -24):
+            tok, near = oracle.invcdf(w, u)
+            want = int(np.nonzero(c > u * c[-1])[0][0])
+            assert (tok == want or near) and w[tok] > 0
+
+
+def test_rejection_with_an_empty_residual_falls_back_to_the_target_law():
+    """sum_x max(0, q(x) - p(x)) = 0 together with a rejection cannot happen in exact arithmetic (Theorem 1's
+    proof: the rejection probability IS that sum).  Constructed here with p == q and a draft token of zero
+    probability under both (0/0 rejects by convention): the token is then drawn from q_t with u_res, the
+    fallback and resampled flags are set, and nothing of zero probability is returned."""
+    lg = np.array([0.3, -np.inf, 1.2, -0.5], dtype=np.float32)
+    q = sm(lg)
+    c = np.cumsum(q)
+    seen = set()
+    for s in range(300):
+        r = oracle.accept_chain(np.stack([lg, lg]), lg[None], [1], 1.0, 17, 2, s)
+        assert r["n_accepted"] == 0
+        assert r["flags"] & oracle.FLAG_FALLBACK and r["flags"] & oracle.FLAG_RESAMPLED
+        assert not r["flags"] & oracle.FLAG_BONUS
+        u_res = oracle.uniforms(17, 2, s, 0)[2]
+        want = int(np.nonzero(c > u_res * c[-1])[0][0])
+        assert r["tokens"][0] == want or r["flags"] & oracle.FLAG_NEAR_CDF
+        assert r["tokens"][0] != 1 and r["tokens"][1] == -1
+        seen.add(int(r["tokens"][0]))
+    assert seen == {0, 2, 3}
+    # an ordinary rejection (p != q) never takes the fallback
+    p = np.array([2.0, 0.1, -1.0, 0.4], dtype=np.float32)
+    for s in range(300):
+        r = oracle.accept_chain(np.stack([lg, lg]), p[None], [0], 1.0, 17, 2, s)
+        assert not r["flags"] & oracle.FLAG_FALLBACK
