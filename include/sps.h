@@ -189,10 +189,22 @@ int sps_generate_adaptive(sps_handle* h, const int32_t* prompt, int32_t prompt_l
                           int32_t K_max, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
 
 /* Same for B sequences with equal prompt lengths, advanced in lock-step with
- * ragged progress; sequence b uses Philox sequence index b.
+ * ragged progress; sequence b uses Philox sequence index index0 + b, index0
+ * being 0 unless sps_set_sequence_index0 changed it.  A sequence that has its
+ * n_new tokens keeps its rows in the later passes (their shape is fixed) but
+ * is no longer advanced, and its overshoot never counts against max_seq:
+ * prompt_len + n_new + K <= max_seq is all that is required.
  *   prompts host [B, prompt_len]; out_tokens host [B, n_new]; out_stats host [B] or NULL. */
 int sps_generate_batch(sps_handle* h, const int32_t* prompts, int32_t B, int32_t prompt_len, int32_t n_new,
                        int32_t K, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
+
+/* Sequence b of the following sps_generate*, sps_step calls draws its random
+ * numbers as Philox sequence index0 + b (counter word c2; the paper runs one
+ * sequence and names no generator -- this is how independent sequences get
+ * independent uniforms here).  With it a batch, or a replica on another GPU,
+ * can carry global sequence numbers and reproduce exactly what each sequence
+ * would have produced alone.  Stays on the handle until changed; default 0. */
+int sps_set_sequence_index0(sps_handle* h, uint32_t index0);
 
 /* Measurement mode (not part of the method): every draft is accepted with the
  * fixed probability alpha instead of min(1, q/p), so that tokens per loop --
@@ -220,22 +232,28 @@ int sps_last_loop_trace(sps_handle* h, float* loop_ms, int32_t* loop_emitted, in
 int sps_reset(sps_handle* h);
 /* make toks[0..n-1] (host) the sequence so far of a batch-1 run; both caches take positions 0..n-2 */
 int sps_prefill(sps_handle* h, const int32_t* toks, int32_t n);
-/* one loop iteration with loop index `step`; out_tokens host [K+1] (emitted first, -1 after),
- * *out_n_emitted = n_accepted + 1, *out_flags SPS_FLAG_* (may be NULL) */
+/* the same for B sequences of their own lengths: sequence b is toks[b * ld .. b * ld + lens[b]) (host, lens[b] >= 1,
+ * lens[b] <= ld); both caches take positions 0 .. lens[b] - 2 of each.  What follows a sequence's length in its
+ * row of toks is ignored.  B <= max_batch. */
+int sps_prefill_batch(sps_handle* h, const int32_t* toks, const int32_t* lens, int32_t B, int32_t ld);
+/* one loop iteration (Algorithm 2's while-body) with loop index `step`, for every sequence the last prefill set:
+ * out_tokens host [B, K+1] (emitted first, -1 after), out_n_emitted host [B] = n_accepted + 1,
+ * out_flags host [B] SPS_FLAG_* (may be NULL); B = 1 after sps_prefill */
 int sps_step(sps_handle* h, int32_t K, float temperature, uint64_t seed, uint32_t step, int32_t* out_tokens,
              int32_t* out_n_emitted, uint32_t* out_flags);
 /* copy what the last sps_step saw to HOST buffers (any may be NULL):
- * q_logits [K+1, V], p_logits [K, V], drafts [K] */
+ * q_logits [B, K+1, V], p_logits [B, K, V], drafts [B, K] */
 int sps_last_logits(sps_handle* h, int32_t K, float* q_logits, float* p_logits, int32_t* drafts);
 
-/* The scoring pass alone ("In parallel, compute K+1 sets of logits from
- * drafts", Algorithm 2): feeds rows[0..K] (host) to the TARGET at positions
+/* The scoring step of Algorithm 2 alone (section Conditional Scoring): one
+ * target pass that yields the K+1 conditional logit rows for the K drafts and
+ * the position after them.  Feeds rows[0..K] (host) to the TARGET at positions
  * len..len+K where len is the target cache's valid length, appends their
  * keys/values, and writes logits.  Does not move the valid length (calling it
  * again overwrites the same positions), so it can be timed repeatedly.
- *   out_logits DEVICE fp32 [K+1, vocab], caller-owned; out_ms host, device time, may be NULL.
- * which: 0 = target, 1 = draft. */
+ *   out_logits DEVICE fp32 [K+1, vocab], caller-owned; out_ms host, device time, may be NULL. */
 int sps_verify(sps_handle* h, const int32_t* rows, int32_t K, float* out_logits, float* out_ms);
+/* The same pass over n_rows rows (1..16) of either model; which: 0 = target, 1 = draft. */
 int sps_score(sps_handle* h, int32_t which, const int32_t* rows, int32_t n_rows, float* out_logits, float* out_ms);
 
 /* The modified rejection sampler alone (Algorithm 2's second for-loop and its
@@ -281,7 +299,8 @@ int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float tempera
  * bytes for the same (dtype, M, N, D), zero-filled once before its first use
  * (the kernel leaves it ready for the next call).
  * out_ms: host, device time of the kernel, may be NULL; when given the call
- * waits for the kernel and returns SPS_ETIMEOUT if a bounded wait inside it ran out.
+ * waits for the kernel and returns SPS_ETIMEOUT if a bounded wait inside it ran out
+ * (Y is then meaningless; the workspace stays usable for the next call).
  * sps_linear_scaled also takes dtype 2: W device int8 [N, D] (signed bytes) with
  * row_scale device fp32 [N], Y[m, n] = row_scale[n] * sum_k X[m, k] W[n, k] -- the
  * weight-only quantisation the paper's closing remark on quantisation refers to
@@ -319,16 +338,37 @@ int64_t sps_linear_wide_workspace_bytes(int32_t N, int32_t D);
  * cudaFree and uses no allocating library routine.
  *   W, X, Y, dtype, M, N, D: as for sps_linear (all device pointers).
  *   stream: cudaStream_t, NULL = default stream; the call only enqueues.
- * Limit: N * splits * 16 <= sps_linear_static_max_floats() (4 Mi floats), where
- * splits = D / 2048 for bf16 with M <= 8, D / 1024 for M > 8, 1 for fp32;
- * larger shapes return SPS_EINVAL with a message.  The first call on a device
- * looks up the array's device address (cudaGetSymbolAddress) with that device
- * current; make that first call before any stream capture begins.
+ * Limit: sps_linear_static_floats_needed(dtype, M, N, D) <=
+ * sps_linear_static_max_floats() (4 Mi floats).  The need is N * 16 * splits,
+ * where splits is how many ranges the kernel cuts D into on the current device
+ * (1 for fp32; for bf16 D over the largest multiple of 128 that divides D and
+ * is at most 2048 -- 1024 for M > 8 or for layers with few rows); ask the
+ * helper rather than redoing that rule.  Larger shapes return SPS_EINVAL with
+ * a message.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that first call
+ * before any stream capture begins.
  * All calls share the one array: two calls whose kernels overlap on the GPU
- * (different streams) race on it -- keep them on one stream or order them. */
+ * (different streams) race on it -- keep them on one stream or order them.
+ * Each call clears the array's counters before its kernel, so a call that
+ * follows an aborted one starts clean.  The call only enqueues and cannot
+ * report a bounded wait that ran out inside the kernel (sps_linear with
+ * out_ms can); Y is then meaningless. */
 int sps_linear_static(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
                       void* stream);
 int64_t sps_linear_static_max_floats(void);
+/* floats of split-K scratch the shape needs on the current device; -1 for arguments sps_linear_static rejects */
+int64_t sps_linear_static_floats_needed(int32_t dtype, int32_t M, int32_t N, int32_t D);
+
+/* Test hook for the give-up path of the kernels' waits.  Every wait inside a
+ * kernel (on a copy, on another CTA, on a tile queue) is bounded by the global
+ * timer: when the bound runs out the kernel records an error, lets the copies
+ * it has in flight land, frees what it holds and returns, and the host call
+ * reports SPS_ETIMEOUT.  limit_us shortens that bound (0 = the default of 2 s;
+ * at most 2 s), and drop_stage >= 0 makes the copy producer of the first CTA
+ * of sps_linear / sps_linear_wide leave out that stage of its ring, so that a
+ * wait runs out on purpose with nothing left in flight (-1 = leave nothing
+ * out).  Process-wide; not thread-safe; meant for tests only. */
+int sps_debug_set_wait(int64_t limit_us, int32_t drop_stage);
 
 /* Philox4x32-10 on the device, for known-answer tests: ctr device uint32 [n,4],
  * key device uint32 [n,2], out device uint32 [n,4]. */

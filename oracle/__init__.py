@@ -81,6 +81,7 @@ def lib():
         L.orc_sps_generate.argtypes = [vp, vp, i32, i32, i32, f64, u64, u32, u32, vp, vp, vp, vp]
         L.orc_sps_generate.restype = i32
         L.orc_sps_trials.argtypes = [vp, vp, vp, i32, i32, i32, f64, u64, u32, i64, i32, vp, vp, vp, vp]
+        L.orc_sps_trials_flagged.argtypes = [vp, vp, vp, i32, i32, i32, f64, u64, u32, i64, vp, vp, vp]
         L.orc_sps_trials_f.argtypes = [vp, vp, vp, i32, i32, i32, f64, i32, f64, u64, u32, i64, vp, vp, vp, vp]
         L.orc_sps_set_sampling.argtypes = [vp, i32, f64]
         L.orc_sample_row_f.argtypes = [vp, i32, f64, i32, f64, f64, vp]
@@ -416,6 +417,19 @@ def trials(target: Model, draft: Model | None, prompt, n_new: int, K: int, T: fl
         lib().orc_sps_trials_f(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
                                int(top_k), float(top_p), seed, b0, n_trials, _p(out), _p(hist), _p(first_acc), _p(first_flags))
     return {"tokens": out, "hist_emitted": hist, "first_n_accepted": first_acc, "first_flags": first_flags}
+
+
+def trials_flagged(target: Model, draft: Model | None, prompt, n_new: int, K: int, T: float, seed: int, n_trials: int,
+                   b0: int = 0):
+    """trials() that also returns, per trial, the flags of all its loops OR-ed together (near ties of draft draws
+    included as FLAG_NEAR_CDF): the trials another implementation may legitimately decide differently."""
+    p = _i32(prompt)
+    out = np.zeros((n_trials, n_new), dtype=np.int32)
+    hist = np.zeros(K + 2, dtype=np.int64)
+    flags = np.zeros(n_trials, dtype=np.uint32)
+    lib().orc_sps_trials_flagged(target._h, draft._h if draft is not None else None, _p(p), p.shape[0], n_new, K, float(T),
+                                 seed, b0, n_trials, _p(out), _p(hist), _p(flags))
+    return {"tokens": out, "hist_emitted": hist, "flags": flags}
 
 
 def trials_adaptive(target: Model, draft: Model, prompt, n_new: int, K_min: int, K_max: int, T: float, seed: int,

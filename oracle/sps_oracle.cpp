@@ -822,7 +822,9 @@ static void sps_trials_impl(OrcModel* target, OrcModel* draft, const int32_t* pr
                             double T, const Filt& filt, uint64_t seed, uint32_t b0, int64_t n_trials, int wrong_rule,
                             int32_t* out_tokens /*[n_trials][n_new]*/, int64_t* emitted_hist /*[K+2]*/,
                             int32_t* first_n_accepted /*[n_trials] or null*/,
-                            uint32_t* first_flags /*[n_trials] or null*/) {
+                            uint32_t* first_flags /*[n_trials] or null*/,
+                            uint32_t* all_flags = nullptr /*[n_trials] or null: flags of every loop of the trial, OR-ed,
+                                                            a draft draw's near tie counted as ORC_NEAR_CDF*/) {
   const int V = target->V;
   for (int i = 0; i < K + 2; ++i) emitted_hist[i] = 0;
   OrcSps* c = orc_sps_create(target, draft);
@@ -834,11 +836,13 @@ static void sps_trials_impl(OrcModel* target, OrcModel* draft, const int32_t* pr
     if (!wrong_rule) {
       orc_sps_reset(c, prompt, P);
       int made = 0; uint32_t s = 0;
+      if (all_flags) all_flags[tr] = 0u;
       while (made < n_new) {
-        int a; uint32_t fl;
-        const int e = orc_sps_loop(c, K, T, seed, b, s, em.data(), &a, &fl, nullptr);
+        int a; uint32_t fl, dnt = 0;
+        const int e = orc_sps_loop(c, K, T, seed, b, s, em.data(), &a, &fl, &dnt);
         if (s == 0 && first_n_accepted) first_n_accepted[tr] = a;
         if (s == 0 && first_flags) first_flags[tr] = fl;
+        if (all_flags) all_flags[tr] |= fl | (dnt ? ORC_NEAR_CDF : 0u);
         ++s;
         emitted_hist[e]++;
         for (int i = 0; i < e && made < n_new; ++i) out[made++] = em[i];
@@ -882,6 +886,14 @@ extern "C" void orc_sps_trials(OrcModel* target, OrcModel* draft, const int32_t*
                                int32_t* out_tokens, int64_t* emitted_hist, int32_t* first_n_accepted, uint32_t* first_flags) {
   sps_trials_impl(target, draft, prompt, P, n_new, K, T, Filt(), seed, b0, n_trials, wrong_rule, out_tokens, emitted_hist,
                   first_n_accepted, first_flags);
+}
+// the same trials, also reporting per trial the flags of all its loops (which trials another implementation may
+// legitimately decide differently)
+extern "C" void orc_sps_trials_flagged(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,
+                                       double T, uint64_t seed, uint32_t b0, int64_t n_trials, int32_t* out_tokens,
+                                       int64_t* emitted_hist, uint32_t* all_flags) {
+  sps_trials_impl(target, draft, prompt, P, n_new, K, T, Filt(), seed, b0, n_trials, 0, out_tokens, emitted_hist, nullptr, nullptr,
+                  all_flags);
 }
 // the same with top-k / nucleus filtering of both models (not with the negative-control chain)
 extern "C" void orc_sps_trials_f(OrcModel* target, OrcModel* draft, const int32_t* prompt, int P, int n_new, int K,

@@ -100,6 +100,11 @@ def lib():
         L.sps_philox.argtypes = [vp, vp, i32, vp, vp]
         L.sps_linear_static.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp]
         L.sps_linear_static_max_floats.restype = i64
+        L.sps_linear_static_floats_needed.argtypes = [i32, i32, i32, i32]
+        L.sps_linear_static_floats_needed.restype = i64
+        L.sps_prefill_batch.argtypes = [vp, vp, vp, i32, i32]
+        L.sps_set_sequence_index0.argtypes = [vp, u32]
+        L.sps_debug_set_wait.argtypes = [i64, i32]
         _lib = L
     return _lib
 
@@ -159,6 +164,7 @@ class Handle:
         self._h = h
         self.vocab = target_cfg["vocab"]
         self.max_K = max_K
+        self.B = 1          # sequences the last prefill set
 
     def close(self):
         if getattr(self, "_h", None):
@@ -204,17 +210,38 @@ class Handle:
 
     def sps_reset(self):
         _check(lib().sps_reset(self._h), self._h)
+        self.B = 1
 
     def sps_prefill(self, toks):
         t = np.ascontiguousarray(toks, dtype=np.int32)
         _check(lib().sps_prefill(self._h, _np_ptr(t), t.shape[0]), self._h)
+        self.B = 1
+
+    def sps_prefill_batch(self, seqs):
+        """seqs: list of B int sequences (their own lengths): the sequences so far of a batch."""
+        lens = np.array([len(x) for x in seqs], dtype=np.int32)
+        ld = int(lens.max())
+        t = np.zeros((len(seqs), ld), dtype=np.int32)
+        for b, x in enumerate(seqs):
+            t[b, :len(x)] = x
+        _check(lib().sps_prefill_batch(self._h, _np_ptr(t), _np_ptr(lens), len(seqs), ld), self._h)
+        self.B = len(seqs)
+
+    def sps_set_sequence_index0(self, index0):
+        """Sequence b of later generate / step calls uses Philox sequence index index0 + b."""
+        _check(lib().sps_set_sequence_index0(self._h, int(index0)), self._h)
 
     def sps_step(self, K, temperature, seed, step):
-        out = np.full(K + 1, -1, dtype=np.int32)
-        n = np.zeros(1, dtype=np.int32)
-        fl = np.zeros(1, dtype=np.uint32)
+        """One loop for every sequence of the last prefill.  Batch 1: (tokens [K+1], n_emitted, flags);
+        batch B > 1: (tokens [B, K+1], n_emitted [B], flags [B])."""
+        B = self.B
+        out = np.full((B, K + 1), -1, dtype=np.int32)
+        n = np.zeros(B, dtype=np.int32)
+        fl = np.zeros(B, dtype=np.uint32)
         _check(lib().sps_step(self._h, K, temperature, seed, step, _np_ptr(out), _np_ptr(n), _np_ptr(fl)), self._h)
-        return out, int(n[0]), int(fl[0])
+        if B == 1:
+            return out[0], int(n[0]), int(fl[0])
+        return out, n, fl
 
     def sps_last_loop_trace(self, cap=4096):
         """(loop_ms, loop_emitted, loop_K) of the last generation, one entry per loop."""
@@ -225,10 +252,14 @@ class Handle:
         return ms[:m], em[:m], kk[:m]
 
     def sps_last_logits(self, K):
-        q = np.zeros((K + 1, self.vocab), dtype=np.float32)
-        p = np.zeros((K, self.vocab), dtype=np.float32)
-        d = np.zeros(K, dtype=np.int32)
+        """(q_logits, p_logits, drafts) of the last step: [K+1, V], [K, V], [K] for batch 1, with a leading B otherwise."""
+        B = self.B
+        q = np.zeros((B, K + 1, self.vocab), dtype=np.float32)
+        p = np.zeros((B, K, self.vocab), dtype=np.float32)
+        d = np.zeros((B, K), dtype=np.int32)
         _check(lib().sps_last_logits(self._h, K, _np_ptr(q), _np_ptr(p) if K else None, _np_ptr(d) if K else None), self._h)
+        if B == 1:
+            return q[0], p[0], d[0]
         return q, p, d
 
     def sps_verify(self, rows, K, out_logits):
@@ -339,3 +370,13 @@ def sps_linear_static(W, X, Y, stream=None):
 
 def sps_linear_static_max_floats():
     return int(lib().sps_linear_static_max_floats())
+
+
+def sps_linear_static_floats_needed(dtype, M, N, D):
+    return int(lib().sps_linear_static_floats_needed(dtype, M, N, D))
+
+
+def sps_debug_set_wait(limit_us=0, drop_stage=-1):
+    """Test hook: bound of the kernels' waits in microseconds (0 = the default 2 s) and the stage the first CTA's copy
+    producer leaves out (-1 = none)."""
+    _check(lib().sps_debug_set_wait(int(limit_us), int(drop_stage)))

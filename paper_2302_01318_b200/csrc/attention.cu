@@ -43,8 +43,11 @@ __global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a) {
       break;
     default: tok = st->row_tok[row]; pos = st->row_pos[row]; break;
   }
-  if (tok < 0 || tok >= a.V) { tok = 0; if (tid == 0) atomicExch(st->err, 1); }
-  if (pos < 0 || pos >= max_seq) { pos = max(0, min(pos, max_seq - 1)); if (tid == 0) atomicExch(st->err, 2); }
+  // A sequence of a batch that has reached its length keeps its slot in every pass (the pass has a fixed shape) but
+  // no longer matters: its rows are parked on a valid position and raise nothing, whatever its overshoot was.
+  const bool dead = a.mode != PASS_PREFILL && a.mode != PASS_EXPLICIT && n >= st->limit[b];
+  if (tok < 0 || tok >= a.V) { tok = 0; if (tid == 0 && !dead) atomicExch(st->err, 1); }
+  if (pos < 0 || pos >= max_seq) { pos = max(0, min(pos, max_seq - 1)); if (tid == 0 && !dead) atomicExch(st->err, 2); }
   if (tid == 0) { st->row_tok[row] = tok; st->row_pos[row] = pos; }
   float local = 0.f;
   float* xr = a.x + (size_t)row * a.d;
@@ -365,13 +368,10 @@ size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh) {
 
 template <int DH, typename CT, int MR>
 static cudaError_t attn_go(const AttnArgs& a, cudaStream_t st) {
-  static size_t cached = 48 * 1024;
+  static DevSmemCache cached{};   // per device, like the attribute itself
   const size_t smem = attn_smem_t<DH, CT, MR>();
-  if (smem > cached) {
-    cudaError_t e = cudaFuncSetAttribute(attn_kernel<DH, CT, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    cached = smem;
-  }
+  cudaError_t e = sps_ensure_smem(attn_kernel<DH, CT, MR>, smem, cached);
+  if (e != cudaSuccess) return e;
   return launch_k(attn_kernel<DH, CT, MR>, dim3(a.H, a.B), dim3(ATTN_THREADS), smem, st, a);
 }
 

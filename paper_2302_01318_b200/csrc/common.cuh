@@ -64,6 +64,43 @@ inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_
 }
 
 // ------------------------------------------------------------------------------------------------
+// cudaFuncSetAttribute is per device: what a launcher remembers about it is kept per device too, so that
+// handles on several GPUs of one process each set the attribute on their own device.
+// ------------------------------------------------------------------------------------------------
+#define SPS_MAX_DEVICES 64
+struct DevSmemCache {
+  size_t bytes[SPS_MAX_DEVICES];
+  bool init;
+};
+template <class Kern>
+inline cudaError_t sps_ensure_smem(Kern k, size_t bytes, DevSmemCache& c) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= SPS_MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (!c.init) { for (size_t& b : c.bytes) b = 48 * 1024; c.init = true; }
+  if (bytes <= c.bytes[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) c.bytes[dev] = bytes;
+  return e;
+}
+// one-time (per device) attribute calls: true the first time on the current device
+struct DevOnce { bool done[SPS_MAX_DEVICES]; };
+inline bool sps_first_on_device(DevOnce& o) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= SPS_MAX_DEVICES) return true;
+  if (o.done[dev]) return false;
+  o.done[dev] = true;
+  return true;
+}
+
+// Bound of every device-side wait, in nanoseconds of %globaltimer (2 s), and the test hook that shortens it and
+// makes one copy producer leave out one stage, so that the give-up path of the kernels can be run on purpose
+// (sps_debug_set_wait in the header).  drop_stage < 0: nothing is left out.
+struct WaitKnobs { unsigned long long limit_ns; int drop_stage; };
+WaitKnobs sps_wait_knobs();
+
+// ------------------------------------------------------------------------------------------------
 // Reductions with a fixed tree (results are bit-reproducible run to run).
 // ------------------------------------------------------------------------------------------------
 __device__ inline float warp_sum(float v) {
@@ -116,7 +153,7 @@ struct DevState {
   uint32_t* flags;    // [B]
   int32_t* err;       // [1] sticky device-side error word (token out of range ...)
   int32_t max_K;
-  int32_t done_counter_pad;
+  uint32_t seq0;      // sequence b draws its random numbers as Philox sequence seq0 + b (sps_set_sequence_index0)
   uint32_t* done_counter;  // [1] CTAs of the accept kernel that finished (for the step advance)
 };
 
@@ -160,6 +197,8 @@ struct LinArgs {
   int PR;                 // rows per shared-memory pass (multiple of 32)      [register-streaming variant]
   int KS, KST, NS, G;     // k-range per CTA, k-range per stage, ring stages, warps per tile [TMA variant]
   int* err;               // sticky error word: set to 3 if a bounded wait ran out
+  unsigned long long wait_ns;   // set by the launcher: bound of every wait inside the kernel
+  int drop_stage;         // set by the launcher: >= 0 makes CTA 0's producer leave out that stage (test hook), -1 = none
   // Packed activations (bf16 TMA kernel only).  A layer may leave, beside Y, the next layer's input ready
   // for the tensor cores: act(y) * gain split into a bf16 high part and a bf16 remainder.  A layer given
   // such an input copies it into shared memory instead of converting X; with PRO_RMSNORM the gain is
@@ -251,6 +290,8 @@ struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(log
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
   int top_k; float top_p;  // used when st == nullptr (0 / 1 = no filtering)
   int smem_weights;        // set by the launcher: weights are staged in shared memory
+  float2* stats;           // when non-null: stats[b * stats_ld] = (row maximum, sum of exp((l - max) / T)) of the row drawn from
+  int stats_ld;
 };
 cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st);
 

@@ -36,6 +36,10 @@ struct HostParams { float temperature, inv_temperature; uint32_t step, pad0; uin
 
 void sps_set_global_error(const char* msg) { g_err = msg ? msg : ""; }
 
+// bound of the kernels' waits and the stage a producer leaves out (test hook, sps_debug_set_wait); process-wide
+static WaitKnobs g_wait_knobs = {2000000000ull, -1};
+WaitKnobs sps_wait_knobs() { return g_wait_knobs; }
+
 struct sps_handle {
   sps_cfg cfg{};
   cudaStream_t stream = nullptr;
@@ -445,24 +449,37 @@ int loop_once(sps_handle* h, int K, bool timed) {
   return SPS_OK;
 }
 
-int set_sequences(sps_handle* h, const int32_t* toks, int B, int n) {
+// toks: host [B][ld]; sequence b is toks[b][0 .. lens[b]) (lens == nullptr: every sequence has n tokens)
+int set_sequences(sps_handle* h, const int32_t* toks, int B, int n, const int32_t* lens = nullptr, int ld = 0) {
   const int max_seq = h->cfg.max_seq;
   if (B < 1 || B > h->cfg.max_batch) return fail(h, SPS_EINVAL, "batch outside 1..max_batch");
-  if (n < 1) return fail(h, SPS_EINVAL, "a sequence needs at least one token");
-  if (n > max_seq) return fail(h, SPS_ERANGE, "sequence longer than max_seq");
+  if (ld <= 0) ld = n;
   const int V = h->tgt.cfg.vocab;
-  for (long long i = 0; i < (long long)B * n; ++i)
-    if (toks[i] < 0 || toks[i] >= V) return fail(h, SPS_ERANGE, "token id outside the vocabulary");
-  h->B = B;
   std::vector<int32_t> nn(B, n);
-  CU(h, cudaMemcpy2DAsync(h->hst.tokens, (size_t)max_seq * 4, toks, (size_t)n * 4, (size_t)n * 4, B, cudaMemcpyHostToDevice, h->stream));
+  int n_max = 0;
+  for (int b = 0; b < B; ++b) {
+    if (lens) nn[b] = lens[b];
+    if (nn[b] < 1) return fail(h, SPS_EINVAL, "a sequence needs at least one token");
+    if (nn[b] > max_seq || nn[b] > ld) return fail(h, SPS_ERANGE, "sequence longer than max_seq (or than its row of the input)");
+    if (nn[b] > n_max) n_max = nn[b];
+  }
+  // what lies beyond a sequence's length is never meaningful: it travels as token 0
+  std::vector<int32_t> stage((size_t)B * n_max, 0);
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < nn[b]; ++i) {
+      const int32_t t = toks[(size_t)b * ld + i];
+      if (t < 0 || t >= V) return fail(h, SPS_ERANGE, "token id outside the vocabulary");
+      stage[(size_t)b * n_max + i] = t;
+    }
+  h->B = B;
+  CU(h, cudaMemcpy2DAsync(h->hst.tokens, (size_t)max_seq * 4, stage.data(), (size_t)n_max * 4, (size_t)n_max * 4, B, cudaMemcpyHostToDevice, h->stream));
   CU(h, cudaMemcpyAsync(h->hst.n, nn.data(), B * 4, cudaMemcpyHostToDevice, h->stream));
   int32_t Bv = B;
   CU(h, cudaMemcpyAsync(&h->dst->B, &Bv, 4, cudaMemcpyHostToDevice, h->stream));
   std::vector<int32_t> lim(B, 0x7fffffff);
   CU(h, cudaMemcpyAsync(h->hst.limit, lim.data(), B * 4, cudaMemcpyHostToDevice, h->stream));
-  CU(h, cudaStreamSynchronize(h->stream));  // nn / lim are stack-lifetime host buffers
-  for (int b = 0; b < B; ++b) h->seq_len[b] = n;
+  CU(h, cudaStreamSynchronize(h->stream));  // stage / nn / lim are stack-lifetime host buffers
+  for (int b = 0; b < B; ++b) h->seq_len[b] = nn[b];
   return SPS_OK;
 }
 
@@ -531,15 +548,20 @@ int prefill_wide(sps_handle* h, ModelDev& m, int n, int seq) {
   return SPS_OK;
 }
 
-int prefill_all(sps_handle* h, int n) {
+// (positions 0 .. seq_len[b] - 2 of sequence b; with ragged lengths the 16-row pass runs every sequence up to the
+// longest one -- the rows beyond a sequence's own length write cache positions that its first loop overwrites
+// before anything reads them)
+int prefill_all(sps_handle* h) {
   const int per = SPS_MAX_ROWS / h->B;
+  int n = 0;
+  for (int b = 0; b < h->B; ++b) n = h->seq_len[b] > n ? h->seq_len[b] : n;
   for (int which = 0; which < 2; ++which) {
     ModelDev& m = which == 0 ? h->tgt : h->drf;
     if (!m.present) continue;
     if (h->wide && m.cfg.dtype >= 1 && n - 1 > SPS_MAX_ROWS / h->B) {
       // one sequence after the other, each in chunks of 128 rows
       for (int b = 0; b < h->B; ++b) {
-        int rc = prefill_wide(h, m, n, b);
+        int rc = prefill_wide(h, m, h->seq_len[b], b);
         if (rc) return rc;
       }
       continue;
@@ -690,7 +712,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   if (cudaMallocHost(&h->h_res, 4 * h->res_words) != cudaSuccess || cudaMallocHost(&h->h_par, sizeof(HostParams)) != cudaSuccess ||
       cudaMallocHost(&h->h_rows, 4 * 2 * SPS_MAX_ROWS) != cudaSuccess)
     return bail(fail(h, SPS_ENOMEM, "pinned host allocation failed"));
-  s.temperature = 1.f; s.inv_temperature = 1.f; s.step = 0; s.seed = 0; s.top_p = 1.f; s.top_k = 0; s.B = 1; s.max_seq = cfg->max_seq; s.max_K = maxK;
+  s.temperature = 1.f; s.inv_temperature = 1.f; s.step = 0; s.seed = 0; s.top_p = 1.f; s.top_k = 0; s.B = 1; s.max_seq = cfg->max_seq; s.max_K = maxK; s.seq0 = 0;
   s.n_acc = h->res;
   s.flags = (uint32_t*)(h->res + MB);
   s.out_tok = h->res + 2 * MB;
@@ -742,8 +764,34 @@ int sps_prefill(sps_handle* h, const int32_t* toks, int32_t n) {
   CU(h, cudaSetDevice(h->cfg.device));
   int rc = set_sequences(h, toks, 1, n);
   if (rc) return rc;
-  if ((rc = prefill_all(h, n))) return rc;
+  if ((rc = prefill_all(h))) return rc;
   CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+int sps_prefill_batch(sps_handle* h, const int32_t* toks, const int32_t* lens, int32_t B, int32_t ld) {
+  if (!h || !toks || !lens) return fail(h, SPS_EINVAL, "null argument");
+  CU(h, cudaSetDevice(h->cfg.device));
+  int rc = set_sequences(h, toks, B, 0, lens, ld);
+  if (rc) return rc;
+  if ((rc = prefill_all(h))) return rc;
+  CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+int sps_set_sequence_index0(sps_handle* h, uint32_t index0) {
+  if (!h) return fail(nullptr, SPS_EINVAL, "null handle");
+  CU(h, cudaSetDevice(h->cfg.device));
+  h->hst.seq0 = index0;
+  CU(h, cudaMemcpyAsync(&h->dst->seq0, &h->hst.seq0, 4, cudaMemcpyHostToDevice, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  return SPS_OK;
+}
+
+int sps_debug_set_wait(int64_t limit_us, int32_t drop_stage) {
+  if (limit_us < 0 || limit_us > 2000000) return fail(nullptr, SPS_EINVAL, "limit_us outside 0..2000000 (0 = the default of 2 s)");
+  g_wait_knobs.limit_ns = limit_us == 0 ? 2000000000ull : (unsigned long long)limit_us * 1000ull;
+  g_wait_knobs.drop_stage = drop_stage < 0 ? -1 : drop_stage;
   return SPS_OK;
 }
 
@@ -824,7 +872,7 @@ static int generate_impl(sps_handle* h, const int32_t* prompts, int B, int P, in
   }
   cudaEvent_t e_pre0 = h->ev[4];
   CU(h, cudaEventRecord(e_pre0, h->stream));
-  if ((rc = prefill_all(h, P))) return rc;
+  if ((rc = prefill_all(h))) return rc;
   // the attention kernel may fetch cache rows of earlier loops before it waits for its predecessor;
   // that is only sound if the host has waited for the stream since those rows were written
   CU(h, cudaStreamSynchronize(h->stream));
@@ -1074,8 +1122,9 @@ int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, cons
   a.part = (float*)(ws + off);
   cudaStream_t st = (cudaStream_t)stream;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaMemsetAsync(a.counters + 2 * LIN_MAX_R + 1, 0, sizeof(int), st);   // the sticky error word starts clear
   if (out_ms) { cudaEventCreate(&e0); cudaEventCreate(&e1); cudaEventRecord(e0, st); }
-  cudaError_t e = lin_launch(dtype, a, p, st);
+  if (e == cudaSuccess) e = lin_launch(dtype, a, p, st);
   if (out_ms) {
     cudaEventRecord(e1, st);
     cudaEventSynchronize(e1);

@@ -470,15 +470,15 @@ __device__ __forceinline__ unsigned long long gtimer() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// wait for a phase with a 2 s bound; false (and error word 3) if it ran out
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err) {
+// wait for a phase, at most limit_ns of the global timer (2 s unless a test shortened it); false (and error word 3) if it ran out
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, unsigned long long limit_ns) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = gtimer();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try(bar, parity)) return true;
-    if (gtimer() - t0 > 2000000000ull) {
+    if (gtimer() - t0 > limit_ns) {
       atomicExch(err, 3);
       return false;
     }
@@ -583,7 +583,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         const int mat = mat_of(a, row0, rin);
         for (int ks = 0; ks < KSUB; ++ks, ++it) {
           const int slot = it % NS, use = it / NS;
-          if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; return; }
+          if (use > 0 && !mbar_wait(bar_empty + 8 * slot, (uint32_t)(use - 1) & 1u, a.err, a.wait_ns)) { ok = false; return; }
+          if (cta == 0 && it == a.drop_stage) continue;   // test hook: this stage is never asked for, its consumer's wait runs out
           mbar_expect_tx(bar_full + 8 * slot, STAGE);
           tma_load_3d(ring + slot * STAGE, &ta.tm[mat], 0, rin, (k_base + ks * KST) / SEGK,
                       bar_full + 8 * slot, policy);
@@ -608,7 +609,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       s_total = local;
       if (!ok || *((volatile int*)&s_abort)) {
         // a wait ran out somewhere: let the copies already issued land before this CTA's memory goes away
-        for (int j = max(0, it - NS); j < it; ++j) mbar_wait(bar_full + 8 * (j % NS), (uint32_t)(j / NS) & 1u, a.err);
+        for (int j = max(0, it - NS); j < it; ++j)
+          if (!(cta == 0 && j == a.drop_stage)) mbar_wait(bar_full + 8 * (j % NS), (uint32_t)(j / NS) & 1u, a.err, a.wait_ns);
       }
     }
     pdl_wait();
@@ -653,7 +655,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           if (lane == 0) s_scale[m] = rsqrtf(tt / (float)D + a.eps);
         }
       }
-      if (!mbar_wait(bar_x, 0u, a.err)) { alive = false; s_abort = 1; }
+      if (!mbar_wait(bar_x, 0u, a.err, a.wait_ns)) { alive = false; s_abort = 1; }
     } else {
     // A thread owns 4 consecutive k (one 16-byte load per row, neighbouring lanes neighbouring addresses)
     // of up to two places of the k-range.  The gain of the norm is a weight: it comes from HBM, and is
@@ -762,7 +764,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           const int tot = s_total;
           if (tot >= 0 && L >= tot) { done = true; break; }
           __nanosleep(32);
-          if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); s_abort = 1; alive = false; break; }
+          if (gtimer() - t0 > a.wait_ns) { atomicExch(a.err, 3); s_abort = 1; alive = false; break; }
         }
         if (done) break;   // every warp of the group sees the same numbers and leaves here together
       }
@@ -778,11 +780,11 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
           const unsigned long long t0 = gtimer();
           while (consumed[slot] < use * GS) {
             __nanosleep(64);
-            if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); alive = false; break; }
+            if (gtimer() - t0 > a.wait_ns) { atomicExch(a.err, 3); alive = false; break; }
           }
           if (!alive) { s_abort = 1; break; }
         }
-        if (!mbar_wait(bar_full + 8 * slot, (uint32_t)use & 1u, a.err)) { alive = false; s_abort = 1; break; }
+        if (!mbar_wait(bar_full + 8 * slot, (uint32_t)use & 1u, a.err, a.wait_ns)) { alive = false; s_abort = 1; break; }
         const uint32_t wrow = ring + slot * STAGE + g * 128;          // row g of slab 0; row g+8 is +1024
         const uint32_t xoff = (uint32_t)(ks * KST) * 2 + (uint32_t)t * 32;  // logical chunk 2t of this stage's k-range
         uint32_t xrow[NT];
@@ -952,7 +954,7 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       while (*((volatile int*)&a.counters[0]) < C) {
         __nanosleep(64);
         if (*((volatile int*)a.err) == 3) { ok = 0; break; }   // another CTA gave up: so do we
-        if (gtimer() - t0 > 2000000000ull) { atomicExch(a.err, 3); ok = 0; break; }
+        if (gtimer() - t0 > a.wait_ns) { atomicExch(a.err, 3); ok = 0; break; }
       }
       __threadfence();
     }
@@ -1184,12 +1186,7 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
 size_t lin_part_floats(int N, int S) { return (size_t)S * SPS_MAX_ROWS * (size_t)N; }
 
 template <class Kern>
-static cudaError_t ensure_smem(Kern k, size_t bytes, size_t& cached) {
-  if (bytes <= cached) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) cached = bytes;
-  return e;
-}
+static cudaError_t ensure_smem(Kern k, size_t bytes, DevSmemCache& cached) { return sps_ensure_smem(k, bytes, cached); }
 
 // A weight matrix [rows][D] bf16 as the copy engine sees it: dims {64 k, rows, D/64} with byte strides
 // {2, D*2, 128}, box {64, 16, KST/64}, 128-byte swizzle.  Descriptors are cached per (pointer, shape).
@@ -1236,7 +1233,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   if ((a.xp_hi || a.yp_hi) && !(dtype >= 1 && p.variant == 2)) return cudaErrorInvalidValue;   // packed activations: TMA kernel only
   if (dtype == 2 && (p.variant != 2 || !a.wscale[0] || (a.D % 128))) return cudaErrorInvalidValue;   // int8 weights: TMA kernel, scales given
   if ((a.xp_hi && !a.xp_lo) || (a.yp_hi && !a.yp_lo)) return cudaErrorInvalidValue;
-  static size_t c_b1 = 48 * 1024, c_b2 = 48 * 1024, c_f1 = 48 * 1024, c_f2 = 48 * 1024, c_t1 = 48 * 1024, c_t2 = 48 * 1024;
+  static DevSmemCache c_b1{}, c_b2{}, c_f1{}, c_f2{}, c_t1{}, c_t2{};   // per device, like the attribute itself
+  { const WaitKnobs wk = sps_wait_knobs(); a.wait_ns = wk.limit_ns; a.drop_stage = wk.drop_stage; }
   cudaError_t e;
   if (dtype == 0) {
     if (p.NT == 1) {
@@ -1258,7 +1256,7 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     }
     ta.a.split_epi = lin_split_epilogue() ? 1 : 0;
     ta.a.q8 = dtype == 2 ? 1 : 0;
-    static size_t c_q1 = 48 * 1024, c_q2 = 48 * 1024;
+    static DevSmemCache c_q1{}, c_q2{};
     if (dtype == 2 && p.NT == 1) {
       if ((e = ensure_smem(lin_bf16_tma_kernel<1, true>, p.smem, c_q1)) != cudaSuccess) return e;
       e = launch_k(lin_bf16_tma_kernel<1, true>, grid, dim3(threads), p.smem, st, ta);
@@ -1275,11 +1273,10 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     if (e == cudaSuccess && ta.a.split_epi) {
       // The epilogue CTAs must fit beside the layer kernel's on the same SM: that needs the same split between
       // L1 and shared memory, i.e. the largest shared-memory carve-out, although they use only 5 KB of it.
-      static bool carve_set = false;
-      if (!carve_set) {
+      static DevOnce carve{};
+      if (sps_first_on_device(carve)) {
         e = cudaFuncSetAttribute(lin_epilogue_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        carve_set = true;
       }
       e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
     }
@@ -1315,6 +1312,13 @@ static __device__ __align__(256) unsigned char g_static_scratch[SPS_STATIC_CTR_B
 
 extern "C" int64_t sps_linear_static_max_floats(void) { return (int64_t)SPS_STATIC_PART_FLOATS; }
 
+extern "C" int64_t sps_linear_static_floats_needed(int32_t dtype, int32_t M, int32_t N, int32_t D) {
+  if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || (dtype != 0 && dtype != 1) || (dtype == 1 && D % 128)) return -1;
+  int dev = 0, num_sm = SPS_NUM_SM_FALLBACK;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&num_sm, cudaDevAttrMultiProcessorCount, dev);
+  return (int64_t)lin_part_floats(N, lin_plan(dtype, M, N, D, num_sm).S);
+}
+
 extern "C" int sps_linear_static(const void* W, int32_t dtype, const float* X, int32_t M, int32_t N, int32_t D, float* Y,
                                  void* stream) {
   if (!W || !X || !Y) { sps_set_global_error("null argument"); return SPS_EINVAL; }
@@ -1327,7 +1331,7 @@ extern "C" int sps_linear_static(const void* W, int32_t dtype, const float* X, i
   cudaDeviceGetAttribute(&num_sm, cudaDevAttrMultiProcessorCount, dev);
   const LinPlan p = lin_plan(dtype, M, N, D, num_sm);
   if (lin_part_floats(N, p.S) > (size_t)SPS_STATIC_PART_FLOATS) {
-    sps_set_global_error("shape needs more split-K scratch than the static array holds (N * splits * 16 floats > 4 Mi floats)");
+    sps_set_global_error("shape needs more split-K scratch than the static array holds (sps_linear_static_floats_needed > sps_linear_static_max_floats)");
     return SPS_EINVAL;
   }
   // set-up, once per device, with that device current: the device address of the static array
@@ -1348,9 +1352,10 @@ extern "C" int sps_linear_static(const void* W, int32_t dtype, const float* X, i
   a.counters = reinterpret_cast<int*>(base[dev]);
   a.part = reinterpret_cast<float*>(base[dev] + SPS_STATIC_CTR_BYTES);
   cudaStream_t st = (cudaStream_t)stream;
-  // The array keeps the last call's contents.  Partial sums are overwritten before they are read and
-  // the kernel re-arms its own counters; the sticky error word is the one thing that must start at zero.
-  e = cudaMemsetAsync(a.counters + 2 * LIN_MAX_R + 1, 0, sizeof(int), st);
+  // The array keeps the last call's contents.  Partial sums are overwritten before they are read.  The
+  // counters (arrival counts, tile queues, the sticky error word) must start at zero: the kernel re-arms
+  // them itself on the way out, but a call that gave up on a wait may not have, so they are cleared here.
+  e = cudaMemsetAsync(a.counters, 0, SPS_STATIC_CTR_BYTES, st);
   if (e == cudaSuccess) e = lin_launch(dtype, a, p, st);
   if (e != cudaSuccess) { sps_set_global_error(cudaGetErrorString(e)); return SPS_ECUDA; }
   return SPS_OK;

@@ -302,10 +302,11 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
   uint32_t step = a.step;
   int top_k = a.top_k;
   float top_p = a.top_p;
-  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; }
+  uint32_t seq = (uint32_t)b;   // Philox sequence index
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; seq += a.st->seq0; }
   const float invT = 1.0f / T;
   const float* row = a.logits + (long long)b * a.ld;
-  const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, a.t);
+  const Uniforms u = sps_uniforms(seed, seq, step, a.t);
   int tok;
   if ((top_k >= 1 && top_k < a.V) || top_p < 1.0f) {
     // filtered draw: tokens under the cut weigh nothing
@@ -366,15 +367,10 @@ static size_t weights_smem(int V) {
   return bytes <= 200 * 1024 ? bytes : 0;
 }
 template <class Kern>
-static cudaError_t sampler_smem_attr(Kern k, size_t bytes, size_t& cached) {
-  if (bytes <= cached) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) cached = bytes;
-  return e;
-}
+static cudaError_t sampler_smem_attr(Kern k, size_t bytes, DevSmemCache& cached) { return sps_ensure_smem(k, bytes, cached); }
 
 cudaError_t sample_launch(const SampleArgs& a_in, cudaStream_t st) {
-  static size_t cached = 48 * 1024;
+  static DevSmemCache cached{};
   SampleArgs a = a_in;
   const size_t smem = weights_smem(a.V);
   a.smem_weights = smem ? 1 : 0;
@@ -407,7 +403,8 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   uint32_t step = a.step;
   int top_k = a.top_k;
   float top_p = a.top_p;
-  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; }
+  uint32_t seq = (uint32_t)b;   // Philox sequence index
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; top_k = a.st->top_k; top_p = a.st->top_p; seq += a.st->seq0; }
   const bool filt = (top_k >= 1 && top_k < V) || top_p < 1.0f;
   const float invT = 1.0f / T;
   const float* qrow = a.q_logits + (long long)b * (K + 1) * V;
@@ -466,7 +463,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     const float pd = lp >= s_cut[K + 1 + t] ? expf((lp - s_max[K + 1 + t]) * invT) / s_sum[K + 1 + t] : 0.f;
     // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
     const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
-    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)t);
+    const Uniforms u = sps_uniforms(seed, seq, step, (uint32_t)t);
     // measurement mode only: accept with a fixed probability whatever the models say (tokens per loop as a function
     // of the acceptance rate alone); the emitted tokens then follow no particular law
     if (forced > 0.f) return u.u_acc < forced;
@@ -501,7 +498,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     const float* pl = prow + (long long)stop * V;
     const float mq = s_max[stop], mp = s_max[K + 1 + stop];
     const float iq = 1.0f / s_sum[stop], ip = 1.0f / s_sum[K + 1 + stop];
-    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)stop);
+    const Uniforms u = sps_uniforms(seed, seq, step, (uint32_t)stop);
     const float cq = s_cut[stop], cp = s_cut[K + 1 + stop];
     auto wres = [&](int i) {
       const float lq = ql[i], lp = pl[i];
@@ -527,7 +524,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
     // ---- every draft accepted: extra token from the (K+1)-th target distribution
     const float* ql = qrow + (long long)K * V;
     const float mq = s_max[K], cq = s_cut[K];
-    const Uniforms u = sps_uniforms(seed, (uint32_t)b, step, (uint32_t)K);
+    const Uniforms u = sps_uniforms(seed, seq, step, (uint32_t)K);
     auto wq = [&](int i) { const float lq = ql[i]; return lq >= cq ? expf((lq - mq) * invT) : 0.f; };
     if (a.smem_weights) {
       for (int i = tid; i < V; i += SAMPLER_THREADS) ws[skew(i)] = wq(i);
@@ -568,7 +565,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
 }
 
 cudaError_t accept_launch(const AcceptArgs& a_in, cudaStream_t st) {
-  static size_t cached = 48 * 1024;
+  static DevSmemCache cached{};
   AcceptArgs a = a_in;
   const size_t smem = weights_smem(a.V);
   a.smem_weights = smem ? 1 : 0;

@@ -69,15 +69,15 @@ __device__ __forceinline__ uint32_t w_mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok;
 }
-// bounded wait: false (and error word 3) after 2 s
-__device__ __forceinline__ bool w_mbar_wait(uint32_t bar, uint32_t parity, int* err) {
+// bounded wait: false (and error word 3) after limit_ns of the global timer (2 s unless a test shortened it)
+__device__ __forceinline__ bool w_mbar_wait(uint32_t bar, uint32_t parity, int* err, unsigned long long limit_ns) {
   if (w_mbar_try(bar, parity)) return true;
   const unsigned long long t0 = w_timer();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 128; ++i)
       if (w_mbar_try(bar, parity)) return true;
-    if (w_timer() - t0 > 2000000000ull) {
+    if (w_timer() - t0 > limit_ns) {
       atomicExch(err, 3);
       return false;
     }
@@ -160,6 +160,8 @@ struct WideGemmArgs {
   __nv_bfloat16 *yhi, *ylo;
   const float* scale[3];
   int* err;
+  unsigned long long wait_ns;   // bound of every wait inside the kernel
+  int drop_stage;               // >= 0: CTA (0, 0)'s producer leaves out that k-block (test hook); -1 = none
 };
 
 template <int MR>
@@ -219,8 +221,9 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
       int issued = 0;
       for (int kb = 0; kb < kb_n && ok; ++kb, ++issued) {
         const int st = kb % WIDE_STAGES, use = kb / WIDE_STAGES;
-        if (use > 0 && !w_mbar_wait(bar_empty + 8 * st, (uint32_t)(use - 1) & 1u, a.err)) { ok = false; break; }
+        if (use > 0 && !w_mbar_wait(bar_empty + 8 * st, (uint32_t)(use - 1) & 1u, a.err, a.wait_ns)) { ok = false; break; }
         if (*s_abort) { ok = false; break; }
+        if (tile == 0 && s == 0 && kb >= pre && kb == a.drop_stage) continue;   // test hook: nothing is asked for, the MMA warp's wait runs out
         const uint32_t dst = ring + st * WIDE_STAGE_BYTES;
         const int k = (kb0 + kb) * WIDE_BK;
         if (kb >= pre) w_mbar_expect_tx(bar_full + 8 * st, WIDE_STAGE_BYTES);
@@ -232,7 +235,8 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
         *s_abort = 1;
         // let the copies already issued land before this CTA's shared memory goes away
         for (int j = max(0, issued - WIDE_STAGES); j < issued; ++j)
-          w_mbar_wait(bar_full + 8 * (j % WIDE_STAGES), (uint32_t)(j / WIDE_STAGES) & 1u, a.err);
+          if (!(tile == 0 && s == 0 && j >= pre && j == a.drop_stage))
+            w_mbar_wait(bar_full + 8 * (j % WIDE_STAGES), (uint32_t)(j / WIDE_STAGES) & 1u, a.err, a.wait_ns);
       }
     }
   } else if (warp == 1) {
@@ -240,7 +244,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
       bool ok = true;
       for (int kb = 0; kb < kb_n && ok; ++kb) {
         const int st = kb % WIDE_STAGES, use = kb / WIDE_STAGES;
-        if (!w_mbar_wait(bar_full + 8 * st, (uint32_t)use & 1u, a.err) || *s_abort) { ok = false; break; }
+        if (!w_mbar_wait(bar_full + 8 * st, (uint32_t)use & 1u, a.err, a.wait_ns) || *s_abort) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = ring + st * WIDE_STAGE_BYTES;
         const uint64_t d_hi = umma_desc(sa), d_lo = umma_desc(sa + WIDE_A_BYTES), d_w = umma_desc(sa + 2 * WIDE_A_BYTES);
@@ -259,7 +263,7 @@ __global__ void __launch_bounds__(192, 1) wide_gemm_kernel(const __grid_constant
     // epilogue warps 2..5: tensor-memory lanes 32 q .. 32 q + 31 with q = warp % 4.  A 128-row accumulator keeps row i
     // in lane i; a 64-row one keeps 16 rows in the first 16 lanes of each of the four lane quarters.
     const int q = warp & 3, row = MR == 128 ? q * 32 + lane : (lane < 16 ? q * 16 + lane : WIDE_M);
-    bool ok = w_mbar_wait(bar_acc, 0u, a.err) && !*s_abort;
+    bool ok = w_mbar_wait(bar_acc, 0u, a.err, a.wait_ns) && !*s_abort;
     ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
@@ -630,6 +634,7 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   }
   a.part = part; a.M = M; a.N = N; a.D = D; a.S = wide_splits_tiles(tiles, D, num_sm); a.err = err;
   a.w_is_output = scales ? 1 : 0;
+  { const WaitKnobs wk = sps_wait_knobs(); a.wait_ns = wk.limit_ns; a.drop_stage = wk.drop_stage; }
   // four columns per access when every matrix, stride and pointer allows 16-byte (8-byte for bf16) accesses
   int vec = ((N | a.rows_mat[0] | a.rows_mat[1] | a.rows_mat[2] | ldp) & 3) == 0 && (ldy & 3) == 0 &&
             (((uintptr_t)part | (uintptr_t)y | (uintptr_t)yhi | (uintptr_t)ylo) & 15) == 0;
@@ -637,12 +642,9 @@ cudaError_t wide_gemm_launch_stacked(const void* const* Ws, const int* rows, int
   a.fused = a.S == 1 ? 1 : 0; a.mode = mode; a.vec = vec; a.ldp = ldp; a.y = y; a.ldy = ldy;
   a.yhi = reinterpret_cast<__nv_bfloat16*>(yhi); a.ylo = reinterpret_cast<__nv_bfloat16*>(ylo);
   for (int i = 0; i < 3; ++i) a.scale[i] = (scales && i < nmat) ? scales[i] : nullptr;
-  static bool attr = false;
-  if (!attr) {
-    if ((e = cudaFuncSetAttribute(wide_gemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<64>::SMEM)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(wide_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WideCfg<128>::SMEM)) != cudaSuccess) return e;
-    attr = true;
-  }
+  static DevSmemCache c64{}, c128{};   // the attribute is per device
+  if ((e = sps_ensure_smem(wide_gemm_kernel<64>, WideCfg<64>::SMEM, c64)) != cudaSuccess) return e;
+  if ((e = sps_ensure_smem(wide_gemm_kernel<128>, WideCfg<128>::SMEM, c128)) != cudaSuccess) return e;
   if (mr == 64) e = launch_k(wide_gemm_kernel<64>, dim3(tiles, a.S), dim3(192), WideCfg<64>::SMEM, st, a);
   else e = launch_k(wide_gemm_kernel<128>, dim3(tiles, a.S), dim3(192), WideCfg<128>::SMEM, st, a);
   if (e != cudaSuccess || a.fused) return e;

@@ -126,11 +126,11 @@ def test_generate_with_filters_matches_oracle_tokens(top_k, top_p, T):
     else:
         osps.set_sampling(top_k, top_p)
         oT = T
+    from gpu_util import oracle_generate, same_or_flagged
     for K in (0, 3):
         got, st = h.sps_generate(prompt, 24, K, T, 11)
-        want = osps.generate(prompt, 24, K, oT, 11)
-        if (got != want["tokens"]).any():
-            assert want["flags"] & NEAR, (K, got, want["tokens"])
+        # a difference is only legitimate from the first flagged near tie (accept test, CDF edge, nucleus cut) on
+        same_or_flagged(got, oracle_generate(osps, prompt, 24, K, oT, 11, near=NEAR))
         if T == 0.0:
             again, _ = h.sps_generate(prompt, 24, K, T, 12345)     # greedy output does not depend on the seed
             assert (again == got).all()
@@ -146,13 +146,8 @@ def test_batch_with_nucleus_equals_independent_sequences():
     got, st = h.sps_generate_batch(prompts, 24, 3, 0.9, 11)
     osps = oracle.Sps(ot, od)
     osps.set_sampling(12, 0.9)
-    ok = 0
-    for b in range(3):
-        want = osps.generate(prompts[b], 24, 3, 0.9, 11, b=b)
-        if (got[b] == want["tokens"]).all():
-            ok += 1
-        else:
-            assert want["flags"] & NEAR
+    from gpu_util import oracle_generate, same_or_flagged
+    ok = sum(same_or_flagged(got[b], oracle_generate(osps, prompts[b], 24, 3, 0.9, 11, b=b, near=NEAR)) for b in range(3))
     assert ok >= 2
     h.close()
 
@@ -183,11 +178,12 @@ def test_adaptive_lookahead_matches_oracle_tokens_and_loop_count():
     prompt = sps_synth.make_prompt(5, 20, V)
     osps = oracle.Sps(ot, od)
     for (kmin, kmax, T) in [(1, 6, 1.0), (2, 4, 0.7), (3, 3, 1.0)]:
+        from gpu_util import oracle_generate, same_or_flagged
         got, st = h.sps_generate_adaptive(prompt, 40, kmin, kmax, T, 21)
         want = osps.generate_adaptive(prompt, 40, kmin, kmax, T, 21)
-        if (got != want["tokens"]).any():
-            assert want["flags"] & NEAR, (kmin, kmax, got, want["tokens"])
-        else:
+        by_loop = oracle_generate(osps, prompt, 40, kmax, T, 21, near=NEAR, K_min=kmin)
+        assert np.array_equal(by_loop["tokens"], want["tokens"]) and by_loop["loops"] == want["loops"]
+        if same_or_flagged(got, by_loop):
             assert st["loops"] == want["loops"] and st["draft_calls"] == want["draft_calls"]
     with pytest.raises(sps.SpsError):
         h.sps_generate_adaptive(prompt, 8, 0, 4, 1.0, 0)

@@ -35,9 +35,42 @@ def test_static_scratch_matches_workspace_version_twice(N, D, M, dt):
         assert torch.equal(got, want)
 
 
+def test_static_scratch_serves_alternating_shapes_without_allocating():
+    """Two shapes with different numbers of k-splits and row ranges take turns on the one shared array: each call
+    must find the counters and tile queues as it needs them, whatever the previous call's shape left behind.  Free
+    device memory does not move across the calls (the entry point allocates nothing)."""
+    g = torch.Generator(device=DEV).manual_seed(99)
+    shapes = [(4099, 2048, 5), (1024, 8192, 3), (777, 1024, 12)]
+    data = []
+    for N, D, M in shapes:
+        W = (torch.randn((N, D), device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+        X = torch.randn((M, D), device=DEV, generator=g)
+        ws = torch.zeros(sps.sps_linear_workspace_bytes(1, M, N, D), dtype=torch.uint8, device=DEV)
+        want = torch.empty((M, N), device=DEV)
+        sps.sps_linear(W, X, want, ws)
+        need = sps.sps_linear_static_floats_needed(1, M, N, D)
+        assert 0 < need <= sps.sps_linear_static_max_floats() and need % (16 * N) == 0
+        data.append((W, X, want, torch.empty((M, N), device=DEV)))
+    sps.sps_linear_static(*data[0][:2], data[0][3])      # first call on the device: resolves the array's address
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for rnd in range(3):
+        for W, X, want, got in data:
+            got.fill_(float("nan"))
+            sps.sps_linear_static(W, X, got)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()     # read before any torch op that might take memory for a temporary
+        assert free1 == free0
+        for W, X, want, got in data:
+            assert torch.equal(got, want), rnd
+        free0, _ = torch.cuda.mem_get_info()
+
+
 def test_static_scratch_rejects_oversized_shapes():
-    # N * splits * 16 floats must fit the array: 65536 rows with 16 splits do not
+    # the split-K scratch the shape needs must fit the array: 65536 rows with 16 splits do not
     assert sps.sps_linear_static_max_floats() == 4 << 20
+    assert sps.sps_linear_static_floats_needed(1, 1, 65536, 32768) > sps.sps_linear_static_max_floats()
+    assert sps.sps_linear_static_floats_needed(1, 1, 8, 100) == -1          # bf16 needs D % 128 == 0
     W = torch.zeros((8, 128), device=DEV, dtype=torch.bfloat16)
     X = torch.zeros((1, 128), device=DEV)
     Y = torch.zeros((1, 8), device=DEV)
