@@ -36,9 +36,6 @@ import sps_synth  # noqa: E402
 
 METRIC = "batch-1 tokens/s SpS vs AR decode; verify-pass HBM GB/s vs peak"
 UNIT = "tokens/s"
-# mean tokens per speculative loop measured by this bench's own arm on each workload (seeded weights and
-# prompts make it repeatable); the CPU arm cannot run whole generations of the 70B pair, so it uses these
-ASSUMED_TOKENS_PER_LOOP = {"70b": 1.295, "mid": 1.9, "tiny": 3.0, "tiny_bf16": 3.0}
 
 
 def measured_peaks():
@@ -114,37 +111,109 @@ def kv_bytes_per_token(cfg):
 
 
 # ----------------------------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample_seconds(c, K, wt_layer, wd_layer, wt_unembed, wd_unembed, P):
-    """Time the oracle, as it stands, on the pieces one loop is made of: one target layer over K+1 rows,
-    the target unembedding over K+1 rows, one draft layer and the draft unembedding over 1 row."""
+class PinnedStage:
+    """Reusable pinned host buffers for reading a layer's matrices back from the device (one per matrix name)."""
+
+    def __init__(self):
+        self.buf = {}
+
+    def numpy(self, name, t):
+        """`t` (device tensor, fp32 or bf16) as the numpy array the oracle reads; the array aliases a pinned buffer that
+        the next call with the same name overwrites."""
+        src = t.view(torch.int16) if t.dtype == torch.bfloat16 else t
+        key = (name, src.dtype)
+        if key not in self.buf or self.buf[key].numel() < src.numel():
+            self.buf[key] = torch.empty(src.numel(), dtype=src.dtype, pin_memory=True)
+        dst = self.buf[key][:src.numel()].view(src.shape)
+        dst.copy_(src)
+        a = dst.numpy()
+        return a.view(np.uint16) if t.dtype == torch.bfloat16 else a
+
+
+def oracle_full_pass(cfg, w_dev, tokens, stage):
+    """One pass of the oracle over ALL layers of a device-resident model, the weights read back one layer at a time:
+    rows `tokens` at positions 0 .. len - 1 with an empty cache.  Returns (logits float64 [rows, V], oracle seconds,
+    read-back seconds).  An int8 model is the fp32 model of its dequantised matrices with a bf16 cache."""
     import oracle
-    tc, dc = c["target"], c["draft"]
-    rng = np.random.default_rng(0)
-    out = {}
-    for tag, mc, lw, un, rows in (("target", tc, wt_layer, wt_unembed, K + 1), ("draft", dc, wd_layer, wd_unembed, 1)):
-        if mc["dtype"] == 2:     # int8 weights: the oracle runs the dequantised fp32 model with a bf16 cache
-            m = oracle.Transformer(dict(mc, n_layers=1, dtype=0), None, P + K + 2, cache_dtype=1)
-        else:
-            m = oracle.Transformer(dict(mc, n_layers=1), None, P + K + 2)
-        emb = un[rng.integers(0, mc["vocab"], rows)]
-        pos = np.arange(P - 1, P - 1 + rows, dtype=np.int32)
-        m.begin_rows(np.ascontiguousarray(emb), pos)
+    q8 = cfg["dtype"] == 2
+    tok = torch.from_numpy(np.asarray(tokens, dtype=np.int64)).to(w_dev["tok_embed"].device)
+    pos = np.arange(len(tokens), dtype=np.int32)
+    emb = w_dev["tok_embed"][tok]
+    m = oracle.Transformer(dict(cfg, dtype=0), None, len(tokens) + 1, cache_dtype=1) if q8 else oracle.Transformer(cfg, None, len(tokens) + 1)
+    t_orc = t_copy = 0.0
+    t0 = time.perf_counter()
+    m.begin_rows(emb.float().cpu().numpy() if q8 else sps_synth.to_numpy(emb), pos)
+    t_orc += time.perf_counter() - t0
+    for l, lw in enumerate(w_dev["layers"]):
         t0 = time.perf_counter()
-        m.layer(0, lw)
+        if q8:
+            one = layer_numpy(lw)
+        else:
+            one = {k: stage.numpy(k, v) for k, v in lw.items()}
         t1 = time.perf_counter()
-        m.end(np.ones(mc["d_model"], dtype=np.float32), un)
+        m.layer(l, one)
         t2 = time.perf_counter()
-        out[tag + "_layer_s"] = t1 - t0
-        out[tag + "_unembed_s"] = t2 - t1
-        m.close()
-    return out
+        t_copy += t1 - t0
+        t_orc += t2 - t1
+    t0 = time.perf_counter()
+    un = unembed_numpy(w_dev) if q8 else stage.numpy("unembed", w_dev["unembed"])
+    t1 = time.perf_counter()
+    out = m.end(w_dev["final_norm"].cpu().numpy(), un)
+    t_orc += time.perf_counter() - t1
+    t_copy += t1 - t0
+    m.close()
+    return out, t_orc, t_copy
 
 
-def oracle_loop_seconds(c, K, s):
-    tc, dc = c["target"], c["draft"]
-    verify = tc["n_layers"] * s["target_layer_s"] + s["target_unembed_s"]
-    draft_row = dc["n_layers"] * s["draft_layer_s"] + s["draft_unembed_s"]
-    return verify + (K + 1) * draft_row if K > 0 else verify / (K + 1)
+def cpu_baseline_full(h, c, wt, wd, K, tokens_per_loop, dev):
+    """The oracle, as it stands, on ONE FULL scoring step of the bench's target (all layers, K + 1 rows) and one full
+    draft step (all layers, one row), on the machine's host cores, with the very weights the GPU arm uses (read back
+    layer by layer); the library scores the same rows so that the logit error is reported beside the time."""
+    import oracle
+    V = c["target"]["vocab"]
+    rows = np.concatenate([sps_synth.make_prompt(0, 1, V), sps_synth.make_prompt(1, K, V)])      # x_0, then K draft tokens
+    stage = PinnedStage()
+    want, t_verify, t_copy = oracle_full_pass(c["target"], wt, rows, stage)
+    h.sps_reset()
+    h.sps_prefill(rows[:1])                      # a one-token sequence: nothing cached, the scoring rows sit at positions 0 .. K
+    out = torch.zeros((K + 1, V), device=dev)
+    h.sps_score(0, rows, out)
+    err = float(np.abs(out.cpu().numpy().astype(np.float64) - want).max())
+    _, t_draft, t_copy_d = oracle_full_pass(c["draft"], wd, rows[:1], stage) if K > 0 else (None, 0.0, 0.0)
+    loop_s = t_verify + K * t_draft
+    tl, dl = c["target"]["n_layers"], c["draft"]["n_layers"]
+    return {"value": tokens_per_loop / loop_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": (f"one full scoring step of the oracle: {tl} of {tl} target layers + unembedding over {K + 1} rows "
+                       f"(positions 0..{K}; the mat-vecs are >99.9% of its work at any context), {t_verify:.1f} s; one full draft step: "
+                       f"{dl} of {dl} layers + unembedding over 1 row, {t_draft:.2f} s, counted {K} times; weights read back from the "
+                       f"device layer by layer ({t_copy + t_copy_d:.1f} s, not counted); divided into the GPU arm's measured "
+                       f"{tokens_per_loop:.3f} tokens per loop on the same models and seeds"),
+            "seconds": {"verify_step": t_verify, "draft_step": t_draft, "loop": loop_s, "weight_readback": t_copy + t_copy_d},
+            "logit_max_abs_err_vs_gpu": err, "logit_tolerance": 5e-2 if c["target"]["dtype"] >= 1 else 1e-3}
+
+
+def oracle_loop_sample(c, K, models, seed, step):
+    """One iteration of Algorithm 2 by the oracle on a depth-reduced pair (full widths and vocabulary), in pieces so that
+    the draft steps and the scoring step are timed apart: K draft steps (one row each after the first), one scoring
+    step over K + 1 rows, then the oracle's accept chain on its own logits.  Returns (draft seconds, scoring seconds,
+    tokens emitted)."""
+    import oracle
+    ot, od, prefix = models
+    n = len(prefix)
+    V = c["target"]["vocab"]
+    drafts, p_rows = [], []
+    t0 = time.perf_counter()
+    for t in range(K):
+        tok = prefix[-1] if t == 0 else drafts[-1]
+        lg = od.forward(np.array([tok], dtype=np.int32), np.array([n - 1 + t], dtype=np.int32))[0]
+        d, _ = oracle.sample_row(lg, 1.0, oracle.uniforms(seed, 0, step, t)[0])
+        drafts.append(d); p_rows.append(lg)
+    t1 = time.perf_counter()
+    rows = np.array([prefix[-1]] + drafts, dtype=np.int32)
+    q = ot.forward(rows, np.arange(n - 1, n + K, dtype=np.int32))
+    t2 = time.perf_counter()
+    r = oracle.accept_chain(q, np.stack(p_rows) if K else np.zeros((0, V), np.float32), drafts, 1.0, seed, 0, step)
+    return t1 - t0, t2 - t1, r["n_accepted"] + 1
 
 
 def layer_numpy(lw):
@@ -167,7 +236,11 @@ DTYPE_NAME = {0: "fp32", 1: "bf16", 2: "int8-weight (row scales, fp16 activation
 
 
 def run_reference(args):
-    """--impl reference: the CPU oracle on the host cores, a bounded sample per step."""
+    """--impl reference: the CPU oracle on the host cores (no GPU work).  Every step is one real iteration of
+    Algorithm 2 by the oracle on a depth-reduced pair -- one target layer and one draft layer at the bench's full
+    widths and vocabulary, random-init by the bench's recipe -- timed in its two phases; each phase is scaled to the
+    full pair by the weight bytes a pass streams (the oracle's time is its mat-vecs'), and the tokens per loop are
+    the oracle's own emitted counts.  Seconds per loop and the scale factors are in the line."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -176,26 +249,39 @@ def run_reference(args):
     c = sps_synth.CONFIGS[cfgname]
     K, P, n_new = args.K, c["prompt_len"], c["n_new"]
     tc, dc = c["target"], c["draft"]
-    one_t = sps_synth.make_weights(dict(tc, n_layers=1), seed=0, tag="target", device="cpu")
-    one_d = sps_synth.make_weights(dict(dc, n_layers=1), seed=0, tag="draft", device="cpu")
-    lt, ld = layer_numpy(one_t["layers"][0]), layer_numpy(one_d["layers"][0])
-    ut, ud = unembed_numpy(one_t), unembed_numpy(one_d)
-    times = []
+    tc1, dc1 = dict(tc, n_layers=min(1, tc["n_layers"])), dict(dc, n_layers=min(1, dc["n_layers"]))
+    one_t = sps_synth.make_weights(tc1, seed=0, tag="target", device="cpu")
+    one_d = sps_synth.make_weights(dc1, seed=0, tag="draft", device="cpu", share_embed_from=one_t if cfgname.startswith("70b") else None)
+
+    def orc(cfg1, w):
+        if cfg1["dtype"] == 2:
+            return oracle.Transformer(dict(cfg1, dtype=0), sps_synth.dequantized_numpy(w), 16 + K, cache_dtype=1)
+        return oracle.Transformer(cfg1, sps_synth.weights_to_numpy(w), 16 + K)
+    ot, od = orc(tc1, one_t), orc(dc1, one_d)
+    prefix = [int(t) for t in sps_synth.make_prompt(0, 4, tc["vocab"])]
+    pre = np.array(prefix[:-1], dtype=np.int32)
+    ot.forward(pre, np.arange(len(pre)), want_logits=False)
+    od.forward(pre, np.arange(len(pre)), want_logits=False)
+    scale_t = sps_synth.weight_bytes(tc) / sps_synth.weight_bytes(tc1)
+    scale_d = sps_synth.weight_bytes(dc) / sps_synth.weight_bytes(dc1)
+    loop_s, emitted = [], []
     for i in range(args.warmup + args.steps):
-        s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
+        td, tv, e = oracle_loop_sample(c, K, (ot, od, prefix), seed=i, step=i)
         if i >= args.warmup:
-            times.append(oracle_loop_seconds(c, K, s))
-    loop_s = statistics.mean(times)
-    tpl = ASSUMED_TOKENS_PER_LOOP.get(cfgname, 1.0) if K > 0 else 1.0
-    value = tpl / loop_s
-    sample = (f"per step: 1 of {tc['n_layers']} target layers over {K + 1} rows + target unembedding + 1 of "
-              f"{dc['n_layers']} draft layers and draft unembedding over 1 row, context {P}; scaled to one loop "
-              f"(x layers, x{K + 1} draft rows) at {tpl} tokens per loop")
+            loop_s.append(td * scale_d + tv * scale_t)
+            emitted.append(e)
+    mean_loop, tpl = statistics.mean(loop_s), statistics.mean(emitted)
+    value = tpl / mean_loop
+    sample = (f"per step: one iteration of Algorithm 2 by the oracle on a depth-reduced pair (1 of {tc['n_layers']} target layers, 1 of "
+              f"{dc['n_layers']} draft layers, full widths and vocabulary, context {len(prefix)}): {K} draft steps, one scoring step over "
+              f"{K + 1} rows, accept chain; phase times scaled by streamed weight bytes (target x{scale_t:.1f}, draft x{scale_d:.1f}); "
+              f"tokens per loop = the oracle's own mean emitted count ({tpl:.2f})")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * loop_s * (n_new / tpl), "higher_is_better": True,
+            "warmup": args.warmup, "ms_per_step": 1e3 * mean_loop * (n_new / tpl), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": workload_name(cfgname, K, P, n_new)},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample,
+                             "seconds_per_loop": mean_loop, "tokens_per_loop": tpl},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -283,8 +369,8 @@ def run_ours(args):
                 "achieved": v_gbs, "peak": peak, "unit": "GB/s", "frac": (v_gbs / peak) if v_gbs else None,
                 "frac_of_8000_nominal": (v_gbs / 8000.0) if v_gbs else None, "peak_source": peak_src,
                 "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
-                # profiles/lin_bf16_tma_32000x8192_M5.md: dram read + write = 1.0096 x the algorithmic bytes of that launch;
-                # traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
+                # one ncu capture of this kernel on the 32000 x 8192 layer: dram read + write = 1.0096 x the algorithmic bytes of
+                # that launch; traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
                 "traffic": args.traffic if args.traffic is not None else
                 (1.0096 * vbytes / n_lin_verify if c["target"]["dtype"] == 1 else None)}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -332,18 +418,7 @@ def run_ours(args):
                           "frac": ar_gbs / peak}
             line["speedup_vs_ar"] = value / ar_tps
         if not args.no_cpu:
-            import oracle
-            lt = layer_numpy(wt["layers"][0])
-            ld = layer_numpy(wd["layers"][0])
-            ut, ud = unembed_numpy(wt), unembed_numpy(wd)
-            s = oracle_sample_seconds(c, K, lt, ld, ut, ud, P)
-            loop_s = oracle_loop_seconds(c, K, s)
-            tpl = emitted / loops if K > 0 else 1.0
-            line["cpu_baseline"] = {"value": tpl / loop_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                                    "sample": (f"oracle timed on 1 of {c['target']['n_layers']} target layers over {K + 1} rows + "
-                                               f"target unembedding + 1 of {c['draft']['n_layers']} draft layers + draft "
-                                               f"unembedding over 1 row (context {P}), scaled to one loop and divided into the "
-                                               f"measured {tpl:.3f} tokens per loop"), "seconds": s}
+            line["cpu_baseline"] = cpu_baseline_full(h, c, wt, wd, K, emitted / loops if K > 0 else 1.0, dev)
     if rank == 0 and world == 1 and args.batch > 1 and c["target"]["dtype"] == 1:
         # the K / batch sweep's corner: `batch` sequences decoded together, batch x (K + 1) rows per scoring pass
         # (above 16 rows the linear layers run as tcgen05 GEMMs); aggregate tokens/s over the batch
@@ -437,6 +512,8 @@ def run_ours(args):
     h.close()
     if rank == 0 and world == 1 and args.sweep and c["target"]["dtype"] == 1:
         line["sweep"] = sweep_bench(sps, c, wt, wd, local, peak)
+    if rank == 0 and world == 1 and args.mid_steps > 0 and cfgname != "mid":
+        line.setdefault("variants", {})["mid"] = pair_variant(sps, "mid", local, peak, args.mid_steps)
     if rank == 0 and world == 1 and not args.no_sampler:
         line["sampler"] = sampler_bench(dev, peak)
     if rank == 0:
@@ -444,6 +521,39 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def pair_variant(sps, cfgname, local, peak, steps):
+    """Another pair of the workload table through the same calls (the mid-size bf16 pair: 24-layer d 2048 target,
+    6-layer d 1024 draft, prompt 128, 256 new tokens, K = 4, batch 1): tokens/s of speculative and autoregressive
+    decoding, the two passes' device times and their weight bytes over time against the measured HBM rate.  At this
+    size a pass is ~120 launches of 8-33 MB each: what it shows is the fixed cost per layer, not the streaming rate."""
+    dev = f"cuda:{local}"
+    c, wt, wd = build_models(cfgname, dev)
+    P, n_new, K, T, V = c["prompt_len"], c["n_new"], c["K"], c["T"], c["target"]["vocab"]
+    h = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=((P + n_new + K + 63) // 64) * 64, max_batch=1, max_K=K, device=local)
+
+    def run(k, n):
+        sts = []
+        for i in range(n):
+            sts.append(h.sps_generate(sps_synth.make_prompt(500 + i, P, V), n_new, k, T, 500 + i)[1])
+        return sts
+    run(K, 2); run(0, 1)
+    st, ar = run(K, steps), run(0, max(1, steps // 2))
+    h.close()
+    loops = sum(x["loops"] for x in st)
+    ms_dec, ms_v, ms_d = sum(x["ms_decode"] for x in st), sum(x["ms_verify"] for x in st), sum(x["ms_draft"] for x in st)
+    tps = len(st) * n_new / (ms_dec / 1e3)
+    ar_tps = len(ar) * n_new / (sum(x["ms_decode"] for x in ar) / 1e3)
+    ctx = P + n_new / 2.0
+    vb = sps_synth.weight_bytes(c["target"]) + kv_bytes_per_token(c["target"]) * ctx
+    db = sps_synth.weight_bytes(c["draft"]) + kv_bytes_per_token(c["draft"]) * ctx
+    v_gbs, d_gbs = vb * loops / (ms_v / 1e3) / 1e9, db * loops * K / (ms_d / 1e3) / 1e9
+    return {"workload": workload_name(cfgname, K, P, n_new), "value": tps, "unit": UNIT, "ar": ar_tps, "speedup_vs_ar": tps / ar_tps,
+            "tokens_per_loop": sum(x["emitted"] for x in st) / loops, "accept_rate": sum(x["accepted"] for x in st) / (loops * K),
+            "ms_verify_per_loop": ms_v / loops, "ms_draft_per_step": ms_d / (loops * K), "ms_accept_per_loop": sum(x["ms_accept"] for x in st) / loops,
+            "verify_gbs": v_gbs, "verify_frac": v_gbs / peak, "draft_gbs": d_gbs, "draft_frac": d_gbs / peak,
+            "ar_frac": sps_synth.weight_bytes(c["target"]) * ar_tps / 1e9 / peak, "kernel_launches_per_loop": sum(x["kernel_launches"] for x in st) / loops}
 
 
 def sweep_bench(sps, c, wt, wd, local, peak):
@@ -477,8 +587,10 @@ def sweep_bench(sps, c, wt, wd, local, peak):
 
 def sampler_bench(dev, peak_gbs):
     """The fused accept / resample / extra-token kernel alone (vocab 32000, K = 4, target logits N(0, 9), draft =
-    target + N(0, 1)): device time per launch against the time its reads, V * (2K + 1) * 4 bytes per sequence, take
-    at the measured HBM rate.  One CTA per sequence: at batch 1 the kernel is a latency chain on one SM, not a
+    target + N(0, 1)): device time per launch against the time its reads take at the measured HBM rate.  The bound used
+    is the bytes the standalone call must read, V * (2K + 1) * 4 per sequence (K + 1 target rows, K draft rows: 1.15 MB
+    at K = 4); the workload table's V * (K + 1) * 8 (1.28 MB) counts a draft row for the extra position too, which does
+    not exist -- `bound_us_table` gives the time for that figure.  One CTA per sequence: at batch 1 the kernel is a latency chain on one SM, not a
     bandwidth problem, and its 1.15 MB of logits were just written by the two models (L2-resident, as here)."""
     import torch
     import paper_2302_01318_b200 as sps
@@ -510,6 +622,7 @@ def sampler_bench(dev, peak_gbs):
         nbytes = B * (2 * K + 1) * V * 4
         bound_us = nbytes / (peak_gbs * 1e9) * 1e6
         out.append({"B": B, "K": K, "V": V, "us": us, "read_bytes": nbytes, "bound_us": bound_us, "frac": bound_us / us,
+                    "bound_us_table": B * (K + 1) * V * 8 / (peak_gbs * 1e9) * 1e6,
                     "mean_accepted": float(na.float().mean().item())})
     return out
 
@@ -531,6 +644,7 @@ def main():
     ap.add_argument("--k-sweep-seeds", type=int, default=8, help="generations per K in --k-sweep")
     ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")
+    ap.add_argument("--mid-steps", type=int, default=3, help="generations of the mid-size pair reported under variants.mid (0 = skip)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="ncu dram bytes per launch of the dominant kernel; default: bytes_per_launch x the ratio measured in profiles/")
     args = ap.parse_args()
