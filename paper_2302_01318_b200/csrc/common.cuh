@@ -211,13 +211,21 @@ struct LinArgs {
   const float* yp_gain;         // [N] multiplied in before packing, null = ones
   int yp_act;                   // PRO_GELU: gelu before packing; PRO_NONE: none
   int split_epi;                // set by the launcher: the split-K epilogue runs as a kernel of its own
+  // Per-tile epilogue (set by the launcher).  Each 16-row output tile is finished as soon as the last of the
+  // warps that hold a share of it (k-splits x warps of a group) has written its partial sums: that warp adds the
+  // k-splits in split order and stores / adds to the residual stream / packs -- no epilogue kernel, no grid-wide
+  // meeting.  tile_ctr counts the arrivals per tile and is left at zero; the sums of squares of a residual
+  // update are then kept per tile: ssq_out[SSQ_IDX(tile, m)].
+  int tile_epi;
+  int* tile_ctr;                // [ceil(N / 16)] arrival counters, zero between launches
   // int8 weights (dtype 2): W holds signed bytes, row n of matrix i is scaled by wscale[i][n] (fp32, applied to
   // the output); the activations' halves are then fp16, not bf16 -- in the slab and in the packed arrays.
   const float* wscale[3];
   int q8;                       // set by the launcher
 };
 
-struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts; size_t smem; };
+struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts, tile_epi; size_t smem; };
+size_t lin_tile_ctr_ints(int N);           // arrival counters a layer of N output features needs
 LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
 int lin_launch_count(const LinPlan& p);   // kernels one lin_launch enqueues
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
@@ -309,6 +317,15 @@ struct AcceptArgs {
   float temperature; uint64_t seed; uint32_t step;  // used when st == nullptr
   int top_k; float top_p;  // used when st == nullptr (0 / 1 = no filtering)
   int smem_weights;        // set by the launcher: weights are staged in shared memory
+  // (row maximum, sum of exp((l - max) / T)) of each draft row, as the kernel that drew the draft tokens left them:
+  // p_stats[b * p_stats_ld + t].  Null: the accept kernel works them out from p_logits itself.
+  const float2* p_stats;
+  int p_stats_ld;
+  // set by the launcher (cluster form of the kernel): CTAs per sequence, tokens per CTA, rows resident in shared memory
+  int csize, slice, resident, chunk, stages;
 };
 cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);
+// the thread-block-cluster form of the same sampler (unfiltered distributions); falls back to the kernel above when
+// `filtered`, for small vocabularies and for shapes it does not take
+cudaError_t accept_launch_fast(const AcceptArgs& a, bool filtered, cudaStream_t st);
 cudaError_t philox_launch(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out, cudaStream_t st);

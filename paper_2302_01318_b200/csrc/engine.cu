@@ -59,6 +59,10 @@ struct sps_handle {
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
+  float2* p_stats = nullptr; // [max_batch][max_K] (row maximum, sum of exponentials) of each draft row, left by the draft sampler
+  bool filtered = false;     // top-k / nucleus / greedy in force for the calls being made (write_params)
+  int* tile_ctr = nullptr;   // per-tile arrival counters of the linear layers' epilogue (zero between launches)
+  size_t tile_ctr_ints = 0;
   int32_t* res = nullptr;    // device: [n_acc B][flags B][out_tok B*(maxK+1)][err 1]
   int32_t* h_res = nullptr;  // pinned mirror
   HostParams* h_par = nullptr;  // pinned
@@ -224,7 +228,7 @@ int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   ea.x = h->x; ea.ssq = h->ssqA;
   CU(h, embed_launch(ea, st)); h->launches++;
   LinArgs base{};
-  base.part = h->part; base.counters = h->counters; base.eps = c.rms_eps;
+  base.part = h->part; base.counters = h->counters; base.tile_ctr = h->tile_ctr; base.eps = c.rms_eps;
   int nA = 1, nB = 1;   // how many partial sums of squares sit in ssqA / ssqB
   base.err = h->hst.err;
   for (int l = 0; l < c.n_layers; ++l) {
@@ -367,6 +371,7 @@ int enqueue_draft(sps_handle* h, int K) {
     SampleArgs sa{};
     sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = V; sa.B = B; sa.t = (uint32_t)t;
     sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
+    sa.stats = h->p_stats + t; sa.stats_ld = h->hst.max_K;
     CU(h, sample_launch(sa, h->stream)); h->launches++;
   }
   return SPS_OK;
@@ -384,7 +389,9 @@ int enqueue_accept(sps_handle* h, int K) {
   aa.st = h->dst; aa.q_logits = h->q_logits; aa.p_logits = h->p_logits; aa.drafts = h->hst.drafts;
   aa.drafts_ld = h->hst.max_K; aa.B = h->B; aa.K = K; aa.V = h->tgt.cfg.vocab;
   aa.n_acc = h->hst.n_acc; aa.out_tok = h->hst.out_tok; aa.out_ld = h->hst.max_K + 1; aa.flags = h->hst.flags;
-  CU(h, accept_launch(aa, h->stream)); h->launches++;
+  // the draft rows' softmax statistics come from the kernel that drew the drafts (the same numbers the draws used)
+  aa.p_stats = K > 0 ? h->p_stats : nullptr; aa.p_stats_ld = h->hst.max_K;
+  CU(h, accept_launch_fast(aa, h->filtered, h->stream)); h->launches++;
   return SPS_OK;
 }
 
@@ -427,6 +434,7 @@ int write_params(sps_handle* h, float T, uint64_t seed, uint32_t step) {
   h->h_par->seed = seed;
   h->h_par->top_k = greedy ? 1 : h->top_k;
   h->h_par->top_p = greedy ? 1.f : h->top_p;
+  h->filtered = greedy || h->top_k >= 1 || h->top_p < 1.f;
   CU(h, cudaMemcpyAsync(h->dst, h->h_par, sizeof(HostParams), cudaMemcpyHostToDevice, h->stream));
   return SPS_OK;
 }
@@ -444,7 +452,14 @@ int loop_once(sps_handle* h, int K, bool timed) {
   CU(h, cudaMemcpyAsync(h->h_res, h->res, h->res_words * 4, cudaMemcpyDeviceToHost, h->stream));
   CU(h, cudaStreamSynchronize(h->stream));
   h->last_K = K;
-  if (h->h_res[h->res_words - 1] == 3) return fail(h, SPS_ETIMEOUT, "a bounded device-side wait ran out");
+  if (h->h_res[h->res_words - 1] == 3) {
+    // a kernel that gave up may have left arrival counters and tile queues half-way: clear them for the next call
+    cudaMemsetAsync(h->counters, 0, sizeof(int) * (2 * LIN_MAX_R + 2), h->stream);
+    cudaMemsetAsync(h->tile_ctr, 0, sizeof(int) * h->tile_ctr_ints, h->stream);
+    cudaMemsetAsync(h->res + (h->res_words - 1), 0, 4, h->stream);
+    cudaStreamSynchronize(h->stream);
+    return fail(h, SPS_ETIMEOUT, "a bounded device-side wait ran out");
+  }
   if (h->h_res[h->res_words - 1] != 0) return fail(h, SPS_ERANGE, "device flagged a token id or position out of range");
   return SPS_OK;
 }
@@ -649,6 +664,12 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   if (part_floats == 0) part_floats = 1;
   h->res_words = (size_t)MB * 2 + (size_t)MB * (maxK + 1) + 1;
   {
+    int n_max = V;
+    for (const ModelDev* m : {&h->tgt, &h->drf})
+      if (m->present) n_max = std::max(n_max, std::max(m->cfg.d_ff, m->cfg.d_model + 2 * kv_width(m->cfg)));
+    h->tile_ctr_ints = lin_tile_ctr_ints(n_max);
+  }
+  {
     // buffers of the 128-row prompt pass, when a bf16 model is there to use it (SPS_WIDE_PREFILL=0 keeps the 16-row pass)
     static const bool off = [] { const char* e = getenv("SPS_WIDE_PREFILL"); return e && atoi(e) == 0; }();
     size_t wd = 0, wf = 0, wpart = 0, wdq = 0;
@@ -695,6 +716,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->p_logits, sizeof(float) * PR * (size_t)V},
       {(void**)&h->part, sizeof(float) * part_floats},
       {(void**)&h->counters, sizeof(int) * (2 * LIN_MAX_R + 2)},
+      {(void**)&h->tile_ctr, sizeof(int) * h->tile_ctr_ints},
+      {(void**)&h->p_stats, sizeof(float2) * (size_t)MB * maxK},
       {(void**)&h->res, 4 * h->res_words},
       {(void**)&h->dst, sizeof(DevState)},
       {(void**)&s.n, 4 * (size_t)MB},
@@ -734,7 +757,7 @@ int sps_destroy(sps_handle* h) {
   free_model(h->tgt);
   free_model(h->drf);
   void* bufs[] = {h->wdq, h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
-                  h->counters, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
+                  h->counters, h->tile_ctr, h->p_stats, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);
   if (h->h_res) cudaFreeHost(h->h_res);
@@ -1022,7 +1045,7 @@ int sps_accept_filtered(const float* q_logits, const float* p_logits, const int3
   a.drafts = draft_tokens ? draft_tokens : out_tokens; a.drafts_ld = K;
   a.B = B; a.K = K; a.V = V; a.n_acc = out_n_accepted; a.out_tok = out_tokens; a.out_ld = K + 1; a.flags = out_flags;
   a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p;
-  cudaError_t e = accept_launch(a, (cudaStream_t)stream);
+  cudaError_t e = accept_launch_fast(a, (top_k >= 1 && top_k < V) || top_p < 1.f, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("accept launch: ") + cudaGetErrorString(e));
   return SPS_OK;
 }
@@ -1056,7 +1079,8 @@ static int cur_num_sm() {
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || dtype < 0 || dtype > 2) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
-  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256);
+  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256 +
+                   ((sizeof(int) * lin_tile_ctr_ints(N) + 255) / 256) * 256);
 }
 
 int64_t sps_linear_wide_workspace_bytes(int32_t N, int32_t D) {
@@ -1118,6 +1142,8 @@ int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, cons
   char* ws = (char*)workspace;
   a.counters = (int*)ws;
   size_t off = ((sizeof(int) * (2 * LIN_MAX_R + 2) + 255) / 256) * 256;
+  a.tile_ctr = (int*)(ws + off);
+  off += ((sizeof(int) * lin_tile_ctr_ints(N) + 255) / 256) * 256;
   off += sizeof(float) * (size_t)LIN_MAX_R * SPS_MAX_ROWS;
   a.part = (float*)(ws + off);
   cudaStream_t st = (cudaStream_t)stream;

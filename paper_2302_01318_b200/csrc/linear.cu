@@ -505,6 +505,60 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 
 #define LIN2_HDR_BYTES 1024
 
+// Finishing one 16-row output tile (per-tile epilogue), by ONE warp.  get(m, n, v0, v1) delivers the finished
+// products of output features n, n + 1 (n even) for activation row m: from shared memory when there is one
+// k-split, else the k-splits' partial sums added in split order.  Then as every epilogue of this file: row
+// scales of int8 weights, the row's 1/rms when the input came packed, store or residual add, the packed copy
+// for the next layer, and -- for a residual update -- this tile's sum of squares per row, reduced over the eight
+// lanes that share a row in a fixed tree.
+template <class Get>
+__device__ __forceinline__ void lin_finish_tile(const LinArgs& a, int tile, const float* row_scale, Get get) {
+  const int lane = threadIdx.x & 31;
+  const bool resid = a.epi == EPI_RESIDUAL;
+  const bool pair_ok = ((a.ldy & 1) == 0) && ((((size_t)a.Y) & 7) == 0) && (!a.yp_hi || (((a.ldyp & 1) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 3) == 0)));
+  const int items = ((a.M * 8 + 31) >> 5) << 5;
+  for (int i = lane; i < items; i += 32) {
+    const int m = i >> 3, p = i & 7, n = tile * 16 + 2 * p;
+    const bool ok0 = m < a.M && n < a.N, ok1 = ok0 && n + 1 < a.N;
+    float y0 = 0.f, y1 = 0.f, sq = 0.f;
+    if (ok0) {
+      get(m, n, ok1, y0, y1);
+      if (a.wscale[0]) {   // int8 weights: the rows' scales (n and n + 1 lie in one matrix: every matrix has a multiple of 16 rows)
+        int rin;
+        const int mat = mat_of(a, n, rin);
+        y0 *= __ldg(a.wscale[mat] + rin);
+        if (ok1) y1 *= __ldg(a.wscale[mat] + rin + 1);
+      }
+      if (row_scale) { const float sc = row_scale[m]; y0 *= sc; y1 *= sc; }
+      float* dst = a.Y + (long long)m * a.ldy + n;
+      if (resid) {
+        if (ok1 && pair_ok) { const float2 o = __ldcg(reinterpret_cast<const float2*>(dst)); y0 += o.x; y1 += o.y; }
+        else { y0 += __ldcg(dst); if (ok1) y1 += __ldcg(dst + 1); }
+        sq = ok1 ? (y0 * y0 + y1 * y1) : y0 * y0;
+      }
+      if (ok1 && pair_ok) *reinterpret_cast<float2*>(dst) = make_float2(y0, y1);
+      else { dst[0] = y0; if (ok1) dst[1] = y1; }
+      if (a.yp_hi) {
+        float z0 = y0, z1 = ok1 ? y1 : 0.f;
+        if (a.yp_act == PRO_GELU) { z0 = gelu_fast(z0); z1 = gelu_fast(z1); }
+        if (a.yp_gain) { z0 *= __ldg(a.yp_gain + n); if (ok1) z1 *= __ldg(a.yp_gain + n + 1); }
+        uint32_t hi, lo;
+        if (a.q8) split_pack_h(z0, z1, hi, lo); else split_pack(z0, z1, hi, lo);
+        unsigned short* ph = reinterpret_cast<unsigned short*>(a.yp_hi) + (long long)m * a.ldyp + n;
+        unsigned short* pl = reinterpret_cast<unsigned short*>(a.yp_lo) + (long long)m * a.ldyp + n;
+        if (ok1 && pair_ok) { *reinterpret_cast<uint32_t*>(ph) = hi; *reinterpret_cast<uint32_t*>(pl) = lo; }
+        else { ph[0] = (unsigned short)(hi & 0xffffu); pl[0] = (unsigned short)(lo & 0xffffu); if (ok1) { ph[1] = (unsigned short)(hi >> 16); pl[1] = (unsigned short)(lo >> 16); } }
+      }
+    }
+    if (resid) {
+      sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+      if (p == 0 && m < a.M) a.ssq_out[SSQ_IDX(tile, m)] = sq;
+    }
+  }
+}
+
 struct LinTmaArgs {
   LinArgs a;
   CUtensorMap tm[3];
@@ -656,6 +710,8 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
         }
       }
       if (!mbar_wait(bar_x, 0u, a.err, a.wait_ns)) { alive = false; s_abort = 1; }
+      // per-tile epilogue: whichever warp finishes a tile multiplies by every row's 1/rms, computed by other warps above
+      if (a.tile_epi && a.pro == PRO_RMSNORM) asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
     } else {
     // A thread owns 4 consecutive k (one 16-byte load per row, neighbouring lanes neighbouring addresses)
     // of up to two places of the k-range.  The gain of the norm is a weight: it comes from HBM, and is
@@ -884,7 +940,77 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[0][i] += __shfl_xor_sync(0xffffffffu, c[0][i], 2);
       }
-      if (G > 1) {
+      if (a.tile_epi) {
+        // ---- per-tile epilogue.  The group's G partial tiles meet in shared memory (element e = col * 16 + row).
+        float* mine = gscr + ((size_t)(round & 1) * NCW + warp) * (NT * 128);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int col = nt * 8 + 2 * t;
+          mine[col * 16 + g] = c[nt][0];
+          mine[(col + 1) * 16 + g] = c[nt][1];
+          mine[col * 16 + g + 8] = c[nt][2];
+          mine[(col + 1) * 16 + g + 8] = c[nt][3];
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(2 + grp), "r"(G * 32) : "memory");
+        if (*((volatile int*)&s_abort)) { alive = false; break; }
+        const float* gbase = gscr + ((size_t)(round & 1) * NCW + grp * G) * (NT * 128);
+        const float* rs = (a.xp_hi && a.pro == PRO_RMSNORM) ? s_scale : nullptr;
+        if (a.S == 1) {
+          // one k-split: the group's sums are the finished products; they meet in the group's slot of `fin`
+          // and the group's first warp finishes the tile (the slot is free again at the next tile's barrier)
+          float* fin = gscr + (size_t)2 * NCW * (NT * 128) + (size_t)grp * (NT * 128);
+          for (int e = rank * 32 + lane; e < NT * 128; e += G * 32) {
+            float sum = 0.f;
+            for (int w = 0; w < G; ++w) sum += gbase[w * (NT * 128) + e];
+            fin[e] = sum;
+          }
+          if (G > 1) asm volatile("bar.sync %0, %1;" ::"r"(2 + grp), "r"(G * 32) : "memory");
+          else __syncwarp();
+          if (rank == 0)
+            lin_finish_tile(a, tile, rs, [&](int m, int n, bool ok1, float& y0, float& y1) {
+              const int r0 = n - tile * 16;
+              y0 = fin[m * 16 + r0];
+              y1 = ok1 ? fin[m * 16 + r0 + 1] : 0.f;
+            });
+        } else {
+          // several k-splits: every warp adds its share of the group's elements to this split's partial sums, then
+          // announces itself on the tile's counter; the last of the S x G warps adds the splits in split order
+          for (int e = rank * 32 + lane; e < NT * 128; e += G * 32) {
+            float sum = 0.f;
+            for (int w = 0; w < G; ++w) sum += gbase[w * (NT * 128) + e];
+            const int col = e >> 4, n = tile * 16 + (e & 15);
+            if (col < a.M && n < a.N) a.part[((size_t)s * SPS_MAX_ROWS + col) * a.N + n] = sum;
+          }
+          __syncwarp();
+          int last = 0;
+          if (lane == 0) {
+            __threadfence();     // this warp's partial sums are visible before its arrival is
+            last = atomicAdd(a.tile_ctr + tile, 1) == a.S * G - 1;
+            if (last) { a.tile_ctr[tile] = 0; __threadfence(); }
+          }
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last) {
+            const bool n_even = (a.N & 1) == 0 && ((((size_t)a.part) & 7) == 0);
+            lin_finish_tile(a, tile, rs, [&](int m, int n, bool ok1, float& y0, float& y1) {
+              const float* src = a.part + (size_t)m * a.N + n;
+              const size_t sstride = (size_t)SPS_MAX_ROWS * a.N;
+              float v0 = 0.f, v1 = 0.f;
+              if (ok1 && n_even) {
+                for (int s0 = 0; s0 < a.S; s0 += 4) {     // four splits in flight, added in split order
+                  float2 v[4];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) v[j] = s0 + j < a.S ? __ldcg(reinterpret_cast<const float2*>(src + (s0 + j) * sstride)) : make_float2(0.f, 0.f);
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) { v0 += v[j].x; v1 += v[j].y; }
+                }
+              } else {
+                for (int sp = 0; sp < a.S; ++sp) { v0 += __ldcg(src + sp * sstride); if (ok1) v1 += __ldcg(src + sp * sstride + 1); }
+              }
+              y0 = v0; y1 = v1;
+            });
+          }
+        }
+      } else if (G > 1) {
         // element e = col * 16 + row of the 16 x (8*NT) tile
         float* mine = gscr + ((size_t)(round & 1) * NCW + warp) * (NT * 128);
 #pragma unroll
@@ -923,13 +1049,14 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
       }
     }
   }
-  if (a.split_epi) {
+  if (a.split_epi || a.tile_epi) {
+    // Per-tile epilogue: every tile this CTA took part in is finished, or will be by the warp that arrives last on it.
     // The split-K epilogue is a kernel of its own (lin_epilogue_kernel): this CTA is done once its partial
     // results are written, and its SM is free for the next layer's CTA, which starts streaming weights
     // while the slower CTAs of this grid are still at work.  The last CTA to leave re-arms the tile queues.
     __syncthreads();
     if (tid == 0) {
-      if (a.xp_hi && a.pro == PRO_RMSNORM && cta == 0)
+      if (!a.tile_epi && a.xp_hi && a.pro == PRO_RMSNORM && cta == 0)
         for (int m = 0; m < a.M; ++m) reinterpret_cast<float*>(a.counters + LIN_SCALE_SLOT)[m] = s_scale[m];
       if (C == 1 || atomicAdd(&a.counters[1], 1) == C - 1) {
         a.counters[0] = 0;
@@ -1077,11 +1204,16 @@ static const size_t kSmemBudget = 200 * 1024;
 // TMA variant: everything a CTA may ask for (227 KB) less the kernel's 1 KB of static shared memory and a little slack
 static const size_t kSmemTma = 225 * 1024;
 
+static bool lin_tile_epilogue() {   // tuning: SPS_LIN_TILE_EPI=0 goes back to the epilogue kernel
+  static const bool on = [] { const char* e = getenv("SPS_LIN_TILE_EPI"); return !(e && atoi(e) == 0); }();
+  return on;
+}
+size_t lin_tile_ctr_ints(int N) { return (size_t)((N + 15) / 16) + 64; }
 static bool lin_split_epilogue() {
   static const bool on = [] { const char* e = getenv("SPS_LIN_SPLIT_EPI"); return !(e && atoi(e) == 0); }();
   return on;
 }
-int lin_launch_count(const LinPlan& p) { return (p.variant == 2 && p.KS > 0 && lin_split_epilogue()) ? 2 : 1; }
+int lin_launch_count(const LinPlan& p) { return (p.variant == 2 && p.KS > 0 && !p.tile_epi && lin_split_epilogue()) ? 2 : 1; }
 
 bool sps_pdl_enabled() {
   static const bool on = [] { const char* e = getenv("SPS_PDL"); return !(e && atoi(e) == 0); }();
@@ -1151,13 +1283,22 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     const int ksub = KS / KST;
     p.G = (ksub % 4 == 0) ? 4 : ((ksub % 2 == 0) ? 2 : 1);
     if (dtype == 2 && ksub == 1) p.G = 2;   // int8, one-stage tiles: the two warps of a group share the stage
-    const size_t gscr = (size_t)2 * LIN_CONSUMER_WARPS * p.NT * 128 * sizeof(float);
+    const size_t gscr = (size_t)3 * LIN_CONSUMER_WARPS * p.NT * 128 * sizeof(float);   // two tile parities per warp + a slot per group
     NS = (int)((kSmemTma - 1024 - xbytes - gscr) / stage);
     if (NS > 24) NS = 24;
     if (NS < 2) NS = 2;
     p.NS = NS;
     p.smem = 1024 + xbytes + (size_t)NS * stage + gscr;
-    p.ssq_parts = p.R * p.S;
+    // Per-tile epilogue: a residual update leaves one sum of squares per 16-row tile, which the next norm must be able
+    // to hold (1), else only plain stores qualify (2).  With several k-splits every tile costs each consumer warp a
+    // fence and an arrival on the tile's counter: that pays where a CTA sees few tiles (the layer is all fixed cost
+    // and this saves a kernel and a grid-wide wait) and costs dearly where it streams many (the consumers fall
+    // behind the copy engine); SPS_LIN_TILE_EPI_MAX moves the limit (work units per CTA; tuning).
+    static const int units_max = [] { const char* e = getenv("SPS_LIN_TILE_EPI_MAX"); return e ? atoi(e) : 0; }();
+    const long long units = (long long)((N + 15) / 16) * p.S;
+    const bool want = lin_tile_epilogue() && (p.S == 1 || units <= (long long)units_max * p.R * p.S);
+    p.tile_epi = !want ? 0 : ((N + 15) / 16 <= LIN_MAX_R ? 1 : 2);
+    p.ssq_parts = p.tile_epi == 1 ? (N + 15) / 16 : p.R * p.S;
     return p;
   }
   const int chunks = D / 128;
@@ -1254,7 +1395,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
       const bool has = i < nmat;   // unused slots repeat the first matrix
       if ((e = weight_tensor_map(a.W[has ? i : 0], has && i > 0 ? a.rows_tail : a.rows_per_mat, a.D, p.KST, dtype == 2, &ta.tm[i])) != cudaSuccess) return e;
     }
-    ta.a.split_epi = lin_split_epilogue() ? 1 : 0;
+    ta.a.tile_epi = (p.tile_epi == 1 || (p.tile_epi == 2 && a.epi != EPI_RESIDUAL)) && a.tile_ctr ? 1 : 0;
+    ta.a.split_epi = (!ta.a.tile_epi && lin_split_epilogue()) ? 1 : 0;
     ta.a.q8 = dtype == 2 ? 1 : 0;
     static DevSmemCache c_q1{}, c_q2{};
     if (dtype == 2 && p.NT == 1) {
@@ -1307,7 +1449,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
 #include "../../include/sps.h"
 
 #define SPS_STATIC_PART_FLOATS (4u << 20)                     /* 16 MiB of partial sums */
-#define SPS_STATIC_CTR_BYTES (((2 * LIN_MAX_R + 2) * 4 + 255) / 256 * 256)
+#define SPS_STATIC_TILE_CTRS 16384                             /* per-tile arrival counters: N up to 262144 */
+#define SPS_STATIC_CTR_BYTES ((((2 * LIN_MAX_R + 2) * 4 + 255) / 256 * 256) + SPS_STATIC_TILE_CTRS * 4)
 static __device__ __align__(256) unsigned char g_static_scratch[SPS_STATIC_CTR_BYTES + 4ull * SPS_STATIC_PART_FLOATS];
 
 extern "C" int64_t sps_linear_static_max_floats(void) { return (int64_t)SPS_STATIC_PART_FLOATS; }
@@ -1350,6 +1493,7 @@ extern "C" int sps_linear_static(const void* W, int32_t dtype, const float* X, i
   a.W[0] = W; a.rows_per_mat = N; a.N = N; a.D = D; a.M = M; a.X = X; a.ldx = D; a.x_row0 = 0; a.x_rowstep = 1;
   a.pro = PRO_NONE; a.epi = EPI_STORE; a.Y = Y; a.ldy = N;
   a.counters = reinterpret_cast<int*>(base[dev]);
+  a.tile_ctr = (lin_tile_ctr_ints(N) <= SPS_STATIC_TILE_CTRS) ? reinterpret_cast<int*>(base[dev] + SPS_STATIC_CTR_BYTES - SPS_STATIC_TILE_CTRS * 4) : nullptr;
   a.part = reinterpret_cast<float*>(base[dev] + SPS_STATIC_CTR_BYTES);
   cudaStream_t st = (cudaStream_t)stream;
   // The array keeps the last call's contents.  Partial sums are overwritten before they are read.  The

@@ -3,6 +3,9 @@
 // warp shuffles plus a block prefix sum over the vocabulary.
 #include <limits.h>
 
+#include <algorithm>
+#include <cstdlib>
+
 #include "common.cuh"
 
 #define SAMPLER_THREADS 1024
@@ -343,20 +346,25 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_kernel(SampleArgs a) {
       if (i < a.V) ws[skew(i)] = expf((l[j] - m) * invT);
     }
     __syncthreads();
-    tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
+    float total;
+    tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, &total);
+    // the row's statistics, for the accept kernel: the very numbers this draw was made with
+    if (a.stats && threadIdx.x == 0) a.stats[(long long)b * a.stats_ld] = make_float2(m, total);
   } else {
     float m = -INFINITY;
     for (int i = threadIdx.x; i < a.V; i += blockDim.x) m = fmaxf(m, row[i]);
     m = block_max_f(m, s_part, &s_val);
+    float total;
     if (a.smem_weights) {
       extern __shared__ float ws[];
       for (int i = threadIdx.x; i < a.V; i += blockDim.x) ws[skew(i)] = expf((row[i] - m) * invT);
       __syncthreads();
-      tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, nullptr);
+      tok = block_invcdf_smem(ws, a.V, u.u_draft, sm, &total);
     } else {
       auto w = [&](int i) { return expf((row[i] - m) * invT); };
-      tok = block_invcdf(w, a.V, u.u_draft, sm, nullptr);
+      tok = block_invcdf(w, a.V, u.u_draft, sm, &total);
     }
+    if (a.stats && threadIdx.x == 0) a.stats[(long long)b * a.stats_ld] = make_float2(m, total);
   }
   if (threadIdx.x == 0) a.out[(long long)b * a.out_ld] = tok;
 }
@@ -564,6 +572,328 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_kernel(AcceptArgs a) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same sampler spread over a thread-block cluster: C CTAs per sequence, CTA c owning tokens
+// [c * slice, (c + 1) * slice) of every row (unfiltered distributions; the filtered ones keep the kernel above).
+//   1. every row whose softmax statistics are needed is read ONCE: its slice goes to shared memory with 16-byte
+//      loads, the CTA takes the slice's maximum and the sum of exp((l - max) / T) from there; the C partial
+//      (max, sum) pairs of a row meet in every CTA's shared memory (distributed shared memory) and are merged
+//      in CTA order.  Draft rows whose statistics the draft sampler left at draft time (p_stats) are not read.
+//   2. every CTA walks the accept chain for itself (same numbers, same decisions): the 2K logits it needs were
+//      asked for at kernel start.
+//   3. the weights of the one distribution that is drawn from -- max(0, q_t - p_t) at the rejected position, or
+//      q_K -- are formed for the CTA's slice (from the rows kept in shared memory when they fit, else re-read),
+//      scanned as in block_invcdf, the CTAs' totals meet as the statistics did, and each CTA looks for the
+//      first running sum above u * total inside its slice; the smallest candidate wins.
+// All sums run in a fixed order (thread chunk, warp scan, warp totals, CTA order): bit-reproducible.
+// ------------------------------------------------------------------------------------------------
+#include <cooperative_groups.h>
+namespace cg = cooperative_groups;
+
+#define ACCF_MAX_C 8
+#define ACCF_MAX_STAGES 32
+// exp((l - m) / T) as 2^((l - m) * c) with c = log2(e) / T: a subtraction, a multiplication and the hardware's
+// base-2 exponential (relative error about 2^-22, plus |argument| * 2^-23 from the product's rounding: below 1e-6 for
+// every weight that carries mass).  The passes over whole rows are bound by instruction issue, and the library
+// exponential costs four times as many instructions.
+__device__ __forceinline__ float exp2_scaled(float l, float m, float c) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"((l - m) * c));
+  return r;
+}
+struct AccfShared {
+  ScanSmem sm;
+  float2 seg[ACC_MAX_ROWS][SAMPLER_WARPS];   // (max, sum) of the segments of each row of the batch in hand
+  float2 part[ACC_MAX_ROWS][ACCF_MAX_C];     // (max, sum) of each row's slice, by CTA rank (filled by all CTAs of the cluster)
+  float row_m[ACC_MAX_ROWS], row_s[ACC_MAX_ROWS];
+  float lq[16], lp[16];                      // logits of the draft tokens in their target / draft rows
+  int dtok[16], okt[16];
+  float tot[ACCF_MAX_C];                     // the CTAs' weight totals
+  int cand[ACCF_MAX_C], lastpos[ACCF_MAX_C];
+  int wcand[SAMPLER_WARPS], wlast[SAMPLER_WARPS];
+  int stop;
+};
+
+__device__ __forceinline__ uint32_t s_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// 16 bytes global -> shared without passing through registers; completion is waited for with cp_async_wait
+__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptArgs a) {
+  __shared__ AccfShared sh;
+  extern __shared__ __align__(128) float dyn[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = a.csize, rank = (int)cluster.block_rank(), b = blockIdx.x / C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = a.K, V = a.V;
+  const int i0 = min(rank * a.slice, V), i1 = min(i0 + a.slice, V), ns = i1 - i0;   // ns is a multiple of 4 (launcher: V % 4 == 0)
+  const bool have_p = a.p_stats != nullptr;
+  const int R = have_p ? K + 1 : 2 * K + 1;       // rows whose statistics are worked out here: q_0..q_K, then p_0..p_{K-1}
+  const int slice_pad = a.slice;                  // a multiple of 4
+  // A row's slice travels in chunks of CH floats (one chunk when the slice is short): unit u = (row u / NCH, chunk u % NCH).
+  // Either every unit has a buffer of its own (`resident`: the rows stay for step 3), or the units go through a ring.
+  const int CH = a.chunk, NCH = (slice_pad + CH - 1) / CH, U = R * NCH, NSTG = a.resident ? U : a.stages;
+  cluster.barrier_arrive();     // its wait stands before the first access to another CTA's shared memory: by then every CTA runs
+  pdl_launch_dependents();
+  pdl_wait();
+  float T = a.temperature;
+  uint64_t seed = a.seed;
+  uint32_t step = a.step;
+  uint32_t seq = (uint32_t)b;
+  if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; seq += a.st->seq0; }
+  const float invT = 1.0f / T;
+  const float c2 = invT * 1.4426950408889634f;    // log2(e) / T
+  const float* qrow = a.q_logits + (long long)b * (K + 1) * V;
+  const float* prow = a.p_logits + (long long)b * K * V;
+  const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
+  auto rowptr = [&](int r) { return r <= K ? qrow + (long long)r * V : prow + (long long)(r - K - 1) * V; };
+  auto unit_floats = [&](int u) { const int ch = u % NCH; return max(0, min(CH, ns - ch * CH)); };
+  // units [u0, u0 + nb) on their way into their buffers: every thread copies its share, 16 bytes at a time, asynchronously
+  auto issue_units = [&](int u0, int nb) {
+    for (int j = 0; j < nb; ++j) {
+      const int u = u0 + j, r = u / NCH, ch = u - r * NCH, n4 = unit_floats(u) >> 2;
+      const float* src = rowptr(r) + i0 + (size_t)ch * CH;
+      float* dst = dyn + (size_t)(u % NSTG) * CH;
+      for (int q4 = tid; q4 < n4; q4 += SAMPLER_THREADS) cp_async16(dst + 4 * q4, src + 4 * q4);
+    }
+    cp_async_commit();
+  };
+  // resident: all units in one batch.  Ring: half the ring at a time, the other half is in flight meanwhile.
+  const int units_at_once = a.resident ? U : max(1, NSTG / 2);
+  issue_units(0, min(units_at_once, U));
+  // the draft tokens' logits: asked for now, used by the chain
+  if (tid >= 32 && tid < 32 + K) {
+    const int t = tid - 32;
+    int d = drafts[t];
+    if (d < 0 || d >= V) { d = 0; if (a.st) atomicExch(a.st->err, 1); }
+    sh.dtok[t] = d;
+    sh.lq[t] = qrow[(long long)t * V + d];
+    sh.lp[t] = prow[(long long)t * V + d];
+  }
+  // ---- 1. statistics.  A warp takes one segment of one unit: its maximum, then the sum of exp((l - max) / T); the
+  // segments are merged by one thread per row, in unit and segment order.
+  if (tid < R) { sh.row_m[tid] = -INFINITY; sh.row_s[tid] = 0.f; }
+  const int NSEG = max(1, SAMPLER_WARPS / units_at_once);
+  for (int u0 = 0; u0 < U; u0 += units_at_once) {
+    const int nb = min(units_at_once, U - u0);
+    // the next batch goes into the other half of the ring (every thread is past the last use of it: see the barrier
+    // at the end of the loop body), then this batch's copies are waited for
+    if (u0 + units_at_once < U) { issue_units(u0 + units_at_once, min(units_at_once, U - u0 - units_at_once)); cp_async_wait<1>(); }
+    else cp_async_wait<0>();
+    __syncthreads();              // everybody's copies of this batch have landed
+    for (int item = warp; item < nb * NSEG; item += SAMPLER_WARPS) {
+      const int j = item / NSEG, sg = item - j * NSEG, u = u0 + j;
+      const float4* src = reinterpret_cast<const float4*>(dyn + (size_t)(u % NSTG) * CH);
+      const int n4 = unit_floats(u) >> 2, per = (n4 + NSEG - 1) / NSEG, q0 = min(sg * per, n4), q1 = min(q0 + per, n4);
+      float m = -INFINITY;
+      for (int q4 = q0 + lane; q4 < q1; q4 += 32) { const float4 v = src[q4]; m = fmaxf(fmaxf(m, fmaxf(v.x, v.y)), fmaxf(v.z, v.w)); }
+      m = warp_max(m);
+      float sum = 0.f;
+      for (int q4 = q0 + lane; q4 < q1; q4 += 32) {
+        const float4 v = src[q4];
+        sum += (exp2_scaled(v.x, m, c2) + exp2_scaled(v.y, m, c2)) + (exp2_scaled(v.z, m, c2) + exp2_scaled(v.w, m, c2));
+      }
+      sum = warp_sum(sum);
+      if (lane == 0) sh.seg[j][sg] = make_float2(q1 > q0 ? m : -INFINITY, q1 > q0 ? sum : 0.f);
+    }
+    __syncthreads();
+    if (warp < nb) {
+      // unit `warp` of the batch: its segments, one per lane, merged with shuffles (a fixed tree)
+      const float2 v = lane < NSEG ? sh.seg[warp][lane] : make_float2(-INFINITY, 0.f);
+      const float mu = warp_max(v.x);
+      const float su = warp_sum(v.y > 0.f ? v.y * expf((v.x - mu) * invT) : 0.f);
+      if (lane == 0) sh.seg[warp][0] = make_float2(mu, su);
+    }
+    __syncthreads();
+    if (tid < R) {
+      // row `tid` takes in its units of this batch, in unit order (this CTA's slice only, for now)
+      float rm = sh.row_m[tid], rs = sh.row_s[tid];
+      for (int j = 0; j < nb; ++j) {
+        const float2 v = sh.seg[j][0];
+        if ((u0 + j) / NCH != tid || !(v.y > 0.f)) continue;
+        const float m = fmaxf(rm, v.x);
+        rs = (rs > 0.f ? rs * expf((rm - m) * invT) : 0.f) + v.y * expf((v.x - m) * invT);
+        rm = m;
+      }
+      sh.row_m[tid] = rm; sh.row_s[tid] = rs;
+    }
+    __syncthreads();              // this batch's buffers and the segment scratch are free again
+  }
+  __syncthreads();
+  // the C partial statistics of every row meet in every CTA
+  cluster.barrier_wait();
+  for (int idx = tid; idx < R * C; idx += SAMPLER_THREADS) {
+    const int r = idx / C, c = idx - r * C;
+    float2* remote = cluster.map_shared_rank(&sh.part[r][rank], c);
+    *remote = make_float2(ns > 0 ? sh.row_m[r] : -INFINITY, ns > 0 ? sh.row_s[r] : 0.f);
+  }
+  cluster.sync();
+  if (tid < 2 * K + 1) {
+    const int r = tid;
+    if (r < R) {
+      float m = -INFINITY;
+      for (int c = 0; c < C; ++c) m = fmaxf(m, sh.part[r][c].x);
+      float sum = 0.f;
+      for (int c = 0; c < C; ++c) { const float2 pc = sh.part[r][c]; if (pc.y > 0.f) sum += pc.y * expf((pc.x - m) * invT); }
+      sh.row_m[r] = m; sh.row_s[r] = sum;
+    } else {
+      const float2 ps = a.p_stats[(long long)b * a.p_stats_ld + (r - K - 1)];
+      sh.row_m[r] = ps.x; sh.row_s[r] = ps.y;
+    }
+  }
+  __syncthreads();
+  // ---- 2. the accept chain: every test on its own thread, the first failure stops the chain (every CTA, identically)
+  if (tid < K) {
+    const int t = tid;
+    const float forced = a.st ? __uint_as_float(a.st->pad0) : 0.f;
+    const float qd = expf((sh.lq[t] - sh.row_m[t]) * invT) / sh.row_s[t];
+    const float pd = expf((sh.lp[t] - sh.row_m[K + 1 + t]) * invT) / sh.row_s[K + 1 + t];
+    // accept with probability min(1, q(d)/p(d)); p == 0 with q > 0 accepts, 0/0 rejects
+    const float ratio = (pd > 0.f) ? fminf(1.0f, qd / pd) : (qd > 0.f ? 1.0f : 0.0f);
+    const Uniforms ut = sps_uniforms(seed, seq, step, (uint32_t)t);
+    sh.okt[t] = forced > 0.f ? (ut.u_acc < forced) : (ut.u_acc < ratio);   // forced: measurement mode only
+  }
+  __syncthreads();
+  int stop = K;
+  for (int t = K - 1; t >= 0; --t) if (!sh.okt[t]) stop = t;
+  const Uniforms u = sps_uniforms(seed, seq, step, (uint32_t)stop);
+  uint32_t fl = stop < K ? 1u : 2u;
+  // ---- 3. the draw: residual at `stop`, or q_K; if the residual sums to nothing, q_stop (flagged)
+  // (resident: one chunk per row, so row r sits at dyn + r * CH)
+  float* wbuf = a.resident ? dyn + (size_t)R * CH : dyn;     // skewed: element i of the slice at i + (i >> 5)
+  const float* ql = (a.resident ? dyn + (size_t)stop * CH : qrow + (long long)stop * V + i0);
+  const float* pl = stop < K ? ((a.resident && !have_p) ? dyn + (size_t)(K + 1 + stop) * CH : prow + (long long)stop * V + i0) : ql;
+  const float mq = sh.row_m[stop], iq = 1.0f / sh.row_s[stop];
+  const float mp = stop < K ? sh.row_m[K + 1 + stop] : 0.f, ip = stop < K ? 1.0f / sh.row_s[K + 1 + stop] : 0.f;
+  int tok = -1;
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    const bool residual = stop < K && attempt == 0;
+    __syncthreads();
+    {
+      const float4* q4p = reinterpret_cast<const float4*>(ql);
+      const float4* p4p = reinterpret_cast<const float4*>(pl);
+      for (int q4 = tid; q4 < (ns >> 2); q4 += SAMPLER_THREADS) {
+        const float4 lq4 = q4p[q4];
+        float w[4] = {exp2_scaled(lq4.x, mq, c2), exp2_scaled(lq4.y, mq, c2), exp2_scaled(lq4.z, mq, c2), exp2_scaled(lq4.w, mq, c2)};
+        if (residual) {
+          const float4 lp4 = p4p[q4];
+          w[0] = fmaxf(0.f, w[0] * iq - exp2_scaled(lp4.x, mp, c2) * ip);
+          w[1] = fmaxf(0.f, w[1] * iq - exp2_scaled(lp4.y, mp, c2) * ip);
+          w[2] = fmaxf(0.f, w[2] * iq - exp2_scaled(lp4.z, mp, c2) * ip);
+          w[3] = fmaxf(0.f, w[3] * iq - exp2_scaled(lp4.w, mp, c2) * ip);
+        }
+        const int i = q4 << 2;                    // four consecutive elements never straddle a skew boundary
+        float* dst = wbuf + skew(i);
+        dst[0] = w[0]; dst[1] = w[1]; dst[2] = w[2]; dst[3] = w[3];
+      }
+    }
+    __syncthreads();
+    // scan of the slice: chunk sums, warp scan, scan of the warp totals (as block_invcdf)
+    const int chunk = (ns + SAMPLER_THREADS - 1) / SAMPLER_THREADS;
+    const int c0 = min(tid * chunk, ns), c1 = min(c0 + chunk, ns);
+    float local = 0.f;
+    for (int i = c0; i < c1; ++i) local += wbuf[skew(i)];
+    float incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) sh.sm.warp_part[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const float v = sh.sm.warp_part[lane];
+      float iv = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float x = __shfl_up_sync(0xffffffffu, iv, o);
+        if (lane >= o) iv += x;
+      }
+      sh.sm.warp_part[lane] = iv - v;
+      const float tot_cta = __shfl_sync(0xffffffffu, iv, 31);
+      if (lane == 31) sh.sm.total = iv;
+      if (lane < C) *cluster.map_shared_rank(&sh.tot[rank], lane) = tot_cta;
+    }
+    cluster.sync();               // also orders this CTA's warp_part / total
+    const float pre_cta = sh.sm.warp_part[warp] + (incl - local);
+    float offset = 0.f, grand = 0.f;
+    for (int c = 0; c < C; ++c) { if (c == rank) offset = grand; grand += sh.tot[c]; }
+    if (residual && !(grand > 0.f)) { fl |= 4u; cluster.sync(); continue; }   // nothing left of q - p: draw from q_stop (every CTA decides the same)
+    const float target = u.u_res * grand;
+    int cand = INT_MAX, last = -1;
+    float cs = offset + pre_cta;
+    for (int i = c0; i < c1; ++i) {
+      const float w = wbuf[skew(i)];
+      cs += w;
+      if (w > 0.f) last = i0 + i;
+      if (cs > target && cand == INT_MAX) cand = i0 + i;
+    }
+    cand = warp_min_int(cand);
+    last = warp_max_int(last);
+    if (lane == 0) { sh.wcand[warp] = cand; sh.wlast[warp] = last; }
+    __syncthreads();
+    if (warp == 0) {
+      cand = warp_min_int(sh.wcand[lane]);
+      last = warp_max_int(sh.wlast[lane]);
+      if (lane == 0) {
+        *cluster.map_shared_rank(&sh.cand[rank], 0) = cand;
+        *cluster.map_shared_rank(&sh.lastpos[rank], 0) = last;
+      }
+    }
+    cluster.sync();
+    if (rank == 0) {
+      int best = INT_MAX, lp = -1;
+      for (int c = 0; c < C; ++c) { best = min(best, sh.cand[c]); lp = max(lp, sh.lastpos[c]); }
+      tok = best != INT_MAX ? best : (lp >= 0 ? lp : V - 1);
+    }
+    break;
+  }
+  if (rank != 0) return;
+  // ---- results (first CTA of the cluster)
+  int32_t* out = a.out_tok + (long long)b * a.out_ld;
+  if (tid <= K) out[tid] = (tid < stop) ? sh.dtok[tid] : (tid == stop ? tok : -1);
+  if (tid == 0) {
+    a.n_acc[b] = stop;
+    a.flags[b] = fl;
+  }
+  if (a.st) {
+    // advance the sequence in place: accepted drafts, then the resampled / extra token
+    DevState* st = a.st;
+    const int n = st->n[b];
+    const bool live = n < st->limit[b];   // a finished sequence of a batch keeps its length
+    __syncthreads();
+    if (live && tid <= stop && n + tid < st->max_seq)
+      st->tokens[(long long)b * st->max_seq + n + tid] = (tid < stop) ? sh.dtok[tid] : tok;
+    __syncthreads();
+    if (tid == 0) {
+      if (live) st->n[b] = n + stop + 1;
+      __threadfence();
+      // the last sequence to finish moves the loop counter
+      const uint32_t done = atomicAdd(st->done_counter, 1u);
+      if (done == (uint32_t)(gridDim.x / C) - 1) {
+        *st->done_counter = 0u;
+        st->step = step + 1u;
+      }
+    }
+  }
+}
+
+// how many CTAs share a sequence: enough to put every SM to work at small batches, one when the batch fills the GPU
+static int accept_cluster_size(int B, int V) {
+  static const int forced = [] { const char* e = getenv("SPS_ACCEPT_CLUSTER"); return e ? atoi(e) : -1; }();   // tuning: 0 = the one-CTA kernel
+  if (forced >= 0) return forced;
+  if (V < 8192) return 0;          // small vocabularies: the one-CTA kernel
+  int num_sm = SPS_NUM_SM_FALLBACK, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&num_sm, cudaDevAttrMultiProcessorCount, dev);
+  // the largest power of two, at most 8 (the portable cluster size), that keeps all the sequences' CTAs on the GPU at once
+  int c = ACCF_MAX_C;
+  while (c > 1 && (long long)B * c > num_sm) c >>= 1;
+  return c;
+}
+
 cudaError_t accept_launch(const AcceptArgs& a_in, cudaStream_t st) {
   static DevSmemCache cached{};
   AcceptArgs a = a_in;
@@ -572,6 +902,51 @@ cudaError_t accept_launch(const AcceptArgs& a_in, cudaStream_t st) {
   cudaError_t e = sampler_smem_attr(accept_kernel, smem, cached);
   if (e != cudaSuccess) return e;
   return launch_k(accept_kernel, dim3(a.B), dim3(SAMPLER_THREADS), smem, st, a);
+}
+
+// the cluster form; `filtered` says whether top-k / nucleus filtering is in force (then the kernel above runs)
+cudaError_t accept_launch_fast(const AcceptArgs& a_in, bool filtered, cudaStream_t st) {
+  const int C = filtered ? 0 : accept_cluster_size(a_in.B, a_in.V);
+  // rows travel as bulk copies: 16-byte aligned row starts and slices
+  const bool aligned = (a_in.V % 4 == 0) && ((((size_t)a_in.q_logits | (size_t)a_in.p_logits) & 15) == 0);
+  if (C < 1 || a_in.K > 15 || !aligned) return accept_launch(a_in, st);
+  static DevSmemCache cached{};
+  AcceptArgs a = a_in;
+  a.csize = C;
+  a.slice = (((a.V + C - 1) / C) + 3) & ~3;
+  const int R = a.p_stats ? a.K + 1 : 2 * a.K + 1;
+  const size_t slice_pad = (size_t)a.slice;
+  const size_t wbytes = sizeof(float) * (slice_pad + slice_pad / 32 + 32);
+  const size_t budget = 196 * 1024;
+  size_t smem;
+  if (sizeof(float) * R * slice_pad + wbytes <= budget && R <= ACCF_MAX_STAGES) {
+    a.resident = 1; a.chunk = a.slice; a.stages = R;             // every row's slice stays in shared memory
+    smem = sizeof(float) * R * slice_pad + wbytes;
+  } else {
+    a.resident = 0;                                              // chunks of at most 32 KB through a ring; the weights reuse it afterwards
+    a.chunk = a.slice < 8192 ? a.slice : 8192;
+    if (wbytes > budget) return accept_launch(a_in, st);         // a slice whose weights do not fit: one-CTA kernel
+    int stages = (int)(budget / (sizeof(float) * a.chunk));
+    const int units = R * ((a.slice + a.chunk - 1) / a.chunk);
+    if (stages > units) stages = units;
+    if (stages > ACCF_MAX_STAGES) stages = ACCF_MAX_STAGES;
+    if (stages < 2) stages = 2;
+    stages &= ~1;                                                // two halves: one being read, one in flight
+    a.stages = stages;
+    smem = std::max(sizeof(float) * (size_t)stages * a.chunk, wbytes);
+  }
+  cudaError_t e = sampler_smem_attr(accept_cluster_kernel, smem, cached);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.B * C); cfg.blockDim = dim3(SAMPLER_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = sps_pdl_enabled() ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, accept_cluster_kernel, a);
 }
 
 __global__ void philox_kernel(const uint32_t* ctr, const uint32_t* key, int n, uint32_t* out) {
