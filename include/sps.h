@@ -51,6 +51,7 @@ extern "C" {
 
 /* sps_cfg.flags */
 #define SPS_CFG_NO_GRAPH 1u   /* launch kernels one by one instead of replaying CUDA graphs  */
+#define SPS_CFG_TENSOR_PARALLEL 2u /* the weights are one rank's shard of both models (see sps_tp_attach) */
 
 typedef struct sps_handle sps_handle;
 
@@ -358,6 +359,40 @@ int sps_linear_static(const void* W, int32_t dtype, const float* X, int32_t M, i
 int64_t sps_linear_static_max_floats(void);
 /* floats of split-K scratch the shape needs on the current device; -1 for arguments sps_linear_static rejects */
 int64_t sps_linear_static_floats_needed(int32_t dtype, int32_t M, int32_t N, int32_t D);
+
+/* Tensor-parallel passes (section Conditional Scoring: the models are served Megatron-style over several chips, the
+ * attention and feed-forward blocks sharded and each followed by an all-reduce of (K + 1) x d_model numbers, which
+ * is latency-bound and about as costly for K + 1 rows as for one; section Choice of Draft Models: the draft is shaped
+ * to be served on the same chips).  One process per GPU; rank r of `world` (<= 8) creates its handle with
+ * SPS_CFG_TENSOR_PARALLEL and ITS SHARD of both models:
+ *   wq, wk, wv, w_up : the shard's output rows -- n_heads / world query heads, n_kv_heads / world key / value heads,
+ *                      d_ff / world feed-forward features (contiguous blocks, rank r the r-th);
+ *   wo, w_down       : the matching input COLUMNS, stored densely: [d_model, n_heads * d_head / world],
+ *                      [d_model, d_ff / world];
+ *   embeddings, unembedding, norm gains: whole, on every rank.
+ * sps_model_cfg then describes the shard: d_model as in the whole model, n_heads / n_kv_heads / d_ff the shard's
+ * (n_heads * d_head < d_model is allowed under this flag).  After every output projection the ranks exchange their
+ * partial updates of the residual stream: each rank stores its partial into a slot of every rank's inbox (plain
+ * stores into peer memory) and raises a flag there; each rank then sums the slots of its OWN inbox in rank order, so
+ * every rank holds the same bits and runs the same loop.  No library collective, no multicast.
+ *
+ * sps_tp_buffers returns this rank's inbox and flag array (device pointers, with their sizes) for export to the
+ * peers (e.g. as CUDA IPC handles, which the caller exchanges however it talks to its peers).
+ * sps_tp_attach gives the handle every rank's inbox and flag array as THIS device addresses them (entry `rank`: its
+ * own); attach every rank before any of them runs a pass.  Afterwards the handle's calls (sps_prefill, sps_step,
+ * sps_generate, ...) are collective: every rank makes the same calls with the same arguments.  Waits on peers are
+ * bounded like every other wait (SPS_ETIMEOUT). */
+int sps_tp_buffers(sps_handle* h, void** inbox, void** flags, int64_t* inbox_bytes, int64_t* flags_bytes);
+int sps_tp_attach(sps_handle* h, int32_t rank, int32_t world, void* const* peer_inbox, void* const* peer_flags);
+/* A whole group emulated on ONE GPU, for checking the sharded arithmetic and the exchange kernels without `world`
+ * GPUs: ranks[r] is rank r's handle, all created on one device with the same cfg.stream and attached to one another
+ * with plain device pointers.  The calls enqueue what the `world` processes would, phase by phase (every rank's
+ * store phase of an exchange before any rank's sum), so nothing ever waits for a kernel that is launched later.
+ * sps_tp_group_prefill: as sps_prefill on every rank.  sps_tp_group_score: as sps_score on every rank; out_logits
+ * host array of `world` DEVICE buffers [n_rows, vocab], which come out identical. */
+int sps_tp_group_prefill(sps_handle* const* ranks, int32_t world, const int32_t* toks, int32_t n);
+int sps_tp_group_score(sps_handle* const* ranks, int32_t world, int32_t which, const int32_t* rows, int32_t n_rows,
+                       float* const* out_logits, float* out_ms);
 
 /* Test hook for the give-up path of the kernels' waits.  Every wait inside a
  * kernel (on a copy, on another CTA, on a tile queue) is bounded by the global

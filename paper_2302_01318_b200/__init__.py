@@ -17,6 +17,7 @@ SPS_OK, SPS_EINVAL, SPS_ENOMEM, SPS_ECUDA, SPS_ERANGE, SPS_ESTATE, SPS_ETIMEOUT 
 SPS_MAX_K = 15
 FLAG_RESAMPLED, FLAG_BONUS, FLAG_FALLBACK = 1, 2, 4
 CFG_NO_GRAPH = 1
+CFG_TENSOR_PARALLEL = 2
 LAYER_KEYS = ("attn_norm", "ffn_norm", "wq", "wk", "wv", "wo", "w_up", "w_down")
 SCALED_KEYS = ("wq", "wk", "wv", "wo", "w_up", "w_down")   # matrices that carry row scales when weights are int8
 
@@ -105,6 +106,10 @@ def lib():
         L.sps_prefill_batch.argtypes = [vp, vp, vp, i32, i32]
         L.sps_set_sequence_index0.argtypes = [vp, u32]
         L.sps_debug_set_wait.argtypes = [i64, i32]
+        L.sps_tp_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64)]
+        L.sps_tp_attach.argtypes = [vp, i32, i32, vp, vp]
+        L.sps_tp_group_prefill.argtypes = [vp, i32, vp, i32]
+        L.sps_tp_group_score.argtypes = [vp, i32, i32, vp, i32, vp, C.POINTER(f32)]
         _lib = L
     return _lib
 
@@ -226,6 +231,18 @@ class Handle:
             t[b, :len(x)] = x
         _check(lib().sps_prefill_batch(self._h, _np_ptr(t), _np_ptr(lens), len(seqs), ld), self._h)
         self.B = len(seqs)
+
+    def tp_buffers(self):
+        """(inbox pointer, flags pointer, inbox bytes, flags bytes) of a tensor-parallel rank's receive buffers."""
+        inbox, flags, nb, nf = C.c_void_p(), C.c_void_p(), C.c_int64(0), C.c_int64(0)
+        _check(lib().sps_tp_buffers(self._h, C.byref(inbox), C.byref(flags), C.byref(nb), C.byref(nf)), self._h)
+        return inbox.value, flags.value, nb.value, nf.value
+
+    def tp_attach(self, rank, world, peer_inbox, peer_flags):
+        """peer_inbox / peer_flags: device addresses (ints) of every rank's buffers as this device sees them."""
+        pi = (C.c_void_p * world)(*peer_inbox)
+        pf = (C.c_void_p * world)(*peer_flags)
+        _check(lib().sps_tp_attach(self._h, rank, world, pi, pf), self._h)
 
     def sps_set_sequence_index0(self, index0):
         """Sequence b of later generate / step calls uses Philox sequence index index0 + b."""

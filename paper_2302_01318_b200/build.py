@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsps_b200.so")
-SOURCES = ["engine.cu", "linear.cu", "attention.cu", "sampler.cu", "wide.cu"]
+SOURCES = ["engine.cu", "linear.cu", "attention.cu", "sampler.cu", "wide.cu", "tp.cu"]
 HEADERS = ["common.cuh", os.path.join("..", "..", "include", "sps.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC",
               "-shared"]

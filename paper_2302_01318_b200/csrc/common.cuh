@@ -287,6 +287,33 @@ cudaError_t wide_gemm_launch(const void* W, const void* hi, const void* lo, int 
 cudaError_t wide_dequant_launch(const void* q, void* out, long long n, int num_sm, cudaStream_t st);
 size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh);
 
+// ------------------------------------------------------------------------------------------------
+// Tensor-parallel exchange (tp.cu): the all-reduce of the partial residual updates as peer stores + a local sum
+// ------------------------------------------------------------------------------------------------
+#define SPS_TP_MAX_WORLD 8
+struct TpArgs {
+  int rank, world, rows, d;         // this rank, ranks, activation rows of the pass, d_model
+  const uint32_t* epoch_ctr;        // device counter of finished exchanges (push works on *ctr + 1 and stores it; reduce reads it)
+  uint32_t* epoch_ctr_w;
+  size_t slot_floats;               // floats of one (parity, rank) slot of an inbox
+  const float* send;                // [rows][d] this rank's partial update
+  float* peer_inbox[SPS_TP_MAX_WORLD];     // every rank's inbox [2][world][slot_floats] as this device addresses it (own included)
+  uint32_t* peer_flags[SPS_TP_MAX_WORLD];  // every rank's flags [world]: flags[r] = last exchange rank r has pushed
+  const float* my_inbox;
+  uint32_t* my_flags;
+  float* x;                         // [rows][d] residual stream, updated in place
+  float* ssq_out;                   // SSQ_IDX(cta, row): per-CTA sums of squares of the updated rows
+  unsigned short* yp_hi;            // packed copy of gain * x for the next layer (null = none): bf16, or fp16 for int8-weight models
+  unsigned short* yp_lo;
+  const float* yp_gain;
+  int half_is_fp16;
+  int* err;
+  unsigned long long wait_ns;
+};
+int tp_reduce_ctas(int d, int num_sm);
+cudaError_t tp_push_launch(const TpArgs& a, cudaStream_t st);
+cudaError_t tp_reduce_launch(const TpArgs& a, int ctas, cudaStream_t st);
+
 struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(logits/T)
   const DevState* st;      // T, seed, step come from here when st != nullptr
   const float* logits;     // row b at logits + b*ld

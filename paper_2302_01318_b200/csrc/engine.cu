@@ -59,6 +59,18 @@ struct sps_handle {
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   int* counters = nullptr;
+  // tensor parallelism (SPS_CFG_TENSOR_PARALLEL): this handle holds one rank's shard of both models
+  bool tp = false;           // the models are shards: n_heads * d_head may be less than d_model
+  bool tp_attached = false;  // sps_tp_attach has given the peers' buffers
+  int tp_rank = 0, tp_world = 1;
+  float* tp_send = nullptr;  // [16][d_model] this rank's partial update of the residual stream
+  float* tp_inbox = nullptr; // [2][SPS_TP_MAX_WORLD][16 * d_model] partial updates received, by exchange parity and rank
+  uint32_t* tp_flags = nullptr;   // [SPS_TP_MAX_WORLD] last exchange each rank has pushed here
+  uint32_t* tp_epoch = nullptr;   // [1] exchanges this rank has opened
+  float* tp_peer_inbox[SPS_TP_MAX_WORLD] = {nullptr};
+  uint32_t* tp_peer_flags[SPS_TP_MAX_WORLD] = {nullptr};
+  size_t tp_slot_floats = 0;
+  int pass_nA = 1, pass_nB = 1;   // partial sums of squares in ssqA / ssqB (carried between the phases of a pass)
   float2* p_stats = nullptr; // [max_batch][max_K] (row maximum, sum of exponentials) of each draft row, left by the draft sampler
   bool filtered = false;     // top-k / nucleus / greedy in force for the calls being made (write_params)
   int* tile_ctr = nullptr;   // per-tile arrival counters of the linear layers' epilogue (zero between launches)
@@ -104,9 +116,12 @@ inline int act_dtype(int dtype) { return dtype == 0 ? 0 : 1; }   // what the emb
 inline int kv_heads(const sps_model_cfg& c) { return c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads; }
 inline int kv_width(const sps_model_cfg& c) { return kv_heads(c) * c.d_head; }   // rows of wk / wv, numbers cached per position
 
-int check_model_cfg(const sps_model_cfg& c, std::string& why) {
+inline int attn_width(const sps_model_cfg& c) { return c.n_heads * c.d_head; }   // rows of wq, columns of wo (= d_model unless the model is a tensor-parallel shard)
+
+int check_model_cfg(const sps_model_cfg& c, std::string& why, bool shard) {
   if (c.n_layers < 0 || c.d_model <= 0 || c.n_heads <= 0 || c.d_ff <= 0 || c.vocab <= 0) { why = "non-positive model dimension"; return 0; }
-  if (c.n_heads * c.d_head != c.d_model) { why = "n_heads * d_head must equal d_model"; return 0; }
+  if (!shard && c.n_heads * c.d_head != c.d_model) { why = "n_heads * d_head must equal d_model"; return 0; }
+  if (shard && (c.n_heads * c.d_head > c.d_model || (c.dtype >= 1 && (c.n_heads * c.d_head) % 128))) { why = "a shard's n_heads * d_head must not exceed d_model (bf16 / int8: a multiple of 128)"; return 0; }
   if (c.d_head != 64 && c.d_head != 128) { why = "d_head must be 64 or 128"; return 0; }
   if (c.n_kv_heads < 0 || c.n_heads % kv_heads(c)) { why = "n_kv_heads must be 0 or a divisor of n_heads"; return 0; }
   if (c.dtype < 0 || c.dtype > 2) { why = "dtype must be 0 (fp32), 1 (bf16) or 2 (int8 weights)"; return 0; }
@@ -133,7 +148,7 @@ int load_model(sps_handle* h, ModelDev& m, const sps_model_cfg& c, const sps_wei
     }
   }
   if (c.dtype == 2) {
-    const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+    const int shapes[5][2] = {{attn_width(c) + 2 * kv_width(c), c.d_model}, {c.d_model, attn_width(c)}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
     for (int M : {1, SPS_MAX_ROWS})
       for (auto& sh : shapes)
         if (lin_plan(2, M, sh[0], sh[1], h->num_sm).variant != 2) return fail(h, SPS_EINVAL, "int8 weights: a layer width splits into more k-ranges than the kernel supports");
@@ -181,7 +196,7 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
   if (!m.present) return 0;
   const sps_model_cfg& c = m.cfg;
   size_t need = 0;
-  const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  const int shapes[5][2] = {{attn_width(c) + 2 * kv_width(c), c.d_model}, {c.d_model, attn_width(c)}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
   for (int M : {1, SPS_MAX_ROWS})
     for (auto& s : shapes) {
       const LinPlan p = lin_plan(c.dtype, M, s[0], s[1], num_sm);
@@ -195,7 +210,7 @@ size_t model_part_floats(const ModelDev& m, int num_sm) {
 bool model_can_pack(const ModelDev& m, int num_sm) {
   const sps_model_cfg& c = m.cfg;
   if (!m.present || c.dtype < 1) return false;
-  const int shapes[5][2] = {{c.d_model + 2 * kv_width(c), c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
+  const int shapes[5][2] = {{attn_width(c) + 2 * kv_width(c), c.d_model}, {c.d_model, attn_width(c)}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}, {c.vocab, c.d_model}};
   for (int M : {1, SPS_MAX_ROWS})
     for (auto& s : shapes)
       if (lin_plan(c.dtype, M, s[0], s[1], num_sm).variant != 2) return false;
@@ -213,99 +228,154 @@ struct PassSpec {
 // one forward pass of a model over the rows `ps` describes, for the handle's B live sequences
 int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps);
 
+// The pass is a list of phases so that the ranks of a tensor-parallel group emulated on one GPU can be stepped
+// through it together: phase 0 = rows + embedding; per layer l, 1 + 4 l = attention block (q | k | v, attention,
+// output projection), + 1 = its exchange's reduction (sharded models only), + 2 = feed-forward block, + 3 = its
+// reduction; the last phase = logits.  An unsharded model's blocks add to the residual stream themselves and its
+// reduction phases are empty.
+int pass_phases(const ModelDev& m) { return 2 + 4 * m.cfg.n_layers; }
+
+TpArgs tp_args(sps_handle* h, const sps_model_cfg& c, int rows) {
+  TpArgs t{};
+  t.rank = h->tp_rank; t.world = h->tp_world; t.rows = rows; t.d = c.d_model;
+  t.epoch_ctr = h->tp_epoch; t.epoch_ctr_w = h->tp_epoch; t.slot_floats = h->tp_slot_floats;
+  t.send = h->tp_send;
+  for (int w = 0; w < h->tp_world; ++w) { t.peer_inbox[w] = h->tp_peer_inbox[w]; t.peer_flags[w] = h->tp_peer_flags[w]; }
+  t.my_inbox = h->tp_inbox; t.my_flags = h->tp_flags;
+  t.x = h->x; t.err = h->hst.err; t.wait_ns = sps_wait_knobs().limit_ns;
+  t.half_is_fp16 = c.dtype == 2 ? 1 : 0;
+  return t;
+}
+
+int run_pass_range(sps_handle* h, ModelDev& m, const PassSpec& ps, int ph0, int ph1) {
+  const sps_model_cfg& c = m.cfg;
+  const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff, da = attn_width(c), dkv = kv_width(c);
+  const bool tp = h->tp && h->tp_world > 1;
+  if (h->tp && !h->tp_attached) return fail(h, SPS_ESTATE, "tensor-parallel handle: sps_tp_attach has not been called");
+  cudaStream_t st = h->stream;
+  LinArgs base{};
+  base.part = h->part; base.counters = h->counters; base.tile_ctr = h->tile_ctr; base.eps = c.rms_eps;
+  base.err = h->hst.err;
+  const int last = pass_phases(m) - 1;
+  for (int ph = ph0; ph < ph1; ++ph) {
+    if (ph == 0) {
+      EmbedArgs ea{};
+      ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
+      ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
+      ea.x = h->x; ea.ssq = h->ssqA;
+      CU(h, embed_launch(ea, st)); h->launches++;
+      h->pass_nA = 1; h->pass_nB = 1;   // how many partial sums of squares sit in ssqA / ssqB
+      continue;
+    }
+    if (ph == last) {
+      if (!ps.logits) continue;
+      LinArgs a = base;
+      a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
+      if (c.dtype == 2) a.wscale[0] = m.unembed_scale;
+      a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
+      a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = h->pass_nA;
+      if (m.packed) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }
+      a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
+      const LinPlan pl = lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm);
+      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+      continue;
+    }
+    const int l = (ph - 1) / 4, sub = (ph - 1) % 4;
+    if (sub == 0) {
+      {  // q, k, v = Wq h, Wk h, Wv h with h = rmsnorm(x, g_attn), one launch over the three matrices
+        LinArgs a = base;
+        a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
+        if (c.dtype == 2) { a.wscale[0] = m.wq_s[l]; a.wscale[1] = m.wk_s[l]; a.wscale[2] = m.wv_s[l]; }
+        a.rows_per_mat = da; a.rows_tail = dkv; a.N = da + 2 * dkv; a.D = d; a.M = rows;
+        a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
+        a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = h->pass_nA;
+        if (m.packed && l > 0) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }   // left there by the layer below
+        a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = a.N;
+        const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+        CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+      }
+      {
+        AttnArgs aa{};
+        aa.st = h->dst; aa.qkv = h->qkv; aa.out = h->attn;
+        aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
+        aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = da;
+        aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
+        aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
+        CU(h, attn_launch(aa, st)); h->launches++;
+      }
+      {  // x += Wo o ; also sum(x^2) for the FFN norm.  A shard's Wo (its columns) gives a partial update instead.
+        LinArgs a = base;
+        a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = da; a.M = rows;
+        if (c.dtype == 2) a.wscale[0] = m.wo_s[l];
+        a.X = h->attn; a.ldx = da; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
+        const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+        if (tp) { a.epi = EPI_STORE; a.Y = h->tp_send; a.ldy = d; }
+        else {
+          a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
+          if (m.packed) { a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_gain = (const float*)m.ffn_norm[l]; a.yp_act = PRO_NONE; }
+          h->pass_nB = pl.ssq_parts;
+        }
+        CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+        if (tp) { CU(h, tp_push_launch(tp_args(h, c, rows), st)); h->launches++; }
+      }
+    } else if (sub == 1 || sub == 3) {
+      if (!tp) continue;
+      // the exchange's second half: x += the ranks' partial updates, sums of squares and packed copy for what follows
+      TpArgs t = tp_args(h, c, rows);
+      const int ctas = tp_reduce_ctas(d, h->num_sm);
+      const void* gain = sub == 1 ? m.ffn_norm[l] : (l + 1 < c.n_layers ? m.attn_norm[l + 1] : m.final_norm);
+      t.ssq_out = sub == 1 ? h->ssqB : h->ssqA;
+      if (m.packed) { t.yp_hi = (unsigned short*)h->xp_hi; t.yp_lo = (unsigned short*)h->xp_lo; t.yp_gain = (const float*)gain; }
+      CU(h, tp_reduce_launch(t, ctas, st)); h->launches++;
+      if (sub == 1) h->pass_nB = ctas; else h->pass_nA = ctas;
+    } else {
+      {  // up = Wup rmsnorm(x, g_ffn)
+        LinArgs a = base;
+        a.W[0] = m.w_up[l]; a.rows_per_mat = dff; a.N = dff; a.D = d; a.M = rows;
+        if (c.dtype == 2) a.wscale[0] = m.w_up_s[l];
+        a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
+        a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB; a.ssq_in_n = h->pass_nB;
+        a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
+        if (m.packed) {
+          a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo;
+          a.yp_hi = h->up_hi; a.yp_lo = h->up_lo; a.ldyp = dff; a.yp_gain = nullptr; a.yp_act = PRO_GELU;
+        }
+        const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+        CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+      }
+      {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm (a shard: a partial update)
+        LinArgs a = base;
+        a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
+        if (c.dtype == 2) a.wscale[0] = m.w_down_s[l];
+        a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
+        if (m.packed) { a.xp_hi = h->up_hi; a.xp_lo = h->up_lo; }
+        const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
+        if (tp) { a.epi = EPI_STORE; a.Y = h->tp_send; a.ldy = d; }
+        else {
+          a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
+          if (m.packed) {
+            a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_act = PRO_NONE;
+            a.yp_gain = (const float*)(l + 1 < c.n_layers ? m.attn_norm[l + 1] : m.final_norm);
+          }
+          h->pass_nA = pl.ssq_parts;
+        }
+        CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
+        if (tp) { CU(h, tp_push_launch(tp_args(h, c, rows), st)); h->launches++; }
+      }
+    }
+  }
+  return SPS_OK;
+}
+
 int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   const sps_model_cfg& c = m.cfg;
-  const int B = h->B, rows = B * ps.rows_per_seq, d = c.d_model, dff = c.d_ff;
+  const int rows = h->B * ps.rows_per_seq;
   // 9..16 rows: the tensor-core GEMM path also beats the 16-row weight-streaming variant (which is bound by shared-memory
   // bandwidth) when the model can take it; SPS_WIDE_MIN_ROWS moves the switch (tuning only)
   static const int wide_min = [] { const char* e = getenv("SPS_WIDE_MIN_ROWS"); return e ? atoi(e) : 9; }();
   if (rows > SPS_MAX_ROWS || (rows >= wide_min && h->wide && c.dtype == 1 && (!ps.logits || (ps.lrow0 == 0 && ps.lrowstep == 1 && ps.lrows == rows))))
     return run_pass_wide(h, m, ps);
-  cudaStream_t st = h->stream;
-  EmbedArgs ea{};
-  ea.st = h->dst; ea.tok_embed = m.tok_embed; ea.dtype = act_dtype(c.dtype); ea.d = d; ea.V = c.vocab;
-  ea.mode = ps.mode; ea.t = ps.t; ea.K = ps.K; ea.c0 = ps.c0; ea.rows_per_seq = ps.rows_per_seq; ea.B = B;
-  ea.x = h->x; ea.ssq = h->ssqA;
-  CU(h, embed_launch(ea, st)); h->launches++;
-  LinArgs base{};
-  base.part = h->part; base.counters = h->counters; base.tile_ctr = h->tile_ctr; base.eps = c.rms_eps;
-  int nA = 1, nB = 1;   // how many partial sums of squares sit in ssqA / ssqB
-  base.err = h->hst.err;
-  for (int l = 0; l < c.n_layers; ++l) {
-    {  // q, k, v = Wq h, Wk h, Wv h with h = rmsnorm(x, g_attn), one launch over the three matrices
-      LinArgs a = base;
-      a.W[0] = m.wq[l]; a.W[1] = m.wk[l]; a.W[2] = m.wv[l];
-      if (c.dtype == 2) { a.wscale[0] = m.wq_s[l]; a.wscale[1] = m.wk_s[l]; a.wscale[2] = m.wv_s[l]; }
-      a.rows_per_mat = d; a.rows_tail = kv_width(c); a.N = d + 2 * kv_width(c); a.D = d; a.M = rows;
-      a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
-      a.pro = PRO_RMSNORM; a.gain = (const float*)m.attn_norm[l]; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
-      if (m.packed && l > 0) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }   // left there by the layer below
-      a.epi = EPI_STORE; a.Y = h->qkv; a.ldy = a.N;
-      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
-    }
-    {
-      AttnArgs aa{};
-      aa.st = h->dst; aa.qkv = h->qkv; aa.out = h->attn;
-      aa.kcache = m.kcache + (size_t)l * m.layer_bytes; aa.vcache = m.vcache + (size_t)l * m.layer_bytes;
-      aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = d;
-      aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
-      aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
-      CU(h, attn_launch(aa, st)); h->launches++;
-    }
-    {  // x += Wo o ; also sum(x^2) for the FFN norm
-      LinArgs a = base;
-      a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = d; a.M = rows;
-      if (c.dtype == 2) a.wscale[0] = m.wo_s[l];
-      a.X = h->attn; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
-      a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqB;
-      if (m.packed) { a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_gain = (const float*)m.ffn_norm[l]; a.yp_act = PRO_NONE; }
-      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      nB = pl.ssq_parts;
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
-    }
-    {  // up = Wup rmsnorm(x, g_ffn)
-      LinArgs a = base;
-      a.W[0] = m.w_up[l]; a.rows_per_mat = dff; a.N = dff; a.D = d; a.M = rows;
-      if (c.dtype == 2) a.wscale[0] = m.w_up_s[l];
-      a.X = h->x; a.ldx = d; a.x_row0 = 0; a.x_rowstep = 1;
-      a.pro = PRO_RMSNORM; a.gain = (const float*)m.ffn_norm[l]; a.ssq_in = h->ssqB; a.ssq_in_n = nB;
-      a.epi = EPI_STORE; a.Y = h->up; a.ldy = dff;
-      if (m.packed) {
-        a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo;
-        a.yp_hi = h->up_hi; a.yp_lo = h->up_lo; a.ldyp = dff; a.yp_gain = nullptr; a.yp_act = PRO_GELU;
-      }
-      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
-    }
-    {  // x += Wdown gelu(up) ; also sum(x^2) for the next norm
-      LinArgs a = base;
-      a.W[0] = m.w_down[l]; a.rows_per_mat = d; a.N = d; a.D = dff; a.M = rows;
-      if (c.dtype == 2) a.wscale[0] = m.w_down_s[l];
-      a.X = h->up; a.ldx = dff; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_GELU;
-      a.epi = EPI_RESIDUAL; a.Y = h->x; a.ldy = d; a.ssq_out = h->ssqA;
-      if (m.packed) {
-        a.xp_hi = h->up_hi; a.xp_lo = h->up_lo;
-        a.yp_hi = h->xp_hi; a.yp_lo = h->xp_lo; a.ldyp = d; a.yp_act = PRO_NONE;
-        a.yp_gain = (const float*)(l + 1 < c.n_layers ? m.attn_norm[l + 1] : m.final_norm);
-      }
-      const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
-      nA = pl.ssq_parts;
-      CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
-    }
-  }
-  if (ps.logits) {
-    LinArgs a = base;
-    a.W[0] = m.unembed; a.rows_per_mat = c.vocab; a.N = c.vocab; a.D = d; a.M = ps.lrows;
-    if (c.dtype == 2) a.wscale[0] = m.unembed_scale;
-    a.X = h->x; a.ldx = d; a.x_row0 = ps.lrow0; a.x_rowstep = ps.lrowstep;
-    a.pro = PRO_RMSNORM; a.gain = (const float*)m.final_norm; a.ssq_in = h->ssqA; a.ssq_in_n = nA;
-    if (m.packed) { a.xp_hi = h->xp_hi; a.xp_lo = h->xp_lo; }
-    a.epi = EPI_STORE; a.Y = ps.logits; a.ldy = ps.logits_ld;
-    const LinPlan pl = lin_plan(c.dtype, ps.lrows, a.N, a.D, h->num_sm);
-    CU(h, lin_launch(c.dtype, a, pl, st)); h->launches += lin_launch_count(pl);
-  }
-  return SPS_OK;
+  return run_pass_range(h, m, ps, 0, pass_phases(m));
 }
 
 // A pass over 17..128 rows (several sequences' K + 1 rows): the same layers, every linear layer as one GEMM on the
@@ -622,9 +692,10 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   if (!target_w || !cfg || !out) return fail(nullptr, SPS_EINVAL, "null argument");
   *out = nullptr;
   std::string why;
-  if (!check_model_cfg(cfg->target, why)) return fail(nullptr, SPS_EINVAL, "target: " + why);
+  const bool shard = (cfg->flags & SPS_CFG_TENSOR_PARALLEL) != 0;
+  if (!check_model_cfg(cfg->target, why, shard)) return fail(nullptr, SPS_EINVAL, "target: " + why);
   if (draft_w) {
-    if (!check_model_cfg(cfg->draft, why)) return fail(nullptr, SPS_EINVAL, "draft: " + why);
+    if (!check_model_cfg(cfg->draft, why, shard)) return fail(nullptr, SPS_EINVAL, "draft: " + why);
     if (cfg->draft.vocab != cfg->target.vocab) return fail(nullptr, SPS_EINVAL, "draft and target vocabularies differ");
   }
   if (cfg->max_K < 0 || cfg->max_K > SPS_MAX_K) return fail(nullptr, SPS_EINVAL, "max_K outside 0..15");
@@ -680,7 +751,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       wd = std::max(wd, (size_t)c.d_model); wf = std::max(wf, (size_t)c.d_ff);
       for (int n_out : {c.d_model + 2 * kv_width(c), c.d_ff, c.vocab}) wpart = std::max(wpart, wide_part_bound(n_out, h->num_sm));
     }
-    if (wd > 0 && !off) {
+    if (wd > 0 && !off && !shard) {     // (a tensor-parallel shard keeps the 16-row passes)
       struct WW { void** p; size_t bytes; };
       const WW ww[] = {{(void**)&h->wx, sizeof(float) * WIDE_ROWS * wd},       {(void**)&h->wqkv, sizeof(float) * WIDE_ROWS * 3 * wd},
                        {(void**)&h->watt, sizeof(float) * WIDE_ROWS * wd},     {(void**)&h->wpart, sizeof(float) * wpart},
@@ -718,6 +789,10 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->counters, sizeof(int) * (2 * LIN_MAX_R + 2)},
       {(void**)&h->tile_ctr, sizeof(int) * h->tile_ctr_ints},
       {(void**)&h->p_stats, sizeof(float2) * (size_t)MB * maxK},
+      {(void**)&h->tp_send, shard ? sizeof(float) * SPS_MAX_ROWS * (size_t)dmax : 16},
+      {(void**)&h->tp_inbox, shard ? sizeof(float) * 2 * SPS_TP_MAX_WORLD * SPS_MAX_ROWS * (size_t)dmax : 16},
+      {(void**)&h->tp_flags, sizeof(uint32_t) * SPS_TP_MAX_WORLD},
+      {(void**)&h->tp_epoch, sizeof(uint32_t) * 4},
       {(void**)&h->res, 4 * h->res_words},
       {(void**)&h->dst, sizeof(DevState)},
       {(void**)&s.n, 4 * (size_t)MB},
@@ -744,6 +819,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       cudaStreamSynchronize(h->stream) != cudaSuccess)
     return bail(fail(h, SPS_ECUDA, "state upload failed"));
   h->B = 1;
+  h->tp = shard;
+  h->tp_slot_floats = (size_t)SPS_MAX_ROWS * dmax;
   *out = h;
   return SPS_OK;
 }
@@ -757,7 +834,7 @@ int sps_destroy(sps_handle* h) {
   free_model(h->tgt);
   free_model(h->drf);
   void* bufs[] = {h->wdq, h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
-                  h->counters, h->tile_ctr, h->p_stats, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
+                  h->counters, h->tile_ctr, h->p_stats, h->tp_send, h->tp_inbox, h->tp_flags, h->tp_epoch, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);
   if (h->h_res) cudaFreeHost(h->h_res);
@@ -1161,6 +1238,117 @@ int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, cons
       return fail(nullptr, SPS_ETIMEOUT, "a bounded device-side wait ran out in the linear kernel");
   }
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("linear launch: ") + cudaGetErrorString(e));
+  return SPS_OK;
+}
+
+int sps_tp_buffers(sps_handle* h, void** inbox, void** flags, int64_t* inbox_bytes, int64_t* flags_bytes) {
+  if (!h || !inbox || !flags) return fail(h, SPS_EINVAL, "null argument");
+  if (!h->tp) return fail(h, SPS_ESTATE, "the handle was not created with SPS_CFG_TENSOR_PARALLEL");
+  *inbox = h->tp_inbox; *flags = h->tp_flags;
+  if (inbox_bytes) *inbox_bytes = (int64_t)(sizeof(float) * 2 * SPS_TP_MAX_WORLD * h->tp_slot_floats);
+  if (flags_bytes) *flags_bytes = (int64_t)(sizeof(uint32_t) * SPS_TP_MAX_WORLD);
+  return SPS_OK;
+}
+
+int sps_tp_attach(sps_handle* h, int32_t rank, int32_t world, void* const* peer_inbox, void* const* peer_flags) {
+  if (!h || !peer_inbox || !peer_flags) return fail(h, SPS_EINVAL, "null argument");
+  if (!h->tp) return fail(h, SPS_ESTATE, "the handle was not created with SPS_CFG_TENSOR_PARALLEL");
+  if (world < 1 || world > SPS_TP_MAX_WORLD || rank < 0 || rank >= world) return fail(h, SPS_EINVAL, "rank / world out of range (world <= 8)");
+  for (int w = 0; w < world; ++w) {
+    if (!peer_inbox[w] || !peer_flags[w]) return fail(h, SPS_EINVAL, "null peer buffer");
+    h->tp_peer_inbox[w] = (float*)peer_inbox[w];
+    h->tp_peer_flags[w] = (uint32_t*)peer_flags[w];
+  }
+  if (peer_inbox[rank] != (void*)h->tp_inbox || peer_flags[rank] != (void*)h->tp_flags)
+    return fail(h, SPS_EINVAL, "entry `rank` of the peer tables must be this handle's own buffers (sps_tp_buffers)");
+  CU(h, cudaSetDevice(h->cfg.device));
+  // exchanges are numbered from zero on every rank: attach all ranks before any of them runs a pass
+  CU(h, cudaMemsetAsync(h->tp_flags, 0, sizeof(uint32_t) * SPS_TP_MAX_WORLD, h->stream));
+  CU(h, cudaMemsetAsync(h->tp_epoch, 0, sizeof(uint32_t) * 4, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  h->tp_rank = rank; h->tp_world = world; h->tp_attached = true;
+  return SPS_OK;
+}
+
+// what the group calls check: `world` attached ranks of one group, in rank order, on one device and one stream
+static int tp_group_check(sps_handle* const* ranks, int world) {
+  if (!ranks || world < 1 || world > SPS_TP_MAX_WORLD) return fail(nullptr, SPS_EINVAL, "bad group");
+  for (int r = 0; r < world; ++r) {
+    sps_handle* h = ranks[r];
+    if (!h || !h->tp || !h->tp_attached || h->tp_world != world || h->tp_rank != r) return fail(h, SPS_EINVAL, "group member is not rank r of `world` attached ranks");
+    if (h->stream != ranks[0]->stream || h->cfg.device != ranks[0]->cfg.device)
+      return fail(h, SPS_EINVAL, "the ranks of an emulated group share one device and one stream");
+  }
+  return SPS_OK;
+}
+
+int sps_tp_group_prefill(sps_handle* const* ranks, int32_t world, const int32_t* toks, int32_t n) {
+  int rc = tp_group_check(ranks, world);
+  if (rc) return rc;
+  if (!toks) return fail(ranks[0], SPS_EINVAL, "null argument");
+  CU(ranks[0], cudaSetDevice(ranks[0]->cfg.device));
+  for (int r = 0; r < world; ++r)
+    if ((rc = set_sequences(ranks[r], toks, 1, n))) return rc;
+  for (int which = 0; which < 2; ++which) {
+    if (!(which == 0 ? ranks[0]->tgt : ranks[0]->drf).present) continue;
+    for (int c0 = 0; c0 < n - 1; c0 += SPS_MAX_ROWS) {
+      PassSpec ps{};
+      ps.mode = PASS_PREFILL; ps.c0 = c0; ps.rows_per_seq = (n - 1 - c0) < SPS_MAX_ROWS ? (n - 1 - c0) : SPS_MAX_ROWS;
+      const int phases = pass_phases(which == 0 ? ranks[0]->tgt : ranks[0]->drf);
+      // what `world` processes would each enqueue on their own GPU, here phase by phase on one stream: every rank's
+      // push of an exchange is enqueued before any rank's reduction of it, so no kernel ever waits on a later one
+      for (int ph = 0; ph < phases; ++ph)
+        for (int r = 0; r < world; ++r)
+          if ((rc = run_pass_range(ranks[r], which == 0 ? ranks[r]->tgt : ranks[r]->drf, ps, ph, ph + 1))) return rc;
+    }
+  }
+  CU(ranks[0], cudaStreamSynchronize(ranks[0]->stream));
+  for (int r = 0; r < world; ++r) ranks[r]->ready = true;
+  return SPS_OK;
+}
+
+int sps_tp_group_score(sps_handle* const* ranks, int32_t world, int32_t which, const int32_t* rows, int32_t n_rows,
+                       float* const* out_logits, float* out_ms) {
+  int rc = tp_group_check(ranks, world);
+  if (rc) return rc;
+  sps_handle* h0 = ranks[0];
+  if (!rows || !out_logits) return fail(h0, SPS_EINVAL, "null argument");
+  if (n_rows < 1 || n_rows > SPS_MAX_ROWS) return fail(h0, SPS_EINVAL, "n_rows outside 1..16");
+  CU(h0, cudaSetDevice(h0->cfg.device));
+  for (int r = 0; r < world; ++r) {
+    sps_handle* h = ranks[r];
+    ModelDev& m = which == 0 ? h->tgt : h->drf;
+    if (!h->ready || h->B != 1 || !m.present || !out_logits[r]) return fail(h, SPS_ESTATE, "group score needs a batch-1 prefill on every rank and a logits buffer per rank");
+    const int len = h->seq_len[0] - 1;
+    if (len + n_rows > h->cfg.max_seq) return fail(h, SPS_ERANGE, "rows would exceed max_seq");
+    for (int i = 0; i < n_rows; ++i) {
+      if (rows[i] < 0 || rows[i] >= m.cfg.vocab) return fail(h, SPS_ERANGE, "token id outside the vocabulary");
+      h->h_rows[i] = rows[i];
+      h->h_rows[SPS_MAX_ROWS + i] = len + i;
+    }
+    CU(h, cudaMemcpyAsync(h->hst.row_tok, h->h_rows, 4 * n_rows, cudaMemcpyHostToDevice, h->stream));
+    CU(h, cudaMemcpyAsync(h->hst.row_pos, h->h_rows + SPS_MAX_ROWS, 4 * n_rows, cudaMemcpyHostToDevice, h->stream));
+  }
+  CU(h0, cudaEventRecord(h0->ev[0], h0->stream));
+  const int phases = pass_phases(which == 0 ? h0->tgt : h0->drf);
+  for (int ph = 0; ph < phases; ++ph)
+    for (int r = 0; r < world; ++r) {
+      sps_handle* h = ranks[r];
+      ModelDev& m = which == 0 ? h->tgt : h->drf;
+      PassSpec ps{};
+      ps.mode = PASS_EXPLICIT; ps.rows_per_seq = n_rows; ps.logits = out_logits[r]; ps.logits_ld = m.cfg.vocab;
+      ps.lrow0 = 0; ps.lrowstep = 1; ps.lrows = n_rows;
+      if ((rc = run_pass_range(h, m, ps, ph, ph + 1))) return rc;
+    }
+  CU(h0, cudaEventRecord(h0->ev[1], h0->stream));
+  CU(h0, cudaStreamSynchronize(h0->stream));
+  if (out_ms) CU(h0, cudaEventElapsedTime(out_ms, h0->ev[0], h0->ev[1]));
+  for (int r = 0; r < world; ++r) {
+    int32_t errw = 0;
+    CU(ranks[r], cudaMemcpy(&errw, ranks[r]->hst.err, 4, cudaMemcpyDeviceToHost));
+    if (errw == 3) return fail(ranks[r], SPS_ETIMEOUT, "a bounded device-side wait ran out");
+    if (errw != 0) return fail(ranks[r], SPS_ERANGE, "device flagged a token id or position out of range");
+  }
   return SPS_OK;
 }
 

@@ -1,0 +1,80 @@
+"""Tensor-parallel scoring on the GPU: a group of rank handles emulated on one GPU (the library's group calls step
+the ranks through every pass phase by phase) against the oracle's UNSHARDED model and against an unsharded handle.
+The real kernels run: every rank streams only its shard of the weights, and the two exchanges per layer go through
+the push / reduce kernels and the inbox / flag buffers, with device pointers in place of peer mappings.
+Tolerances: logits within 1e-3 (fp32) / 5e-2 (bf16, int8) of the oracle; every rank's logits bit-identical."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_01318_b200 as sps
+import sps_synth
+from gpu_util import oracle_model
+from paper_2302_01318_b200 import tensor_parallel as tpar
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+TOL = {"tiny": 1e-3, "tiny_bf16": 5e-2, "tiny_q8": 5e-2, "tiny_gqa": 1e-3}
+
+
+@pytest.mark.parametrize("name,world,with_draft", [("tiny", 2, True), ("tiny", 4, False), ("tiny_bf16", 2, False),
+                                                   ("tiny_q8", 2, False), ("tiny_gqa", 2, False)])
+def test_group_scoring_equals_the_unsharded_model(name, world, with_draft):
+    c = sps_synth.CONFIGS[name]
+    wt = sps_synth.make_weights(c["target"], tag="target")
+    wd = sps_synth.make_weights(c["draft"], tag="draft") if with_draft else None
+    gt = sps_synth.weights_to(wt, DEV)
+    gd = sps_synth.weights_to(wd, DEV) if with_draft else None
+    g = tpar.Group(world, c["target"], gt, c["draft"] if with_draft else None, gd, max_seq=96, max_K=4)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(0, 40, V)                 # three prompt passes of up to 16 rows
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(1, 4, V)])
+    g.prefill(prompt)
+    outs = [torch.zeros((5, V), device=DEV) for _ in range(world)]
+    for which, cfg, w in ((0, c["target"], wt), (1, c["draft"], wd)):
+        if w is None:
+            continue
+        g.score(which, rows, outs)
+        torch.cuda.synchronize()
+        om = oracle_model(cfg, w, 96)
+        om.forward(prompt[:-1], np.arange(39), want_logits=False)
+        want = om.forward64(rows, np.arange(39, 44))
+        got = outs[0].cpu().numpy()
+        err = np.abs(got - want).max()
+        print(f"{name} x{world} model {which}: logit error vs the oracle {err:.2e}")
+        assert err < TOL[name], err
+        for r in range(1, world):
+            assert torch.equal(outs[r], outs[0])             # same summation order on every rank
+    # the unsharded handle on the same weights, same rows
+    h = sps.Handle(c["target"], gt, None, None, max_seq=96, max_K=4)
+    h.sps_prefill(prompt)
+    ref = torch.zeros((5, V), device=DEV)
+    g.score(0, rows, outs)
+    h.sps_score(0, rows, ref)
+    torch.cuda.synchronize()
+    assert (outs[0] - ref).abs().max().item() < TOL[name] * 0.1
+    # scoring again rewrites the same positions: same bits (exchange numbering carries on)
+    again = [torch.zeros((5, V), device=DEV) for _ in range(world)]
+    g.score(0, rows, again)
+    torch.cuda.synchronize()
+    assert torch.equal(again[0], outs[0])
+    h.close()
+    g.close()
+
+
+def test_tensor_parallel_handles_state_their_requirements():
+    c = sps_synth.CONFIGS["tiny"]
+    gt = sps_synth.weights_to(sps_synth.make_weights(c["target"], tag="target"), DEV)
+    sw = tpar.shard_weights(c["target"], gt, 0, 2)
+    sc = tpar.shard_config(c["target"], 2)
+    with pytest.raises(sps.SpsError):                         # a shard's shape without the flag
+        sps.Handle(sc, sw, None, None, max_seq=64)
+    h = sps.Handle(sc, sw, None, None, max_seq=64, flags=sps.CFG_TENSOR_PARALLEL)
+    with pytest.raises(sps.SpsError) as e:                    # a pass before the peers are attached
+        h.sps_prefill(sps_synth.make_prompt(0, 8, c["target"]["vocab"]))
+    assert e.value.code == sps.SPS_ESTATE
+    inbox, flags, nb, nf = h.tp_buffers()
+    assert inbox and flags and nb > 0 and nf > 0
+    with pytest.raises(sps.SpsError):                         # the own entry must be the own buffers
+        h.tp_attach(0, 2, [flags, inbox], [flags, flags])
+    h.close()
