@@ -48,6 +48,8 @@ extern "C" {
 #define SPS_FLAG_RESAMPLED 1u /* a draft was rejected; token drawn from norm(max(0, q - p)) */
 #define SPS_FLAG_BONUS 2u     /* all K drafts accepted; extra token drawn from q_{K+1}       */
 #define SPS_FLAG_FALLBACK 4u  /* rejected with sum max(0, q - p) == 0: token drawn from q_t  */
+#define SPS_FLAG_TIMEOUT 8u   /* sps_accept only: a bounded wait inside the kernel ran out; this
+                                 sequence's outputs are meaningless (handle calls return SPS_ETIMEOUT) */
 
 /* sps_cfg.flags */
 #define SPS_CFG_NO_GRAPH 1u   /* launch kernels one by one instead of replaying CUDA graphs  */

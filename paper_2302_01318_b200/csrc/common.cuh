@@ -350,6 +350,7 @@ struct AcceptArgs {
   int p_stats_ld;
   // set by the launcher (cluster form of the kernel): CTAs per sequence, tokens per CTA, rows resident in shared memory
   int csize, slice, resident, chunk, stages;
+  unsigned long long wait_ns;   // bound of the waits on the row copies
 };
 cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);
 // the thread-block-cluster form of the same sampler (unfiltered distributions); falls back to the kernel above when

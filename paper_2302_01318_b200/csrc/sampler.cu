@@ -611,7 +611,8 @@ struct AccfShared {
   float tot[ACCF_MAX_C];                     // the CTAs' weight totals
   int cand[ACCF_MAX_C], lastpos[ACCF_MAX_C];
   int wcand[SAMPLER_WARPS], wlast[SAMPLER_WARPS];
-  int stop;
+  int stop, timeout;
+  unsigned long long bar[ACCF_MAX_STAGES];   // one mbarrier per unit buffer
 };
 
 __device__ __forceinline__ uint32_t s_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -621,6 +622,25 @@ __device__ __forceinline__ void cp_async16(float* dst, const float* src) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// wait for a phase of an mbarrier, at most limit_ns of the global timer; false when the bound ran out
+__device__ __forceinline__ bool s_mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+  unsigned long long t0 = 0;
+  for (int spin = 0;; ++spin) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((spin & 63) == 63) {
+      unsigned long long t;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+      if (t0 == 0) t0 = t;
+      else if (t - t0 > limit_ns) return false;
+    }
+  }
+}
 
 __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptArgs a) {
   __shared__ AccfShared sh;
@@ -636,7 +656,13 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
   // A row's slice travels in chunks of CH floats (one chunk when the slice is short): unit u = (row u / NCH, chunk u % NCH).
   // Either every unit has a buffer of its own (`resident`: the rows stay for step 3), or the units go through a ring.
   const int CH = a.chunk, NCH = (slice_pad + CH - 1) / CH, U = R * NCH, NSTG = a.resident ? U : a.stages;
+  if (tid == 0) {
+    for (int i = 0; i < NSTG; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(s_smem_u32(&sh.bar[i])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    sh.timeout = 0;
+  }
   cluster.barrier_arrive();     // its wait stands before the first access to another CTA's shared memory: by then every CTA runs
+  __syncthreads();
   pdl_launch_dependents();
   pdl_wait();
   float T = a.temperature;
@@ -651,19 +677,21 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
   const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
   auto rowptr = [&](int r) { return r <= K ? qrow + (long long)r * V : prow + (long long)(r - K - 1) * V; };
   auto unit_floats = [&](int u) { const int ch = u % NCH; return max(0, min(CH, ns - ch * CH)); };
-  // units [u0, u0 + nb) on their way into their buffers: every thread copies its share, 16 bytes at a time, asynchronously
+  // units [u0, u0 + nb) on their way into their buffers: one bulk copy each (the copy engine works while the warps
+  // compute), completion counted on the buffer's mbarrier.  Issued by thread 0.
   auto issue_units = [&](int u0, int nb) {
     for (int j = 0; j < nb; ++j) {
-      const int u = u0 + j, r = u / NCH, ch = u - r * NCH, n4 = unit_floats(u) >> 2;
-      const float* src = rowptr(r) + i0 + (size_t)ch * CH;
-      float* dst = dyn + (size_t)(u % NSTG) * CH;
-      for (int q4 = tid; q4 < n4; q4 += SAMPLER_THREADS) cp_async16(dst + 4 * q4, src + 4 * q4);
+      const int u = u0 + j, r = u / NCH, ch = u - r * NCH;
+      const uint32_t bar = s_smem_u32(&sh.bar[u % NSTG]), bytes = (uint32_t)unit_floats(u) * 4u;
+      if (bytes == 0) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory"); continue; }
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(s_smem_u32(dyn + (size_t)(u % NSTG) * CH)), "l"(rowptr(r) + i0 + (size_t)ch * CH), "r"(bytes), "r"(bar) : "memory");
     }
-    cp_async_commit();
   };
   // resident: all units in one batch.  Ring: half the ring at a time, the other half is in flight meanwhile.
   const int units_at_once = a.resident ? U : max(1, NSTG / 2);
-  issue_units(0, min(units_at_once, U));
+  if (tid == 0) issue_units(0, min(U, a.resident ? U : NSTG));
   // the draft tokens' logits: asked for now, used by the chain
   if (tid >= 32 && tid < 32 + K) {
     const int t = tid - 32;
@@ -679,13 +707,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
   const int NSEG = max(1, SAMPLER_WARPS / units_at_once);
   for (int u0 = 0; u0 < U; u0 += units_at_once) {
     const int nb = min(units_at_once, U - u0);
-    // the next batch goes into the other half of the ring (every thread is past the last use of it: see the barrier
-    // at the end of the loop body), then this batch's copies are waited for
-    if (u0 + units_at_once < U) { issue_units(u0 + units_at_once, min(units_at_once, U - u0 - units_at_once)); cp_async_wait<1>(); }
-    else cp_async_wait<0>();
-    __syncthreads();              // everybody's copies of this batch have landed
     for (int item = warp; item < nb * NSEG; item += SAMPLER_WARPS) {
       const int j = item / NSEG, sg = item - j * NSEG, u = u0 + j;
+      // a warp waits for its own unit only: units that have landed are worked on while the others are in flight
+      if (!s_mbar_wait(s_smem_u32(&sh.bar[u % NSTG]), (uint32_t)((u / NSTG) & 1), a.wait_ns)) sh.timeout = 1;
       const float4* src = reinterpret_cast<const float4*>(dyn + (size_t)(u % NSTG) * CH);
       const int n4 = unit_floats(u) >> 2, per = (n4 + NSEG - 1) / NSEG, q0 = min(sg * per, n4), q1 = min(q0 + per, n4);
       float m = -INFINITY;
@@ -721,6 +746,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
       sh.row_m[tid] = rm; sh.row_s[tid] = rs;
     }
     __syncthreads();              // this batch's buffers and the segment scratch are free again
+    if (!a.resident && tid == 0 && u0 + NSTG < U) issue_units(u0 + NSTG, min(nb, U - u0 - NSTG));   // the units that take these buffers next
   }
   __syncthreads();
   // the C partial statistics of every row meet in every CTA
@@ -851,6 +877,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
     }
     break;
   }
+  if (sh.timeout) {   // a copy never arrived within the bound: the outputs mean nothing; say so
+    fl |= 8u;         // SPS_FLAG_TIMEOUT
+    if (a.st && tid == 0) atomicExch(a.st->err, 3);
+  }
   if (rank != 0) return;
   // ---- results (first CTA of the cluster)
   int32_t* out = a.out_tok + (long long)b * a.out_ld;
@@ -914,6 +944,7 @@ cudaError_t accept_launch_fast(const AcceptArgs& a_in, bool filtered, cudaStream
   AcceptArgs a = a_in;
   a.csize = C;
   a.slice = (((a.V + C - 1) / C) + 3) & ~3;
+  a.wait_ns = sps_wait_knobs().limit_ns;
   const int R = a.p_stats ? a.K + 1 : 2 * a.K + 1;
   const size_t slice_pad = (size_t)a.slice;
   const size_t wbytes = sizeof(float) * (slice_pad + slice_pad / 32 + 32);
