@@ -329,6 +329,8 @@ struct SampleArgs {        // one inverse-CDF draw per sequence from softmax(log
   int stats_ld;
 };
 cudaError_t sample_launch(const SampleArgs& a, cudaStream_t st);
+// the draw spread over a thread-block cluster (unfiltered distributions, large vocabularies); else the kernel above
+cudaError_t sample_launch_fast(const SampleArgs& a, bool filtered, cudaStream_t st);
 
 struct AcceptArgs {
   DevState* st;            // when non-null: T/seed/step from the state, and the loop is advanced
@@ -351,6 +353,12 @@ struct AcceptArgs {
   // set by the launcher (cluster form of the kernel): CTAs per sequence, tokens per CTA, rows resident in shared memory
   int csize, slice, resident, chunk, stages;
   unsigned long long wait_ns;   // bound of the waits on the row copies
+  // The cluster kernel as the draft sampler: K = 0, one row per sequence (q_logits, row stride q_ld), the draw uses
+  // u_draft of position sample_t, the token goes to out_tok[b * out_ld] and the row's (max, sum) to stats_out.
+  int sample_t;                 // < 0: accept mode
+  long long q_ld;               // sample mode: floats between consecutive sequences' rows
+  float2* stats_out;
+  int stats_ld;
 };
 cudaError_t accept_launch(const AcceptArgs& a, cudaStream_t st);
 // the thread-block-cluster form of the same sampler (unfiltered distributions); falls back to the kernel above when

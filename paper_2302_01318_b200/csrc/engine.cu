@@ -442,7 +442,7 @@ int enqueue_draft(sps_handle* h, int K) {
     sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = V; sa.B = B; sa.t = (uint32_t)t;
     sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
     sa.stats = h->p_stats + t; sa.stats_ld = h->hst.max_K;
-    CU(h, sample_launch(sa, h->stream)); h->launches++;
+    CU(h, sample_launch_fast(sa, h->filtered, h->stream)); h->launches++;
   }
   return SPS_OK;
 }
@@ -460,7 +460,7 @@ int enqueue_accept(sps_handle* h, int K) {
   aa.drafts_ld = h->hst.max_K; aa.B = h->B; aa.K = K; aa.V = h->tgt.cfg.vocab;
   aa.n_acc = h->hst.n_acc; aa.out_tok = h->hst.out_tok; aa.out_ld = h->hst.max_K + 1; aa.flags = h->hst.flags;
   // the draft rows' softmax statistics come from the kernel that drew the drafts (the same numbers the draws used)
-  aa.p_stats = K > 0 ? h->p_stats : nullptr; aa.p_stats_ld = h->hst.max_K;
+  aa.p_stats = K > 0 ? h->p_stats : nullptr; aa.p_stats_ld = h->hst.max_K; aa.sample_t = -1;
   CU(h, accept_launch_fast(aa, h->filtered, h->stream)); h->launches++;
   return SPS_OK;
 }
@@ -1121,7 +1121,7 @@ int sps_accept_filtered(const float* q_logits, const float* p_logits, const int3
   a.st = nullptr; a.q_logits = q_logits; a.p_logits = p_logits ? p_logits : q_logits;
   a.drafts = draft_tokens ? draft_tokens : out_tokens; a.drafts_ld = K;
   a.B = B; a.K = K; a.V = V; a.n_acc = out_n_accepted; a.out_tok = out_tokens; a.out_ld = K + 1; a.flags = out_flags;
-  a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p;
+  a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p; a.sample_t = -1;
   cudaError_t e = accept_launch_fast(a, (top_k >= 1 && top_k < V) || top_p < 1.f, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("accept launch: ") + cudaGetErrorString(e));
   return SPS_OK;
@@ -1142,7 +1142,7 @@ int sps_sample_filtered(const float* logits, int32_t B, int32_t V, float tempera
   SampleArgs a{};
   a.st = nullptr; a.logits = logits; a.ld = V; a.V = V; a.B = B; a.t = t; a.out = out_tokens; a.out_ld = 1;
   a.temperature = temperature; a.seed = seed; a.step = step; a.top_k = top_k; a.top_p = top_p;
-  cudaError_t e = sample_launch(a, (cudaStream_t)stream);
+  cudaError_t e = sample_launch_fast(a, (top_k >= 1 && top_k < V) || top_p < 1.f, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(nullptr, SPS_ECUDA, std::string("sample launch: ") + cudaGetErrorString(e));
   return SPS_OK;
 }

@@ -672,7 +672,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
   if (a.st) { T = a.st->temperature; seed = a.st->seed; step = a.st->step; seq += a.st->seq0; }
   const float invT = 1.0f / T;
   const float c2 = invT * 1.4426950408889634f;    // log2(e) / T
-  const float* qrow = a.q_logits + (long long)b * (K + 1) * V;
+  const float* qrow = a.sample_t >= 0 ? a.q_logits + (long long)b * a.q_ld : a.q_logits + (long long)b * (K + 1) * V;
   const float* prow = a.p_logits + (long long)b * K * V;
   const int32_t* drafts = a.drafts + (long long)b * a.drafts_ld;
   auto rowptr = [&](int r) { return r <= K ? qrow + (long long)r * V : prow + (long long)(r - K - 1) * V; };
@@ -848,7 +848,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
     float offset = 0.f, grand = 0.f;
     for (int c = 0; c < C; ++c) { if (c == rank) offset = grand; grand += sh.tot[c]; }
     if (residual && !(grand > 0.f)) { fl |= 4u; cluster.sync(); continue; }   // nothing left of q - p: draw from q_stop (every CTA decides the same)
-    const float target = u.u_res * grand;
+    const float target = (a.sample_t >= 0 ? sps_uniforms(seed, seq, step, (uint32_t)a.sample_t).u_draft : u.u_res) * grand;
     int cand = INT_MAX, last = -1;
     float cs = offset + pre_cta;
     for (int i = c0; i < c1; ++i) {
@@ -883,6 +883,13 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) accept_cluster_kernel(AcceptA
   }
   if (rank != 0) return;
   // ---- results (first CTA of the cluster)
+  if (a.sample_t >= 0) {   // the draft sampler: the token, and the row's statistics for the accept kernel
+    if (tid == 0) {
+      a.out_tok[(long long)b * a.out_ld] = tok;
+      if (a.stats_out) a.stats_out[(long long)b * a.stats_ld] = make_float2(sh.row_m[0], sh.row_s[0]);
+    }
+    return;
+  }
   int32_t* out = a.out_tok + (long long)b * a.out_ld;
   if (tid <= K) out[tid] = (tid < stop) ? sh.dtok[tid] : (tid == stop ? tok : -1);
   if (tid == 0) {
@@ -934,12 +941,28 @@ cudaError_t accept_launch(const AcceptArgs& a_in, cudaStream_t st) {
   return launch_k(accept_kernel, dim3(a.B), dim3(SAMPLER_THREADS), smem, st, a);
 }
 
+// the cluster form of the draft draw: the accept kernel with K = 0 and one row
+cudaError_t sample_launch_fast(const SampleArgs& s, bool filtered, cudaStream_t st) {
+  const int C = filtered ? 0 : accept_cluster_size(s.B, s.V);
+  const bool aligned = (s.V % 4 == 0) && ((s.ld & 3) == 0) && ((((size_t)s.logits) & 15) == 0);
+  if (C < 1 || !aligned) return sample_launch(s, st);
+  AcceptArgs a{};
+  a.st = const_cast<DevState*>(s.st); a.q_logits = s.logits; a.p_logits = s.logits; a.drafts = s.out; a.drafts_ld = 0;
+  a.B = s.B; a.K = 0; a.V = s.V; a.out_tok = s.out; a.out_ld = s.out_ld;
+  a.temperature = s.temperature; a.seed = s.seed; a.step = s.step;
+  a.sample_t = (int)s.t; a.q_ld = s.ld; a.stats_out = s.stats; a.stats_ld = s.stats_ld;
+  const cudaError_t e = accept_launch_fast(a, false, st);
+  if (e != cudaErrorInvalidValue) return e;
+  (void)cudaGetLastError();          // a shape the cluster kernel does not take: the one-CTA kernel
+  return sample_launch(s, st);
+}
+
 // the cluster form; `filtered` says whether top-k / nucleus filtering is in force (then the kernel above runs)
 cudaError_t accept_launch_fast(const AcceptArgs& a_in, bool filtered, cudaStream_t st) {
   const int C = filtered ? 0 : accept_cluster_size(a_in.B, a_in.V);
   // rows travel as bulk copies: 16-byte aligned row starts and slices
   const bool aligned = (a_in.V % 4 == 0) && ((((size_t)a_in.q_logits | (size_t)a_in.p_logits) & 15) == 0);
-  if (C < 1 || a_in.K > 15 || !aligned) return accept_launch(a_in, st);
+  if (C < 1 || a_in.K > 15 || !aligned) return a_in.sample_t >= 0 ? cudaErrorInvalidValue : accept_launch(a_in, st);
   static DevSmemCache cached{};
   AcceptArgs a = a_in;
   a.csize = C;
@@ -956,7 +979,7 @@ cudaError_t accept_launch_fast(const AcceptArgs& a_in, bool filtered, cudaStream
   } else {
     a.resident = 0;                                              // chunks of at most 32 KB through a ring; the weights reuse it afterwards
     a.chunk = a.slice < 8192 ? a.slice : 8192;
-    if (wbytes > budget) return accept_launch(a_in, st);         // a slice whose weights do not fit: one-CTA kernel
+    if (wbytes > budget) return a_in.sample_t >= 0 ? cudaErrorInvalidValue : accept_launch(a_in, st);   // a slice whose weights do not fit: one-CTA kernel
     int stages = (int)(budget / (sizeof(float) * a.chunk));
     const int units = R * ((a.slice + a.chunk - 1) / a.chunk);
     if (stages > units) stages = units;
