@@ -7,7 +7,12 @@
 // this pass's keys for itself and the group's first head alone appends them to the cache.  Rejected drafts are never erased: a row only
 // ever reads positions <= its own, and the next pass overwrites the stale ones ("rollback" is the
 // sequence length moving back, nothing else).
+#include <cooperative_groups.h>
+
+#include <cstdlib>
+
 #include "common.cuh"
+namespace cg = cooperative_groups;
 
 template <typename CT> struct CacheIO;
 template <> struct CacheIO<float> {
@@ -149,11 +154,20 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   float* row_a = row_l + MR;                                     // [MR] rescale of this tile
   int* pos_s = reinterpret_cast<int*>(row_a + MR);               // [MR]
   uint64_t* bar = reinterpret_cast<uint64_t*>(pos_s + MR);       // 8-byte aligned by construction
+  // split context: the first CTA of the cluster receives every CTA's (max, sum, unnormalised output) here
+  float* xo = reinterpret_cast<float*>(bar + 2);                 // [SPLIT][MR][DH]
+  float* xm = xo + (size_t)a.split * MR * DH;                    // [SPLIT][MR]
+  float* xl = xm + a.split * MR;                                 // [SPLIT][MR]
 
+  // The context of a (head, sequence) may be split over the `split` CTAs of a thread-block cluster (grid z): CTA c
+  // attends over positions [c * chunk, (c + 1) * chunk) and the partial results -- running maximum, sum and
+  // unnormalised output per query row -- meet in the first CTA's shared memory, where they are merged in CTA order.
+  const int SPLIT = a.split, crank = SPLIT > 1 ? (int)cg::this_cluster().block_rank() : 0;
+  if (SPLIT > 1) cg::this_cluster().barrier_arrive();   // waited for before the first remote store: by then every CTA runs
   const int h = blockIdx.x, b = a.seq0 + blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int Mb = a.rows_per_seq, row0 = blockIdx.y * Mb, d = a.d, max_seq = a.max_seq;
   const int group = a.H / a.Hkv, hk = h / group;   // the key / value head this query head reads
-  const bool appends = (h - hk * group) == 0;       // one head of a group writes the cache
+  const bool appends = (h - hk * group) == 0 && crank == 0;   // one CTA of one head of a group writes the cache
   const int ldq = d + 2 * a.Hkv * DH;                // row stride of the q | k | v buffer
   CT* kc = reinterpret_cast<CT*>(a.kcache) + ((size_t)b * a.Hkv + hk) * (size_t)max_seq * DH;
   CT* vc = reinterpret_cast<CT*>(a.vcache) + ((size_t)b * a.Hkv + hk) * (size_t)max_seq * DH;
@@ -172,6 +186,13 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   __syncthreads();
   int n_ctx = 0, n_old = max_seq;
   for (int i = 0; i < Mb; ++i) { n_ctx = max(n_ctx, pos_s[i] + 1); n_old = min(n_old, pos_s[i]); }
+  // this CTA's share of the context: [p0, p1) (a multiple of 8 positions per CTA, at least 32)
+  int p0 = 0, p1 = n_ctx;
+  if (SPLIT > 1) {
+    const int chunk = max(32, (((n_ctx + SPLIT - 1) / SPLIT) + 7) & ~7);
+    p0 = min(crank * chunk, n_ctx);
+    p1 = min(p0 + chunk, n_ctx);
+  }
   // Rows [0, n_old) were cached by earlier passes; rows >= n_old of a tile come from knew / vnew.
   // Of the old rows, [0, n_safe) were written before the host last waited for the stream (the host
   // waits once per loop and after the prompt pass), so they may be fetched before this kernel waits
@@ -181,35 +202,36 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   if (a.mode == PASS_VERIFY) n_safe = max(a.st->n[b] - 1, 0);
   else if (a.mode == PASS_DRAFT0 || a.mode == PASS_DRAFT_T) n_safe = max(a.st->n[b] - 2, 0);
   n_safe = min(n_safe, n_old);
-  auto copy_rows = [&](int r0, int r1) {   // cache rows [r0, r1) of tile 0 .. into the tile buffers
+  auto copy_rows = [&](int t0, int r0, int r1) {   // cache rows [r0, r1) into rows r0 - t0 .. of the tile buffers
     const uint32_t bytes = (uint32_t)(r1 - r0) * DH * (uint32_t)sizeof(CT);
-    const int tr = r0 % TP;
+    const int tr = r0 - t0;
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(a_smem_u32(Ks + tr * DH)), "l"(kc + (size_t)r0 * DH), "r"(bytes), "r"(bar_addr) : "memory");
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(a_smem_u32(Vs + tr * DH)), "l"(vc + (size_t)r0 * DH), "r"(bytes), "r"(bar_addr) : "memory");
     return 2 * bytes;
   };
-  // the part of a tile that is fetched after the wait; it also arrives on the tile's barrier
+  // the part of the tile that starts at t0 which is fetched after the wait; it also arrives on the tile's barrier
   auto issue_tile = [&](int t0, int from) {
-    const int r1 = min(t0 + TP, n_old);
+    const int r1 = min(min(t0 + TP, n_old), p1);
     if (r1 > from) {
       const uint32_t bytes = 2u * (uint32_t)(r1 - from) * DH * (uint32_t)sizeof(CT);
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
-      copy_rows(from, r1);
+      copy_rows(t0, from, r1);
     } else {
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
     }
   };
-  const int pre = min(TP, n_safe);   // rows of tile 0 fetched right away
+  const int pre_end = min(min(p0 + TP, n_safe), p1);   // rows [p0, pre_end) of the first tile are fetched right away
+  const int pre = max(pre_end - p0, 0);
   if (tid == 0 && pre > 0) {
     const uint32_t bytes = 2u * (uint32_t)pre * DH * (uint32_t)sizeof(CT);
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_addr), "r"(bytes) : "memory");
-    copy_rows(0, pre);
+    copy_rows(p0, p0, p0 + pre);
   }
   pdl_launch_dependents();
   pdl_wait();
-  if (tid == 0) issue_tile(0, pre);
+  if (tid == 0 && p1 > p0) issue_tile(p0, p0 + pre);
 
   // ---- rotary on q and k (adjacent pairs, angle = pos * base^(-2i/dh)); append k, v at the row's position
   for (int idx = tid; idx < Mb * (DH / 2); idx += ATTN_THREADS) {
@@ -242,8 +264,8 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
   float qreg[MR][DPL];   // this lane's dims of every query row (score phase)
   bool ok = true;
   int phase = 0;
-  for (int t0 = 0; t0 < n_ctx; t0 += TP, phase ^= 1) {
-    const int tn = min(TP, n_ctx - t0);   // positions of this tile
+  for (int t0 = p0; t0 < p1; t0 += TP, phase ^= 1) {
+    const int tn = min(TP, p1 - t0);   // positions of this tile
     if (!a_mbar_wait(bar_addr, (uint32_t)phase, a.st->err)) ok = false;
     __syncthreads();   // also: phase A's shared writes are visible
     // patch in the rows of this pass that fall into the tile
@@ -252,7 +274,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
       const int j = pos_s[i] - t0;
       if (j >= 0 && j < TP) { Ks[j * DH + e] = knew[idx]; Vs[j * DH + e] = vnew[idx]; }
     }
-    if (t0 == 0) {
+    if (t0 == p0) {
 #pragma unroll
       for (int i = 0; i < MR; ++i)
 #pragma unroll
@@ -331,18 +353,55 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
       }
     }
     __syncthreads();   // the tile buffers and sc are free again
-    if (tid == 0 && t0 + TP < n_ctx) issue_tile(t0 + TP, t0 + TP);
+    if (tid == 0 && t0 + TP < p1) issue_tile(t0 + TP, t0 + TP);
   }
 #pragma unroll
   for (int i = 0; i < MR; ++i)
     if (i < Mb) { red[(pg * MR + i) * DH + 2 * dp] = o[i][0]; red[(pg * MR + i) * DH + 2 * dp + 1] = o[i][1]; }
   __syncthreads();
+  if (SPLIT > 1) {
+    // every CTA's partial result goes to the first CTA of the cluster (distributed shared memory)
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.barrier_wait();
+    float* rxo = cluster.map_shared_rank(xo, 0) + (size_t)crank * MR * DH;
+    for (int idx = tid; idx < Mb * DH; idx += ATTN_THREADS) {
+      const int i = idx / DH, e = idx - i * DH;
+      float t = 0.f;
+#pragma unroll
+      for (int g = 0; g < PG; ++g) t += red[(g * MR + i) * DH + e];
+      rxo[i * DH + e] = ok ? t : 0.f;
+    }
+    if (tid < Mb) {
+      cluster.map_shared_rank(xm, 0)[crank * MR + tid] = (ok && p1 > p0) ? row_m[tid] : -INFINITY;
+      cluster.map_shared_rank(xl, 0)[crank * MR + tid] = (ok && p1 > p0) ? row_l[tid] : 0.f;
+    }
+    cluster.sync();
+    if (crank != 0) return;
+    // merge in CTA order: o = sum_c e^(m_c - M) o_c / sum_c e^(m_c - M) l_c
+    if (tid < Mb) {
+      float M = -INFINITY;
+      for (int c = 0; c < SPLIT; ++c) M = fmaxf(M, xm[c * MR + tid]);
+      float den = 0.f;
+      for (int c = 0; c < SPLIT; ++c) {
+        const float mc = xm[c * MR + tid];
+        const float w = (mc == -INFINITY) ? 0.f : expf(mc - M);
+        xm[c * MR + tid] = w;             // from here on: the CTA's weight
+        den += w * xl[c * MR + tid];
+      }
+      row_l[tid] = den;
+    }
+    __syncthreads();
+  }
   for (int idx = tid; idx < Mb * DH; idx += ATTN_THREADS) {
     const int i = idx / DH, e = idx - i * DH;
     float t = 0.f;
+    if (SPLIT > 1) {
+      for (int c = 0; c < SPLIT; ++c) t += xm[c * MR + i] * xo[((size_t)c * MR + i) * DH + e];
+    } else {
 #pragma unroll
-    for (int g = 0; g < PG; ++g) t += red[(g * MR + i) * DH + e];
-    const float val = ok ? t / row_l[i] : 0.f;
+      for (int g = 0; g < PG; ++g) t += red[(g * MR + i) * DH + e];
+    }
+    const float val = (ok && row_l[i] > 0.f) ? t / row_l[i] : 0.f;
     const size_t oi = (size_t)(row0 + i) * d + h * DH + e;
     a.out[oi] = val;
     if (a.out_hi) {
@@ -354,25 +413,50 @@ __global__ void __launch_bounds__(ATTN_THREADS) attn_kernel(AttnArgs a) {
 }
 
 template <int DH, typename CT, int MR>
-static size_t attn_smem_t() {
+static size_t attn_smem_t(int split) {
   constexpr int TP = ATTN_TILE_BYTES / (DH * (int)sizeof(CT));
   constexpr int PG = ATTN_THREADS / (DH / 2);
   return 2 * (size_t)ATTN_TILE_BYTES + 2 * (size_t)MR * DH * sizeof(CT) + sizeof(float) * ((size_t)MR * DH + (size_t)MR * TP + (size_t)PG * MR * DH + 3 * MR) +
-         sizeof(int) * MR + 16;
+         sizeof(int) * MR + 16 + sizeof(float) * (size_t)split * ((size_t)MR * DH + 2 * MR);
 }
 
 size_t attn_smem_bytes(int rows_per_seq, int max_seq, int dh) {
   (void)rows_per_seq; (void)max_seq; (void)dh;
-  return attn_smem_t<128, float, 16>();   // the largest instantiation
+  return attn_smem_t<128, float, 16>(1);   // the largest instantiation
+}
+
+// CTAs a (head, sequence) is split over: enough to put the SMs to work, as far as the exchange buffer (32 KB) allows
+static int attn_split(int heads_x_seqs, int MR, int DH) {
+  static const int forced = [] { const char* e = getenv("SPS_ATTN_SPLIT"); return e ? atoi(e) : 0; }();   // tuning: 1 = never split
+  int num_sm = SPS_NUM_SM_FALLBACK, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&num_sm, cudaDevAttrMultiProcessorCount, dev);
+  int s = num_sm / (heads_x_seqs > 0 ? heads_x_seqs : 1);
+  const int cap = 8192 / (MR * DH);        // exchange buffer: split x MR x DH floats <= 32 KB
+  if (s > cap) s = cap;
+  if (s > 8) s = 8;
+  if (forced > 0 && forced < s) s = forced;
+  return s < 1 ? 1 : s;
 }
 
 template <int DH, typename CT, int MR>
-static cudaError_t attn_go(const AttnArgs& a, cudaStream_t st) {
+static cudaError_t attn_go(const AttnArgs& a_in, cudaStream_t st) {
   static DevSmemCache cached{};   // per device, like the attribute itself
-  const size_t smem = attn_smem_t<DH, CT, MR>();
+  AttnArgs a = a_in;
+  a.split = attn_split(a.H * a.B, MR, DH);
+  const size_t smem = attn_smem_t<DH, CT, MR>(a.split);
   cudaError_t e = sps_ensure_smem(attn_kernel<DH, CT, MR>, smem, cached);
   if (e != cudaSuccess) return e;
-  return launch_k(attn_kernel<DH, CT, MR>, dim3(a.H, a.B), dim3(ATTN_THREADS), smem, st, a);
+  if (a.split == 1) return launch_k(attn_kernel<DH, CT, MR>, dim3(a.H, a.B), dim3(ATTN_THREADS), smem, st, a);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.H, a.B, a.split); cfg.blockDim = dim3(ATTN_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = a.split;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = sps_pdl_enabled() ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, attn_kernel<DH, CT, MR>, a);
 }
 
 template <int DH, typename CT>

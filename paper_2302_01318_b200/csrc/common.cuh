@@ -264,6 +264,7 @@ struct AttnArgs {
   int Hkv;                // key / value heads: query head h uses head h / (H / Hkv)
   int seq0;               // grid row y works on sequence seq0 + y (its cache and state) and on rows y * rows_per_seq .. of qkv / out
   int mode, t, c0;        // which rows the pass feeds (PassMode), as in EmbedArgs
+  int split;              // set by the launcher: CTAs (one thread-block cluster) that share a (head, sequence)'s context
 };
 cudaError_t attn_launch(const AttnArgs& a, cudaStream_t st);
 
