@@ -391,8 +391,13 @@ int sps_tp_attach(sps_handle* h, int32_t rank, int32_t world, void* const* peer_
  * with plain device pointers.  The calls enqueue what the `world` processes would, phase by phase (every rank's
  * store phase of an exchange before any rank's sum), so nothing ever waits for a kernel that is launched later.
  * sps_tp_group_prefill: as sps_prefill on every rank.  sps_tp_group_score: as sps_score on every rank; out_logits
- * host array of `world` DEVICE buffers [n_rows, vocab], which come out identical. */
+ * host array of `world` DEVICE buffers [n_rows, vocab], which come out identical.  sps_tp_group_generate: below. */
 int sps_tp_group_prefill(sps_handle* const* ranks, int32_t world, const int32_t* toks, int32_t n);
+/* sps_generate for the emulated group (one sequence): every rank drafts, scores and runs the accept kernel on its own
+ * copy of the logits; the ranks' decisions are compared after every loop (SPS_ESTATE if they ever differ) and rank 0's
+ * tokens are returned.  out_stats: counts and the decode time only. */
+int sps_tp_group_generate(sps_handle* const* ranks, int32_t world, const int32_t* prompt, int32_t prompt_len, int32_t n_new,
+                          int32_t K, float temperature, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats);
 int sps_tp_group_score(sps_handle* const* ranks, int32_t world, int32_t which, const int32_t* rows, int32_t n_rows,
                        float* const* out_logits, float* out_ms);
 

@@ -110,6 +110,7 @@ def lib():
         L.sps_tp_attach.argtypes = [vp, i32, i32, vp, vp]
         L.sps_tp_group_prefill.argtypes = [vp, i32, vp, i32]
         L.sps_tp_group_score.argtypes = [vp, i32, i32, vp, i32, vp, C.POINTER(f32)]
+        L.sps_tp_group_generate.argtypes = [vp, i32, vp, i32, i32, i32, f32, u64, vp, C.POINTER(sps_stats)]
         _lib = L
     return _lib
 

@@ -429,30 +429,42 @@ int run_pass_wide(sps_handle* h, ModelDev& m, const PassSpec& ps) {
 
 // K draft steps: step 0 feeds two rows per sequence (positions n-2, n-1) so that a draft cache left
 // one token behind by a fully accepted loop catches up in the same fixed-shape pass
+PassSpec draft_spec(sps_handle* h, int K, int t) {
+  const int V = h->tgt.cfg.vocab;
+  PassSpec ps{};
+  ps.mode = t == 0 ? PASS_DRAFT0 : PASS_DRAFT_T; ps.t = t; ps.K = K; ps.rows_per_seq = t == 0 ? 2 : 1;
+  ps.logits = h->p_logits + (size_t)t * V; ps.logits_ld = (long long)K * V;
+  ps.lrow0 = t == 0 ? 1 : 0; ps.lrowstep = t == 0 ? 2 : 1; ps.lrows = h->B;
+  return ps;
+}
+
+int enqueue_sample(sps_handle* h, int K, int t) {
+  const PassSpec ps = draft_spec(h, K, t);
+  SampleArgs sa{};
+  sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = h->tgt.cfg.vocab; sa.B = h->B; sa.t = (uint32_t)t;
+  sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
+  sa.stats = h->p_stats + t; sa.stats_ld = h->hst.max_K;
+  CU(h, sample_launch_fast(sa, h->filtered, h->stream)); h->launches++;
+  return SPS_OK;
+}
+
 int enqueue_draft(sps_handle* h, int K) {
-  const int V = h->tgt.cfg.vocab, B = h->B;
   for (int t = 0; t < K; ++t) {
-    PassSpec ps{};
-    ps.mode = t == 0 ? PASS_DRAFT0 : PASS_DRAFT_T; ps.t = t; ps.K = K; ps.rows_per_seq = t == 0 ? 2 : 1;
-    ps.logits = h->p_logits + (size_t)t * V; ps.logits_ld = (long long)K * V;
-    ps.lrow0 = t == 0 ? 1 : 0; ps.lrowstep = t == 0 ? 2 : 1; ps.lrows = B;
-    int rc = run_pass(h, h->drf, ps);
+    int rc = run_pass(h, h->drf, draft_spec(h, K, t));
     if (rc) return rc;
-    SampleArgs sa{};
-    sa.st = h->dst; sa.logits = ps.logits; sa.ld = ps.logits_ld; sa.V = V; sa.B = B; sa.t = (uint32_t)t;
-    sa.out = h->hst.drafts + t; sa.out_ld = h->hst.max_K;
-    sa.stats = h->p_stats + t; sa.stats_ld = h->hst.max_K;
-    CU(h, sample_launch_fast(sa, h->filtered, h->stream)); h->launches++;
+    if ((rc = enqueue_sample(h, K, t))) return rc;
   }
   return SPS_OK;
 }
 
-int enqueue_verify(sps_handle* h, int K) {
+PassSpec verify_spec(sps_handle* h, int K) {
   PassSpec ps{};
   ps.mode = PASS_VERIFY; ps.K = K; ps.rows_per_seq = K + 1;
   ps.logits = h->q_logits; ps.logits_ld = h->tgt.cfg.vocab; ps.lrow0 = 0; ps.lrowstep = 1; ps.lrows = h->B * (K + 1);
-  return run_pass(h, h->tgt, ps);
+  return ps;
 }
+
+int enqueue_verify(sps_handle* h, int K) { return run_pass(h, h->tgt, verify_spec(h, K)); }
 
 int enqueue_accept(sps_handle* h, int K) {
   AcceptArgs aa{};
@@ -1304,6 +1316,78 @@ int sps_tp_group_prefill(sps_handle* const* ranks, int32_t world, const int32_t*
   }
   CU(ranks[0], cudaStreamSynchronize(ranks[0]->stream));
   for (int r = 0; r < world; ++r) ranks[r]->ready = true;
+  return SPS_OK;
+}
+
+// one pass of every rank, phase by phase
+static int tp_group_pass(sps_handle* const* ranks, int world, int which, PassSpec (*spec)(sps_handle*, int, int), int K, int t) {
+  const int phases = pass_phases(which == 0 ? ranks[0]->tgt : ranks[0]->drf);
+  for (int ph = 0; ph < phases; ++ph)
+    for (int r = 0; r < world; ++r) {
+      const int rc = run_pass_range(ranks[r], which == 0 ? ranks[r]->tgt : ranks[r]->drf, spec(ranks[r], K, t), ph, ph + 1);
+      if (rc) return rc;
+    }
+  return SPS_OK;
+}
+static PassSpec verify_spec_t(sps_handle* h, int K, int) { return verify_spec(h, K); }
+
+int sps_tp_group_generate(sps_handle* const* ranks, int32_t world, const int32_t* prompt, int32_t P, int32_t n_new, int32_t K,
+                          float T, uint64_t seed, int32_t* out_tokens, sps_stats* out_stats) {
+  int rc = tp_group_check(ranks, world);
+  if (rc) return rc;
+  sps_handle* h0 = ranks[0];
+  if (!prompt || !out_tokens || n_new < 1 || P < 1 || !(T >= 0.f)) return fail(h0, SPS_EINVAL, "bad argument");
+  if ((long long)P + n_new + K > h0->cfg.max_seq) return fail(h0, SPS_ERANGE, "prompt_len + n_new + K exceeds max_seq");
+  CU(h0, cudaSetDevice(h0->cfg.device));
+  for (int r = 0; r < world; ++r) {
+    if ((rc = sps_reset(ranks[r]))) return rc;
+    if ((rc = check_K(ranks[r], K))) return rc;
+  }
+  if ((rc = sps_tp_group_prefill(ranks, world, prompt, P))) return rc;
+  for (int r = 0; r < world; ++r) {
+    int32_t lim = P + n_new;
+    CU(ranks[r], cudaMemcpy(ranks[r]->hst.limit, &lim, 4, cudaMemcpyHostToDevice));
+    if ((rc = write_params(ranks[r], T, seed, 0u))) return rc;
+  }
+  sps_stats st;
+  std::memset(&st, 0, sizeof(st));
+  const int MB = h0->cfg.max_batch, ld = h0->hst.max_K + 1;
+  int made = 0;
+  CU(h0, cudaEventRecord(h0->ev[5], h0->stream));
+  while (made < n_new) {
+    // what each rank's process would enqueue for one loop, interleaved phase by phase
+    for (int t = 0; t < K; ++t) {
+      if ((rc = tp_group_pass(ranks, world, 1, draft_spec, K, t))) return rc;
+      for (int r = 0; r < world; ++r) if ((rc = enqueue_sample(ranks[r], K, t))) return rc;
+    }
+    if ((rc = tp_group_pass(ranks, world, 0, verify_spec_t, K, 0))) return rc;
+    for (int r = 0; r < world; ++r) {
+      sps_handle* h = ranks[r];
+      if ((rc = enqueue_accept(h, K))) return rc;
+      CU(h, cudaMemcpyAsync(h->h_res, h->res, h->res_words * 4, cudaMemcpyDeviceToHost, h->stream));
+    }
+    CU(h0, cudaStreamSynchronize(h0->stream));
+    for (int r = 0; r < world; ++r) {
+      sps_handle* h = ranks[r];
+      h->last_K = K;
+      if (h->h_res[h->res_words - 1] == 3) return fail(h, SPS_ETIMEOUT, "a bounded device-side wait ran out");
+      if (h->h_res[h->res_words - 1] != 0) return fail(h, SPS_ERANGE, "device flagged a token id or position out of range");
+      // every rank holds the same residual stream bit for bit, hence the same logits, hence the same decisions
+      if (std::memcmp(h->h_res, h0->h_res, 4 * (h->res_words - 1)) != 0) return fail(h, SPS_ESTATE, "the ranks of the group decided differently");
+    }
+    const int a = h0->h_res[0];
+    add_loop_stats(&st, K, a, (uint32_t)h0->h_res[MB]);
+    for (int i = 0; i <= a; ++i) {
+      if (made < n_new) out_tokens[made++] = h0->h_res[2 * MB + i];
+      else st.overshoot += 1;
+    }
+    for (int r = 0; r < world; ++r) ranks[r]->seq_len[0] += a + 1;
+  }
+  CU(h0, cudaEventRecord(h0->ev[6], h0->stream));
+  CU(h0, cudaEventSynchronize(h0->ev[6]));
+  CU(h0, cudaEventElapsedTime(&st.ms_decode, h0->ev[5], h0->ev[6]));
+  if (out_stats) *out_stats = st;
+  (void)ld;
   return SPS_OK;
 }
 

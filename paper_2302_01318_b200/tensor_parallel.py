@@ -13,7 +13,7 @@ import ctypes as C
 
 import numpy as np
 
-from . import CFG_TENSOR_PARALLEL, Handle, _check, lib
+from . import CFG_TENSOR_PARALLEL, Handle, _check, lib, sps_stats
 
 ROW_SHARDED = ("wq", "wk", "wv", "w_up")       # by output rows
 COL_SHARDED = ("wo", "w_down")                 # by input columns
@@ -97,6 +97,15 @@ class Group:
         _check(lib().sps_tp_group_score(self._arr, self.world, which, r.ctypes.data_as(C.c_void_p), r.shape[0], outs, C.byref(ms)),
                self.ranks[0]._h)
         return ms.value
+
+    def generate(self, prompt, n_new, K, temperature, seed):
+        """The whole speculative loop on the emulated group: (tokens, stats of rank 0)."""
+        p = np.ascontiguousarray(prompt, dtype=np.int32)
+        out = np.zeros(n_new, dtype=np.int32)
+        st = sps_stats()
+        _check(lib().sps_tp_group_generate(self._arr, self.world, p.ctypes.data_as(C.c_void_p), p.shape[0], n_new, K, temperature, seed,
+                                           out.ctypes.data_as(C.c_void_p), C.byref(st)), self.ranks[0]._h)
+        return out, st.as_dict()
 
     def close(self):
         for h in self.ranks:

@@ -62,6 +62,31 @@ def test_group_scoring_equals_the_unsharded_model(name, world, with_draft):
     g.close()
 
 
+@pytest.mark.parametrize("name,world", [("tiny", 2), ("tiny", 4)])
+def test_group_generation_equals_the_oracle_loop(name, world):
+    """The whole loop under tensor parallelism (both models sharded, every rank drafting, scoring and sampling on its
+    own copy of the logits): rank 0's tokens equal the UNSHARDED oracle's outside flagged near ties, and the ranks never
+    decide differently (the call itself checks that after every loop)."""
+    import oracle
+    from gpu_util import oracle_generate, same_or_flagged
+    c = sps_synth.CONFIGS[name]
+    # four ranks need a draft with four heads: one layer of the target's width stands in for the two-head draft
+    dcfg = c["draft"] if c["draft"]["n_heads"] % world == 0 else dict(c["target"], n_layers=1, d_ff=512)
+    wt = sps_synth.make_weights(c["target"], tag="target")
+    wd = sps_synth.make_weights(dcfg, tag="draft")
+    g = tpar.Group(world, c["target"], sps_synth.weights_to(wt, DEV), dcfg, sps_synth.weights_to(wd, DEV), max_seq=128, max_K=4)
+    osps = oracle.Sps(oracle_model(c["target"], wt, 128), oracle_model(dcfg, wd, 128))
+    V = c["target"]["vocab"]
+    ok = 0
+    for seed in range(4):
+        prompt = sps_synth.make_prompt(seed, 16, V)
+        got, st = g.generate(prompt, 32, 4, 1.0, seed)
+        assert st["emitted"] - st["overshoot"] == 32 and st["loops"] == sum(st["hist_emitted"])
+        ok += same_or_flagged(got, oracle_generate(osps, prompt, 32, 4, 1.0, seed))
+    assert ok >= 3
+    g.close()
+
+
 def test_tensor_parallel_handles_state_their_requirements():
     c = sps_synth.CONFIGS["tiny"]
     gt = sps_synth.weights_to(sps_synth.make_weights(c["target"], tag="target"), DEV)
