@@ -1,7 +1,9 @@
-"""Multi-GPU = independent replicas.  A batch-1 speculative loop is a chain of dependent passes and does
-not shard; independent sequences do, trivially: rank r of W takes sequences r, r+W, ... (their Philox
-sequence index is the global sequence number, so results equal a single-GPU run), there is no collective
-on the data path, and the job's time is the maximum over ranks."""
+"""Multi-GPU throughput = independent replicas.  A batch-1 speculative loop is a chain of dependent passes;
+independent sequences shard trivially: rank r of W takes the global sequences r, r+W, ...  A sequence's
+global number selects its prompt and its seed (and, for batches, its Philox sequence index through
+`sps_set_sequence_index0`), so what a sequence generates does not depend on which rank ran it; there is no
+collective on the data path, and the job's time is the maximum over ranks.  (Sharding ONE sequence over
+GPUs is tensor parallelism: `tensor_parallel.py`.)"""
 from __future__ import annotations
 
 
