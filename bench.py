@@ -371,8 +371,9 @@ def run_ours(args):
                 "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
                 # one ncu capture of this kernel on the 32000 x 8192 layer: dram read + write = 1.0096 x the algorithmic bytes of
                 # that launch; traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
+                # (int8 weights: the capture of the 32768 x 8192 int8 layer gives 272.90 MB for 268.44 MB of weights, 1.0166 x)
                 "traffic": args.traffic if args.traffic is not None else
-                (1.0096 * vbytes / n_lin_verify if c["target"]["dtype"] == 1 else None)}
+                ({1: 1.0096, 2: 1.0166}.get(c["target"]["dtype"], 0) * vbytes / n_lin_verify or None)}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dec_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {0: "f32", 1: "bf16", 2: "f16"}[c["target"]["dtype"]], "data": "synthetic",
@@ -512,6 +513,8 @@ def run_ours(args):
     h.close()
     if rank == 0 and world == 1 and args.sweep and c["target"]["dtype"] == 1:
         line["sweep"] = sweep_bench(sps, c, wt, wd, local, peak)
+        # the variants above damp both models' output projections in place, so that is the pair the sweep ran on
+        line["sweep_models"] = "damped pair (acceptance in the paper's regime)" if args.aligned_steps > 0 else "random-init pair (natural acceptance)"
     if rank == 0 and world == 1 and args.mid_steps > 0 and cfgname != "mid":
         line.setdefault("variants", {})["mid"] = pair_variant(sps, "mid", local, peak, args.mid_steps)
     if rank == 0 and world == 1 and not args.no_sampler:

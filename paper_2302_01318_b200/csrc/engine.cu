@@ -507,6 +507,22 @@ int launch_phase(sps_handle* h, std::map<int, cudaGraphExec_t>& cache, int K, in
   return SPS_OK;
 }
 
+// the device's sticky status word after a pass the host has waited for: 0, 3 (a bounded wait ran out), else a range error
+int check_device_status(sps_handle* h) {
+  int32_t errw = 0;
+  CU(h, cudaMemcpy(&errw, h->hst.err, 4, cudaMemcpyDeviceToHost));
+  if (errw == 0) return SPS_OK;
+  if (errw == 3) {
+    // a kernel that gave up may have left arrival counters and tile queues half-way: clear them for the next call
+    cudaMemsetAsync(h->counters, 0, sizeof(int) * (2 * LIN_MAX_R + 2), h->stream);
+    cudaMemsetAsync(h->tile_ctr, 0, sizeof(int) * h->tile_ctr_ints, h->stream);
+    cudaMemsetAsync(h->res + (h->res_words - 1), 0, 4, h->stream);
+    cudaStreamSynchronize(h->stream);
+    return fail(h, SPS_ETIMEOUT, "a bounded device-side wait ran out");
+  }
+  return fail(h, SPS_ERANGE, "device flagged a token id or position out of range");
+}
+
 int write_params(sps_handle* h, float T, uint64_t seed, uint32_t step) {
   // temperature 0 = greedy decoding: the one-token limit of top-k, applied to both models
   const bool greedy = T == 0.f;
@@ -878,7 +894,7 @@ int sps_prefill(sps_handle* h, const int32_t* toks, int32_t n) {
   if (rc) return rc;
   if ((rc = prefill_all(h))) return rc;
   CU(h, cudaStreamSynchronize(h->stream));
-  return SPS_OK;
+  return check_device_status(h);
 }
 
 int sps_prefill_batch(sps_handle* h, const int32_t* toks, const int32_t* lens, int32_t B, int32_t ld) {
@@ -888,7 +904,7 @@ int sps_prefill_batch(sps_handle* h, const int32_t* toks, const int32_t* lens, i
   if (rc) return rc;
   if ((rc = prefill_all(h))) return rc;
   CU(h, cudaStreamSynchronize(h->stream));
-  return SPS_OK;
+  return check_device_status(h);
 }
 
 int sps_set_sequence_index0(sps_handle* h, uint32_t index0) {
@@ -1088,7 +1104,7 @@ int sps_score(sps_handle* h, int32_t which, const int32_t* rows, int32_t n_rows,
   CU(h, cudaEventRecord(h->ev[1], h->stream));
   CU(h, cudaStreamSynchronize(h->stream));
   if (out_ms) CU(h, cudaEventElapsedTime(out_ms, h->ev[0], h->ev[1]));
-  return SPS_OK;
+  return check_device_status(h);
 }
 
 int sps_verify(sps_handle* h, const int32_t* rows, int32_t K, float* out_logits, float* out_ms) {

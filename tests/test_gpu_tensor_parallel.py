@@ -87,6 +87,35 @@ def test_group_generation_equals_the_oracle_loop(name, world):
     g.close()
 
 
+def test_a_rank_whose_peer_never_arrives_gives_up_within_the_bound():
+    """The per-process form of a pass on rank 0 alone: its peer never stores its partial update nor raises its flag,
+    so the reduction's wait on that flag runs out (bound shortened to 3 ms), the kernel returns and the call reports
+    SPS_ETIMEOUT -- nothing hangs, and the group works afterwards."""
+    c = sps_synth.CONFIGS["tiny"]
+    wt = sps_synth.make_weights(c["target"], tag="target")
+    g = tpar.Group(2, c["target"], sps_synth.weights_to(wt, DEV), None, None, max_seq=64, max_K=4)
+    V = c["target"]["vocab"]
+    prompt = sps_synth.make_prompt(0, 8, V)
+    sps.sps_debug_set_wait(3000, -1)
+    try:
+        with pytest.raises(sps.SpsError) as e:
+            g.ranks[0].sps_prefill(prompt)          # a collective call made by one rank only
+        assert e.value.code == sps.SPS_ETIMEOUT
+    finally:
+        sps.sps_debug_set_wait(0, -1)
+    g.close()
+    # a fresh group on the same device is unaffected
+    g = tpar.Group(2, c["target"], sps_synth.weights_to(wt, DEV), None, None, max_seq=64, max_K=4)
+    g.prefill(prompt)
+    outs = [torch.zeros((1, V), device=DEV) for _ in range(2)]
+    g.score(0, prompt[-1:], outs)
+    torch.cuda.synchronize()
+    om = oracle_model(c["target"], wt, 64)
+    om.forward(prompt[:-1], np.arange(7), want_logits=False)
+    assert np.abs(outs[0].cpu().numpy() - om.forward64(prompt[-1:], [7])).max() < 1e-3
+    g.close()
+
+
 def test_tensor_parallel_handles_state_their_requirements():
     c = sps_synth.CONFIGS["tiny"]
     gt = sps_synth.weights_to(sps_synth.make_weights(c["target"], tag="target"), DEV)
