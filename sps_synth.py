@@ -27,6 +27,10 @@ CONFIGS = {
     # same pair with a 16-token vocabulary: exact end-to-end distribution tests
     "tiny16": dict(target=_cfg(2, 256, 4, 64, 1024, 16, 0), draft=_cfg(1, 128, 2, 64, 512, 16, 0),
                    prompt_len=16, n_new=3, K=4, T=1.0),
+    # the fp32 pair with a vocabulary of 8192: large enough for the samplers that spread a sequence over a thread-block
+    # cluster, small enough for token-exact parity against the oracle
+    "tiny_v8k": dict(target=_cfg(2, 256, 4, 64, 1024, 8192, 0), draft=_cfg(1, 128, 2, 64, 512, 8192, 0),
+                     prompt_len=16, n_new=48, K=4, T=1.0),
     # tiny shapes with bf16 storage: exercises the bf16 kernels at oracle-friendly size
     "tiny_bf16": dict(target=_cfg(2, 256, 2, 128, 1024, 1024, 1), draft=_cfg(1, 128, 1, 128, 512, 1024, 1),
                       prompt_len=16, n_new=64, K=4, T=1.0),

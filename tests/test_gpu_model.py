@@ -122,6 +122,32 @@ def test_token_parity_tiny_fp32(K):
     h.close()
 
 
+@pytest.mark.parametrize("K", [4, 1])
+def test_token_parity_with_the_cluster_samplers(K):
+    """Vocabulary 8192 (fp32 pair): the draft draws and the accept step run as thread-block-cluster kernels (a
+    sequence spread over 8 CTAs, the draft rows' softmax statistics handed from the draw to the accept step), inside
+    the loop and token-exact against the oracle per loop, outside flagged near ties.  Then three sequences at once
+    (clusters of 8 per sequence) with ragged progress."""
+    h, ot, od, c = make_pair("tiny_v8k")
+    V = c["target"]["vocab"]
+    loops = near = 0
+    worst = 0.0
+    for seed in range(4):
+        prompt = sps_synth.make_prompt(seed, c["prompt_len"], V)
+        l, n, w = teacher_forced(h, ot, od, prompt, c["n_new"], K, c["T"], seed)
+        loops += l; near += n; worst = max(worst, w)
+    print(f"V=8192 K={K}: {loops} loops, {near} near-tie mismatches, worst logit error {worst:.2e}")
+    assert worst < 1e-3 and near <= max(2, loops // 25)
+    h.close()
+    if K == 4:
+        hb, ots, ods, _ = make_pair_multi("tiny_v8k", 3, max_seq=128, max_K=K)
+        prompts = [sps_synth.make_prompt(40 + b, 10 + 2 * b, V) for b in range(3)]
+        loops, resyncs, worst, bad = teacher_forced_batch(hb, ots, ods, prompts, 20, K, 1.0, 9, 1e-3, index0=5, exact_tokens=True)
+        print(f"V=8192 batch 3: {loops} loops, {resyncs} re-syncs, {bad} unflagged decisions")
+        assert bad == 0
+        hb.close()
+
+
 @pytest.mark.parametrize("name", ["tiny_gqa", "tiny_mqa_bf16"])
 def test_grouped_key_value_heads(name):
     """Fewer key / value heads than query heads (grouped-query target 4 -> 2 and multi-query draft 2 -> 1 in fp32,

@@ -135,6 +135,53 @@ def test_accept_identical_models_and_zero_probabilities():
     compare_accept(q2, p, d2, 1.0, 8, 0)
 
 
+@pytest.mark.parametrize("B", [16, 4096])
+def test_cluster_sampler_joint_law_and_oracle_trials(B):
+    """Theorem 1 through the cluster kernels (vocabulary 8192; B = 16: eight CTAs per sequence, B = 4096: one, rows
+    through the chunk ring): six tokens carry all the mass, spread over the CTAs' slices, so the 2 x 6 cells
+    min(p, q) / max(0, q - p) are checked by chi-square over 2^17 trials (launch = loop index, row = sequence index),
+    and every trial is compared with the oracle's chain on the same uniforms."""
+    V, n = 8192, 1 << 17
+    live = np.array([5, 1030, 2047, 4100, 6000, 8191])
+    rng = np.random.default_rng(B)
+    p6, q6 = sm(rng.normal(size=6) * 1.5), sm(rng.normal(size=6) * 1.5)
+    lq = np.full(V, -1e4, dtype=np.float32); lq[live] = np.log(q6)
+    lp = np.full(V, -1e4, dtype=np.float32); lp[live] = np.log(p6)
+    ql = torch.from_numpy(np.tile(lq, (B, 2, 1))).to(DEV)
+    pl = torch.from_numpy(np.tile(lp, (B, 1, 1))).to(DEV)
+    d = torch.zeros((B, 1), dtype=torch.int32, device=DEV)
+    n_acc = torch.zeros(B, dtype=torch.int32, device=DEV)
+    toks = torch.zeros((B, 2), dtype=torch.int32, device=DEV)
+    flags = torch.zeros(B, dtype=torch.int32, device=DEV)
+    acc_all, tok_all, d_all = [], [], []
+    for step in range(n // B):
+        sps.sps_sample(pl.view(B, V), 1.0, 42, step, 0, d.view(B))
+        sps.sps_accept(ql, pl, d, 1.0, 42, step, n_acc, toks, flags)
+        acc_all.append(n_acc.cpu().numpy() == 1); tok_all.append(toks.cpu().numpy()[:, 0].copy()); d_all.append(d.cpu().numpy()[:, 0].copy())
+    acc, tok, dd = np.concatenate(acc_all), np.concatenate(tok_all), np.concatenate(d_all)
+    assert np.isin(tok, live).all() and np.isin(dd, live).all()
+    idx = np.searchsorted(live, tok)
+    cells = np.zeros((2, 6))
+    np.add.at(cells[0], idx[acc], 1)
+    np.add.at(cells[1], idx[~acc], 1)
+    assert chi_square_p(cells, np.stack([np.minimum(p6, q6), np.maximum(0, q6 - p6)])) > 1e-3
+    assert chi_square_p(cells.sum(0), q6) > 1e-3
+    assert chi_square_p(np.bincount(np.searchsorted(live, dd), minlength=6), p6) > 1e-3     # the drafts follow p
+    beta = np.minimum(p6, q6).sum()
+    assert abs(acc.mean() - beta) < 4 * np.sqrt(beta * (1 - beta) / n)
+    # trial by trial against the oracle (sampled: the oracle walks 8192-token rows)
+    bad = 0
+    for i in range(0, n, max(1, n // 3000)):
+        step, b = divmod(i, B)
+        tok_d, near_d = oracle.sample_row(lp, 1.0, oracle.uniforms(42, b, step, 0)[0])
+        r = oracle.accept_chain(np.stack([lq, lq]), lp[None], [int(dd[i])], 1.0, 42, b, step)
+        if dd[i] != tok_d and not near_d:
+            bad += 1
+        if (acc[i] != (r["n_accepted"] == 1) or tok[i] != r["tokens"][0]) and not r["flags"] & (oracle.FLAG_NEAR_ACCEPT | oracle.FLAG_NEAR_CDF):
+            bad += 1
+    assert bad == 0
+
+
 def test_accept_joint_law_on_gpu_million_trials():
     """Theorem 1 on the GPU path: 2^20 trials as batch rows (sequence index = trial), V = 16.
     Drafts come from sps_sample, the chain from sps_accept; cells follow min(p,q) / max(0,q-p)."""
