@@ -1258,7 +1258,12 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm) {
     int KS = 128;
     for (int k = 128; k <= ks_max && k <= D; k += 128) if (D % k == 0) KS = k;
     // a small layer (few 16-row tiles) leaves SMs idle with one long k-range: halve it while that doubles the work units
-    if (dtype == 1 && KS > 1024 && KS % 256 == 0 && (long long)((N + 15) / 16) * (D / KS) < 2LL * num_sm) KS /= 2;
+    // -- unless the layer has a single k-range, whose tiles are finished inside the kernel (per-tile epilogue): a second
+    // k-range would bring the epilogue kernel and its grid-wide wait back (SPS_LIN_HALVE_SINGLE=1: halve those too; tuning)
+    static const bool halve_single = [] { const char* e = getenv("SPS_LIN_HALVE_SINGLE"); return e && atoi(e) == 1; }();
+    if (dtype == 1 && KS > 1024 && KS % 256 == 0 && (long long)((N + 15) / 16) * (D / KS) < 2LL * num_sm &&
+        (D / KS > 1 || halve_single || !lin_tile_epilogue()))
+      KS /= 2;
     static const int kst_env = [] { const char* e = getenv("SPS_LIN_KST"); return e ? atoi(e) : 1024; }();
     int KST = 128;
     for (int k : {256, 512, 1024}) if (KS % k == 0 && k <= kst_env) KST = k;
