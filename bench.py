@@ -511,9 +511,12 @@ def run_ours(args):
                                                    "min": float(t.min()), "max": float(t.max())}})
             line["variants"]["k_sweep"] = sweep
     h.close()
+    if rank == 0 and world == 1 and args.mini_sweep and not args.sweep and c["target"]["dtype"] == 1 and cfgname.startswith("70b"):
+        line["sweep_mini"] = mini_sweep(sps, c, wt, wd, local, peak)
     if rank == 0 and world == 1 and args.sweep and c["target"]["dtype"] == 1:
         line["sweep"] = sweep_bench(sps, c, wt, wd, local, peak)
         # the variants above damp both models' output projections in place, so that is the pair the sweep ran on
+    if rank == 0 and world == 1 and ("sweep" in line or "sweep_mini" in line):
         line["sweep_models"] = "damped pair (acceptance in the paper's regime)" if args.aligned_steps > 0 else "random-init pair (natural acceptance)"
     if rank == 0 and world == 1 and args.mid_steps > 0 and cfgname != "mid":
         line.setdefault("variants", {})["mid"] = pair_variant(sps, "mid", local, peak, args.mid_steps)
@@ -557,6 +560,33 @@ def pair_variant(sps, cfgname, local, peak, steps):
             "ms_verify_per_loop": ms_v / loops, "ms_draft_per_step": ms_d / (loops * K), "ms_accept_per_loop": sum(x["ms_accept"] for x in st) / loops,
             "verify_gbs": v_gbs, "verify_frac": v_gbs / peak, "draft_gbs": d_gbs, "draft_frac": d_gbs / peak,
             "ar_frac": sps_synth.weight_bytes(c["target"]) * ar_tps / 1e9 / peak, "kernel_launches_per_loop": sum(x["kernel_launches"] for x in st) / loops}
+
+
+def mini_sweep(sps, c, wt, wd, local, peak):
+    """A compact cut of the K x batch sweep for the default line (the full one, `--sweep`, takes minutes): prompt 512,
+    64 new tokens, temperature 1, K in {1, 2, 4, 8} at batch 1 and 8, against autoregressive decoding at that batch;
+    per cell tokens/s over the batch, accepted drafts per target call and the scoring pass's time."""
+    P, n_new, V, T = 512, 64, c["target"]["vocab"], 1.0
+    out = []
+    for Bn in (1, 8):
+        hs = sps.Handle(c["target"], wt, c["draft"], wd, max_seq=((P + n_new + 8 + 63) // 64) * 64, max_batch=Bn, max_K=8, device=local)
+        prompts = np.stack([sps_synth.make_prompt(2000 + b, P, V) for b in range(Bn)])
+        ar = None
+        for K in (0, 1, 2, 4, 8):
+            hs.sps_generate_batch(prompts[:, :32], 8, K, T, 1)      # first use of (K, batch): eager run, then graph capture
+            _, st = hs.sps_generate_batch(prompts, n_new, K, T, 7)
+            ms, loops = st[0]["ms_decode"], max(s["loops"] for s in st)
+            tps = Bn * n_new / (ms / 1e3)
+            if K == 0:
+                ar = tps
+                continue
+            ms_v = st[0]["ms_verify"] / loops
+            out.append({"batch": Bn, "K": K, "value": tps, "ar": ar, "vs_ar": tps / ar,
+                        "accepted_per_call": sum(s["accepted"] for s in st) / sum(s["loops"] for s in st),
+                        "ms_verify": ms_v, "verify_frac": sps_synth.weight_bytes(c["target"]) / (ms_v / 1e3) / 1e9 / peak,
+                        "ms_draft_per_step": st[0]["ms_draft"] / (loops * K)})
+        hs.close()
+    return out
 
 
 def sweep_bench(sps, c, wt, wd, local, peak):
@@ -653,6 +683,8 @@ def main():
     ap.add_argument("--aligned-gamma", type=float, default=1e-4)
     ap.add_argument("--batch", type=int, default=8, help="also decode this many sequences together (0 / 1 = skip)")
     ap.add_argument("--sweep", action="store_true", help="also run the K x temperature x batch sweep (prompt 512, 256 tokens; minutes)")
+    ap.add_argument("--no-mini-sweep", dest="mini_sweep", action="store_false",
+                    help="skip the compact K x batch sweep of the default line (prompt 512, 64 tokens, K in {1,2,4,8}, batch 1 and 8)")
     ap.add_argument("--k-sweep-seeds", type=int, default=8, help="generations per K in --k-sweep")
     ap.add_argument("--k-sweep", action="store_true", help="also run the damped pair at K = 1, 2, 3, 4, 6, 8")
     ap.add_argument("--no-sampler", action="store_true", help="skip the standalone accept-kernel timings")

@@ -94,23 +94,21 @@ def test_linear_fp32(M, N, D):
 
 @pytest.mark.parametrize("N,D", [(8192, 8192), (8192, 32768), (32000, 8192), (24576, 6144)])
 def test_linear_full_size_sampled_rows(N, D):
-    """the 70B-shaped layers at full size, M = 5 as in the bench: 64 sampled output rows checked
-    one by one against the oracle's double dot products"""
+    """the 70B-shaped layers at full size, M = 5 as in the bench: EVERY output feature of every row against the
+    oracle's double dot products (the oracle splits the rows over the host's cores: a second or two per matrix)"""
     g = torch.Generator(device=DEV).manual_seed(N + D)
     W = torch.empty((N, D), device=DEV, dtype=torch.bfloat16).normal_(0, 0.02, generator=g)
     X = torch.randn((5, D), device=DEV, generator=g)
     got = run_linear(W, X)
-    rows = np.unique(np.concatenate([[0, 1, 15, 16, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 58)]))
-    Wr = sps_synth.to_numpy(W[torch.from_numpy(rows).to(DEV)])
-    want = oracle.linear(Wr, X.cpu().numpy())
-    assert np.abs(got[:, rows] - want).max() <= tol(W[:64].float(), X, D)
+    want = oracle.linear(sps_synth.to_numpy(W), X.cpu().numpy())
     assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= tol(W[:64].float(), X, D)
 
 
 @pytest.mark.parametrize("N,D", [(32768, 8192), (8192, 32768)])
 def test_linear_int8_full_size_sampled_rows(N, D):
-    """the 70B-shaped feed-forward matrices as int8 at full size (268 MB each), M = 5 as in the bench: sampled
-    output rows against the oracle's double dot products on the dequantised rows"""
+    """the 70B-shaped feed-forward matrices as int8 at full size (268 MB each), M = 5 as in the bench: every
+    output feature against the oracle's double dot products on the dequantised matrix"""
     g = torch.Generator(device=DEV).manual_seed(N + D)
     q = torch.randint(-127, 128, (N, D), device=DEV, generator=g, dtype=torch.int32).to(torch.int8)
     scale = (torch.rand(N, device=DEV, generator=g) * 1e-3 + 1e-4).float()
@@ -120,12 +118,10 @@ def test_linear_int8_full_size_sampled_rows(N, D):
     sps.sps_linear_scaled(q, scale, X, Y, ws)
     torch.cuda.synchronize()
     got = Y.cpu().numpy()
-    rows = np.unique(np.concatenate([[0, 1, 15, 16, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 58)]))
-    idx = torch.from_numpy(rows).to(DEV)
-    Wd = (q[idx].double() * scale[idx].double()[:, None]).float().cpu()
+    Wd = (q.double() * scale.double()[:, None]).float().cpu()     # the dequantised matrix the oracle's model is defined on
     want = oracle.linear(Wd.numpy(), X.cpu().numpy())
-    assert np.abs(got[:, rows] - want).max() <= tol(Wd, X.cpu(), D)
     assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= tol(Wd[:4096], X.cpu(), D)
 
 
 
@@ -156,13 +152,15 @@ def test_linear_wide_small(M, N, D):
 
 @pytest.mark.parametrize("N,D", [(32768, 8192), (8192, 32768)])
 def test_linear_wide_full_size_sampled_rows(N, D):
-    """the 70B-shaped feed-forward matrices at full size with the prompt's 127 rows: sampled output features of
-    every row against the oracle's double dot products"""
+    """the 70B-shaped feed-forward matrices at full size with the prompt's 127 rows: every 16th output feature (one
+    per 16-row group of every 256-row tile, plus the tiles' edges) of every row against the oracle's double dot
+    products -- all of them would be 34 G multiply-adds of oracle time per matrix"""
     g = torch.Generator(device=DEV).manual_seed(N + D)
     W = torch.empty((N, D), device=DEV, dtype=torch.bfloat16).normal_(0, 0.02, generator=g)
     X = torch.randn((127, D), device=DEV, generator=g)
     got = run_linear_wide(W, X)
-    rows = np.unique(np.concatenate([[0, 1, 255, 256, N - 1, N - 2], np.random.default_rng(0).integers(0, N, 26)]))
+    rows = np.unique(np.concatenate([[0, 1, 255, 256, N - 1, N - 2], np.arange(0, N, 16) + (np.arange(0, N, 16) // 16) % 16]))
+    rows = rows[rows < N]
     Wr = sps_synth.to_numpy(W[torch.from_numpy(rows).to(DEV)])
     want = oracle.linear(Wr, X.cpu().numpy())
     assert np.abs(got[:, rows] - want).max() <= tol(W[:64].float(), X.cpu(), D)
