@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsps_b200.so")
-SOURCES = ["engine.cu", "linear.cu", "attention.cu", "sampler.cu", "wide.cu", "tp.cu"]
+SOURCES = ["engine.cu", "linear.cu", "linear_tc.cu", "attention.cu", "sampler.cu", "wide.cu", "tp.cu"]
 HEADERS = ["common.cuh", os.path.join("..", "..", "include", "sps.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC",
               "-shared"]
@@ -24,7 +24,8 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+        extra = os.environ.get("SPS_NVCC_EXTRA", "").split()   # e.g. -D switches of a debugging build
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
         subprocess.check_call(cmd)
     return LIB
 

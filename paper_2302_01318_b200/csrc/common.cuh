@@ -78,7 +78,8 @@ inline cudaError_t sps_ensure_smem(Kern k, size_t bytes, DevSmemCache& c) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= SPS_MAX_DEVICES) return cudaErrorInvalidDevice;
-  if (!c.init) { for (size_t& b : c.bytes) b = 48 * 1024; c.init = true; }
+  // 48 KB is the limit for static and dynamic shared memory TOGETHER unless the attribute says more: set it from 32 KB on
+  if (!c.init) { for (size_t& b : c.bytes) b = 32 * 1024; c.init = true; }
   if (bytes <= c.bytes[dev]) return cudaSuccess;
   e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
   if (e == cudaSuccess) c.bytes[dev] = bytes;
@@ -222,6 +223,11 @@ struct LinArgs {
   // the output); the activations' halves are then fp16, not bf16 -- in the slab and in the packed arrays.
   const float* wscale[3];
   int q8;                       // set by the launcher
+  // Tensor-core kernel (lin_tc_kernel; set by the launcher, sk_R = 0 otherwise).  Within a k-split the sk_tot stages of
+  // the layer (sk_SPT per 128-row tile) are cut into sk_R equal pieces, one per CTA; a piece that starts inside a
+  // tile leaves its partial sums in carry[cta][m][row of the tile] instead of part, and the epilogue adds them in.
+  float* carry;                 // [LIN_TC_MAX_CTAS][SPS_MAX_ROWS][128], null = the kernel is not used
+  int sk_R, sk_SPT, sk_tot, sk_BR;   // sk_BR: weight rows per tile (64 or 128)
 };
 
 struct LinPlan { int R, S, WC, PR, NT, variant, KS, KST, NS, G, ssq_parts, tile_epi; size_t smem; };
@@ -230,6 +236,11 @@ LinPlan lin_plan(int dtype, int M, int N, int D, int num_sm);
 int lin_launch_count(const LinPlan& p);   // kernels one lin_launch enqueues
 cudaError_t lin_launch(int dtype, const LinArgs& a, const LinPlan& p, cudaStream_t st);
 size_t lin_part_floats(int N, int S_max);
+#define LIN_TC_MAX_CTAS 160
+inline size_t lin_carry_floats() { return (size_t)LIN_TC_MAX_CTAS * SPS_MAX_ROWS * 128; }
+struct LinTcPlan { int KBS, KBX, NS, NGRP, BR, R, SPT, tot; size_t smem; };
+bool lin_tc_plan(const LinArgs& a, const LinPlan& p, LinTcPlan* out);     // can the layer run on the tcgen05 kernel, and how
+cudaError_t lin_tc_launch(const LinArgs& a, const LinTcPlan& t, cudaStream_t st);
 void sps_set_global_error(const char* msg);   // text returned by sps_last_error(NULL)
 #define LIN_MAX_R 512
 // partial sums of squares: the partials of one row are neighbours, so a warp fetches them with a few coalesced loads

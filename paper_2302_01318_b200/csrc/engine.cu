@@ -58,6 +58,7 @@ struct sps_handle {
   void* wdq = nullptr;   // bf16 copy of the int8 matrix (or q | k | v) the prompt-pass GEMM is reading
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
+  size_t part_floats = 0;   // floats of `part` ahead of the carry tiles
   int* counters = nullptr;
   // tensor parallelism (SPS_CFG_TENSOR_PARALLEL): this handle holds one rank's shard of both models
   bool tp = false;           // the models are shards: n_heads * d_head may be less than d_model
@@ -254,7 +255,7 @@ int run_pass_range(sps_handle* h, ModelDev& m, const PassSpec& ps, int ph0, int 
   if (h->tp && !h->tp_attached) return fail(h, SPS_ESTATE, "tensor-parallel handle: sps_tp_attach has not been called");
   cudaStream_t st = h->stream;
   LinArgs base{};
-  base.part = h->part; base.counters = h->counters; base.tile_ctr = h->tile_ctr; base.eps = c.rms_eps;
+  base.part = h->part; base.carry = h->part + h->part_floats; base.counters = h->counters; base.tile_ctr = h->tile_ctr; base.eps = c.rms_eps;
   base.err = h->hst.err;
   const int last = pass_phases(m) - 1;
   for (int ph = ph0; ph < ph1; ++ph) {
@@ -370,9 +371,9 @@ int run_pass_range(sps_handle* h, ModelDev& m, const PassSpec& ps, int ph0, int 
 int run_pass(sps_handle* h, ModelDev& m, const PassSpec& ps) {
   const sps_model_cfg& c = m.cfg;
   const int rows = h->B * ps.rows_per_seq;
-  // 9..16 rows: the tensor-core GEMM path also beats the 16-row weight-streaming variant (which is bound by shared-memory
-  // bandwidth) when the model can take it; SPS_WIDE_MIN_ROWS moves the switch (tuning only)
-  static const int wide_min = [] { const char* e = getenv("SPS_WIDE_MIN_ROWS"); return e ? atoi(e) : 9; }();
+  // Up to 16 rows stream the weights once (for bf16 models through the tcgen05 weight-streaming kernel, which carries 16 rows
+  // at the cost of one); the GEMM path takes over above that.  SPS_WIDE_MIN_ROWS moves the switch (tuning only).
+  static const int wide_min = [] { const char* e = getenv("SPS_WIDE_MIN_ROWS"); return e ? atoi(e) : 17; }();
   if (rows > SPS_MAX_ROWS || (rows >= wide_min && h->wide && c.dtype == 1 && (!ps.logits || (ps.lrow0 == 0 && ps.lrowstep == 1 && ps.lrows == rows))))
     return run_pass_wide(h, m, ps);
   return run_pass_range(h, m, ps, 0, pass_phases(m));
@@ -761,6 +762,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
   const size_t pf2 = model_part_floats(h->drf, h->num_sm);
   if (pf2 > part_floats) part_floats = pf2;
   if (part_floats == 0) part_floats = 1;
+  part_floats = (part_floats + 63) / 64 * 64;
+  h->part_floats = part_floats;
   h->res_words = (size_t)MB * 2 + (size_t)MB * (maxK + 1) + 1;
   {
     int n_max = V;
@@ -813,7 +816,7 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->ssqB, sizeof(float) * LIN_MAX_R * SPS_MAX_ROWS},
       {(void**)&h->q_logits, sizeof(float) * MR * (size_t)V},
       {(void**)&h->p_logits, sizeof(float) * PR * (size_t)V},
-      {(void**)&h->part, sizeof(float) * part_floats},
+      {(void**)&h->part, sizeof(float) * (part_floats + lin_carry_floats())},   // split-K partial sums, then the tensor-core kernel's carry tiles
       {(void**)&h->counters, sizeof(int) * (2 * LIN_MAX_R + 2)},
       {(void**)&h->tile_ctr, sizeof(int) * h->tile_ctr_ints},
       {(void**)&h->p_stats, sizeof(float2) * (size_t)MB * maxK},
@@ -1184,8 +1187,8 @@ static int cur_num_sm() {
 int64_t sps_linear_workspace_bytes(int32_t dtype, int32_t M, int32_t N, int32_t D) {
   if (M < 1 || M > SPS_MAX_ROWS || N < 1 || D < 1 || dtype < 0 || dtype > 2) return -1;
   const LinPlan p = lin_plan(dtype, M, N, D, cur_num_sm());
-  return (int64_t)(sizeof(float) * (lin_part_floats(N, p.S) + (size_t)LIN_MAX_R * SPS_MAX_ROWS) + sizeof(int) * (2 * LIN_MAX_R + 2) + 256 +
-                   ((sizeof(int) * lin_tile_ctr_ints(N) + 255) / 256) * 256);
+  return (int64_t)(sizeof(float) * ((lin_part_floats(N, p.S) + 63) / 64 * 64 + lin_carry_floats() + (size_t)LIN_MAX_R * SPS_MAX_ROWS) +
+                   sizeof(int) * (2 * LIN_MAX_R + 2) + 256 + ((sizeof(int) * lin_tile_ctr_ints(N) + 255) / 256) * 256);
 }
 
 int64_t sps_linear_wide_workspace_bytes(int32_t N, int32_t D) {
@@ -1251,6 +1254,7 @@ int sps_linear_scaled(const void* W, int32_t dtype, const float* row_scale, cons
   off += ((sizeof(int) * lin_tile_ctr_ints(N) + 255) / 256) * 256;
   off += sizeof(float) * (size_t)LIN_MAX_R * SPS_MAX_ROWS;
   a.part = (float*)(ws + off);
+  a.carry = a.part + (lin_part_floats(N, p.S) + 63) / 64 * 64;
   cudaStream_t st = (cudaStream_t)stream;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   cudaError_t e = cudaMemsetAsync(a.counters + 2 * LIN_MAX_R + 1, 0, sizeof(int), st);   // the sticky error word starts clear

@@ -177,6 +177,142 @@ __device__ void lin_epilogue(const LinArgs& a, int r, int row_begin, int nrows, 
 // order afterwards; ssq_s: 16 shared floats that carry the per-row sums across chunks.
 __device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 
+// Tensor-core kernel: CTA r of a k-split owns stages [r tot / R, (r + 1) tot / R).  If such a boundary lies strictly inside
+// the tile (sk_BR weight rows) of output feature n, the CTA that starts there left its piece in carry[(r S + s)][m][n mod 128]; this
+// returns the address for k-split 0, activation row 0 (k-splits are SPS_MAX_ROWS * 128 floats apart), or null.
+__device__ __forceinline__ const float* lin_carry_of(const LinArgs& a, int n) {
+  // 32-bit arithmetic: stages of a k-split x row ranges stays far below 2^31 (the launcher checks)
+  const uint32_t t = (uint32_t)n / (uint32_t)a.sk_BR;
+  const uint32_t end = (t + 1u) * (uint32_t)a.sk_SPT;                       // one past the tile's last stage
+  const uint32_t r_hi = (end * (uint32_t)a.sk_R - 1u) / (uint32_t)a.sk_tot;  // the CTA that owns that last stage
+  const uint32_t b = (r_hi * (uint32_t)a.sk_tot) / (uint32_t)a.sk_R;         // where its piece starts
+  if (b <= t * (uint32_t)a.sk_SPT) return nullptr;
+  return a.carry + (size_t)r_hi * a.S * SPS_MAX_ROWS * 128 + ((uint32_t)n - t * (uint32_t)a.sk_BR);
+}
+
+// The epilogue kernel's slice: output features [n_first, n_first + rows_all) of every activation row, 16 warps.  Warps
+// 2 m' and 2 m' + 1 finish rows m' and m' + 8: a lane of half h takes the work items (4 features, or 1) 32 h + lane,
+// + 64, ... of its row.  Everything an item needs -- the row's 1/rms, the old value of a residual update, the S partial
+// sums, the carry pieces of the tensor-core kernel, the gain of the packed copy -- is asked for before any of it is
+// used: the slice costs one trip to L2.  A row's sum of squares is the lanes' sums (items in index order) added in the
+// fixed shuffle tree, first half then second: it depends neither on the number of rows nor on which row it is.
+__device__ void lin_epilogue_rows(const LinArgs& a, int part_idx, int n_first, int rows_all, const float* row_scale, float (*s_half)[2]) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, half = warp & 1;
+  const int S = a.S, N = a.N;
+  const bool resid = a.epi == EPI_RESIDUAL;
+  const bool vec = (((N | n_first | rows_all | a.rows_per_mat | a.rows_tail) & 3) == 0) && ((a.ldy & 3) == 0) &&
+                   (!a.wscale[0] || (((size_t)a.wscale[0] | (size_t)a.wscale[1] | (size_t)a.wscale[2]) & 15) == 0) &&
+                   ((((size_t)a.Y | (size_t)a.part) & 15) == 0) &&
+                   (!a.yp_hi || (((a.ldyp & 3) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 7) == 0) &&
+                                 (!a.yp_gain || (((size_t)a.yp_gain & 15) == 0))));
+  const size_t sstride = (size_t)SPS_MAX_ROWS * N, cstride = (size_t)SPS_MAX_ROWS * 128;
+  for (int m = warp >> 1; m < a.M; m += 8) {
+    float ssq = 0.f;
+    const float rs = row_scale ? __ldcg(row_scale + m) : 1.f;
+    if (vec) {
+      const int items = rows_all >> 2;
+      for (int i = half * 32 + lane; i < items; i += 64) {
+        const int n = n_first + 4 * i;
+        float* dst = a.Y + (long long)m * a.ldy + n;
+        const float* src = a.part + (size_t)m * N + n;
+        const float* cp = a.sk_R ? lin_carry_of(a, n) : nullptr;
+        float4 old = make_float4(0.f, 0.f, 0.f, 0.f), gn = make_float4(1.f, 1.f, 1.f, 1.f), ws = gn, y = old;
+        if (resid) old = __ldcg(reinterpret_cast<const float4*>(dst));
+        if (a.yp_hi && a.yp_gain) gn = __ldg(reinterpret_cast<const float4*>(a.yp_gain + n));
+        if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: every matrix has a multiple of 4 rows)
+          int rin;
+          const int mat = mat_of(a, n, rin);
+          ws = __ldg(reinterpret_cast<const float4*>(a.wscale[mat] + rin));
+        }
+        if (S <= 4) {
+          float4 v[4], c[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            v[j] = j < S ? __ldcg(reinterpret_cast<const float4*>(src + j * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            c[j] = (cp && j < S) ? __ldcg(reinterpret_cast<const float4*>(cp + (size_t)m * 128 + j * cstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          y = f4_add(f4_add(f4_add(v[0], v[1]), v[2]), v[3]);
+          if (cp) y = f4_add(f4_add(f4_add(f4_add(y, c[0]), c[1]), c[2]), c[3]);
+        } else {
+          for (int s0 = 0; s0 < S; s0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              v[j] = s0 + j < S ? __ldcg(reinterpret_cast<const float4*>(src + (s0 + j) * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
+          }
+          if (cp)
+            for (int s0 = 0; s0 < S; s0 += 8) {
+              float4 c[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                c[j] = s0 + j < S ? __ldcg(reinterpret_cast<const float4*>(cp + (size_t)m * 128 + (s0 + j) * cstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) y = f4_add(y, c[j]);
+            }
+        }
+        if (a.wscale[0]) { y.x *= ws.x; y.y *= ws.y; y.z *= ws.z; y.w *= ws.w; }
+        if (row_scale) { y.x *= rs; y.y *= rs; y.z *= rs; y.w *= rs; }
+        if (resid) {
+          y = f4_add(y, old);
+          ssq += ((y.x * y.x + y.y * y.y) + y.z * y.z) + y.w * y.w;
+        }
+        *reinterpret_cast<float4*>(dst) = y;
+        if (a.yp_hi) {
+          if (a.yp_act == PRO_GELU) { y.x = gelu_fast(y.x); y.y = gelu_fast(y.y); y.z = gelu_fast(y.z); y.w = gelu_fast(y.w); }
+          if (a.yp_gain) { y.x *= gn.x; y.y *= gn.y; y.z *= gn.z; y.w *= gn.w; }
+          uint2 hi, lo;
+          if (a.q8) { split_pack_h(y.x, y.y, hi.x, lo.x); split_pack_h(y.z, y.w, hi.y, lo.y); }
+          else { split_pack(y.x, y.y, hi.x, lo.x); split_pack(y.z, y.w, hi.y, lo.y); }
+          *reinterpret_cast<uint2*>(a.yp_hi + (long long)m * a.ldyp + n) = hi;
+          *reinterpret_cast<uint2*>(a.yp_lo + (long long)m * a.ldyp + n) = lo;
+        }
+      }
+    } else {
+      for (int i = half * 32 + lane; i < rows_all; i += 64) {
+        const int n = n_first + i;
+        const float* cp = a.sk_R ? lin_carry_of(a, n) : nullptr;
+        const float old = resid ? __ldcg(a.Y + (long long)m * a.ldy + n) : 0.f;
+        float y = 0.f;
+        for (int s0 = 0; s0 < S; s0 += 16) {
+          float v[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = (s0 + j < S) ? __ldcg(a.part + ((size_t)(s0 + j) * SPS_MAX_ROWS + m) * N + n) : 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) y += v[j];
+        }
+        if (cp) for (int sp = 0; sp < S; ++sp) y += __ldcg(cp + ((size_t)sp * SPS_MAX_ROWS + m) * 128);
+        if (a.wscale[0]) { int rin; const int mat = mat_of(a, n, rin); y *= __ldg(a.wscale[mat] + rin); }
+        if (row_scale) y *= rs;
+        if (resid) { y += old; ssq += y * y; }
+        a.Y[(long long)m * a.ldy + n] = y;
+        if (a.yp_hi) {
+          if (a.yp_act == PRO_GELU) y = gelu_fast(y);
+          if (a.yp_gain) y *= __ldg(a.yp_gain + n);
+          if (a.q8) {
+            const __half h = __float2half_rn(y);
+            reinterpret_cast<__half*>(a.yp_hi)[(long long)m * a.ldyp + n] = h;
+            reinterpret_cast<__half*>(a.yp_lo)[(long long)m * a.ldyp + n] = __float2half_rn(y - __half2float(h));
+          } else {
+            const __nv_bfloat16 h = __float2bfloat16_rn(y);
+            a.yp_hi[(long long)m * a.ldyp + n] = h;
+            a.yp_lo[(long long)m * a.ldyp + n] = __float2bfloat16_rn(y - __bfloat162float(h));
+          }
+        }
+      }
+    }
+    if (resid) {
+      ssq = warp_sum(ssq);
+      if (lane == 0) s_half[m][half] = ssq;
+    }
+  }
+  if (resid) {
+    __syncthreads();
+    if (tid < a.M) a.ssq_out[SSQ_IDX(part_idx, tid)] = s_half[tid][0] + s_half[tid][1];
+  }
+}
+
 __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, int rows_all, float* sq_s, int sq_cap,
                                    float* ssq_s, const float* row_scale) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
@@ -223,6 +359,14 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
             for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
           }
         }
+        if (a.sk_R) {
+          // tensor-core kernel: the one CTA boundary that may fall inside this 128-row tile left its piece in `carry`
+          const float* cp = lin_carry_of(a, n);
+          if (cp) {
+            cp += (size_t)m * 128;
+            for (int sp = 0; sp < S; ++sp) y = f4_add(y, __ldcg(reinterpret_cast<const float4*>(cp + (size_t)sp * SPS_MAX_ROWS * 128)));
+          }
+        }
         if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: every matrix has a multiple of 4 rows)
           int rin;
           const int mat = mat_of(a, n, rin);
@@ -259,6 +403,10 @@ __device__ void lin_epilogue_slice(const LinArgs& a, int part_idx, int n_first, 
           for (int j = 0; j < 16; ++j) v[j] = (s0 + j < S) ? __ldcg(a.part + ((size_t)(s0 + j) * SPS_MAX_ROWS + m) * N + n) : 0.f;
 #pragma unroll
           for (int j = 0; j < 16; ++j) y += v[j];
+        }
+        if (a.sk_R) {
+          const float* cp = lin_carry_of(a, n);
+          if (cp) for (int sp = 0; sp < S; ++sp) y += __ldcg(cp + ((size_t)sp * SPS_MAX_ROWS + m) * 128);
         }
         if (a.wscale[0]) { int rin; const int mat = mat_of(a, n, rin); y *= __ldg(a.wscale[mat] + rin); }
         if (row_scale) y *= row_scale[m];
@@ -563,6 +711,7 @@ struct LinTmaArgs {
   LinArgs a;
   CUtensorMap tm[3];
 };
+
 
 // Q8: int8 weights (one byte per k, 128 k per 128-byte row segment), converted to fp16 in registers; the
 // activations' halves are fp16 too.  Otherwise bf16 weights and halves.
@@ -1112,10 +1261,9 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 // ---- the split-K epilogue of the TMA kernel as a kernel of its own.  Its CTAs are small enough to sit
 // beside the layer kernel's on the same SMs: they wait for that grid to complete (the hardware's grid-wide
 // meeting), then each finishes its slice of the output columns.
-__global__ void __launch_bounds__(256, 5) lin_epilogue_kernel(const LinArgs a, int C) {   // <= 48 registers: it has to fit beside the layer kernel
-  __shared__ float sq_s[1024];
-  __shared__ float ssq_s[SPS_MAX_ROWS];
-  __shared__ float row_scale[SPS_MAX_ROWS];
+// 512 threads, <= 64 registers and ~130 bytes of shared memory: one CTA of it fits beside a layer kernel's CTA on an SM
+__global__ void __launch_bounds__(512, 2) lin_epilogue_kernel(const LinArgs a, int C) {
+  __shared__ float s_half[SPS_MAX_ROWS][2];
   const int cta = blockIdx.x, tid = threadIdx.x;
   pdl_launch_dependents();
   const int quads = (a.N + 3) >> 2;
@@ -1127,10 +1275,8 @@ __global__ void __launch_bounds__(256, 5) lin_epilogue_kernel(const LinArgs a, i
     if (n < b1) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.yp_gain + n));
   }
   pdl_wait();
-  const bool scaled = a.xp_hi && a.pro == PRO_RMSNORM;
-  if (scaled && tid < a.M) row_scale[tid] = __ldcg(reinterpret_cast<const float*>(a.counters + LIN_SCALE_SLOT) + tid);
-  __syncthreads();
-  lin_epilogue_slice(a, cta, b0, b1 - b0, sq_s, 1024, ssq_s, scaled ? row_scale : nullptr);
+  const bool scaled = a.xp_hi && a.pro == PRO_RMSNORM;   // the layer kernel left the rows' 1/rms for us
+  lin_epilogue_rows(a, cta, b0, b1 - b0, scaled ? reinterpret_cast<const float*>(a.counters + LIN_SCALE_SLOT) : nullptr, s_half);
 }
 
 // ---- fp32 weights: one warp per output row, X (after the prologue) in shared memory ---------------
@@ -1382,6 +1528,8 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
   static DevSmemCache c_b1{}, c_b2{}, c_f1{}, c_f2{}, c_t1{}, c_t2{};   // per device, like the attribute itself
   { const WaitKnobs wk = sps_wait_knobs(); a.wait_ns = wk.limit_ns; a.drop_stage = wk.drop_stage; }
   cudaError_t e;
+  LinTcPlan tcp{};
+  a.sk_R = 0;
   if (dtype == 0) {
     if (p.NT == 1) {
       if ((e = ensure_smem(lin_f32_kernel<1>, p.smem, c_f1)) != cudaSuccess) return e;
@@ -1390,11 +1538,24 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
       if ((e = ensure_smem(lin_f32_kernel<2>, p.smem, c_f2)) != cudaSuccess) return e;
       e = launch_k(lin_f32_kernel<2>, dim3(p.R), dim3(256), p.smem, st, a);
     }
+  } else if (p.variant == 2 && dtype == 1 && !p.tile_epi && lin_split_epilogue() && lin_tc_plan(a, p, &tcp)) {
+    // bf16 weights, several k-splits: the tcgen05 kernel, then the same split-K epilogue kernel
+    a.sk_R = tcp.R; a.sk_SPT = tcp.SPT; a.sk_tot = tcp.tot; a.sk_BR = tcp.BR; a.split_epi = 1; a.tile_epi = 0; a.q8 = 0;
+    e = lin_tc_launch(a, tcp, st);
+    if (e == cudaSuccess) {
+      static DevOnce carve{};
+      if (sps_first_on_device(carve)) {
+        e = cudaFuncSetAttribute(lin_epilogue_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+      }
+      e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(512), 0, st, a, p.R * p.S);
+    }
   } else if (p.variant == 2) {
     dim3 grid(p.R, p.S);
     const int threads = (LIN_CONSUMER_WARPS + 1) * 32;
     LinTmaArgs ta;
     ta.a = a;
+    ta.a.sk_R = 0;
     const int nmat = a.N > a.rows_per_mat ? 1 + (a.N - a.rows_per_mat + a.rows_tail - 1) / a.rows_tail : 1;
     for (int i = 0; i < 3; ++i) {
       const bool has = i < nmat;   // unused slots repeat the first matrix
@@ -1425,7 +1586,7 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
         e = cudaFuncSetAttribute(lin_epilogue_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
       }
-      e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
+      e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(512), 0, st, ta.a, p.R * p.S);
     }
   } else {
     dim3 grid(p.R, p.S);

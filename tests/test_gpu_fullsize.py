@@ -65,8 +65,29 @@ def test_scoring_pass_at_70b_layer_shapes(name):
         assert worst[which] < 5e-2, worst
     print("worst logit error target / draft:", worst)
     # the whole loop runs at these shapes and keeps its invariants
-    toks, st = h.sps_generate(prompt, 12, 4, 1.0, 3)
-    assert ((toks >= 0) & (toks < V)).all() and st["loops"] == sum(st["hist_emitted"]) and st["emitted"] - st["overshoot"] == 12
+    for K in (4, 1, 2):   # K = 1, 2: other shared-memory sizes of the cluster sampler at this vocabulary
+        toks, st = h.sps_generate(prompt, 12, K, 1.0, 3)
+        assert ((toks >= 0) & (toks < V)).all() and st["loops"] == sum(st["hist_emitted"]) and st["emitted"] - st["overshoot"] == 12
+    h.close()
+
+
+def test_scoring_pass_of_twelve_rows_at_70b_layer_shapes():
+    """9..16 rows per pass (two or three sequences' K + 1 rows) stream the weights through the same tcgen05 kernel with
+    a 32-column activation operand: twelve rows against the oracle, same tolerance."""
+    c = sps_synth.CONFIGS["70b"]
+    tc = dict(c["target"], n_layers=2)
+    wt = sps_synth.make_weights(tc, tag="target", device=DEV)
+    h = sps.Handle(tc, wt, None, None, max_seq=64, max_K=11)
+    V = tc["vocab"]
+    prompt = sps_synth.make_prompt(0, 9, V)
+    rows = np.concatenate([prompt[-1:], sps_synth.make_prompt(1, 11, V)])
+    h.sps_prefill(prompt)
+    out = torch.zeros((12, V), device=DEV)
+    h.sps_score(0, rows, out)
+    got = out.cpu().numpy().astype(np.float64)
+    want = oracle_logits(tc, wt, prompt[:-1], None, rows)
+    err = float(np.abs(got - want).max())
+    assert np.isfinite(got).all() and err < 5e-2, err
     h.close()
 
 

@@ -23,9 +23,11 @@ def restore_knobs():
     sps.sps_debug_set_wait(0, -1)
 
 
-@pytest.mark.parametrize("drop", [1, 3])     # stages of the first CTA's first two tiles (both are always its own)
-def test_linear_wait_runs_out_and_the_next_call_is_clean(drop):
-    M, N, D = 5, 4096, 4096
+# five rows: the tcgen05 kernel (the MMA lane's wait on the missing stage runs out); two rows: the mma.sync kernel (a
+# consumer warp's wait does).  Stages 1 and 3 are always among the first CTA's own.
+@pytest.mark.parametrize("drop,M", [(1, 5), (3, 5), (1, 2), (3, 2)])
+def test_linear_wait_runs_out_and_the_next_call_is_clean(drop, M):
+    N, D = 4096, 4096
     g = torch.Generator().manual_seed(3)
     W = (torch.randn((N, D), generator=g) * 0.05).to(torch.bfloat16)
     X = torch.randn((M, D), generator=g)
