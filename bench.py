@@ -365,15 +365,15 @@ def run_ours(args):
     v_gbs = vbytes * loops / (ms_verify / 1e3) / 1e9 if ms_verify > 0 else None
     d_gbs = dbytes * loops * K / (ms_draft / 1e3) / 1e9 if ms_draft > 0 and K > 0 else None
     n_lin_verify = 5 * c["target"]["n_layers"] + 1
-    roofline = {"bound": "hbm", "kernel": "lin_bf16_tma_kernel (weight-streaming linear layer) averaged over the scoring pass",
+    roofline = {"bound": "hbm", "kernel": ("lin_tc_kernel (tcgen05 weight-streaming linear layer)" if (c["target"]["dtype"] == 1 and K + 1 >= 5) else "lin_bf16_tma_kernel (weight-streaming linear layer)") + " averaged over the scoring pass",
                 "achieved": v_gbs, "peak": peak, "unit": "GB/s", "frac": (v_gbs / peak) if v_gbs else None,
                 "frac_of_8000_nominal": (v_gbs / 8000.0) if v_gbs else None, "peak_source": peak_src,
                 "bytes_per_launch": vbytes / n_lin_verify, "avg_launch_us": 1e3 * ms_verify / loops / n_lin_verify if loops else None,
-                # one ncu capture of this kernel on the 32000 x 8192 layer: dram read + write = 1.0096 x the algorithmic bytes of
+                # one ncu capture of this kernel on the 32000 x 8192 layer: dram read + write = 1.0088 x the algorithmic bytes of
                 # that launch; traffic grows with the bytes of the matrix, so the ratio is applied to the average launch of a pass
                 # (int8 weights: the capture of the 32768 x 8192 int8 layer gives 272.90 MB for 268.44 MB of weights, 1.0166 x)
                 "traffic": args.traffic if args.traffic is not None else
-                ({1: 1.0096, 2: 1.0166}.get(c["target"]["dtype"], 0) * vbytes / n_lin_verify or None)}
+                ({1: 1.0088, 2: 1.0166}.get(c["target"]["dtype"], 0) * vbytes / n_lin_verify or None)}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dec_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": {0: "f32", 1: "bf16", 2: "f16"}[c["target"]["dtype"]], "data": "synthetic",

@@ -476,6 +476,7 @@ bool lin_tc_plan(const LinArgs& a, const LinPlan& p, LinTcPlan* out) {
   t.NS = NS;
   t.smem = 512 + xbytes + (size_t)NS * stage;
   t.R = p.R < T ? p.R : T;
+  if (t.R * 10 < p.R * 9) return false;   // a layer of few 128-row tiles would leave SMs idle: the 16-row tiles of the mma.sync kernel
   if (t.R < 1 || (long long)t.R * p.S > LIN_TC_MAX_CTAS) return false;
   t.SPT = t.KBS / t.KBX;
   t.tot = T * t.SPT;
