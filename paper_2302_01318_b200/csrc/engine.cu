@@ -57,6 +57,7 @@ struct sps_handle {
   void *wa_hi = nullptr, *wa_lo = nullptr, *wu_hi = nullptr, *wu_lo = nullptr;
   void* wdq = nullptr;   // bf16 copy of the int8 matrix (or q | k | v) the prompt-pass GEMM is reading
   __nv_bfloat16 *xp_hi = nullptr, *xp_lo = nullptr, *up_hi = nullptr, *up_lo = nullptr;   // packed activations (bf16 models)
+  __nv_bfloat16 *ap_hi = nullptr, *ap_lo = nullptr;   // the attention output, packed by the attention kernel for the output projection
   float *q_logits = nullptr, *p_logits = nullptr, *part = nullptr;
   size_t part_floats = 0;   // floats of `part` ahead of the carry tiles
   int* counters = nullptr;
@@ -302,6 +303,8 @@ int run_pass_range(sps_handle* h, ModelDev& m, const PassSpec& ps, int ph0, int 
         aa.rope = m.rope; aa.dtype = act_dtype(c.dtype); aa.H = c.n_heads; aa.Hkv = kv_heads(c); aa.dh = c.d_head; aa.d = da;
         aa.max_seq = h->cfg.max_seq; aa.rows_per_seq = ps.rows_per_seq; aa.B = B;
         aa.mode = ps.mode; aa.t = ps.t; aa.c0 = ps.c0;
+        // bf16 models: the output also as bf16 halves, ready for the output projection's tensor-core operand
+        if (m.packed && c.dtype == 1) { aa.out_hi = h->ap_hi; aa.out_lo = h->ap_lo; }
         CU(h, attn_launch(aa, st)); h->launches++;
       }
       {  // x += Wo o ; also sum(x^2) for the FFN norm.  A shard's Wo (its columns) gives a partial update instead.
@@ -309,6 +312,7 @@ int run_pass_range(sps_handle* h, ModelDev& m, const PassSpec& ps, int ph0, int 
         a.W[0] = m.wo[l]; a.rows_per_mat = d; a.N = d; a.D = da; a.M = rows;
         if (c.dtype == 2) a.wscale[0] = m.wo_s[l];
         a.X = h->attn; a.ldx = da; a.x_row0 = 0; a.x_rowstep = 1; a.pro = PRO_NONE;
+        if (m.packed && c.dtype == 1) { a.xp_hi = h->ap_hi; a.xp_lo = h->ap_lo; }
         const LinPlan pl = lin_plan(c.dtype, rows, a.N, a.D, h->num_sm);
         if (tp) { a.epi = EPI_STORE; a.Y = h->tp_send; a.ldy = d; }
         else {
@@ -810,6 +814,8 @@ int sps_create(const sps_weights* target_w, const sps_weights* draft_w, const sp
       {(void**)&h->up, sizeof(float) * SPS_MAX_ROWS * (size_t)fmax},
       {(void**)&h->xp_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
       {(void**)&h->xp_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->ap_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
+      {(void**)&h->ap_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)dmax},
       {(void**)&h->up_hi, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
       {(void**)&h->up_lo, sizeof(__nv_bfloat16) * SPS_MAX_ROWS * (size_t)fmax},
       {(void**)&h->ssqA, sizeof(float) * LIN_MAX_R * MR},
@@ -864,7 +870,7 @@ int sps_destroy(sps_handle* h) {
   for (auto& kv : h->g_verify) cudaGraphExecDestroy(kv.second);
   free_model(h->tgt);
   free_model(h->drf);
-  void* bufs[] = {h->wdq, h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
+  void* bufs[] = {h->wdq, h->wx, h->wqkv, h->watt, h->wpart, h->wa_hi, h->wa_lo, h->wu_hi, h->wu_lo, h->xp_hi, h->xp_lo, h->ap_hi, h->ap_lo, h->up_hi, h->up_lo, h->x, h->qkv, h->attn, h->up, h->ssqA, h->ssqB, h->q_logits, h->p_logits, h->part,
                   h->counters, h->tile_ctr, h->p_stats, h->tp_send, h->tp_inbox, h->tp_flags, h->tp_epoch, h->res, h->dst, h->hst.n, h->hst.limit, h->hst.tokens, h->hst.drafts, h->hst.row_tok,
                   h->hst.row_pos, h->hst.done_counter};
   for (void* p : bufs) if (p) cudaFree(p);

@@ -206,52 +206,59 @@ __device__ void lin_epilogue_rows(const LinArgs& a, int part_idx, int n_first, i
                    (!a.yp_hi || (((a.ldyp & 3) == 0) && ((((size_t)a.yp_hi | (size_t)a.yp_lo) & 7) == 0) &&
                                  (!a.yp_gain || (((size_t)a.yp_gain & 15) == 0))));
   const size_t sstride = (size_t)SPS_MAX_ROWS * N, cstride = (size_t)SPS_MAX_ROWS * 128;
-  for (int m = warp >> 1; m < a.M; m += 8) {
+  for (int m = warp >> 1; m < a.M; m += (int)(blockDim.x >> 6)) {
     float ssq = 0.f;
     const float rs = row_scale ? __ldcg(row_scale + m) : 1.f;
     if (vec) {
-      const int items = rows_all >> 2;
-      for (int i = half * 32 + lane; i < items; i += 64) {
-        const int n = n_first + 4 * i;
+      // More than four k-splits: four neighbouring lanes share an item, each adds a quarter of the splits (and of the
+      // carry pieces), and the quarters meet in lane order -- so that a slice of few items still costs one trip to L2.
+      const int items = rows_all >> 2, SG = S > 4 ? 4 : 1, PL = (S + SG - 1) / SG, sub = SG == 4 ? (lane & 3) : 0;
+      const int per_warp = 32 / SG, mine = SG == 4 ? (lane >> 2) : lane;
+      const int iters = (items + 2 * per_warp - 1) / (2 * per_warp);
+      for (int it = 0; it < iters; ++it) {
+        const int i = it * 2 * per_warp + half * per_warp + mine;
+        const bool live = i < items;
+        const int n = n_first + 4 * (live ? i : 0);
         float* dst = a.Y + (long long)m * a.ldy + n;
         const float* src = a.part + (size_t)m * N + n;
-        const float* cp = a.sk_R ? lin_carry_of(a, n) : nullptr;
+        const float* cp = (a.sk_R && live) ? lin_carry_of(a, n) : nullptr;
         float4 old = make_float4(0.f, 0.f, 0.f, 0.f), gn = make_float4(1.f, 1.f, 1.f, 1.f), ws = gn, y = old;
-        if (resid) old = __ldcg(reinterpret_cast<const float4*>(dst));
-        if (a.yp_hi && a.yp_gain) gn = __ldg(reinterpret_cast<const float4*>(a.yp_gain + n));
-        if (a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: every matrix has a multiple of 4 rows)
+        const bool fin = live && sub == 0;     // the lane that finishes the item
+        if (fin && resid) old = __ldcg(reinterpret_cast<const float4*>(dst));
+        if (fin && a.yp_hi && a.yp_gain) gn = __ldg(reinterpret_cast<const float4*>(a.yp_gain + n));
+        if (fin && a.wscale[0]) {   // int8 weights: the rows' scales (n..n+3 lie in one matrix: every matrix has a multiple of 4 rows)
           int rin;
           const int mat = mat_of(a, n, rin);
           ws = __ldg(reinterpret_cast<const float4*>(a.wscale[mat] + rin));
         }
-        if (S <= 4) {
-          float4 v[4], c[4];
+        if (live) {
+          const int s_lo = sub * PL, s_hi = min(S, s_lo + PL);
+          for (int s0 = s_lo; s0 < s_hi; s0 += 4) {
+            float4 v[4], c[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            v[j] = j < S ? __ldcg(reinterpret_cast<const float4*>(src + j * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            c[j] = (cp && j < S) ? __ldcg(reinterpret_cast<const float4*>(cp + (size_t)m * 128 + j * cstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-          y = f4_add(f4_add(f4_add(v[0], v[1]), v[2]), v[3]);
-          if (cp) y = f4_add(f4_add(f4_add(f4_add(y, c[0]), c[1]), c[2]), c[3]);
-        } else {
-          for (int s0 = 0; s0 < S; s0 += 8) {
-            float4 v[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              v[j] = s0 + j < S ? __ldcg(reinterpret_cast<const float4*>(src + (s0 + j) * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) y = f4_add(y, v[j]);
-          }
-          if (cp)
-            for (int s0 = 0; s0 < S; s0 += 8) {
-              float4 c[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                c[j] = s0 + j < S ? __ldcg(reinterpret_cast<const float4*>(cp + (size_t)m * 128 + (s0 + j) * cstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) y = f4_add(y, c[j]);
+            for (int j = 0; j < 4; ++j) {
+              v[j] = s0 + j < s_hi ? __ldcg(reinterpret_cast<const float4*>(src + (s0 + j) * sstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+              c[j] = (cp && s0 + j < s_hi) ? __ldcg(reinterpret_cast<const float4*>(cp + (size_t)m * 128 + (s0 + j) * cstride)) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) y = f4_add(y, v[j]);
+            if (cp) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) y = f4_add(y, c[j]);
+            }
+          }
         }
+        if (SG == 4) {
+          // quarters 1, 2, 3 join quarter 0 in that order
+#pragma unroll
+          for (int q = 1; q < 4; ++q) {
+            float4 o;
+            o.x = __shfl_down_sync(0xffffffffu, y.x, q, 4); o.y = __shfl_down_sync(0xffffffffu, y.y, q, 4);
+            o.z = __shfl_down_sync(0xffffffffu, y.z, q, 4); o.w = __shfl_down_sync(0xffffffffu, y.w, q, 4);
+            if (sub == 0) y = f4_add(y, o);
+          }
+        }
+        if (!fin) continue;
         if (a.wscale[0]) { y.x *= ws.x; y.y *= ws.y; y.z *= ws.z; y.w *= ws.w; }
         if (row_scale) { y.x *= rs; y.y *= rs; y.z *= rs; y.w *= rs; }
         if (resid) {
@@ -1261,9 +1268,10 @@ __global__ void __launch_bounds__((LIN_CONSUMER_WARPS + 1) * 32, 1) lin_bf16_tma
 // ---- the split-K epilogue of the TMA kernel as a kernel of its own.  Its CTAs are small enough to sit
 // beside the layer kernel's on the same SMs: they wait for that grid to complete (the hardware's grid-wide
 // meeting), then each finishes its slice of the output columns.
-// 512 threads, <= 64 registers and ~130 bytes of shared memory: one CTA of it fits beside a layer kernel's CTA on an SM
-__global__ void __launch_bounds__(512, 2) lin_epilogue_kernel(const LinArgs a, int C) {
-  __shared__ float s_half[SPS_MAX_ROWS][2];
+// 512 threads, ~130 bytes of shared memory, and between 65 and 96 registers: one CTA of it fits beside a layer kernel's
+// CTA on an SM (96 x 512 + the layer's 64 x 192 registers), but never two on one SM, not even on an SM the layer's grid
+// left idle -- two would keep the next layer's CTA off that SM until the epilogue is over.
+__device__ __forceinline__ void lin_epilogue_body(const LinArgs& a, int C, float (*s_half)[2]) {
   const int cta = blockIdx.x, tid = threadIdx.x;
   pdl_launch_dependents();
   const int quads = (a.N + 3) >> 2;
@@ -1277,6 +1285,16 @@ __global__ void __launch_bounds__(512, 2) lin_epilogue_kernel(const LinArgs a, i
   pdl_wait();
   const bool scaled = a.xp_hi && a.pro == PRO_RMSNORM;   // the layer kernel left the rows' 1/rms for us
   lin_epilogue_rows(a, cta, b0, b1 - b0, scaled ? reinterpret_cast<const float*>(a.counters + LIN_SCALE_SLOT) : nullptr, s_half);
+}
+__global__ void __maxnreg__(96) lin_epilogue_kernel(const LinArgs a, int C) {
+  __shared__ float s_half[SPS_MAX_ROWS][2];
+  lin_epilogue_body(a, C, s_half);
+}
+// The same with 256 threads and at most 88 registers, beside the mma.sync layer kernel (288 threads x 144 registers):
+// eight warps finish four rows at a time.
+__global__ void __maxnreg__(88) lin_epilogue_small_kernel(const LinArgs a, int C) {
+  __shared__ float s_half[SPS_MAX_ROWS][2];
+  lin_epilogue_body(a, C, s_half);
 }
 
 // ---- fp32 weights: one warp per output row, X (after the prologue) in shared memory ---------------
@@ -1348,7 +1366,7 @@ __global__ void __launch_bounds__(256) lin_f32_kernel(const LinArgs a) {
 // ------------------------------------------------------------------------------------------------
 static const size_t kSmemBudget = 200 * 1024;
 // TMA variant: everything a CTA may ask for (227 KB) less the kernel's 1 KB of static shared memory and a little slack
-static const size_t kSmemTma = 225 * 1024;
+static const size_t kSmemTma = 224 * 1024;
 
 static bool lin_tile_epilogue() {   // tuning: SPS_LIN_TILE_EPI=0 goes back to the epilogue kernel
   static const bool on = [] { const char* e = getenv("SPS_LIN_TILE_EPI"); return !(e && atoi(e) == 0); }();
@@ -1580,13 +1598,13 @@ cudaError_t lin_launch(int dtype, const LinArgs& a_in, const LinPlan& p, cudaStr
     }
     if (e == cudaSuccess && ta.a.split_epi) {
       // The epilogue CTAs must fit beside the layer kernel's on the same SM: that needs the same split between
-      // L1 and shared memory, i.e. the largest shared-memory carve-out, although they use only 5 KB of it.
+      // L1 and shared memory, i.e. the largest shared-memory carve-out, although they use next to none of it.
       static DevOnce carve{};
       if (sps_first_on_device(carve)) {
-        e = cudaFuncSetAttribute(lin_epilogue_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(lin_epilogue_small_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
       }
-      e = launch_k(lin_epilogue_kernel, dim3(p.R * p.S), dim3(512), 0, st, ta.a, p.R * p.S);
+      e = launch_k(lin_epilogue_small_kernel, dim3(p.R * p.S), dim3(256), 0, st, ta.a, p.R * p.S);
     }
   } else {
     dim3 grid(p.R, p.S);
