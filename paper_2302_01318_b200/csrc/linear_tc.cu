@@ -56,12 +56,14 @@ __device__ __forceinline__ void t_mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void t_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// one try: the thread sleeps in hardware until the phase completes or about a microsecond has passed (no busy polling:
+// the kernel runs at the board's power cap, and what idle lanes burn comes off the clock)
 __device__ __forceinline__ uint32_t t_mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(1000u)
       : "memory");
   return ok;
 }
@@ -352,7 +354,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) lin_tc_kernel(const __grid_cons
     for (int xa = x0; xa < x1 && ok; ++seg, buf ^= 1) {
       const int tile = xa / SPT, xe = min(x1, (tile + 1) * SPT);
       const bool mid = xa != tile * SPT;      // the tile was begun by the CTA before this one
-      ok = t_mbar_wait(bar_acc + 8 * buf, (uint32_t)(seg >> 1) & 1u, a.err, a.wait_ns, s_abort);
+      ok = lane != 0 || t_mbar_wait(bar_acc + 8 * buf, (uint32_t)(seg >> 1) & 1u, a.err, a.wait_ns, s_abort);   // one lane waits, the warp follows
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
