@@ -47,11 +47,12 @@ def test_linear_bf16_small(M, N, D):
 
 
 @pytest.mark.parametrize("M", [5, 7, 8, 9, 13, 16])
-@pytest.mark.parametrize("N,D", [(8000, 4096), (2304, 8192), (4224, 3072), (1100, 6144), (16384, 16384)])
+@pytest.mark.parametrize("N,D", [(8000, 4096), (9001, 4096), (2304, 8192), (4224, 3072), (1100, 6144), (16384, 16384)])
 def test_linear_bf16_tensor_core_kernel_pieces(M, N, D):
     """Shapes the tcgen05 weight-streaming kernel takes (bf16, five rows or more, several k-splits): tiles of 128
     weight rows cut into equal pieces per CTA, so most tiles are shared by two CTAs and meet again in the epilogue
-    kernel (partial sums + carry); N = 8000 and 1100 end in a ragged tile, 4224 x 3072 has k-ranges of 24 k-blocks,
+    kernel (partial sums + carry); N = 8000 and 1100 end in a ragged tile, N = 9001 also takes the epilogue's
+    one-feature-at-a-time path, 4224 x 3072 has k-ranges of 24 k-blocks,
     1100 rows are fewer tiles than the grid has row ranges, 16384 x 16384 has eight k-splits; 9..16 rows use the
     32-column form of the operand."""
     g = torch.Generator().manual_seed(7 * N + D + M)
